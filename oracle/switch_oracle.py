@@ -1,0 +1,210 @@
+"""CPU oracle for one Switch FFN layer (Switch Transformer, arxiv 2101.03961): forward and backward.
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT.  This file is the slow, plain definition the CUDA library is
+checked against.  Only the test-suite, the smoke check and the benchmark's CPU-baseline leg may import
+it; nothing in the product path does, and it shares no code with the CUDA path (it imports numpy only).
+
+Everything is float64 and written in the paper's notation and order:
+  h = x . W_r, p = softmax(h)                                   (Section 2.1, Eq. 1)
+  top-1 expert e_t = argmax_i p_i(x_t), gate g_t = p_{e_t}(x_t)  (Section 2.1, "Switch Routing")
+  expert capacity C = (tokens / experts) x capacity factor       (Section 2.2, Eq. 3)
+  slots in token order, tokens beyond the capacity are dropped   (Section 2.2, Fig. 3; appendix router pseudo-code)
+  auxiliary loss alpha . N . sum_i f_i P_i                       (Section 2.2, Eq. 4-6)
+  expert FFN  y = ReLU(x W_in) W_out, no bias                    (Section 5, "Reviewing the FFN layer")
+  layer output y_t = g_t . E_{e_t}(x_t)                          (Section 2.1, Eq. 2 with k = 1; Fig. 2)
+The backward pass is the derivative of exactly those formulas (the paper leaves it to autodiff): the
+gate keeps the router differentiable (Section 2.1), P is differentiable and f is not (Section 2.2).
+
+Readings taken where the paper is silent or its listing is garbled (each is checked by a pin test):
+  * capacity is floor(T * cf / E); positions are 0-based counts of earlier tokens with the same expert, and
+    an expert keeps its first C tokens in token order (the listing's 1-based cumsum compared with `less`
+    would keep C - 1, whereas Fig. 3 gives every expert a batch of exactly the capacity of Eq. 3);
+  * f_i counts the argmax before the capacity cut (Eq. 5 is the argmax indicator);
+  * argmax ties go to the lowest expert index;
+  * a dropped token's output row is 0 (its gate is masked to 0; the residual add belongs to the caller);
+  * the gate multiplies in full precision (no bfloat16 rounding of the combine weights);
+  * one call is one routing group; the row order of x is the token order;
+  * ReLU'(0) = 0;
+  * an optional constant per-expert bias may be added to the logits (used by the overflow-stress
+    workload only; the paper's router has none).
+
+All functions here are pinned by tests/test_oracle_pins.py: none is "parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+F64 = np.float64
+
+
+def expert_capacity(T: int, E: int, capacity_factor: float) -> int:
+    """Eq. 3: expert capacity = (tokens per batch / number of experts) x capacity factor, floored, at most T."""
+    C = int(math.floor(float(T) * float(capacity_factor) / float(E)))
+    return min(C, T)
+
+
+def router_logits(x, W_r, router_bias=None):
+    """Section 2.1: h(x) = W_r . x for every token; x [T, d], W_r [d, E] -> h [T, E] (float64)."""
+    h = np.asarray(x, dtype=F64) @ np.asarray(W_r, dtype=F64)
+    if router_bias is not None:
+        h = h + np.asarray(router_bias, dtype=F64)[None, :]
+    return h
+
+
+def router_probs(h):
+    """Eq. 1: p_i(x) = exp(h_i) / sum_j exp(h_j), evaluated with the row maximum subtracted."""
+    z = h - h.max(axis=1, keepdims=True)
+    ez = np.exp(z)
+    return ez / ez.sum(axis=1, keepdims=True)
+
+
+def top1(p):
+    """Switch routing (k = 1): expert index e_t = argmax_i p[t, i] (lowest index on ties), gate g_t = p[t, e_t]."""
+    e = np.argmax(p, axis=1).astype(np.int64)
+    g = p[np.arange(p.shape[0]), e]
+    return e, g
+
+
+def load_balance_loss(p, e, alpha: float):
+    """Eq. 4-6: alpha . N . sum_i f_i . P_i with f_i the argmax fraction and P_i the mean probability."""
+    T, N = p.shape
+    f = np.bincount(e, minlength=N).astype(F64) / T        # Eq. 5
+    P = p.sum(axis=0) / T                                    # Eq. 6
+    return float(alpha * N * np.dot(f, P)), f, P             # Eq. 4
+
+
+def dispatch_plan(e, E: int, C: int):
+    """Slot assignment in token order with the capacity cut (Section 2.2, Fig. 3).
+
+    pos[t]  = number of earlier tokens routed to the same expert (0-based)
+    keep[t] = pos[t] < C
+    slot[t] = e[t] * C + pos[t] for kept tokens, -1 for dropped ones
+    token_of_slot[s] = the token stored in slot s, -1 for an empty slot
+    count[i] = tokens whose argmax is expert i (before the cut); kept[i] = min(count[i], C)
+    """
+    e = np.asarray(e, dtype=np.int64)
+    T = e.shape[0]
+    pos = np.zeros(T, dtype=np.int64)
+    running = np.zeros(E, dtype=np.int64)
+    for t in range(T):
+        pos[t] = running[e[t]]
+        running[e[t]] += 1
+    count = running.copy()
+    keep = pos < C
+    slot = np.where(keep, e * C + pos, -1)
+    token_of_slot = np.full(E * C, -1, dtype=np.int64)
+    token_of_slot[slot[keep]] = np.flatnonzero(keep)
+    kept = np.minimum(count, C)
+    return {"pos": pos, "keep": keep, "slot": slot, "token_of_slot": token_of_slot, "count": count, "kept": kept}
+
+
+def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None,
+                   capacity: int | None = None, expert_index=None, experts=None):
+    """Forward of the Switch FFN layer for one routing group.
+
+    x [T, d]; W_r [d, E]; W_in [E, d, f]; W_out [E, f, d].  `capacity` overrides Eq. 3 when given.
+    `expert_index`, when given, replaces the argmax (used to follow a legitimate near-tie flip of the
+    device router); the gate is then p[t, expert_index[t]].  `experts`, when given, restricts the
+    expert FFN work to that subset (rows of y for other experts' tokens stay 0): the router, plan and
+    loss are always computed for every token.  W_in / W_out may be any object indexable by expert.
+    Returns a dict with every intermediate the staged comparisons need.
+    """
+    x64 = np.asarray(x, dtype=F64)
+    T, d = x64.shape
+    E = np.asarray(W_r).shape[1]
+    h = router_logits(x64, W_r, router_bias)
+    p = router_probs(h)
+    if expert_index is None:
+        e, g = top1(p)
+    else:
+        e = np.asarray(expert_index, dtype=np.int64)
+        g = p[np.arange(T), e]
+    aux, f, P = load_balance_loss(p, e, alpha)
+    C = expert_capacity(T, E, capacity_factor) if capacity is None else int(capacity)
+    plan = dispatch_plan(e, E, C)
+    keep = plan["keep"]
+
+    y = np.zeros((T, d), dtype=F64)
+    u = {}                                   # per expert: pre-activation of its kept tokens
+    o = np.zeros((T, d), dtype=F64)          # un-gated expert output E_i(x_t); 0 for dropped tokens
+    todo = range(E) if experts is None else experts
+    for i in todo:
+        tok = np.flatnonzero(keep & (e == i))            # kept tokens of expert i, in token order
+        if tok.size == 0:
+            continue
+        u_i = x64[tok] @ np.asarray(W_in[i], dtype=F64)          # h = x W_in
+        a_i = np.maximum(u_i, 0.0)                               # ReLU(h)
+        o_i = a_i @ np.asarray(W_out[i], dtype=F64)              # y = ReLU(h) W_out
+        u[i] = u_i
+        o[tok] = o_i
+        y[tok] = g[tok, None] * o_i                              # Eq. 2 with one selected expert
+    out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "y": y, "o": o, "u": u,
+           "T": T, "E": E, "alpha": alpha}
+    out.update(plan)
+    return out
+
+
+def switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=None, want_weight_grads=True):
+    """Backward of switch_forward for upstream gradients dy [T, d] (of y) and d_aux (of the auxiliary loss).
+
+    Returns dx [T, d], dW_r [d, E], db [E] (router-bias gradient), dW_in / dW_out as dicts expert -> array
+    (experts with no kept token get zeros), plus dgate [T] and dh [T, E] for staged comparisons.
+    """
+    x64 = np.asarray(x, dtype=F64)
+    dy64 = np.asarray(dy, dtype=F64)
+    W_r64 = np.asarray(W_r, dtype=F64)
+    T, d = x64.shape
+    E = W_r64.shape[1]
+    p, e, g, keep, alpha = fwd["p"], fwd["e"], fwd["g"], fwd["keep"], fwd["alpha"]
+
+    dx = np.zeros((T, d), dtype=F64)
+    dgate = np.zeros(T, dtype=F64)
+    dW_in, dW_out = {}, {}
+    todo = range(E) if experts is None else experts
+    for i in todo:
+        tok = np.flatnonzero(keep & (e == i))
+        W_in_i = np.asarray(W_in[i], dtype=F64)
+        W_out_i = np.asarray(W_out[i], dtype=F64)
+        if tok.size == 0:
+            if want_weight_grads:
+                dW_in[i] = np.zeros_like(W_in_i)
+                dW_out[i] = np.zeros_like(W_out_i)
+            continue
+        u_i = fwd["u"][i]
+        a_i = np.maximum(u_i, 0.0)
+        do_i = g[tok, None] * dy64[tok]                 # y = g . o        =>  do = g . dy
+        dgate[tok] = np.sum(dy64[tok] * fwd["o"][tok], axis=1)   #          =>  dg = <dy, o>
+        da_i = do_i @ W_out_i.T                         # o = a W_out
+        du_i = da_i * (u_i > 0.0)                       # a = ReLU(u), ReLU'(0) = 0
+        dx[tok] = du_i @ W_in_i.T                       # u = x W_in
+        if want_weight_grads:
+            dW_out[i] = a_i.T @ do_i
+            dW_in[i] = x64[tok].T @ du_i
+
+    # Router: total loss depends on p through the kept tokens' gates and through P in the auxiliary loss
+    # (f is piecewise constant, hence no gradient).  aux = alpha . E . sum_i f_i . (1/T) sum_t p[t, i].
+    G = np.broadcast_to((d_aux * alpha * E / T) * fwd["f"][None, :], (T, E)).copy()
+    kept_tok = np.flatnonzero(keep)
+    G[kept_tok, e[kept_tok]] += dgate[kept_tok]
+    dh = p * (G - np.sum(p * G, axis=1, keepdims=True))     # softmax Jacobian applied to G
+    dW_r = x64.T @ dh
+    db = dh.sum(axis=0)
+    dx_router = dh @ W_r64.T
+    dx = dx + dx_router
+    return {"dx": dx, "dW_r": dW_r, "db": db, "dW_in": dW_in, "dW_out": dW_out, "dgate": dgate, "dh": dh,
+            "dx_router": dx_router, "G": G}
+
+
+def router_backward_given_dgate(p, e, keep, count, dgate, x, W_r, alpha: float, d_aux: float = 1.0):
+    """The router's part of the backward pass alone, for a caller-supplied gate gradient dgate [T]."""
+    p = np.asarray(p, dtype=F64)
+    T, E = p.shape
+    f = np.asarray(count, dtype=F64) / T
+    G = np.broadcast_to((d_aux * alpha * E / T) * f[None, :], (T, E)).copy()
+    kept_tok = np.flatnonzero(keep)
+    G[kept_tok, np.asarray(e)[kept_tok]] += np.asarray(dgate, dtype=F64)[kept_tok]
+    dh = p * (G - np.sum(p * G, axis=1, keepdims=True))
+    x64 = np.asarray(x, dtype=F64)
+    return {"dh": dh, "dW_r": x64.T @ dh, "dx_router": dh @ np.asarray(W_r, dtype=F64).T}

@@ -1,0 +1,347 @@
+"""Pins for the CPU oracle: each test checks oracle/switch_oracle.py against something other than itself.
+
+What the paper and the mathematics fix: Eq. 3 values, a hand-worked example, a literal one-hot
+dispatch/combine formulation (the appendix pseudo-code's data flow, rebuilt here with dense tensors),
+brute-force position counting, the E = 1 reduction to a dense FFN, the closed forms of the auxiliary
+loss, constructed routings with a known answer, and central finite differences for the backward pass.
+"""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import switch_oracle as so
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand_layer(T, d, f, E, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((T, d))
+    W_r = rng.standard_normal((d, E)) * scale / math.sqrt(d)
+    W_in = rng.standard_normal((E, d, f)) / math.sqrt(d)
+    W_out = rng.standard_normal((E, f, d)) / math.sqrt(f)
+    return x, W_r, W_in, W_out
+
+
+# ------------------------------------------------------------------ Eq. 3
+def test_capacity_matches_eq3_table():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "capacity_eq3.txt")) if l.strip() and not l.startswith("#")]
+    assert len(rows) >= 5
+    for T, E, cf, C in rows:
+        assert so.expert_capacity(int(T), int(E), float(cf)) == int(C)
+
+
+def test_capacity_floor_and_cap():
+    assert so.expert_capacity(10, 4, 1.0) == 2          # 2.5 floored
+    assert so.expert_capacity(10, 4, 1.25) == 3         # 3.125 floored
+    assert so.expert_capacity(8, 1, 2.0) == 8           # never more slots than tokens
+
+
+# ------------------------------------------------------------------ hand-worked example
+def test_hand_worked_example():
+    g = json.load(open(os.path.join(GOLDEN, "hand_example.json")))
+    W_r = np.array(g["W_r_times_1_over_ln3"], dtype=float) * math.log(3.0)
+    out = so.switch_forward(np.array(g["x"], float), W_r, np.array(g["W_in"], float), np.array(g["W_out"], float),
+                            g["capacity_factor"], g["alpha"])
+    ex = g["expect"]
+    np.testing.assert_allclose(out["p"], ex["p"], rtol=0, atol=1e-14)
+    assert out["e"].tolist() == ex["e"]
+    np.testing.assert_allclose(out["g"], ex["g"], atol=1e-14)
+    assert out["C"] == ex["C"]
+    assert out["pos"].tolist() == ex["pos"]
+    assert out["keep"].astype(int).tolist() == ex["keep"]
+    assert out["slot"].tolist() == ex["slot"]
+    assert out["count"].tolist() == ex["count"]
+    assert out["kept"].tolist() == ex["kept"]
+    np.testing.assert_allclose(out["y"], ex["y"], atol=1e-13)
+    np.testing.assert_allclose(out["f"], ex["f"], atol=1e-15)
+    np.testing.assert_allclose(out["P"], ex["P"], atol=1e-14)
+    assert abs(out["aux"] - ex["aux"]) < 1e-15
+
+
+# ------------------------------------------------------------------ softmax / gate
+def test_softmax_rows_sum_to_one_and_gate_bounds():
+    x, W_r, _, _ = _rand_layer(200, 16, 8, 12, seed=1, scale=3.0)
+    p = so.router_probs(so.router_logits(x, W_r))
+    np.testing.assert_allclose(p.sum(1), 1.0, atol=1e-14)
+    e, g = so.top1(p)
+    assert np.all(g >= 1.0 / 12 - 1e-15) and np.all(g <= 1.0)
+    assert np.all(p[np.arange(200), e] == p.max(1))
+
+
+def test_softmax_against_direct_formula_and_shift_invariance():
+    rng = np.random.default_rng(2)
+    h = rng.standard_normal((7, 5))
+    direct = np.array([[math.exp(h[t, i]) / sum(math.exp(h[t, j]) for j in range(5)) for i in range(5)]
+                       for t in range(7)])
+    np.testing.assert_allclose(so.router_probs(h), direct, rtol=1e-14)
+    np.testing.assert_allclose(so.router_probs(h + 1000.0), direct, rtol=1e-12)   # no overflow, same value
+
+
+def test_logits_orientation_and_bias():
+    # h[t, i] = sum_k x[t, k] W_r[k, i] (+ b_i): a transposed operand or dropped bias changes these numbers.
+    x = np.array([[1.0, 2.0, 3.0]])
+    W_r = np.array([[1.0, 0.0], [0.0, 10.0], [100.0, 0.0]])
+    np.testing.assert_array_equal(so.router_logits(x, W_r), [[301.0, 20.0]])
+    np.testing.assert_array_equal(so.router_logits(x, W_r, np.array([0.5, -1.0])), [[301.5, 19.0]])
+
+
+def test_argmax_tie_goes_to_lowest_index():
+    p = np.array([[0.4, 0.4, 0.2], [0.1, 0.45, 0.45]])
+    e, g = so.top1(p)
+    assert e.tolist() == [0, 1] and g.tolist() == [0.4, 0.45]
+
+
+# ------------------------------------------------------------------ dispatch plan
+def _brute_force_plan(e, E, C):
+    T = len(e)
+    pos = [sum(1 for s in range(t) if e[s] == e[t]) for t in range(T)]          # O(T^2) definition
+    keep = [pos[t] < C for t in range(T)]
+    slot = [e[t] * C + pos[t] if keep[t] else -1 for t in range(T)]
+    tos = [-1] * (E * C)
+    for t in range(T):
+        if keep[t]:
+            tos[slot[t]] = t
+    count = [sum(1 for t in range(T) if e[t] == i) for i in range(E)]
+    return pos, keep, slot, tos, count
+
+
+@pytest.mark.parametrize("T,E,C,seed", [(97, 5, 11, 0), (64, 8, 8, 1), (200, 3, 50, 2), (33, 7, 1, 3)])
+def test_dispatch_plan_matches_brute_force(T, E, C, seed):
+    rng = np.random.default_rng(seed)
+    e = rng.integers(0, E, size=T)
+    e[rng.random(T) < 0.4] = 0                      # skew so that expert 0 overflows
+    plan = so.dispatch_plan(e, E, C)
+    pos, keep, slot, tos, count = _brute_force_plan(e.tolist(), E, C)
+    assert plan["pos"].tolist() == pos
+    assert plan["keep"].tolist() == keep
+    assert plan["slot"].tolist() == slot
+    assert plan["token_of_slot"].tolist() == tos
+    assert plan["count"].tolist() == count
+    assert plan["kept"].tolist() == [min(c, C) for c in count]
+    # invariants: kept slots of an expert are 0..kept-1 in increasing token order
+    for i in range(E):
+        toks = [t for t in plan["token_of_slot"][i * C:(i + 1) * C] if t >= 0]
+        assert toks == sorted(toks) and len(toks) == plan["kept"][i]
+        assert all(plan["token_of_slot"][i * C + j] >= 0 for j in range(plan["kept"][i]))
+    assert plan["kept"].sum() <= min(T, E * C)
+
+
+def test_round_robin_routing_has_no_drops_and_uniform_f():
+    # x_t = c * unit(t mod E), W_r = identity block  =>  e_t = t mod E, pos_t = floor(t / E), nothing dropped at cf = 1
+    T, E, d = 64, 8, 8
+    x = np.zeros((T, d))
+    x[np.arange(T), np.arange(T) % E] = 5.0
+    W_r = np.eye(d, E)
+    W_in = np.ones((E, d, 4))
+    W_out = np.ones((E, 4, d))
+    out = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01)
+    assert out["e"].tolist() == [t % E for t in range(T)]
+    assert out["pos"].tolist() == [t // E for t in range(T)]
+    assert out["keep"].all() and out["C"] == 8
+    assert abs(out["aux"] - 0.01) < 1e-15            # f uniform => aux = alpha whatever P is (sum P = 1)
+
+
+def test_zero_router_sends_everything_to_expert_zero():
+    T, E, d, f = 40, 4, 6, 5
+    x, _, W_in, W_out = _rand_layer(T, d, f, E, seed=3)
+    out = so.switch_forward(x, np.zeros((d, E)), W_in, W_out, 1.0, 0.01)
+    C = out["C"]
+    assert C == 10 and (out["e"] == 0).all()
+    assert out["keep"].tolist() == [t < C for t in range(T)]         # exactly the first C tokens are kept
+    np.testing.assert_allclose(out["g"], 0.25)
+    assert abs(out["aux"] - 0.01) < 1e-15            # P uniform => aux = alpha whatever f is (sum f = 1)
+    assert np.all(out["y"][C:] == 0.0)               # dropped tokens: no computation, zero rows
+    dense = np.maximum(x[:C] @ W_in[0], 0) @ W_out[0]
+    np.testing.assert_allclose(out["y"][:C], 0.25 * dense, rtol=1e-13)
+
+
+def test_aux_loss_upper_bound_and_definition():
+    x, W_r, W_in, W_out = _rand_layer(128, 8, 4, 6, seed=4, scale=4.0)
+    out = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.03)
+    T, E = 128, 6
+    # Eq. 4-6 written as explicit loops
+    f = [sum(1 for t in range(T) if out["e"][t] == i) / T for i in range(E)]
+    P = [sum(out["p"][t, i] for t in range(T)) / T for i in range(E)]
+    assert abs(out["aux"] - 0.03 * E * sum(fi * Pi for fi, Pi in zip(f, P))) < 1e-15
+    assert out["aux"] <= 0.03 * E + 1e-15
+    assert abs(sum(f) - 1) < 1e-15 and abs(sum(P) - 1) < 1e-14
+    # f is counted before the capacity cut: it does not change when the capacity shrinks
+    out_small = so.switch_forward(x, W_r, W_in, W_out, 0.25, 0.03)
+    assert not out_small["keep"].all()
+    assert out_small["aux"] == out["aux"]
+
+
+# ------------------------------------------------------------------ whole forward
+def test_single_expert_reduces_to_dense_ffn():
+    T, d, f = 24, 10, 14
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, 1, seed=5)
+    out = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01)
+    np.testing.assert_allclose(out["g"], 1.0, atol=0)
+    np.testing.assert_allclose(out["y"], np.maximum(x @ W_in[0], 0) @ W_out[0], rtol=1e-13)
+    assert abs(out["aux"] - 0.01) < 1e-16
+    half = so.switch_forward(x, W_r, W_in, W_out, 0.5, 0.01)     # capacity 12: first 12 rows, rest zero
+    np.testing.assert_allclose(half["y"][:12], out["y"][:12], rtol=1e-13)
+    assert np.all(half["y"][12:] == 0)
+
+
+def _literal_one_hot_layer(x, W_r, W_in, W_out, cf, alpha):
+    """The layer as dense one-hot dispatch / combine tensors and einsums (the appendix's data flow)."""
+    T, d = x.shape
+    E = W_r.shape[1]
+    C = int(math.floor(T * cf / E))
+    logits = np.einsum("td,de->te", x, W_r)
+    probs = np.exp(logits - logits.max(1, keepdims=True))
+    probs /= probs.sum(1, keepdims=True)
+    index = probs.argmax(1)
+    gate = probs.max(1)
+    mask = np.eye(E)[index]                                        # [T, E] one-hot
+    density = mask.mean(0)
+    density_proxy = probs.mean(0)
+    aux = alpha * np.mean(density * density_proxy) * E * E
+    position = (np.cumsum(mask, axis=0) - 1.0) * mask              # 0-based position inside the expert
+    mask = mask * (position < C)
+    mask_flat = mask.sum(1)
+    gate = gate * mask_flat
+    pos_index = position.sum(1).astype(int)
+    pos_one_hot = np.zeros((T, C))
+    ok = pos_index < C
+    pos_one_hot[np.flatnonzero(ok), pos_index[ok]] = 1.0
+    combine = gate[:, None, None] * mask[:, :, None] * pos_one_hot[:, None, :]    # [T, E, C]
+    dispatch = (combine != 0).astype(float)
+    expert_inputs = np.einsum("td,tec->ecd", x, dispatch)
+    hidden = np.maximum(np.einsum("ecd,edf->ecf", expert_inputs, W_in), 0.0)
+    expert_outputs = np.einsum("ecf,efd->ecd", hidden, W_out)
+    y = np.einsum("ecd,tec->td", expert_outputs, combine)
+    return y, aux, dispatch
+
+
+@pytest.mark.parametrize("T,d,f,E,cf,seed", [(48, 6, 10, 4, 1.0, 0), (64, 8, 12, 8, 1.25, 1), (40, 5, 7, 5, 0.5, 2)])
+def test_index_formulation_equals_literal_one_hot_formulation(T, d, f, E, cf, seed):
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=seed, scale=2.0)
+    out = so.switch_forward(x, W_r, W_in, W_out, cf, 0.01)
+    y, aux, dispatch = _literal_one_hot_layer(x, W_r, W_in, W_out, cf, 0.01)
+    np.testing.assert_allclose(out["y"], y, rtol=1e-12, atol=1e-13)
+    assert abs(out["aux"] - aux) < 1e-15
+    C = out["C"]
+    mine = np.zeros((T, E, C))
+    for t in range(T):
+        if out["keep"][t]:
+            mine[t, out["e"][t], out["pos"][t]] = 1.0
+    np.testing.assert_array_equal(mine, dispatch)
+
+
+def test_large_capacity_is_plain_top1_mixture():
+    T, d, f, E = 50, 6, 9, 5
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=6, scale=2.0)
+    out = so.switch_forward(x, W_r, W_in, W_out, float(E), 0.01)       # capacity = T: nothing can drop
+    assert out["keep"].all()
+    for t in range(T):
+        i = out["e"][t]
+        ref = out["p"][t, i] * (np.maximum(x[t] @ W_in[i], 0) @ W_out[i])
+        np.testing.assert_allclose(out["y"][t], ref, rtol=1e-12, atol=1e-14)
+
+
+def test_expert_subset_restricts_only_ffn_work():
+    x, W_r, W_in, W_out = _rand_layer(60, 6, 8, 4, seed=7, scale=2.0)
+    full = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01)
+    part = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01, experts=[1, 3])
+    sel = np.isin(full["e"], [1, 3])
+    np.testing.assert_array_equal(part["y"][sel], full["y"][sel])
+    assert np.all(part["y"][~sel] == 0)
+    assert part["aux"] == full["aux"] and part["slot"].tolist() == full["slot"].tolist()
+
+
+# ------------------------------------------------------------------ backward
+def _loss(x, W_r, b, W_in, W_out, cf, alpha, R, d_aux, expert_index):
+    out = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_bias=b, expert_index=expert_index)
+    return float(np.sum(out["y"] * R) + d_aux * out["aux"])
+
+
+def test_backward_matches_central_finite_differences():
+    T, d, f, E, cf, alpha, d_aux = 16, 8, 16, 4, 0.75, 0.05, 1.7
+    rng = np.random.default_rng(11)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=11, scale=2.0)
+    b = rng.standard_normal(E) * 0.3
+    R = rng.standard_normal((T, d))
+    fwd = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_bias=b)
+    assert (~fwd["keep"]).sum() >= 2                       # some tokens are dropped in this case
+    srt = np.sort(fwd["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-3          # no argmax boundary within reach of the step
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    e_frozen = fwd["e"]
+    eps = 1e-6
+
+    def fd(arr, idx):
+        old = arr[idx]
+        arr[idx] = old + eps
+        lp = _loss(x, W_r, b, W_in, W_out, cf, alpha, R, d_aux, e_frozen)
+        arr[idx] = old - eps
+        lm = _loss(x, W_r, b, W_in, W_out, cf, alpha, R, d_aux, e_frozen)
+        arr[idx] = old
+        return (lp - lm) / (2 * eps)
+
+    for name, arr, grad in [("dx", x, bwd["dx"]), ("dW_r", W_r, bwd["dW_r"]), ("db", b, bwd["db"])]:
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            num[idx] = fd(arr, idx)
+        err = np.linalg.norm(num - grad) / np.linalg.norm(grad)
+        assert err < 1e-7, (name, err)
+    dW_in = np.stack([bwd["dW_in"][i] for i in range(E)])
+    dW_out = np.stack([bwd["dW_out"][i] for i in range(E)])
+    for name, arr, grad in [("dW_in", W_in, dW_in), ("dW_out", W_out, dW_out)]:
+        idxs = [tuple(rng.integers(0, s) for s in arr.shape) for _ in range(150)]
+        num = np.array([fd(arr, i) for i in idxs])
+        ana = np.array([grad[i] for i in idxs])
+        assert np.linalg.norm(num - ana) / np.linalg.norm(ana) < 1e-7, name
+
+
+def test_backward_invariants():
+    T, d, f, E = 40, 6, 8, 5
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=12, scale=3.0)
+    rng = np.random.default_rng(12)
+    dy = rng.standard_normal((T, d))
+    # make expert 4 unreachable (huge negative bias) so that it has no tokens
+    b = np.array([0.0, 0.0, 0.0, 0.0, -50.0])
+    fwd = so.switch_forward(x, W_r, W_in, W_out, 0.5, 0.0, router_bias=b)       # alpha = 0
+    assert fwd["count"][4] == 0 and (~fwd["keep"]).any()
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, dy)
+    np.testing.assert_allclose(bwd["dh"].sum(1), 0.0, atol=1e-14)            # softmax gradient sums to zero per token
+    assert np.all(bwd["dx"][~fwd["keep"]] == 0.0)                            # dropped token, alpha = 0: no gradient at all
+    assert np.all(bwd["dgate"][~fwd["keep"]] == 0.0)
+    assert np.all(bwd["dW_in"][4] == 0) and np.all(bwd["dW_out"][4] == 0)    # expert without tokens
+    # with alpha > 0 a dropped token still gets the auxiliary-loss gradient through P
+    fwd2 = so.switch_forward(x, W_r, W_in, W_out, 0.5, 0.1, router_bias=b)
+    bwd2 = so.switch_backward(fwd2, x, W_r, W_in, W_out, dy)
+    assert np.abs(bwd2["dx"][~fwd2["keep"]]).max() > 0
+
+
+def test_single_expert_backward_is_dense_ffn_backward():
+    T, d, f = 12, 5, 7
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, 1, seed=13)
+    dy = np.random.default_rng(13).standard_normal((T, d))
+    fwd = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01)
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, dy)
+    u = x @ W_in[0]
+    a = np.maximum(u, 0)
+    da = dy @ W_out[0].T
+    du = da * (u > 0)
+    np.testing.assert_allclose(bwd["dW_out"][0], a.T @ dy, rtol=1e-12)
+    np.testing.assert_allclose(bwd["dW_in"][0], x.T @ du, rtol=1e-12)
+    np.testing.assert_allclose(bwd["dx"], du @ W_in[0].T, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(bwd["dW_r"], 0.0, atol=1e-14)                 # p == 1 identically
+
+
+def test_router_backward_helper_agrees_with_full_backward():
+    T, d, f, E = 30, 6, 8, 4
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=14, scale=2.0)
+    dy = np.random.default_rng(14).standard_normal((T, d))
+    fwd = so.switch_forward(x, W_r, W_in, W_out, 0.75, 0.02)
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux=0.5)
+    rb = so.router_backward_given_dgate(fwd["p"], fwd["e"], fwd["keep"], fwd["count"], bwd["dgate"], x, W_r,
+                                        0.02, d_aux=0.5)
+    np.testing.assert_allclose(rb["dW_r"], bwd["dW_r"], rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(rb["dx_router"], bwd["dx_router"], rtol=1e-13, atol=1e-15)
