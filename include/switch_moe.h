@@ -1,0 +1,168 @@
+/*
+ * switch_moe.h -- C ABI of the Switch FFN layer (Switch Transformer, arxiv 2101.03961) for one NVIDIA B200.
+ *
+ * One call = one routing group of T tokens (rows of x, in token order).  The layer is
+ *   router      h = x . W_r (+ b), p = softmax(h) in float32          (Section 2.1, Eq. 1; Section 2.4 selective precision)
+ *   top-1       e_t = argmax_i p[t,i], gate g_t = p[t,e_t]            (Section 2.1, "Switch Routing")
+ *   capacity    C = floor(T * capacity_factor / E)                    (Section 2.2, Eq. 3)
+ *   dispatch    expert i keeps its first C tokens in token order, later ones are dropped (Section 2.2, Fig. 3)
+ *   expert FFN  o_t = ReLU(x_t W_in[e_t]) W_out[e_t], no bias         (Section 5, FFN review)
+ *   combine     y_t = g_t . o_t ; y_t = 0 for a dropped token         (Section 2.1, Eq. 2 with k = 1; Fig. 2)
+ *   aux loss    alpha . E . sum_i f_i . P_i                           (Section 2.2, Eq. 4-6)
+ * and its backward pass (derivative of the above; f carries no gradient, Section 2.2).
+ *
+ * Conventions for every entry point
+ *   - Plain C, no exceptions.  Return value: SWITCH_MOE_OK (0) or a negative switch_moe_status.
+ *   - Unless a parameter says HOST, every data pointer is a DEVICE pointer owned by the caller; the library
+ *     never allocates or frees device memory and keeps no state between calls other than what it writes into
+ *     the caller's workspace.  All tensors are dense, row-major, 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue work; they do
+ *     not synchronise unless stated.  Calls sharing one workspace must be ordered on one stream.
+ *   - dtype SWITCH_MOE_BF16: x, W_in, W_out, y, dy, dx, dW_in, dW_out are bfloat16; the router (W_r, bias, probs,
+ *     gate, dW_r, aux loss) is float32.  dtype SWITCH_MOE_F32: everything is float32.
+ *   - Gradients are overwritten, not accumulated.
+ *   - Limits: 1 <= E <= 256; d_model and d_ff multiples of 8 (bf16: multiples of 64 for the tensor-core path);
+ *     T * capacity_factor / E >= 1.
+ */
+#ifndef SWITCH_MOE_H_
+#define SWITCH_MOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum switch_moe_dtype { SWITCH_MOE_BF16 = 0, SWITCH_MOE_F32 = 1 };
+
+enum switch_moe_gemm_path {
+  SWITCH_MOE_GEMM_DEFAULT = 0, /* bf16: tcgen05 tensor-core grouped GEMM; f32: plain FP32 FMA grouped GEMM */
+  SWITCH_MOE_GEMM_SIMT = 1     /* validation only: FP32-FMA grouped GEMM for either dtype */
+};
+
+typedef enum switch_moe_status {
+  SWITCH_MOE_OK = 0,
+  SWITCH_MOE_INVALID_ARGUMENT = -1,    /* null pointer, non-positive size, capacity 0 */
+  SWITCH_MOE_UNSUPPORTED_SHAPE = -2,   /* E > 256, d_model / d_ff not a supported multiple, misaligned pointer */
+  SWITCH_MOE_WORKSPACE_TOO_SMALL = -3,
+  SWITCH_MOE_CUDA_ERROR = -4,          /* a CUDA runtime / driver call or a kernel launch failed */
+  SWITCH_MOE_DEVICE_TIMEOUT = -5       /* a bounded device-side wait gave up (see switch_moe_check_device_status) */
+} switch_moe_status;
+
+typedef struct switch_moe_config {
+  int32_t T;                 /* tokens in this routing group */
+  int32_t d_model;
+  int32_t d_ff;
+  int32_t E;                 /* number of experts (the paper's N) */
+  float capacity_factor;     /* Eq. 3 */
+  float alpha;               /* Eq. 4 coefficient */
+  int32_t capacity_override; /* 0: use Eq. 3; > 0: use this expert capacity instead */
+  int32_t dtype;             /* switch_moe_dtype */
+  int32_t gemm_path;         /* switch_moe_gemm_path */
+  int32_t reserved[5];       /* must be 0 */
+  void* const* stage_events; /* HOST array of SWITCH_MOE_STAGE_EVENTS cudaEvent_t handles, or NULL (default).
+                                When set, fwd records event i on the stream before its stage i (0 router, 1 dispatch
+                                plan, 2 gather, 3 GEMM1+ReLU, 4 GEMM2+combine) and event 5 after the last one; bwd
+                                records events 6..11 before (6 gather dy, 7 dgrad2, 8 wgrad2, 9 dgrad1, 10 wgrad1,
+                                11 router backward) and event 12 after.  For per-kernel timing only. */
+} switch_moe_config;
+
+#define SWITCH_MOE_STAGE_EVENTS 13
+
+/* Regions of the workspace that switch_moe_workspace_view can expose (all written by the library). */
+enum switch_moe_ws_region {
+  SWITCH_MOE_WS_STATUS = 0,         /* int32[16]; [0] != 0 after a device-side timeout */
+  SWITCH_MOE_WS_EXPERT_INDEX = 1,   /* int32[T]   e_t */
+  SWITCH_MOE_WS_GATE = 2,           /* float[T]   g_t (the un-masked top-1 probability, also for dropped tokens) */
+  SWITCH_MOE_WS_SLOT = 3,           /* int32[T]   e_t * C + pos_t, or -1 if dropped */
+  SWITCH_MOE_WS_TOKEN_OF_SLOT = 4,  /* int32[E*C] token stored in each slot, or -1 */
+  SWITCH_MOE_WS_COUNT = 5,          /* int32[E]   tokens whose argmax is expert i, before the capacity cut */
+  SWITCH_MOE_WS_KEPT = 6,           /* int32[E]   min(count, C) */
+  SWITCH_MOE_WS_PSUM = 7,           /* float[E]   sum_t p[t,i] */
+  SWITCH_MOE_WS_PROBS = 8,          /* float[T,E] router probabilities */
+  SWITCH_MOE_WS_XD = 9,             /* [E,C,d_model] dispatched tokens (dtype of x) */
+  SWITCH_MOE_WS_H = 10,             /* [E,C,d_ff]    ReLU(x W_in) per slot */
+  SWITCH_MOE_WS_DYD = 11,           /* [E,C,d_model] g . dy per slot (backward) */
+  SWITCH_MOE_WS_DH = 12,            /* [E,C,d_ff]    gradient of the pre-activation per slot (backward) */
+  SWITCH_MOE_WS_DGATE = 13,         /* float[T]   <dy_t, o_t> for kept tokens (backward) */
+  SWITCH_MOE_WS_DLOGITS = 14,       /* float[T,E] gradient of the router logits (backward) */
+  SWITCH_MOE_WS_REGION_COUNT = 15
+};
+
+/* Eq. 3.  HOST call.  *C_out = capacity_override if > 0, else floor(T * capacity_factor / E) capped at T.
+ * Errors: INVALID_ARGUMENT for null pointers, non-positive sizes or a resulting capacity of 0. */
+int switch_moe_capacity(const switch_moe_config* cfg, int32_t* C_out);
+
+/* HOST call.  Bytes of device workspace that fwd/bwd need for this config (a few hundred MB at Switch-Base
+ * shapes: the per-slot buffers X_d, H, dY_d, dH dominate).  The workspace must be 1024-byte aligned. */
+int switch_moe_workspace_bytes(const switch_moe_config* cfg, size_t* bytes_out);
+
+/* HOST call.  Device address and size of one workspace region (switch_moe_ws_region), for diagnostics and
+ * staged tests.  Nothing is copied. */
+int switch_moe_workspace_view(const switch_moe_config* cfg, void* workspace, int32_t region, void** ptr_out,
+                              size_t* bytes_out);
+
+/* Forward of the whole layer (all of: router, Eq. 1; top-1; Eq. 3 capacity and token-order dispatch, Fig. 3;
+ * expert FFN; gate-scaled combine, Eq. 2; auxiliary loss, Eq. 4-6).
+ *   x [T,d_model]; W_r [d_model,E] float32; router_bias float32[E] or NULL (constant added to the logits; the
+ *   paper's router has none); W_in [E,d_model,d_ff]; W_out [E,d_ff,d_model];
+ *   y [T,d_model] (out; rows of dropped tokens are written as 0); aux_loss device float[1] (out).
+ * The workspace keeps what backward needs (probs, expert index, gate, slots, X_d, H). */
+int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r, const float* router_bias,
+                   const void* W_in, const void* W_out, void* y, float* aux_loss, void* workspace,
+                   size_t workspace_bytes, void* stream);
+
+/* Backward of the whole layer, for upstream gradients dy [T,d_model] of y and the scalar d_aux of the auxiliary
+ * loss (1.0 when that loss is simply added to the model loss, Section 2.2).  `workspace` must be the one the
+ * matching switch_moe_fwd call filled, and x, W_r, W_in, W_out, y the same buffers with unchanged contents.
+ *   dx [T,d_model], dW_r [d_model,E] float32, dW_in [E,d_model,d_ff], dW_out [E,d_ff,d_model] (all out).
+ * The gate gradient uses o_t = y_t / g_t (g_t >= 1/E > 0).  f carries no gradient (Section 2.2). */
+int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, const void* x, const float* W_r,
+                   const void* W_in, const void* W_out, const void* y, void* workspace, size_t workspace_bytes,
+                   void* dx, float* dW_r, void* dW_in, void* dW_out, void* stream);
+
+/* Staged: the router alone (Eq. 1, top-1, the P-sums of Eq. 6).  Fills the workspace regions PROBS, EXPERT_INDEX,
+ * GATE and the per-block partial sums that the dispatch plan reduces into PSUM. */
+int switch_moe_router_fwd(const switch_moe_config* cfg, const void* x, const float* W_r, const float* router_bias,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* Staged: the dispatch plan alone (Eq. 3, Fig. 3, Eq. 4-6) for a caller-supplied expert index (device int32[T],
+ * e.g. the oracle's).  If expert_index is NULL the workspace's EXPERT_INDEX is used.  Fills COUNT, KEPT, SLOT,
+ * TOKEN_OF_SLOT, PSUM (from whatever partial sums the workspace holds) and, if aux_loss != NULL, the loss. */
+int switch_moe_dispatch_plan(const switch_moe_config* cfg, const int32_t* expert_index, float* aux_loss,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Staged: the router's backward alone for a caller-supplied gate gradient (device float[T]; entries of dropped
+ * tokens are ignored): G = d_aux.alpha.E.f_i/T + [i = e_t, kept].dgate_t, dh = p (G - <p,G>), dW_r = x^T dh,
+ * dx_router = dh W_r^T.  Uses PROBS, EXPERT_INDEX, SLOT, COUNT of the workspace.  dx_router [T,d_model] is written
+ * in the config's dtype (not accumulated). */
+int switch_moe_router_bwd(const switch_moe_config* cfg, const void* x, const float* W_r, const float* dgate,
+                          float d_aux, void* workspace, size_t workspace_bytes, void* dx_router, float* dW_r,
+                          void* stream);
+
+/* One training step with HOST activations: copies x_host and dy_host (pinned host memory, [T,d_model]) to the
+ * device buffers x_dev / dy_dev, runs switch_moe_fwd and switch_moe_bwd, and copies y, dx and the auxiliary loss
+ * back to y_host, dx_host, aux_host.  Weights and weight gradients stay on the device.  Synchronises the stream
+ * before returning.  x_dev, dy_dev, y_dev, dx_dev, aux_dev are caller-owned device staging buffers. */
+int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const void* dy_host, float d_aux,
+                         const float* W_r, const float* router_bias, const void* W_in, const void* W_out,
+                         void* x_dev, void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r,
+                         void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream`, reads the workspace's status word and returns SWITCH_MOE_DEVICE_TIMEOUT if a kernel
+ * gave up on a bounded wait (its results are then invalid), SWITCH_MOE_CUDA_ERROR if the stream reports an
+ * error, else SWITCH_MOE_OK.  info_out (HOST int32[16], may be NULL) receives the raw status words. */
+int switch_moe_check_device_status(const switch_moe_config* cfg, void* workspace, int32_t* info_out, void* stream);
+
+/* HOST call.  Number of this library's kernels that one switch_moe_fwd plus one switch_moe_bwd launch. */
+int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches_out);
+
+/* HOST call.  Static description of a status code. */
+const char* switch_moe_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWITCH_MOE_H_ */

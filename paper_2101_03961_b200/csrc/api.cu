@@ -1,0 +1,240 @@
+// C ABI of the Switch FFN library: argument checks, workspace planning and the launch sequences of the forward and
+// backward passes.  Every step of the layer runs in this library's own kernels; nothing here allocates device memory.
+#include <cstring>
+
+#include "switch_common.cuh"
+
+using namespace swmoe;
+
+namespace {
+
+struct Ctx {
+  Shape s;
+  Plan p;
+};
+
+int prepare(const switch_moe_config* cfg, const void* workspace, size_t workspace_bytes, bool need_ws, Ctx* c) {
+  int rc = resolve_shape(cfg, &c->s);
+  if (rc != SWITCH_MOE_OK) return rc;
+  make_plan(c->s, &c->p);
+  if (need_ws) {
+    if (workspace == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 1023u) != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+    if (workspace_bytes < c->p.total) return SWITCH_MOE_WORKSPACE_TOO_SMALL;
+  }
+  return SWITCH_MOE_OK;
+}
+
+int run_gemm(GemmOp op, const Ctx& c, const GemmArgs& a, void* ws, cudaStream_t st) {
+  return c.s.gemm_path == 0 ? launch_tc_gemm(op, c.s, c.p, a, ws, st) : launch_simt_gemm(op, c.s, c.p, a, ws, st);
+}
+
+// Optional per-stage timing: records the caller's event `i` on the stream (see switch_moe_config::stage_events).
+int mark(const switch_moe_config* cfg, int i, cudaStream_t st) {
+  if (cfg->stage_events == nullptr) return SWITCH_MOE_OK;
+  return cudaEventRecord(static_cast<cudaEvent_t>(cfg->stage_events[i]), st) == cudaSuccess ? SWITCH_MOE_OK
+                                                                                             : SWITCH_MOE_CUDA_ERROR;
+}
+
+#define SWMOE_TRY(expr)                    \
+  do {                                     \
+    int rc__ = (expr);                     \
+    if (rc__ != SWITCH_MOE_OK) return rc__; \
+  } while (0)
+
+}  // namespace
+
+extern "C" {
+
+int switch_moe_capacity(const switch_moe_config* cfg, int32_t* C_out) {
+  if (C_out == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
+  Shape s;
+  SWMOE_TRY(resolve_shape(cfg, &s));
+  *C_out = s.C;
+  return SWITCH_MOE_OK;
+}
+
+int switch_moe_workspace_bytes(const switch_moe_config* cfg, size_t* bytes_out) {
+  if (bytes_out == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, nullptr, 0, false, &c));
+  *bytes_out = c.p.total;
+  return SWITCH_MOE_OK;
+}
+
+int switch_moe_workspace_view(const switch_moe_config* cfg, void* workspace, int32_t region, void** ptr_out,
+                              size_t* bytes_out) {
+  if (ptr_out == nullptr || bytes_out == nullptr || workspace == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, nullptr, 0, false, &c));
+  const Shape& s = c.s;
+  const Plan& p = c.p;
+  const size_t T = s.T, E = s.E, C = s.C;
+  size_t off, bytes;
+  switch (region) {
+    case SWITCH_MOE_WS_STATUS: off = p.status; bytes = 16 * 4; break;
+    case SWITCH_MOE_WS_EXPERT_INDEX: off = p.expert_index; bytes = T * 4; break;
+    case SWITCH_MOE_WS_GATE: off = p.gate; bytes = T * 4; break;
+    case SWITCH_MOE_WS_SLOT: off = p.slot; bytes = T * 4; break;
+    case SWITCH_MOE_WS_TOKEN_OF_SLOT: off = p.token_of_slot; bytes = E * C * 4; break;
+    case SWITCH_MOE_WS_COUNT: off = p.count; bytes = E * 4; break;
+    case SWITCH_MOE_WS_KEPT: off = p.kept; bytes = E * 4; break;
+    case SWITCH_MOE_WS_PSUM: off = p.psum; bytes = E * 4; break;
+    case SWITCH_MOE_WS_PROBS: off = p.probs; bytes = T * E * 4; break;
+    case SWITCH_MOE_WS_XD: off = p.xd; bytes = E * C * s.d * s.elt; break;
+    case SWITCH_MOE_WS_H: off = p.h; bytes = E * C * s.f * s.elt; break;
+    case SWITCH_MOE_WS_DYD: off = p.dyd; bytes = E * C * s.d * s.elt; break;
+    case SWITCH_MOE_WS_DH: off = p.dh; bytes = E * C * s.f * s.elt; break;
+    case SWITCH_MOE_WS_DGATE: off = p.dgate; bytes = T * 4; break;
+    case SWITCH_MOE_WS_DLOGITS: off = p.dlogits; bytes = T * E * 4; break;
+    default: return SWITCH_MOE_INVALID_ARGUMENT;
+  }
+  *ptr_out = static_cast<char*>(workspace) + off;
+  *bytes_out = bytes;
+  return SWITCH_MOE_OK;
+}
+
+int switch_moe_router_fwd(const switch_moe_config* cfg, const void* x, const float* W_r, const float* router_bias,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
+  if (x == nullptr || W_r == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (!aligned16(x) || !aligned16(W_r)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  return launch_router_fwd(c.s, c.p, x, W_r, router_bias, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int switch_moe_dispatch_plan(const switch_moe_config* cfg, const int32_t* expert_index, float* aux_loss,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
+  return launch_dispatch_plan(c.s, c.p, expert_index, aux_loss, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r, const float* router_bias,
+                   const void* W_in, const void* W_out, void* y, float* aux_loss, void* workspace,
+                   size_t workspace_bytes, void* stream) {
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
+  if (!x || !W_r || !W_in || !W_out || !y || !aux_loss) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (!aligned16(x) || !aligned16(W_r) || !aligned16(W_in) || !aligned16(W_out) || !aligned16(y))
+    return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(ws_ptr<char>(workspace, c.p.status), 0, 16 * 4, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  SWMOE_TRY(mark(cfg, 0, st));
+  SWMOE_TRY(launch_router_fwd(c.s, c.p, x, W_r, router_bias, workspace, st));
+  SWMOE_TRY(mark(cfg, 1, st));
+  SWMOE_TRY(launch_dispatch_plan(c.s, c.p, nullptr, aux_loss, workspace, st));
+  SWMOE_TRY(mark(cfg, 2, st));
+  SWMOE_TRY(launch_gather_x(c.s, c.p, x, y, workspace, st));
+  GemmArgs a{};
+  a.W_in = W_in; a.W_out = W_out; a.y = y;
+  SWMOE_TRY(mark(cfg, 3, st));
+  SWMOE_TRY(run_gemm(kGemm1Relu, c, a, workspace, st));
+  SWMOE_TRY(mark(cfg, 4, st));
+  SWMOE_TRY(run_gemm(kGemm2Combine, c, a, workspace, st));
+  SWMOE_TRY(mark(cfg, 5, st));
+  return SWITCH_MOE_OK;
+}
+
+int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, const void* x, const float* W_r,
+                   const void* W_in, const void* W_out, const void* y, void* workspace, size_t workspace_bytes,
+                   void* dx, float* dW_r, void* dW_in, void* dW_out, void* stream) {
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
+  if (!dy || !x || !W_r || !W_in || !W_out || !y || !dx || !dW_r || !dW_in || !dW_out)
+    return SWITCH_MOE_INVALID_ARGUMENT;
+  if (!aligned16(dy) || !aligned16(x) || !aligned16(W_r) || !aligned16(W_in) || !aligned16(W_out) || !aligned16(y) ||
+      !aligned16(dx) || !aligned16(dW_r) || !aligned16(dW_in) || !aligned16(dW_out))
+    return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  GemmArgs a{};
+  a.W_in = W_in; a.W_out = W_out; a.dx = dx; a.dW_in = dW_in; a.dW_out = dW_out;
+  SWMOE_TRY(mark(cfg, 6, st));
+  SWMOE_TRY(launch_gather_dy(c.s, c.p, dy, y, workspace, st));
+  SWMOE_TRY(mark(cfg, 7, st));
+  SWMOE_TRY(run_gemm(kDgrad2Mask, c, a, workspace, st));
+  SWMOE_TRY(mark(cfg, 8, st));
+  SWMOE_TRY(run_gemm(kWgrad2, c, a, workspace, st));
+  SWMOE_TRY(mark(cfg, 9, st));
+  SWMOE_TRY(run_gemm(kDgrad1Scatter, c, a, workspace, st));
+  SWMOE_TRY(mark(cfg, 10, st));
+  SWMOE_TRY(run_gemm(kWgrad1, c, a, workspace, st));
+  SWMOE_TRY(mark(cfg, 11, st));
+  SWMOE_TRY(launch_router_bwd(c.s, c.p, x, W_r, ws_ptr<float>(workspace, c.p.dgate), d_aux, workspace, dx, true, dW_r,
+                              st));
+  SWMOE_TRY(mark(cfg, 12, st));
+  return SWITCH_MOE_OK;
+}
+
+int switch_moe_router_bwd(const switch_moe_config* cfg, const void* x, const float* W_r, const float* dgate,
+                          float d_aux, void* workspace, size_t workspace_bytes, void* dx_router, float* dW_r,
+                          void* stream) {
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
+  if (!x || !W_r || !dgate || !dx_router || !dW_r) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (!aligned16(x) || !aligned16(W_r) || !aligned16(dx_router) || !aligned16(dW_r))
+    return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  return launch_router_bwd(c.s, c.p, x, W_r, dgate, d_aux, workspace, dx_router, false, dW_r,
+                           static_cast<cudaStream_t>(stream));
+}
+
+int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const void* dy_host, float d_aux,
+                         const float* W_r, const float* router_bias, const void* W_in, const void* W_out,
+                         void* x_dev, void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r,
+                         void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
+  if (!x_host || !dy_host || !x_dev || !dy_dev || !y_dev || !dx_dev || !aux_dev || !y_host || !dx_host || !aux_host)
+    return SWITCH_MOE_INVALID_ARGUMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t act = (size_t)c.s.T * c.s.d * c.s.elt;
+  if (cudaMemcpyAsync(x_dev, x_host, act, cudaMemcpyHostToDevice, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  if (cudaMemcpyAsync(dy_dev, dy_host, act, cudaMemcpyHostToDevice, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  SWMOE_TRY(switch_moe_fwd(cfg, x_dev, W_r, router_bias, W_in, W_out, y_dev, aux_dev, workspace, workspace_bytes,
+                           stream));
+  if (cudaMemcpyAsync(y_host, y_dev, act, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  if (cudaMemcpyAsync(aux_host, aux_dev, sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return SWITCH_MOE_CUDA_ERROR;
+  SWMOE_TRY(switch_moe_bwd(cfg, dy_dev, d_aux, x_dev, W_r, W_in, W_out, y_dev, workspace, workspace_bytes, dx_dev, dW_r,
+                           dW_in, dW_out, stream));
+  if (cudaMemcpyAsync(dx_host, dx_dev, act, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  return SWITCH_MOE_OK;
+}
+
+int switch_moe_check_device_status(const switch_moe_config* cfg, void* workspace, int32_t* info_out, void* stream) {
+  Ctx c;
+  SWMOE_TRY(prepare(cfg, workspace, ~(size_t)0, true, &c));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t host[16];
+  if (cudaMemcpyAsync(host, ws_ptr<char>(workspace, c.p.status), sizeof(host), cudaMemcpyDeviceToHost, st) !=
+      cudaSuccess)
+    return SWITCH_MOE_CUDA_ERROR;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  if (info_out != nullptr) std::memcpy(info_out, host, sizeof(host));
+  return host[0] != 0 ? SWITCH_MOE_DEVICE_TIMEOUT : SWITCH_MOE_OK;
+}
+
+int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches_out) {
+  if (launches_out == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
+  Shape s;
+  SWMOE_TRY(resolve_shape(cfg, &s));
+  // fwd: router, 3 plan kernels, gather, 2 GEMMs; bwd: gather, 4 GEMMs, 4 router-backward kernels
+  *launches_out = 7 + 9;
+  return SWITCH_MOE_OK;
+}
+
+const char* switch_moe_status_string(int status) {
+  switch (status) {
+    case SWITCH_MOE_OK: return "ok";
+    case SWITCH_MOE_INVALID_ARGUMENT: return "invalid argument (null pointer, non-positive size, or capacity 0)";
+    case SWITCH_MOE_UNSUPPORTED_SHAPE: return "unsupported shape or misaligned pointer";
+    case SWITCH_MOE_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case SWITCH_MOE_CUDA_ERROR: return "CUDA error";
+    case SWITCH_MOE_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,228 @@
+// Capacity-limited dispatch of the Switch FFN layer (Section 2.2, Eq. 3 and Fig. 3) and the load-balancing loss
+// (Eq. 4-6), as integer index work: no one-hot dispatch / combine tensor is ever built.
+//   plan   : count_i, pos_t = number of earlier tokens with the same expert, keep_t = pos_t < C,
+//            slot_t = e_t * C + pos_t, token_of_slot, kept_i = min(count_i, C), token-tile list for the grouped GEMMs,
+//            P-sums and aux = alpha . E . sum_i (count_i / T)(Psum_i / T)
+//   gather : X_d[slot] = x[token]   (forward)        dY_d[slot] = g_token . dy[token], dgate_token (backward)
+// Positions are deterministic (token order): block histograms -> column scan -> stable in-block rank. No atomics
+// decide a position.
+#include "switch_common.cuh"
+
+namespace swmoe {
+namespace {
+
+// hist[b][e] = number of tokens of block b routed to expert e
+__global__ void __launch_bounds__(kPlanBlockTokens)
+plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int* __restrict__ hist) {
+  __shared__ int h[kMaxExperts];
+  for (int e = threadIdx.x; e < E; e += blockDim.x) h[e] = 0;
+  __syncthreads();
+  const int t = blockIdx.x * kPlanBlockTokens + threadIdx.x;
+  if (t < T) atomicAdd(&h[expert_index[t]], 1);              // integer counts: order-independent
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) hist[(size_t)blockIdx.x * E + e] = h[e];
+}
+
+// One block.  Column scan of the histograms, counts, kept, P-sums, the auxiliary loss and the token-tile list.
+__global__ void __launch_bounds__(kMaxExperts)
+plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __restrict__ psum_partial,
+                 int router_blocks, int T, int E, int C, float alpha, int* __restrict__ hist_base,
+                 int* __restrict__ count, int* __restrict__ kept, float* __restrict__ psum,
+                 float* __restrict__ aux_loss, int* __restrict__ tile_expert, int* __restrict__ tile_row0) {
+  __shared__ float term[kMaxExperts];
+  __shared__ int kept_s[kMaxExperts];
+  const int e = threadIdx.x;
+  if (e < E) {
+    int run = 0;
+    for (int b = 0; b < plan_blocks; ++b) {
+      hist_base[(size_t)b * E + e] = run;
+      run += hist[(size_t)b * E + e];
+    }
+    count[e] = run;
+    const int k = min(run, C);
+    kept[e] = k;
+    kept_s[e] = k;
+    float ps = 0.f;
+    for (int b = 0; b < router_blocks; ++b) ps += psum_partial[(size_t)b * E + e];   // fixed order
+    psum[e] = ps;
+    term[e] = ((float)run / (float)T) * (ps / (float)T);                              // f_i . P_i  (Eq. 5, 6)
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float s = 0.f;
+    for (int i = 0; i < E; ++i) s += term[i];
+    if (aux_loss != nullptr) *aux_loss = alpha * (float)E * s;                        // Eq. 4
+    int n = 0;
+    for (int i = 0; i < E; ++i)
+      for (int r = 0; r < kept_s[i]; r += kTileM) {
+        tile_expert[1 + n] = i;
+        tile_row0[1 + n] = r;
+        ++n;
+      }
+    tile_expert[0] = n;
+    tile_row0[0] = n;
+  }
+}
+
+// pos_t = base[block][e] + (tokens of earlier warps with e) + (earlier lanes with e); slot, token_of_slot.
+__global__ void __launch_bounds__(kPlanBlockTokens)
+plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__ hist_base,
+                   const int* __restrict__ kept, int T, int E, int C, int* __restrict__ slot,
+                   int* __restrict__ token_of_slot) {
+  __shared__ int warp_cnt[kPlanBlockTokens / 32][kMaxExperts];
+  constexpr int kWarps = kPlanBlockTokens / 32;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  for (int i = tid; i < kWarps * kMaxExperts; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
+  __syncthreads();
+  const int t = blockIdx.x * kPlanBlockTokens + tid;
+  const int e = t < T ? expert_index[t] : -1 - lane;          // distinct dummies for out-of-range lanes
+  const unsigned same = __match_any_sync(0xffffffffu, e);
+  const int rank = __popc(same & ((1u << lane) - 1u));
+  if (t < T && rank == 0) warp_cnt[warp][e] = __popc(same);
+  __syncthreads();
+  if (t < T) {
+    int pos = hist_base[(size_t)blockIdx.x * E + e] + rank;
+    for (int w = 0; w < warp; ++w) pos += warp_cnt[w][e];
+    const int s = pos < C ? e * C + pos : -1;
+    slot[t] = s;
+    if (s >= 0) token_of_slot[s] = t;
+  }
+  // empty slots of every expert: -1 (disjoint from the kept slots written above)
+  const int total = E * C;
+  for (int s = blockIdx.x * blockDim.x + tid; s < total; s += gridDim.x * blockDim.x) {
+    const int ex = s / C, pos = s - ex * C;
+    if (pos >= kept[ex]) token_of_slot[s] = -1;
+  }
+}
+
+// Forward gather.  Part 1 (blockIdx.x < slot_blocks): one warp per slot row; kept slots copy the token's row
+// with 128-bit loads and stores, slots in [kept_i, roundup(kept_i, kTileM)) are zero-filled so that tensor-core
+// tiles never read stale rows.  Part 2: one warp per token; dropped tokens get a zero output row (their
+// representation reaches the next layer only through the caller's residual connection, Section 2.2).
+__global__ void __launch_bounds__(256)
+gather_x_kernel(const uint4* __restrict__ x, const int* __restrict__ token_of_slot, const int* __restrict__ kept,
+                const int* __restrict__ slot, int T, int E, int C, int row_vec, int slot_blocks,
+                uint4* __restrict__ xd, uint4* __restrict__ y) {
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  if ((int)blockIdx.x < slot_blocks) {
+    const int s = blockIdx.x * 8 + wib;
+    if (s >= E * C) return;
+    const int ex = s / C, pos = s - ex * C, k = kept[ex];
+    uint4* dst = xd + (size_t)s * row_vec;
+    if (pos < k) {
+      const uint4* src = x + (size_t)token_of_slot[s] * row_vec;
+      for (int v = lane; v < row_vec; v += 32) dst[v] = src[v];
+    } else if (pos < (k + kTileM - 1) / kTileM * kTileM) {
+      for (int v = lane; v < row_vec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+    }
+  } else {
+    const int t = (blockIdx.x - slot_blocks) * 8 + wib;
+    if (t >= T || slot[t] >= 0) return;
+    uint4* dst = y + (size_t)t * row_vec;
+    for (int v = lane; v < row_vec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+  }
+}
+
+__device__ __forceinline__ float dot_scale8(const uint4& a, const uint4& b, float g, uint4* out) {
+  const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+  const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+  __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(out);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 fa = __bfloat1622float2(pa[i]), fb = __bfloat1622float2(pb[i]);
+    s = fmaf(fa.x, fb.x, s);
+    s = fmaf(fa.y, fb.y, s);
+    po[i] = __floats2bfloat162_rn(g * fa.x, g * fa.y);
+  }
+  return s;
+}
+__device__ __forceinline__ float dot_scale4(const uint4& a, const uint4& b, float g, uint4* out) {
+  const float* fa = reinterpret_cast<const float*>(&a);
+  const float* fb = reinterpret_cast<const float*>(&b);
+  float* fo = reinterpret_cast<float*>(out);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { s = fmaf(fa[i], fb[i], s); fo[i] = g * fa[i]; }
+  return s;
+}
+
+// Backward gather: dY_d[slot] = g . dy[token] (derivative of Eq. 2 w.r.t. the expert output) and
+// dgate[token] = <dy, o> with o = y / g (derivative w.r.t. the gate).  Tail rows are zero-filled as in forward.
+template <bool kBf16>
+__global__ void __launch_bounds__(256)
+gather_dy_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ y, const float* __restrict__ gate,
+                 const int* __restrict__ token_of_slot, const int* __restrict__ kept, int E, int C, int row_vec,
+                 uint4* __restrict__ dyd, float* __restrict__ dgate) {
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int s = blockIdx.x * 8 + wib;
+  if (s >= E * C) return;
+  const int ex = s / C, pos = s - ex * C, k = kept[ex];
+  uint4* dst = dyd + (size_t)s * row_vec;
+  if (pos < k) {
+    const int t = token_of_slot[s];
+    const float g = gate[t];
+    const uint4* src = dy + (size_t)t * row_vec;
+    const uint4* ysrc = y + (size_t)t * row_vec;
+    float dot = 0.f;
+    for (int v = lane; v < row_vec; v += 32) {
+      uint4 o;
+      dot += kBf16 ? dot_scale8(src[v], ysrc[v], g, &o) : dot_scale4(src[v], ysrc[v], g, &o);
+      dst[v] = o;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    if (lane == 0) dgate[t] = dot / g;
+  } else if (pos < (k + kTileM - 1) / kTileM * kTileM) {
+    for (int v = lane; v < row_vec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+  }
+}
+
+}  // namespace
+
+int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_index, float* aux_loss, void* ws,
+                         cudaStream_t st) {
+  int* ei = ws_ptr<int>(ws, p.expert_index);
+  if (expert_index != nullptr && expert_index != ei) {
+    if (cudaMemcpyAsync(ei, expert_index, (size_t)s.T * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return SWITCH_MOE_CUDA_ERROR;
+  }
+  plan_hist_kernel<<<s.plan_blocks, kPlanBlockTokens, 0, st>>>(ei, s.T, s.E, ws_ptr<int>(ws, p.hist));
+  plan_scan_kernel<<<1, kMaxExperts, 0, st>>>(ws_ptr<int>(ws, p.hist), s.plan_blocks,
+                                              ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, s.C,
+                                              s.alpha, ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count),
+                                              ws_ptr<int>(ws, p.kept), ws_ptr<float>(ws, p.psum), aux_loss,
+                                              ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0));
+  plan_assign_kernel<<<s.plan_blocks, kPlanBlockTokens, 0, st>>>(ei, ws_ptr<int>(ws, p.hist_base),
+                                                                 ws_ptr<int>(ws, p.kept), s.T, s.E, s.C,
+                                                                 ws_ptr<int>(ws, p.slot),
+                                                                 ws_ptr<int>(ws, p.token_of_slot));
+  return launch_status();
+}
+
+int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void* ws, cudaStream_t st) {
+  const int row_vec = (int)((size_t)s.d * s.elt / 16);
+  const int slot_blocks = (s.E * s.C + 7) / 8, tok_blocks = (s.T + 7) / 8;
+  gather_x_kernel<<<slot_blocks + tok_blocks, 256, 0, st>>>(
+      static_cast<const uint4*>(x), ws_ptr<int>(ws, p.token_of_slot), ws_ptr<int>(ws, p.kept),
+      ws_ptr<int>(ws, p.slot), s.T, s.E, s.C, row_vec, slot_blocks, ws_ptr<uint4>(ws, p.xd), static_cast<uint4*>(y));
+  return launch_status();
+}
+
+int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* ws, cudaStream_t st) {
+  const int row_vec = (int)((size_t)s.d * s.elt / 16);
+  const int blocks = (s.E * s.C + 7) / 8;
+  if (s.dtype == SWITCH_MOE_BF16)
+    gather_dy_kernel<true><<<blocks, 256, 0, st>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(y),
+                                                   ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
+                                                   ws_ptr<int>(ws, p.kept), s.E, s.C, row_vec,
+                                                   ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate));
+  else
+    gather_dy_kernel<false><<<blocks, 256, 0, st>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(y),
+                                                    ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
+                                                    ws_ptr<int>(ws, p.kept), s.E, s.C, row_vec,
+                                                    ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate));
+  return launch_status();
+}
+
+}  // namespace swmoe

@@ -1,0 +1,138 @@
+// Shared host-side plumbing of the Switch FFN library: shape derivation, workspace layout, launch checks.
+// Nothing here is shared with the CPU oracle.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "switch_moe.h"
+
+namespace swmoe {
+
+constexpr int kMaxExperts = 256;        // router kernels keep ceil(E/32) <= 8 experts per lane
+constexpr int kRouterBlockTokens = 64;  // tokens per router-forward block (one partial P-sum row each)
+constexpr int kPlanBlockTokens = 256;   // tokens per dispatch-plan block (one histogram row each)
+constexpr int kTileM = 128;             // token rows per tensor-core tile; tails are zero-filled to this
+constexpr int kDwrChunkTokens = 512;    // tokens per split of the dW_r reduction
+
+struct Shape {
+  int T, d, f, E, C;
+  int dtype;        // switch_moe_dtype
+  int gemm_path;    // resolved: 0 = tcgen05, 1 = SIMT
+  float alpha;
+  size_t elt;       // bytes per activation / expert-weight element
+  int Epad;         // E rounded up to 32 * {1,2,4,8}
+  int router_blocks, plan_blocks, max_mtiles, dwr_chunks;
+};
+
+// Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
+struct Plan {
+  size_t status, expert_index, gate, slot, token_of_slot, count, kept, psum, psum_partial, hist, hist_base,
+      tile_expert, tile_row0, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, total;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
+  if (!cfg) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (cfg->T <= 0 || cfg->d_model <= 0 || cfg->d_ff <= 0 || cfg->E <= 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (cfg->capacity_override < 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (cfg->capacity_override == 0 && !(cfg->capacity_factor > 0.f)) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (cfg->dtype != SWITCH_MOE_BF16 && cfg->dtype != SWITCH_MOE_F32) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (cfg->gemm_path != SWITCH_MOE_GEMM_DEFAULT && cfg->gemm_path != SWITCH_MOE_GEMM_SIMT)
+    return SWITCH_MOE_INVALID_ARGUMENT;
+  for (int i = 0; i < 5; ++i)
+    if (cfg->reserved[i] != 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (cfg->E > kMaxExperts) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  if (cfg->d_model % 8 != 0 || cfg->d_ff % 8 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->T = cfg->T; s->d = cfg->d_model; s->f = cfg->d_ff; s->E = cfg->E;
+  s->dtype = cfg->dtype; s->alpha = cfg->alpha;
+  long long C;
+  if (cfg->capacity_override > 0) {
+    C = cfg->capacity_override;
+  } else {
+    double c = (double)cfg->T * (double)cfg->capacity_factor / (double)cfg->E;   // Eq. 3, floored
+    C = (long long)c;
+  }
+  if (C > cfg->T) C = cfg->T;
+  if (C <= 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if ((long long)cfg->E * C > 0x7fffffffLL) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->C = (int)C;
+  s->elt = cfg->dtype == SWITCH_MOE_BF16 ? 2 : 4;
+  s->gemm_path = (cfg->dtype == SWITCH_MOE_F32 || cfg->gemm_path == SWITCH_MOE_GEMM_SIMT) ? 1 : 0;
+  if (s->gemm_path == 0 && (cfg->d_model % 64 != 0 || cfg->d_ff % 64 != 0)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  int ne = (cfg->E + 31) / 32;
+  int ne_pow2 = 1;
+  while (ne_pow2 < ne) ne_pow2 *= 2;
+  s->Epad = 32 * ne_pow2;
+  s->router_blocks = (cfg->T + kRouterBlockTokens - 1) / kRouterBlockTokens;
+  s->plan_blocks = (cfg->T + kPlanBlockTokens - 1) / kPlanBlockTokens;
+  s->max_mtiles = cfg->E * ((s->C + kTileM - 1) / kTileM);
+  s->dwr_chunks = (cfg->T + kDwrChunkTokens - 1) / kDwrChunkTokens;
+  return SWITCH_MOE_OK;
+}
+
+inline void make_plan(const Shape& s, Plan* p) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+  const size_t T = s.T, E = s.E, C = s.C, d = s.d, f = s.f;
+  p->status = take(16 * sizeof(int32_t));
+  p->expert_index = take(T * 4);
+  p->gate = take(T * 4);
+  p->slot = take(T * 4);
+  p->token_of_slot = take(E * C * 4);
+  p->count = take(E * 4);
+  p->kept = take(E * 4);
+  p->psum = take(E * 4);
+  p->psum_partial = take((size_t)s.router_blocks * E * 4);
+  p->hist = take((size_t)s.plan_blocks * E * 4);
+  p->hist_base = take((size_t)s.plan_blocks * E * 4);
+  p->tile_expert = take(((size_t)s.max_mtiles + 4) * 4);   // [0] = number of token tiles, then one entry per tile
+  p->tile_row0 = take(((size_t)s.max_mtiles + 4) * 4);
+  p->probs = take(T * E * 4);
+  p->dlogits = take(T * E * 4);
+  p->xd = take(E * C * d * s.elt);
+  p->h = take(E * C * f * s.elt);
+  p->dyd = take(E * C * d * s.elt);
+  p->dh = take(E * C * f * s.elt);
+  p->dgate = take(T * 4);
+  p->dwr_partial = take((size_t)s.dwr_chunks * d * E * 4);
+  p->total = off;
+}
+
+template <typename T>
+inline T* ws_ptr(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
+
+inline int launch_status() { return cudaGetLastError() == cudaSuccess ? SWITCH_MOE_OK : SWITCH_MOE_CUDA_ERROR; }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- kernels' host launchers (each returns a switch_moe_status) ----------------------------------------
+int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
+                      cudaStream_t st);
+int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_index, float* aux_loss, void* ws,
+                         cudaStream_t st);
+int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void* ws, cudaStream_t st);
+int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* ws, cudaStream_t st);
+int launch_router_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* dgate, float d_aux,
+                      void* ws, void* dx, bool accumulate_dx, float* dW_r, cudaStream_t st);
+
+// The six expert GEMMs (Section 5: h = x W_in, y = ReLU(h) W_out, and their derivatives).
+enum GemmOp {
+  kGemm1Relu = 0,     // H = ReLU(X_d W_in)
+  kGemm2Combine = 1,  // y[token] = g . (H W_out)[slot]
+  kDgrad2Mask = 2,    // dH = (dY_d W_out^T) * [H > 0]
+  kDgrad1Scatter = 3, // dx[token] = (dH W_in^T)[slot]
+  kWgrad2 = 4,        // dW_out = H^T dY_d
+  kWgrad1 = 5         // dW_in = X_d^T dH
+};
+struct GemmArgs {
+  const void* W_in; const void* W_out;   // expert weights
+  void* y; void* dx; void* dW_in; void* dW_out;
+};
+int launch_simt_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
+int launch_tc_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
+
+}  // namespace swmoe

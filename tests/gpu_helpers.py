@@ -1,0 +1,108 @@
+"""Shared plumbing of the GPU parity tests: upload seeded inputs, run the CUDA library through its C ABI, fetch
+results as float64 numpy arrays, and compare with the CPU oracle."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import switch_oracle as so
+from paper_2101_03961_b200 import build as sbuild
+from paper_2101_03961_b200 import inputs as si
+from paper_2101_03961_b200 import switch_moe as sm
+
+# Tolerances (relative Frobenius error per tensor).  The fp32 router: 1e-5.  bf16 layer outputs and weight
+# gradients: 2e-2 (one bf16 rounding is 2^-9 = 2e-3 relative; H, dY_d, dH and the result are each rounded once
+# and the products accumulate in fp32).  All-fp32 configuration: 2e-4 (fp32 accumulation over d_ff terms).
+TOL_ROUTER = 1e-5
+TOL_BF16 = 2e-2
+TOL_F32 = 2e-4
+FLIP_GAP = 1e-4
+
+
+def rel_err(a, b) -> float:
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    den = np.linalg.norm(b)
+    return float(np.linalg.norm(a - b) / den) if den > 0 else float(np.linalg.norm(a - b))
+
+
+def to_dev(a: np.ndarray, dtype: int) -> torch.Tensor:
+    """float32 numpy -> device tensor in the layer's activation dtype (bf16 bits uploaded as-is)."""
+    if dtype == sm.BF16:
+        bits = si.to_bf16_bits(a)
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16).reshape(a.shape)
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+
+
+def to_np(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+class GpuLayer:
+    """Device buffers of one layer call plus the library calls on them."""
+
+    def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0):
+        sbuild.build()
+        self.scfg = cfg
+        self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
+                                  dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path)
+        dt = cfg.dtype
+        self.x = to_dev(data["x"], dt)
+        self.dy = to_dev(data["dy"], dt)
+        self.W_r = torch.from_numpy(np.ascontiguousarray(data["W_r"], dtype=np.float32)).cuda()
+        b = data.get("router_bias")
+        self.bias = None if b is None else torch.from_numpy(np.ascontiguousarray(b, dtype=np.float32)).cuda()
+        self.W_in = to_dev(data["W_in"], dt)
+        self.W_out = to_dev(data["W_out"], dt)
+        tdt = torch.bfloat16 if dt == sm.BF16 else torch.float32
+        # outputs start as NaN so that any element the library fails to write shows up
+        self.y = torch.full_like(self.x, float("nan"))
+        self.dx = torch.full_like(self.x, float("nan"))
+        self.dW_in = torch.full_like(self.W_in, float("nan"))
+        self.dW_out = torch.full_like(self.W_out, float("nan"))
+        self.dW_r = torch.full_like(self.W_r, float("nan"))
+        self.aux = torch.full((1,), float("nan"), dtype=torch.float32, device="cuda")
+        self.ws = sm.allocate_workspace(self.cfg)
+        self.ws.fill_(0xFF)                       # stale workspace contents must never leak into results
+        self.C = sm.switch_moe_capacity(self.cfg)
+        self.view(sm.WS_STATUS).zero_()
+        assert tdt == self.x.dtype
+
+    def view(self, region):
+        return sm.switch_moe_workspace_view(self.cfg, self.ws, region)
+
+    def fwd(self):
+        sm.switch_moe_fwd(self.cfg, self.x, self.W_r, self.bias, self.W_in, self.W_out, self.y, self.aux, self.ws)
+        sm.switch_moe_check_device_status(self.cfg, self.ws)
+
+    def bwd(self, d_aux=1.0):
+        sm.switch_moe_bwd(self.cfg, self.dy, d_aux, self.x, self.W_r, self.W_in, self.W_out, self.y, self.ws, self.dx,
+                          self.dW_r, self.dW_in, self.dW_out)
+        sm.switch_moe_check_device_status(self.cfg, self.ws)
+
+    def expert_index(self) -> np.ndarray:
+        return self.view(sm.WS_EXPERT_INDEX).cpu().numpy().astype(np.int64)
+
+
+def check_flips(gpu_e: np.ndarray, ora: dict) -> int:
+    """Argmax flips are legitimate only where the oracle's top-2 probability gap is below FLIP_GAP."""
+    diff = np.flatnonzero(gpu_e != ora["e"])
+    if diff.size:
+        srt = np.sort(ora["p"][diff], axis=1)
+        gap = srt[:, -1] - srt[:, -2]
+        assert np.all(gap < FLIP_GAP), f"{diff.size} flips, largest gap {gap.max():.3e}"
+        # the expert the device picked must be the oracle's runner-up-or-tied maximum
+        assert np.all(ora["p"][diff, gpu_e[diff]] >= srt[:, -2] - 1e-12)
+    return int(diff.size)
+
+
+def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capacity=None, experts=None):
+    """Oracle forward with the device's expert choice (identical unless a near-tie flipped), after checking flips."""
+    first = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
+                              router_bias=data.get("router_bias"), capacity=capacity, experts=[])
+    flips = check_flips(gpu_e, first)
+    fwd = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
+                            router_bias=data.get("router_bias"), capacity=capacity, expert_index=gpu_e,
+                            experts=experts)
+    fwd["flips"] = flips
+    return fwd

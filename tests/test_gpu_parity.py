@@ -1,0 +1,248 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs.
+
+Integer work (expert counts, slots, drop masks, inverse maps) must match bit for bit.  Floating point is held to
+the tolerances in gpu_helpers (router 1e-5; bf16 tensors 2e-2 relative Frobenius error; all-fp32 layer 2e-4).
+Argmax flips are counted and allowed only inside a top-2 probability gap of 1e-4; the oracle then follows the
+device's expert choice, because a single flip moves every later slot of two experts.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import switch_oracle as so
+from paper_2101_03961_b200 import inputs as si
+from paper_2101_03961_b200 import switch_moe as sm
+from tests.gpu_helpers import (TOL_BF16, TOL_F32, TOL_ROUTER, GpuLayer, check_flips, oracle_following, rel_err, to_np)
+
+pytestmark = pytest.mark.gpu
+
+TINY = si.CONFIGS["tiny"]
+# bf16 cases that span several tiles and ragged tails in every dimension (T, C, d, f not multiples of the tiles)
+MID = si.SwitchConfig("mid", 2048, 128, 256, 8, 1.25)
+RAGGED = si.SwitchConfig("ragged", 1999, 192, 320, 5, 1.25, bias_std=0.3)
+MANY = si.SwitchConfig("many_experts", 4096, 64, 128, 96, 1.0, bias_std=0.2)
+
+
+def _stack(d):
+    return np.stack([d[i] for i in range(len(d))])
+
+
+# ---------------------------------------------------------------------------------------------- router (staged)
+@pytest.mark.parametrize("cfg", [TINY, MID, RAGGED, MANY, si.SwitchConfig("e1", 300, 64, 64, 1, 1.0),
+                                 si.SwitchConfig("e256", 1024, 64, 64, 256, 2.0)], ids=lambda c: c.name)
+def test_router_forward_matches_oracle(cfg):
+    data = si.gen_layer(cfg, seed=0)
+    g = GpuLayer(cfg, data)
+    sm.switch_moe_router_fwd(g.cfg, g.x, g.W_r, g.bias, g.ws)
+    torch.cuda.synchronize()
+    h = so.router_logits(data["x"], data["W_r"], data.get("router_bias"))
+    p = so.router_probs(h)
+    e, gate = so.top1(p)
+    probs = to_np(g.view(sm.WS_PROBS)).reshape(cfg.T, cfg.E)
+    assert np.abs(probs - p).max() <= TOL_ROUTER
+    assert rel_err(probs, p) <= TOL_ROUTER
+    np.testing.assert_allclose(probs.sum(1), 1.0, atol=1e-5)
+    gpu_e = g.expert_index()
+    flips = check_flips(gpu_e, {"e": e, "p": p})
+    assert flips <= max(2, cfg.T // 1000)
+    gpu_gate = to_np(g.view(sm.WS_GATE))
+    np.testing.assert_allclose(gpu_gate, p[np.arange(cfg.T), gpu_e], rtol=TOL_ROUTER, atol=1e-7)
+
+
+def test_router_ties_go_to_lowest_expert():
+    cfg = si.SwitchConfig("ties", 256, 64, 64, 16, 1.0)
+    data = si.gen_layer(cfg, seed=1)
+    data["W_r"][:] = 0.0
+    g = GpuLayer(cfg, data)
+    g.fwd()
+    assert (g.expert_index() == 0).all()
+    np.testing.assert_allclose(to_np(g.view(sm.WS_GATE)), 1.0 / 16, rtol=1e-6)
+    slot = g.view(sm.WS_SLOT).cpu().numpy()
+    C = g.C
+    assert slot.tolist() == [t if t < C else -1 for t in range(cfg.T)]          # exactly the first C tokens kept
+    assert abs(float(g.aux.item()) - cfg.alpha) <= 1e-6 * cfg.alpha + 1e-9        # P uniform => aux = alpha
+    y = to_np(g.y)
+    assert np.all(y[C:] == 0.0) and np.isfinite(y).all()
+
+
+# ---------------------------------------------------------------------------------------------- dispatch (staged)
+def _plan_case(name, T, E, C, e):
+    return name, T, E, C, np.asarray(e, dtype=np.int32)
+
+
+def _plan_cases():
+    rng = np.random.default_rng(0)
+    cases = [
+        _plan_case("uniform", 4096, 16, 256, rng.integers(0, 16, 4096)),
+        _plan_case("ragged_T", 1999, 5, 499, rng.integers(0, 5, 1999)),
+        _plan_case("all_one_expert", 3000, 8, 375, np.full(3000, 3)),
+        _plan_case("round_robin", 2048, 64, 32, np.arange(2048) % 64),
+        _plan_case("capacity_1", 700, 7, 1, rng.integers(0, 7, 700)),
+        _plan_case("e256", 5000, 256, 19, rng.integers(0, 256, 5000)),
+    ]
+    skew = rng.integers(0, 32, 32768)
+    skew[rng.random(32768) < 0.5] = 7
+    cases.append(_plan_case("skewed_32k", 32768, 32, 1024, skew))
+    return cases
+
+
+@pytest.mark.parametrize("case", _plan_cases(), ids=lambda c: c[0])
+def test_dispatch_plan_is_bit_exact_given_oracle_routing(case):
+    _, T, E, C, e = case
+    cfg = sm.make_config(T, 64, 64, E, 1.0, capacity_override=C)
+    ws = sm.allocate_workspace(cfg)
+    ws.fill_(0xFF)
+    sm.switch_moe_dispatch_plan(cfg, torch.from_numpy(e).cuda(), None, ws)
+    torch.cuda.synchronize()
+    plan = so.dispatch_plan(e, E, C)
+    v = lambda r: sm.switch_moe_workspace_view(cfg, ws, r).cpu().numpy().astype(np.int64)
+    np.testing.assert_array_equal(v(sm.WS_COUNT), plan["count"])
+    np.testing.assert_array_equal(v(sm.WS_KEPT), plan["kept"])
+    np.testing.assert_array_equal(v(sm.WS_SLOT), plan["slot"])
+    np.testing.assert_array_equal(v(sm.WS_TOKEN_OF_SLOT), plan["token_of_slot"])
+    np.testing.assert_array_equal(v(sm.WS_SLOT) >= 0, plan["keep"])
+
+
+def test_dispatch_plan_is_deterministic():
+    rng = np.random.default_rng(5)
+    e = torch.from_numpy(rng.integers(0, 128, 32768).astype(np.int32)).cuda()
+    cfg = sm.make_config(32768, 64, 64, 128, 1.0)
+    ws = sm.allocate_workspace(cfg)
+    outs = []
+    for _ in range(3):
+        ws.fill_(0xFF)
+        sm.switch_moe_dispatch_plan(cfg, e, None, ws)
+        torch.cuda.synchronize()
+        outs.append(sm.switch_moe_workspace_view(cfg, ws, sm.WS_SLOT).clone())
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+
+
+# ---------------------------------------------------------------------------------------------- whole layer
+def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0):
+    data = si.gen_layer(cfg, seed=seed)
+    g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override)
+    g.fwd()
+    gpu_e = g.expert_index()
+    cap = capacity_override if capacity_override else None
+    fwd = oracle_following(cfg, data, gpu_e, capacity=cap)
+    E, C = cfg.E, g.C
+    assert C == fwd["C"]
+    # integer state: bit exact
+    np.testing.assert_array_equal(g.view(sm.WS_SLOT).cpu().numpy(), fwd["slot"])
+    np.testing.assert_array_equal(g.view(sm.WS_COUNT).cpu().numpy(), fwd["count"])
+    np.testing.assert_array_equal(g.view(sm.WS_KEPT).cpu().numpy(), fwd["kept"])
+    np.testing.assert_array_equal(g.view(sm.WS_TOKEN_OF_SLOT).cpu().numpy(), fwd["token_of_slot"])
+    # router and loss
+    assert rel_err(to_np(g.view(sm.WS_PROBS)).reshape(cfg.T, E), fwd["p"]) <= TOL_ROUTER
+    assert abs(float(g.aux.item()) - fwd["aux"]) <= TOL_ROUTER * abs(fwd["aux"])
+    np.testing.assert_allclose(to_np(g.view(sm.WS_PSUM)), fwd["p"].sum(0), rtol=TOL_ROUTER)
+    # dispatched tokens and hidden activations, slot by slot
+    xd = to_np(g.view(sm.WS_XD)).reshape(E, C, cfg.d_model)
+    hid = to_np(g.view(sm.WS_H)).reshape(E, C, cfg.d_ff)
+    x64 = np.asarray(data["x"], dtype=np.float64)
+    errs = {}
+    for i in range(E):
+        k = int(fwd["kept"][i])
+        if k == 0:
+            continue
+        tok = fwd["token_of_slot"][i * C:i * C + k]
+        np.testing.assert_array_equal(xd[i, :k], x64[tok])
+        errs[f"H[{i}]"] = rel_err(hid[i, :k], np.maximum(fwd["u"][i], 0.0))
+    y = to_np(g.y)
+    assert np.isfinite(y).all()
+    assert np.all(y[~fwd["keep"]] == 0.0)                      # dropped tokens: zero rows
+    errs["y"] = rel_err(y, fwd["y"])
+
+    g.bwd(d_aux=d_aux)
+    bwd = so.switch_backward(fwd, data["x"], data["W_r"], data["W_in"], data["W_out"], data["dy"], d_aux=d_aux)
+    kept_tok = np.flatnonzero(fwd["keep"])
+    errs["dgate"] = rel_err(to_np(g.view(sm.WS_DGATE))[kept_tok], bwd["dgate"][kept_tok])
+    errs["dx"] = rel_err(to_np(g.dx), bwd["dx"])
+    errs["dW_r"] = rel_err(to_np(g.dW_r), bwd["dW_r"])
+    dW_in, dW_out = to_np(g.dW_in), to_np(g.dW_out)
+    assert np.isfinite(dW_in).all() and np.isfinite(dW_out).all() and np.isfinite(to_np(g.dx)).all()
+    errs["dW_in"] = rel_err(dW_in, _stack(bwd["dW_in"]))
+    errs["dW_out"] = rel_err(dW_out, _stack(bwd["dW_out"]))
+    for i in range(E):
+        if fwd["kept"][i] == 0:                                # expert without tokens: exactly zero gradients
+            assert np.all(dW_in[i] == 0) and np.all(dW_out[i] == 0)
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, (bad, errs)
+    return errs
+
+
+def test_tiny_fp32_layer_matches_oracle():
+    _check_layer(TINY, sm.GEMM_DEFAULT, TOL_F32)
+
+
+@pytest.mark.parametrize("cfg", [MID, RAGGED, MANY], ids=lambda c: c.name)
+def test_bf16_layer_on_fp32_fma_path_matches_oracle(cfg):
+    _check_layer(cfg, sm.GEMM_SIMT, TOL_BF16)
+
+
+@pytest.mark.parametrize("cfg", [MID, RAGGED, MANY], ids=lambda c: c.name)
+def test_bf16_layer_on_tensor_cores_matches_oracle(cfg):
+    _check_layer(cfg, sm.GEMM_DEFAULT, TOL_BF16, d_aux=0.5)
+
+
+def test_tensor_core_layer_with_empty_and_overflowing_experts():
+    # a strong bias leaves some experts empty and overflows others; capacity not a multiple of any tile
+    cfg = si.SwitchConfig("skewed", 3000, 128, 192, 12, 1.0, bias_std=2.0)
+    errs = _check_layer(cfg, sm.GEMM_DEFAULT, TOL_BF16, seed=3)
+    assert errs
+
+
+def test_tensor_core_layer_single_expert_is_dense_ffn():
+    cfg = si.SwitchConfig("dense", 512, 128, 256, 1, 1.0)
+    data = si.gen_layer(cfg, seed=2)
+    g = GpuLayer(cfg, data)
+    g.fwd()
+    x, W_in, W_out = (np.asarray(data[k], dtype=np.float64) for k in ("x", "W_in", "W_out"))
+    dense = np.maximum(x @ W_in[0], 0) @ W_out[0]
+    assert rel_err(to_np(g.y), dense) <= TOL_BF16
+    np.testing.assert_allclose(to_np(g.view(sm.WS_GATE)), 1.0)
+
+
+def test_capacity_override_is_honoured():
+    _check_layer(MID, sm.GEMM_DEFAULT, TOL_BF16, capacity_override=200)
+
+
+# ---------------------------------------------------------------------------------------------- router backward (staged)
+@pytest.mark.parametrize("cfg", [TINY, MID.with_(dtype=si.DTYPE_F32), RAGGED], ids=lambda c: c.name)
+def test_router_backward_given_identical_gate_gradient(cfg):
+    data = si.gen_layer(cfg, seed=4)
+    g = GpuLayer(cfg, data, gemm_path=sm.GEMM_SIMT)
+    g.fwd()
+    gpu_e = g.expert_index()
+    fwd = oracle_following(cfg, data, gpu_e, experts=[])
+    rng = np.random.default_rng(4)
+    dgate = rng.standard_normal(cfg.T).astype(np.float32)
+    dxr = torch.full_like(g.x, float("nan"))
+    sm.switch_moe_router_bwd(g.cfg, g.x, g.W_r, torch.from_numpy(dgate).cuda(), 0.7, g.ws, dxr, g.dW_r)
+    torch.cuda.synchronize()
+    p_gpu = to_np(g.view(sm.WS_PROBS)).reshape(cfg.T, cfg.E)
+    ref = so.router_backward_given_dgate(p_gpu, gpu_e, fwd["keep"], fwd["count"], dgate, data["x"], data["W_r"],
+                                         cfg.alpha, d_aux=0.7)
+    assert rel_err(to_np(g.view(sm.WS_DLOGITS)).reshape(cfg.T, cfg.E), ref["dh"]) <= TOL_ROUTER
+    assert rel_err(to_np(g.dW_r), ref["dW_r"]) <= TOL_ROUTER
+    tol_dx = TOL_ROUTER if cfg.dtype == si.DTYPE_F32 else 4e-3          # bf16 output rounding
+    assert rel_err(to_np(dxr), ref["dx_router"]) <= tol_dx
+
+
+# ---------------------------------------------------------------------------------------------- error paths
+def test_undersized_workspace_and_misaligned_pointers_are_rejected():
+    import ctypes
+    cfg = sm.make_config(512, 64, 256, 8, 1.0)
+    ws = sm.allocate_workspace(cfg)
+    lib = sm.load_library()
+    x = torch.zeros(512, 64, dtype=torch.bfloat16, device="cuda")
+    W_r = torch.zeros(64, 8, device="cuda")
+    rc = lib.switch_moe_router_fwd(ctypes.byref(cfg), x.data_ptr(), W_r.data_ptr(), None, ws.data_ptr(),
+                                   ws.numel() - 1, None)
+    assert rc == sm.WORKSPACE_TOO_SMALL
+    rc = lib.switch_moe_router_fwd(ctypes.byref(cfg), x.data_ptr() + 2, W_r.data_ptr(), None, ws.data_ptr(),
+                                   ws.numel(), None)
+    assert rc == sm.UNSUPPORTED_SHAPE
+    rc = lib.switch_moe_router_fwd(ctypes.byref(cfg), x.data_ptr(), W_r.data_ptr(), None, ws.data_ptr() + 16,
+                                   ws.numel(), None)
+    assert rc == sm.UNSUPPORTED_SHAPE
