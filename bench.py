@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the Switch FFN layer (forward + backward) on B200: tokens/s, roofline fraction, CPU-oracle baseline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload switch_base]
+
+One step = one switch_moe_fwd + one switch_moe_bwd over a batch of T synthetic tokens (every hot-path stage).
+With N > 1 (launched by torchrun) every rank runs an independent replica on its own GPU: the layer has no
+exchange step on one device, so there is no collective on the data path ("replicas only", weak scaling).
+`--impl reference` times the CPU oracle on a bounded sample of the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2101_03961_b200 import inputs as si  # noqa: E402
+
+METRIC = "switch_moe_layer_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return json.load(open(path)), "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle arm
+class OracleSample:
+    """The CPU oracle (as it stands) on a bounded sample of the workload: router, plan and loss forward and backward
+    on all T tokens, the expert FFN forward + backward on the first `n_experts` experts only; the expert time is
+    scaled to all experts by kept-token count.  Inputs are generated once, outside the timed part."""
+
+    def __init__(self, cfg: si.SwitchConfig, seed: int, n_experts: int):
+        self.cfg = cfg
+        self.x, self.dy = si.gen_x(cfg, seed), si.gen_dy(cfg, seed)
+        self.W_r, self.b = si.gen_W_r(cfg, seed), si.gen_router_bias(cfg, seed)
+        self.sample = list(range(min(n_experts, cfg.E)))
+        self.W_in = {e: si.gen_W_in_expert(cfg, e, seed) for e in self.sample}
+        self.W_out = {e: si.gen_W_out_expert(cfg, e, seed) for e in self.sample}
+        self.desc = ""
+
+    def step(self, reps: int = 3) -> float:
+        """One timed pass; returns the seconds one whole fwd+bwd of the workload would take at this rate.
+        Each of the four passes is timed `reps` times and the minimum kept (host timing noise is large)."""
+        from oracle import switch_oracle as so
+        cfg, a = self.cfg, (self.x, self.W_r, self.W_in, self.W_out)
+        kw = dict(router_bias=self.b)
+        t_rf, t_af, t_ab, t_rb = [], [], [], []
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            so.switch_forward(*a, cfg.capacity_factor, cfg.alpha, experts=[], **kw)
+            t_rf.append(time.perf_counter() - t0)
+            t0 = time.perf_counter()
+            fwd = so.switch_forward(*a, cfg.capacity_factor, cfg.alpha, experts=self.sample, **kw)
+            t_af.append(time.perf_counter() - t0)
+            t0 = time.perf_counter()
+            so.switch_backward(fwd, *a, self.dy, experts=self.sample)
+            t_ab.append(time.perf_counter() - t0)
+            t0 = time.perf_counter()
+            so.switch_backward(fwd, *a, self.dy, experts=[])
+            t_rb.append(time.perf_counter() - t0)
+        kept_sample, kept_all = int(fwd["kept"][self.sample].sum()), int(fwd["kept"].sum())
+        t_router = min(t_rf) + min(t_rb)
+        t_experts = max(min(t_af) - min(t_rf), 0.0) + max(min(t_ab) - min(t_rb), 0.0)
+        self.desc = (f"router+dispatch+loss fwd/bwd on all {cfg.T} tokens; expert FFN fwd+bwd on {len(self.sample)} of "
+                     f"{cfg.E} experts ({kept_sample} of {kept_all} kept tokens), expert time scaled by kept tokens; "
+                     f"min of {reps} repetitions per pass")
+        return t_router + t_experts * kept_all / max(kept_sample, 1)
+
+    @staticmethod
+    def cores() -> int:
+        try:
+            from threadpoolctl import threadpool_info
+            return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        except Exception:
+            return os.cpu_count() or 1
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    # the router part alone costs seconds per step on the host, so the reference arm samples few experts
+    sample = OracleSample(cfg, args.seed, max(1, min(args.oracle_experts, 2)))
+    per_step = []
+    for i in range(args.warmup + args.steps):
+        t = sample.step()
+        if i >= args.warmup:
+            per_step.append(t)
+    t = max(statistics.mean(per_step), 1e-12)
+    value = cfg.T / t
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "T": cfg.T, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "E": cfg.E,
+                   "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": sample.cores(), "kind": "oracle", "sample": sample.desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.thread = [], None, None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0])); smax.append(float(r[1])); power.append(float(r[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------- GPU arm
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    from paper_2101_03961_b200 import build as sbuild
+    from paper_2101_03961_b200 import switch_moe as sm
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the layer has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    sbuild.build()
+    sm.load_library()
+
+    def dev(a):
+        if cfg.dtype == si.DTYPE_BF16:
+            return torch.from_numpy(si.to_bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16).reshape(a.shape)
+        return torch.from_numpy(a).cuda()
+
+    seed = args.seed + rank                                   # each replica routes its own batch
+    x_np, dy_np = si.gen_x(cfg, seed), si.gen_dy(cfg, seed)
+    as_bits = cfg.dtype == si.DTYPE_BF16
+    W_in_np = si.gen_W_in(cfg, args.seed, as_bits=as_bits)
+    W_out_np = si.gen_W_out(cfg, args.seed, as_bits=as_bits)
+    if as_bits:
+        W_in = torch.from_numpy(W_in_np.view(np.int16)).cuda().view(torch.bfloat16)
+        W_out = torch.from_numpy(W_out_np.view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        W_in, W_out = torch.from_numpy(W_in_np).cuda(), torch.from_numpy(W_out_np).cuda()
+    del W_in_np, W_out_np
+    x, dy = dev(x_np), dev(dy_np)
+    W_r = torch.from_numpy(si.gen_W_r(cfg, args.seed)).cuda()
+    b_np = si.gen_router_bias(cfg, args.seed)
+    bias = None if b_np is None else torch.from_numpy(b_np).cuda()
+
+    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype)
+    ws = sm.allocate_workspace(mcfg)
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    dW_in, dW_out, dW_r = torch.empty_like(W_in), torch.empty_like(W_out), torch.empty_like(W_r)
+    aux = torch.zeros(1, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        sm.switch_moe_fwd(mcfg, x, W_r, bias, W_in, W_out, y, aux, ws, stream)
+        sm.switch_moe_bwd(mcfg, dy, 1.0, x, W_r, W_in, W_out, y, ws, dx, dW_r, dW_in, dW_out, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sm.switch_moe_check_device_status(mcfg, ws, stream)
+
+    # ---- timed region: K steps, device-timed; per-stage events recorded inside the same region
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(sm.STAGE_EVENTS)] for _ in range(args.steps)]
+    for evs in events:
+        for ev in evs:
+            ev.record(stream)                                 # creates the underlying cudaEvent_t handles
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    t_start.record(stream)
+    for k in range(args.steps):
+        sm.set_stage_events(mcfg, events[k])
+        step()
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    sm.set_stage_events(mcfg, None)
+    sm.switch_moe_check_device_status(mcfg, ws, stream)
+    elapsed_ms = t_start.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * cfg.T / (ms_per_step * 1e-3)
+
+    stage_ms = {}
+    for i, name in enumerate(sm.STAGE_NAMES):
+        if name is None:
+            continue
+        stage_ms[name] = statistics.mean(events[k][i].elapsed_time(events[k][i + 1]) for k in range(args.steps))
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    kept = int(sm.switch_moe_workspace_view(mcfg, ws, sm.WS_KEPT).sum().item())
+    peaks, peak_kind = load_peaks()
+    gemm_names = ["gemm1_relu", "gemm2_combine", "dgrad2_mask", "wgrad2", "dgrad1_scatter", "wgrad1"]
+    gemm_ms_avg = statistics.mean(stage_ms[n] for n in gemm_names)
+    flops_per_launch = 2.0 * kept * cfg.d_model * cfg.d_ff           # useful flops of one expert GEMM (kept rows only)
+    achieved_tf = flops_per_launch / (gemm_ms_avg * 1e-3) / 1e12
+    if cfg.dtype == si.DTYPE_BF16:
+        peak_tf = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+        roofline = {"bound": "tensor", "kernel": "grouped_gemm_tc_kernel (6 launches per step)",
+                    "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
+                    "traffic": None, "peak_source": f"{peak_kind} bf16 sustained (kernel timed inside a long step)",
+                    "flops_per_launch": flops_per_launch, "avg_launch_ms": gemm_ms_avg}
+    else:
+        peak_tf = 148 * 128 * 2 * 1.965e9 / 1e12
+        roofline = {"bound": "alu", "kernel": "simt_grouped_gemm_kernel", "achieved": achieved_tf, "peak": peak_tf,
+                    "unit": "TFLOP/s", "frac": achieved_tf / peak_tf, "traffic": None,
+                    "peak_source": "148 SMs x 128 FP32 lanes x 2 x 1.965 GHz"}
+    hbm = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+    elt = 2 if cfg.dtype == si.DTYPE_BF16 else 4
+    row_bytes = cfg.d_model * elt
+    stages = {n: {"ms": stage_ms[n]} for n in stage_ms}
+    for n in gemm_names:
+        stages[n]["tflops"] = flops_per_launch / (stage_ms[n] * 1e-3) / 1e12
+    stages["gather_x"]["gbs"] = (2 * kept * row_bytes) / (stage_ms["gather_x"] * 1e-3) / 1e9
+    stages["gather_dy"]["gbs"] = (3 * kept * row_bytes) / (stage_ms["gather_dy"] * 1e-3) / 1e9
+    stages["router_fwd"]["gbs"] = (cfg.T * row_bytes + cfg.T * cfg.E * 4) / (stage_ms["router_fwd"] * 1e-3) / 1e9
+    stages["router_fwd"]["fp32_tflops"] = 2.0 * cfg.T * cfg.d_model * cfg.E / (stage_ms["router_fwd"] * 1e-3) / 1e12
+    stages["router_bwd"]["fp32_tflops"] = 4.0 * cfg.T * cfg.d_model * cfg.E / (stage_ms["router_bwd"] * 1e-3) / 1e12
+    for n in ("gather_x", "gather_dy", "router_fwd"):
+        stages[n]["hbm_frac"] = stages[n]["gbs"] / hbm
+
+    # ---- end to end through the C ABI with HOST activations (pinned), copies inside the timed region
+    xh, dyh = x.cpu().pin_memory(), dy.cpu().pin_memory()
+    yh, dxh = torch.empty_like(xh).pin_memory(), torch.empty_like(xh).pin_memory()
+    auxh = torch.zeros(1).pin_memory()
+    e2e_steps = max(2, min(args.steps, 10))
+
+    def host_step():
+        sm.switch_moe_step_host(mcfg, xh, dyh, 1.0, W_r, bias, W_in, W_out, x, dy, y, dx, aux, dW_r, dW_in, dW_out,
+                                yh, dxh, auxh, ws, stream)
+
+    host_step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        host_step()                                           # synchronises the stream before returning
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    act_bytes = cfg.T * row_bytes
+    e2e = {"value": world * cfg.T / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 2 * act_bytes,
+           "d2h_bytes_per_step": 2 * act_bytes + 4, "ms_per_step": e2e_s * 1e3,
+           "note": "x, dy copied from pinned host memory; y, dx, aux copied back; weights and weight gradients resident"}
+
+    # ---- CPU baseline: the oracle on a bounded sample, this machine's host cores
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        osample = OracleSample(cfg, args.seed, args.oracle_experts)
+        osample.step(reps=1)                                  # warm-up (BLAS threads, page faults)
+        t = osample.step()
+        cpu = {"value": cfg.T / t, "unit": UNIT, "cores": osample.cores(), "kind": "oracle", "sample": osample.desc,
+               "seconds_scaled": t}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == si.DTYPE_BF16 else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "T": cfg.T, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "E": cfg.E,
+                   "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha, "capacity": sm.switch_moe_capacity(mcfg),
+                   "kept_tokens": kept, "parallelism": "replicas" if world > 1 else "single",
+                   "l2": "inputs larger than L2 (weights 2 x %.0f MB per pass), no flush" %
+                         (cfg.E * cfg.d_model * cfg.d_ff * elt / 1e6)},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": sm.switch_moe_launches_per_step(mcfg) * args.steps,
+        "roofline": roofline, "cpu_baseline": cpu, "stages": stages,
+        "aux_loss": float(aux.item()),
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="switch_base", choices=sorted(si.CONFIGS))
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--oracle-experts", type=int, default=None,
+                    help="experts whose FFN the CPU oracle runs in its bounded sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = si.CONFIGS[args.workload]
+    if args.oracle_experts is None:
+        # about 10-30 s of host work in total: ~1e11 flops of fp64 matmul per pass, a few passes
+        per_expert = 12.0 * (cfg.T / cfg.E) * cfg.d_model * cfg.d_ff
+        args.oracle_experts = int(max(1, min(cfg.E, round(1.0e11 / per_expert))))
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,126 @@
+"""Full-size parity in the launch configuration the benchmark times: the whole layer runs on the device at the
+workload's real shape; the oracle checks everything it can afford exactly -- the router and the dispatch plan for
+all tokens (bit-exact integers), the auxiliary loss, and, for a sample of experts (the fullest, the emptiest
+non-empty one and two others), every output row and gradient those experts produce.  Properties that hold at any
+size cover the rest: dropped tokens give zero rows, experts without tokens give zero gradients, nothing is NaN.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import switch_oracle as so
+from paper_2101_03961_b200 import build as sbuild
+from paper_2101_03961_b200 import inputs as si
+from paper_2101_03961_b200 import switch_moe as sm
+from tests.gpu_helpers import TOL_BF16, TOL_ROUTER, check_flips, rel_err, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def _bits_to_dev(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _run_fullsize(name, seed=0, n_extra=2):
+    sbuild.build()
+    cfg = si.CONFIGS[name]
+    assert cfg.dtype == si.DTYPE_BF16
+    x_np, dy_np = si.gen_x(cfg, seed), si.gen_dy(cfg, seed)
+    W_r_np, b_np = si.gen_W_r(cfg, seed), si.gen_router_bias(cfg, seed)
+    x, dy = _bits_to_dev(si.to_bf16_bits(x_np)), _bits_to_dev(si.to_bf16_bits(dy_np))
+    W_in = _bits_to_dev(si.gen_W_in(cfg, seed, as_bits=True, threads=16))
+    W_out = _bits_to_dev(si.gen_W_out(cfg, seed, as_bits=True, threads=16))
+    W_r = torch.from_numpy(W_r_np).cuda()
+    bias = None if b_np is None else torch.from_numpy(b_np).cuda()
+    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha)
+    ws = sm.allocate_workspace(mcfg)
+    ws.fill_(0xFF)
+    y, dx = torch.full_like(x, float("nan")), torch.full_like(x, float("nan"))
+    dW_in, dW_out = torch.full_like(W_in, float("nan")), torch.full_like(W_out, float("nan"))
+    dW_r = torch.full_like(W_r, float("nan"))
+    aux = torch.zeros(1, device="cuda")
+    sm.switch_moe_fwd(mcfg, x, W_r, bias, W_in, W_out, y, aux, ws)
+    sm.switch_moe_bwd(mcfg, dy, 1.0, x, W_r, W_in, W_out, y, ws, dx, dW_r, dW_in, dW_out)
+    sm.switch_moe_check_device_status(mcfg, ws)
+    view = lambda r: sm.switch_moe_workspace_view(mcfg, ws, r)
+    T, E, C = cfg.T, cfg.E, sm.switch_moe_capacity(mcfg)
+
+    # router for all tokens; flips only inside the allowed gap; then the oracle follows the device's choice
+    gpu_e = view(sm.WS_EXPERT_INDEX).cpu().numpy().astype(np.int64)
+    h = so.router_logits(x_np, W_r_np, b_np)
+    p = so.router_probs(h)
+    e0, _ = so.top1(p)
+    flips = check_flips(gpu_e, {"e": e0, "p": p})
+    assert flips <= 8
+    assert np.abs(to_np(view(sm.WS_PROBS)).reshape(T, E) - p).max() <= TOL_ROUTER
+    plan = so.dispatch_plan(gpu_e, E, so.expert_capacity(T, E, cfg.capacity_factor))
+    assert C == so.expert_capacity(T, E, cfg.capacity_factor)
+    np.testing.assert_array_equal(view(sm.WS_SLOT).cpu().numpy(), plan["slot"])
+    np.testing.assert_array_equal(view(sm.WS_TOKEN_OF_SLOT).cpu().numpy(), plan["token_of_slot"])
+    np.testing.assert_array_equal(view(sm.WS_COUNT).cpu().numpy(), plan["count"])
+    np.testing.assert_array_equal(view(sm.WS_KEPT).cpu().numpy(), plan["kept"])
+    aux_ref, _, _ = so.load_balance_loss(p, gpu_e, cfg.alpha)
+    assert abs(float(aux.item()) - aux_ref) <= TOL_ROUTER * aux_ref
+
+    # sampled experts: fullest, emptiest non-empty, and a few fixed ones
+    count = plan["count"]
+    nonempty = np.flatnonzero(count > 0)
+    sample = {int(np.argmax(count)), int(nonempty[np.argmin(count[nonempty])])}
+    rng = np.random.default_rng(seed)
+    sample.update(int(v) for v in rng.choice(nonempty, size=min(n_extra, nonempty.size), replace=False))
+    sample = sorted(sample)
+    W_in_s = {i: si.gen_W_in_expert(cfg, i, seed) for i in sample}
+    W_out_s = {i: si.gen_W_out_expert(cfg, i, seed) for i in sample}
+    fwd = so.switch_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, router_bias=b_np,
+                            expert_index=gpu_e, experts=sample)
+    bwd = so.switch_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
+    keep = plan["keep"]
+    hid = view(sm.WS_H).view(E, C, cfg.d_ff)
+    errs = {}
+    for i in sample:
+        tok = np.flatnonzero(keep & (gpu_e == i))
+        k = tok.size
+        assert k == plan["kept"][i]
+        tt = torch.from_numpy(tok).cuda()
+        errs[f"H[{i}]"] = rel_err(to_np(hid[i, :k]), np.maximum(fwd["u"][i], 0.0))
+        errs[f"y[{i}]"] = rel_err(to_np(y[tt]), fwd["y"][tok])
+        errs[f"dx[{i}]"] = rel_err(to_np(dx[tt]), bwd["dx"][tok])
+        errs[f"dW_in[{i}]"] = rel_err(to_np(dW_in[i]), bwd["dW_in"][i])
+        errs[f"dW_out[{i}]"] = rel_err(to_np(dW_out[i]), bwd["dW_out"][i])
+        errs[f"dgate[{i}]"] = rel_err(to_np(view(sm.WS_DGATE)[tt]), bwd["dgate"][tok])
+    bad = {k: v for k, v in errs.items() if not v <= TOL_BF16}
+    assert not bad, (bad, errs)
+
+    # properties that hold at any size
+    dropped = torch.from_numpy(np.flatnonzero(~keep)).cuda()
+    if dropped.numel():
+        assert bool((y[dropped] == 0).all())
+    assert bool(torch.isfinite(y).all()) and bool(torch.isfinite(dx).all()) and bool(torch.isfinite(dW_r).all())
+    assert bool(torch.isfinite(dW_in).all()) and bool(torch.isfinite(dW_out).all())
+    for i in np.flatnonzero(count == 0):
+        assert bool((dW_in[int(i)] == 0).all()) and bool((dW_out[int(i)] == 0).all())
+    # dropped tokens receive only the router's gradient: finite and small, never the expert path
+    return {"flips": flips, "dropped": int((~keep).sum()), "errs": errs}
+
+
+def test_switch_base_full_size():
+    out = _run_fullsize("switch_base")
+    assert out["dropped"] < 0.01 * 32768                     # well-balanced routing: under 1% dropped
+
+
+def test_overflow_stress_calibrated_full_size():
+    out = _run_fullsize("stress_calibrated")
+    assert 0.15 * 32768 < out["dropped"] < 0.40 * 32768
+
+
+def test_overflow_stress_literal_full_size():
+    out = _run_fullsize("stress_literal")
+    assert out["dropped"] > 0.8 * 32768                      # a N(0, 2^2) bias overflows almost everything
+
+
+def test_switch_large_full_size():
+    _run_fullsize("switch_large")
+
+
+def test_wide_expert_full_size():
+    _run_fullsize("wide", n_extra=1)
