@@ -141,6 +141,25 @@ int switch_moe_router_bwd(const switch_moe_config* cfg, const void* x, const flo
                           float d_aux, void* workspace, size_t workspace_bytes, void* dx_router, float* dW_r,
                           void* stream);
 
+/* The dispatch plan for callers that cannot allocate device memory and have no workspace to pass.  (The paper has
+ * no counterpart: this is a packaging variant of switch_moe_dispatch_plan, not a step of the method.)
+ * Meant for a process whose device heap is owned entirely by another allocator (a serving arena, a framework's
+ * caching pool), or a call site where cudaMalloc's device-wide synchronisation cannot be tolerated.  The only
+ * scratch the plan needs -- per-block expert histograms and their scan -- is a 512 KiB array compiled into the
+ * library, resident on every GPU that loads it until the process exits; the call itself allocates and frees
+ * nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *   expert_index device int32[T] (in).  Outputs, all caller-owned device buffers: count int32[E], kept int32[E],
+ *   slot int32[T] (e*C + position, or -1 if dropped), token_of_slot int32[E*C] (-1 for empty slots) -- the same
+ *   values switch_moe_dispatch_plan leaves in its workspace regions of those names.
+ * Limits: T <= SWITCH_MOE_STATIC_PLAN_MAX_TOKENS (else SWITCH_MOE_UNSUPPORTED_SHAPE), E <= 256.
+ * The first call on each device looks up the array's device address (with that device current); make that first
+ * call before starting any stream capture.  All calls on a device share the one array: nothing in it needs
+ * clearing between calls (every word read is written earlier in the same call), but two calls whose kernels
+ * overlap on the GPU (different streams, or several host threads) race on it -- serialise them. */
+#define SWITCH_MOE_STATIC_PLAN_MAX_TOKENS 65536
+int switch_moe_dispatch_plan_static(const switch_moe_config* cfg, const int32_t* expert_index, int32_t* count,
+                                    int32_t* kept, int32_t* slot, int32_t* token_of_slot, void* stream);
+
 /* One training step with HOST activations: copies x_host and dy_host (pinned host memory, [T,d_model]) to the
  * device buffers x_dev / dy_dev, runs switch_moe_fwd and switch_moe_bwd, and copies y, dx and the auxiliary loss
  * back to y_host, dx_host, aux_host.  Weights and weight gradients stay on the device.  Synchronises the stream

@@ -28,7 +28,7 @@ WS_STATUS, WS_EXPERT_INDEX, WS_GATE, WS_SLOT, WS_TOKEN_OF_SLOT, WS_COUNT, WS_KEP
 EXPORTED_SYMBOLS = [
     "switch_moe_capacity", "switch_moe_workspace_bytes", "switch_moe_workspace_view", "switch_moe_fwd",
     "switch_moe_bwd", "switch_moe_router_fwd", "switch_moe_dispatch_plan", "switch_moe_router_bwd",
-    "switch_moe_step_host", "switch_moe_check_device_status", "switch_moe_launches_per_step",
+    "switch_moe_dispatch_plan_static", "switch_moe_step_host", "switch_moe_check_device_status", "switch_moe_launches_per_step",
     "switch_moe_status_string",
 ]
 
@@ -72,6 +72,7 @@ def load_library() -> ctypes.CDLL:
     lib.switch_moe_bwd.argtypes = [cp, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp, vp, vp, vp, vp]
     lib.switch_moe_router_fwd.argtypes = [cp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.switch_moe_dispatch_plan.argtypes = [cp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.switch_moe_dispatch_plan_static.argtypes = [cp, vp, vp, vp, vp, vp, vp]
     lib.switch_moe_router_bwd.argtypes = [cp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp, vp, vp]
     lib.switch_moe_step_host.argtypes = [cp, vp, vp, ctypes.c_float] + [vp] * 15 + [vp, ctypes.c_size_t, vp]
     lib.switch_moe_check_device_status.argtypes = [cp, vp, i32p, vp]
@@ -191,6 +192,14 @@ def switch_moe_dispatch_plan(cfg, expert_index, aux_loss, workspace, stream=None
     _check(load_library().switch_moe_dispatch_plan(ctypes.byref(cfg), _ptr(expert_index), _ptr(aux_loss),
                                                    _ptr(workspace), workspace.numel(), _stream(stream)),
            "switch_moe_dispatch_plan")
+
+
+def switch_moe_dispatch_plan_static(cfg, expert_index, count, kept, slot, token_of_slot, stream=None) -> None:
+    """Dispatch plan without a workspace and without any allocation (scratch is a static array inside the library);
+    for callers that cannot call cudaMalloc.  Outputs go to the four caller-owned int32 tensors."""
+    _check(load_library().switch_moe_dispatch_plan_static(ctypes.byref(cfg), _ptr(expert_index), _ptr(count),
+                                                          _ptr(kept), _ptr(slot), _ptr(token_of_slot),
+                                                          _stream(stream)), "switch_moe_dispatch_plan_static")
 
 
 def switch_moe_router_bwd(cfg, x, W_r, dgate, d_aux, workspace, dx_router, dW_r, stream=None) -> None:
