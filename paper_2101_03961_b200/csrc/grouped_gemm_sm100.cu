@@ -5,10 +5,10 @@
 //   dH = (dY_d W_out^T) * [H > 0]            dx[token] = (dH W_in^T)[slot]
 //   dW_out = H^T dY_d                        dW_in     = X_d^T dH                     (contraction over kept tokens)
 //
-// One persistent CTA per SM, 192 threads: warp 0 issues TMA loads into a 4-stage ring of 128B-swizzled tiles
+// One persistent CTA per SM, 320 threads: warp 0 issues TMA loads into a 4-stage ring of 128B-swizzled tiles
 // (A 128x64, B 256x64 per stage), warp 1 issues tcgen05.mma (M=128, N=256, K=16) into one of two 128x256 float32
-// accumulators in tensor memory, warps 2-5 drain the other accumulator (tcgen05.ld), apply the epilogue and write
-// full 128-byte row segments.  Operands may be K-major or MN-major (the weight matrices are used both ways), chosen
+// accumulators in tensor memory, warps 2-9 drain the other accumulator (tcgen05.ld; each warp owns one 32-lane group
+// and one half of the columns), apply the epilogue and write full 128-byte row segments.  Operands may be K-major or MN-major (the weight matrices are used both ways), chosen
 // per product by descriptor bits only.  No TMA multicast is used anywhere.
 //
 // Every wait on an mbarrier is bounded in time; a wait that gives up records a code in the workspace status word,
@@ -25,10 +25,10 @@ constexpr int kABytes = kTileM * kBK * 2;            // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;               // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;       // 48 KB
 constexpr int kAtomBytes = 64 * kBK * 2;             // one 64(MN) x 64(K) MN-major box: 8 KB
-constexpr int kOutStageBytes = 4 * 32 * 128;         // 4 epilogue warps x 32 rows x 128 B
+constexpr int kOutStageBytes = 8 * 32 * 128;         // 8 epilogue warps x 32 rows x 128 B
 constexpr int kBarBytes = 128;
 constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kOutStageBytes + kBarBytes;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                        // TMA warp, MMA warp, 8 epilogue warps
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
@@ -200,7 +200,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -293,7 +293,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   } else {
     // ------------------------------------------------------------------------------------------ epilogue warps
     const int lg = warp & 3;                                  // TMEM lane group this warp may read
-    const uint32_t my_stage = out_stage_base + (uint32_t)(warp - 2) * 4096u;
+    const int half = (warp - 2) >> 2;                         // which pair of 64-column chunks this warp drains
     uint8_t* my_stage_gen = smem_gen + kStages * kStageBytes + (warp - 2) * 4096;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -316,13 +316,27 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       } else if (t.m0 + r < p.M) {
         row_off = ((long long)t.e * p.M + t.m0 + r) * p.ld_out;
       }
+      // write-out assignment: instruction `it` covers rows it*4 + lane/8, 16-byte column (lane & 7)
+      long long offs[8];
+#pragma unroll
+      for (int it = 0; it < 8; ++it) offs[it] = __shfl_sync(0xffffffffu, row_off, it * 4 + (lane >> 3));
+      // ReLU mask of the first chunk, fetched while the accumulator is still being produced
+      uint4 hm[8];
+      if (p.op == kDgrad2Mask) {
+        const int col = t.n0 + (2 * half) * 64 + (lane & 7) * 8;
+#pragma unroll
+        for (int it = 0; it < 8; ++it)
+          hm[it] = (offs[it] >= 0 && col < p.N) ? *reinterpret_cast<const uint4*>(p.mask_src + offs[it] + col)
+                                                : make_uint4(0, 0, 0, 0);
+      }
       ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)acc * kBN;
 #pragma unroll 1
-      for (int c = 0; c < kBN / 64; ++c) {
+      for (int cc = 0; cc < 2; ++cc) {
+        const int c = 2 * half + cc;
         uint32_t v[64];
         if (t.k_blocks > 0) {
           tc_ld32(t_addr + c * 64, v);
@@ -332,7 +346,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 #pragma unroll
           for (int i = 0; i < 64; ++i) v[i] = 0u;
         }
-        if (c == kBN / 64 - 1) {                              // accumulator fully read: hand it back to the MMA warp
+        if (cc == 1) {                                        // this warp's share is read: hand it back to the MMA warp
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -355,29 +369,39 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         __syncwarp();
         // coalesced write-out: each instruction covers 4 rows x 128 bytes
         const int col = t.n0 + c * 64 + (lane & 7) * 8;
+        uint4 val[8];
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
           const int rr = it * 4 + (lane >> 3);
-          const long long off = __shfl_sync(0xffffffffu, row_off, rr);
-          uint4 val = *reinterpret_cast<const uint4*>(my_stage_gen + rr * 128 + (((lane & 7) ^ (rr & 7)) << 4));
-          if (off >= 0 && col < p.N) {
-            if (p.op == kDgrad2Mask) {                        // ReLU'(u) = [u > 0], read from the saved activation
-              const uint4 hm = *reinterpret_cast<const uint4*>(p.mask_src + off + col);
-              const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hm);
-              __nv_bfloat162* vp = reinterpret_cast<__nv_bfloat162*>(&val);
-              const __nv_bfloat16 zero = __float2bfloat16(0.f);
+          val[it] = *reinterpret_cast<const uint4*>(my_stage_gen + rr * 128 + (((lane & 7) ^ (rr & 7)) << 4));
+        }
+        if (p.op == kDgrad2Mask) {                            // ReLU'(u) = [u > 0], read from the saved activation
+          const __nv_bfloat16 zero = __float2bfloat16(0.f);
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                if (!(__low2float(hp[q]) > 0.f)) vp[q].x = zero;
-                if (!(__high2float(hp[q]) > 0.f)) vp[q].y = zero;
-              }
+          for (int it = 0; it < 8; ++it) {
+            const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hm[it]);
+            __nv_bfloat162* vp = reinterpret_cast<__nv_bfloat162*>(&val[it]);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              if (!(__low2float(hp[q]) > 0.f)) vp[q].x = zero;
+              if (!(__high2float(hp[q]) > 0.f)) vp[q].y = zero;
             }
-            *reinterpret_cast<uint4*>(p.out + off + col) = val;
           }
+          if (cc == 0) {                                      // fetch the second chunk's mask behind this chunk's stores
+            const int col2 = col + 64;
+#pragma unroll
+            for (int it = 0; it < 8; ++it)
+              hm[it] = (offs[it] >= 0 && col2 < p.N) ? *reinterpret_cast<const uint4*>(p.mask_src + offs[it] + col2)
+                                                     : make_uint4(0, 0, 0, 0);
+          }
+        }
+        if (col < p.N) {
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            if (offs[it] >= 0) *reinterpret_cast<uint4*>(p.out + offs[it] + col) = val[it];
         }
         __syncwarp();
       }
-      (void)my_stage;
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }

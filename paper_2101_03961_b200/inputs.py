@@ -56,6 +56,9 @@ CONFIGS = {
     "stress_literal": SwitchConfig("stress_literal", 32768, 768, 3072, 64, 1.0, bias_std=2.0),
     "switch_large": SwitchConfig("switch_large", 32768, 1024, 4096, 128, 1.25),
     "wide": SwitchConfig("wide", 16384, 4096, 10240, 64, 1.25),
+    # a quarter of switch_base (same tokens per expert, same d_model / d_ff): small enough for profiler captures,
+    # still larger than L2 (2 x 151 MB of weights)
+    "switch_base_quarter": SwitchConfig("switch_base_quarter", 8192, 768, 3072, 32, 1.25),
 }
 
 
