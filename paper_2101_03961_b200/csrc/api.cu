@@ -220,8 +220,9 @@ int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches
   if (launches_out == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
   Shape s;
   SWMOE_TRY(resolve_shape(cfg, &s));
-  // fwd: router, 3 plan kernels, gather, 2 GEMMs; bwd: gather, 4 GEMMs, 4 router-backward kernels
-  *launches_out = 7 + 9;
+  // fwd: router, 3 plan kernels, gather, 2 GEMMs; bwd: gather, 4 GEMMs, 4 router-backward kernels.
+  // The tensor-core router adds an operand-split kernel in forward and two in backward.
+  *launches_out = s.router_tc ? (8 + 11) : (7 + 9);
   return SWITCH_MOE_OK;
 }
 

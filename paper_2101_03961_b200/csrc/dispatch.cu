@@ -23,29 +23,64 @@ plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int* __rest
   for (int e = threadIdx.x; e < E; e += blockDim.x) hist[(size_t)blockIdx.x * E + e] = h[e];
 }
 
-// One block.  Column scan of the histograms, counts, kept, P-sums, the auxiliary loss and the token-tile list.
-__global__ void __launch_bounds__(kMaxExperts)
+// One block of 4 x 256 threads: thread (g, e) owns quarter g of the rows of column e.  Column scan of the
+// histograms, counts, kept, P-sums (all in a fixed order), the auxiliary loss and the token-tile list.
+constexpr int kScanGroups = 4;
+__global__ void __launch_bounds__(kScanGroups * kMaxExperts)
 plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __restrict__ psum_partial,
                  int router_blocks, int T, int E, int C, float alpha, int* __restrict__ hist_base,
                  int* __restrict__ count, int* __restrict__ kept, float* __restrict__ psum,
                  float* __restrict__ aux_loss, int* __restrict__ tile_expert, int* __restrict__ tile_row0) {
+  __shared__ int qsum[kScanGroups][kMaxExperts];
+  __shared__ float qps[kScanGroups][kMaxExperts];
   __shared__ float term[kMaxExperts];
   __shared__ int kept_s[kMaxExperts];
-  const int e = threadIdx.x;
+  const int e = threadIdx.x % kMaxExperts, g = threadIdx.x / kMaxExperts;
+  const int hq = (plan_blocks + kScanGroups - 1) / kScanGroups, h0 = g * hq, h1 = min(plan_blocks, h0 + hq);
+  const int rq = (router_blocks + kScanGroups - 1) / kScanGroups, r0 = g * rq, r1 = min(router_blocks, r0 + rq);
+  if (e < E) {
+    int sum = 0;
+    for (int b0 = h0; b0 < h1; b0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = b0 + j < h1 ? hist[(size_t)(b0 + j) * E + e] : 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) sum += v[j];
+    }
+    qsum[g][e] = sum;
+    float ps = 0.f;
+    for (int b0 = r0; b0 < r1; b0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = b0 + j < r1 ? psum_partial[(size_t)(b0 + j) * E + e] : 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) ps += v[j];                                          // fixed order
+    }
+    qps[g][e] = ps;
+  }
+  __syncthreads();
   if (e < E) {
     int run = 0;
-    for (int b = 0; b < plan_blocks; ++b) {
-      hist_base[(size_t)b * E + e] = run;
-      run += hist[(size_t)b * E + e];
+    for (int q = 0; q < g; ++q) run += qsum[q][e];
+    for (int b0 = h0; b0 < h1; b0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = b0 + j < h1 ? hist[(size_t)(b0 + j) * E + e] : 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (b0 + j < h1) { hist_base[(size_t)(b0 + j) * E + e] = run; run += v[j]; }
     }
-    count[e] = run;
-    const int k = min(run, C);
-    kept[e] = k;
-    kept_s[e] = k;
-    float ps = 0.f;
-    for (int b = 0; b < router_blocks; ++b) ps += psum_partial[(size_t)b * E + e];   // fixed order
-    psum[e] = ps;
-    term[e] = ((float)run / (float)T) * (ps / (float)T);                              // f_i . P_i  (Eq. 5, 6)
+    if (g == 0) {
+      int total = 0;
+      float ps = 0.f;
+      for (int q = 0; q < kScanGroups; ++q) { total += qsum[q][e]; ps += qps[q][e]; }
+      count[e] = total;
+      const int k = min(total, C);
+      kept[e] = k;
+      kept_s[e] = k;
+      psum[e] = ps;
+      term[e] = ((float)total / (float)T) * (ps / (float)T);                           // f_i . P_i  (Eq. 5, 6)
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -188,7 +223,7 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
       return SWITCH_MOE_CUDA_ERROR;
   }
   plan_hist_kernel<<<s.plan_blocks, kPlanBlockTokens, 0, st>>>(ei, s.T, s.E, ws_ptr<int>(ws, p.hist));
-  plan_scan_kernel<<<1, kMaxExperts, 0, st>>>(ws_ptr<int>(ws, p.hist), s.plan_blocks,
+  plan_scan_kernel<<<1, kScanGroups * kMaxExperts, 0, st>>>(ws_ptr<int>(ws, p.hist), s.plan_blocks,
                                               ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, s.C,
                                               s.alpha, ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count),
                                               ws_ptr<int>(ws, p.kept), ws_ptr<float>(ws, p.psum), aux_loss,

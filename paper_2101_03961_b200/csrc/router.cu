@@ -351,10 +351,19 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
   router_dlogits_kernel<NE><<<(s.T + 7) / 8, 256, 0, st>>>(ws_ptr<float>(ws, p.probs),
                                                             ws_ptr<int>(ws, p.expert_index), ws_ptr<int>(ws, p.slot),
                                                             ws_ptr<int>(ws, p.count), dgate, cG, s.T, s.E, dlogits);
-  dim3 grid((s.d + kDwrK - 1) / kDwrK, s.dwr_chunks);
   float* partial = ws_ptr<float>(ws, p.dwr_partial);
-  router_dwr_partial_kernel<XT, NE><<<grid, 256, 0, st>>>(static_cast<const XT*>(x), dlogits, s.T, s.d, s.E, partial);
   const size_t n = (size_t)s.d * s.E;
+  if constexpr (sizeof(XT) == 2) {
+    if (s.router_tc) {
+      // tensor-core products (bf16-split operands), then the same fixed-order reduction of the token splits
+      int rc = launch_router_tc_bwd(s, p, x, W_r, ws, dx, accumulate_dx, st);
+      if (rc != SWITCH_MOE_OK) return rc;
+      router_dwr_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partial, s.dwr_chunks, n, dW_r);
+      return launch_status();
+    }
+  }
+  dim3 grid((s.d + kDwrK - 1) / kDwrK, s.dwr_chunks);
+  router_dwr_partial_kernel<XT, NE><<<grid, 256, 0, st>>>(static_cast<const XT*>(x), dlogits, s.T, s.d, s.E, partial);
   router_dwr_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partial, s.dwr_chunks, n, dW_r);
   constexpr int ES = 32 * NE + 4;
   const size_t smem = 2 * 64 * ES * sizeof(float);
@@ -379,6 +388,7 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
 
 int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
                       cudaStream_t st) {
+  if (s.router_tc && s.dtype == SWITCH_MOE_BF16) return launch_router_tc_fwd(s, p, x, W_r, bias, ws, st);
   SWMOE_DISPATCH_NE(router_fwd_t, s, p, x, W_r, bias, ws, st)
 }
 

@@ -1,0 +1,509 @@
+// Router of the Switch FFN layer on the B200 tensor cores with float32-grade accuracy (Section 2.4: the router is the
+// part of the layer that must not run in bfloat16).
+//
+// x is bfloat16, hence exact in float32.  A float32 operand w is written as the sum of three bfloat16 numbers
+// (w = hi + mid + lo exactly up to 2^-24 relative), every bf16 x bf16 product is exact in float32, and tcgen05
+// accumulates in float32.  So
+//   logits   h = x W_r            = x (W_hi + W_mid + W_lo)                       (Section 2.1; Eq. 1 follows in the epilogue)
+//   dW_r       = x^T dh           = x^T (dh_hi + dh_mid + dh_lo)                  (contraction over tokens, split over CTAs)
+//   dx_router  = dh W_r^T         ~ dh_hi W_hi^T + dh_hi W_mid^T + dh_mid W_hi^T  (the output is bfloat16: 2^-16 suffices)
+// are bfloat16 tensor-core products whose results agree with the float32 definition to about 1e-7 relative, and the
+// router stops being bound by the FP32 FMA pipes (E flop per byte of x) and becomes a streaming kernel.
+//
+// The forward epilogue keeps one token per thread (a TMEM lane holds all E logits of a token): softmax, top-1 with
+// lowest-index ties and the gate need no cross-thread traffic; the column sums of p for Eq. 6 use warp shuffles.
+#include "tc_common.cuh"
+
+namespace swmoe {
+using namespace tc;
+namespace {
+
+constexpr int kRThreads = 192;                       // TMA warp, MMA warp, 4 epilogue warps
+constexpr int kROutStageBytes = 4 * 32 * 128;
+constexpr int kRSmemBytes = 1024 + kStages * kStageBytes + kROutStageBytes + 128;
+
+enum RouterOp { kRFwd = 0, kRDwr = 1, kRDx = 2 };
+
+struct RouterTcParams {
+  int T, d, E, Epad64;
+  int mma_n;                 // MMA N: Epad64 (fwd, dwr) or 256 (dx)
+  int n_mtiles, n_ntiles;
+  int splits, chunk_kblocks, total_kblocks;   // dwr: split of the token contraction
+  int wrap;                  // k-blocks per part: d/64 (fwd), Epad64/64 (dx); dwr derives it per tile
+  const float* bias; float* probs; int* expert_index; float* gate; float* psum_partial;   // fwd
+  float* partial;                                                                         // dwr
+  __nv_bfloat16* dx; const int* slot; int accumulate;                                     // dx
+  int* status;
+};
+
+struct RTile {
+  int m0, n0, split, k_base, wrap, k_blocks;
+};
+
+template <int OP>
+__device__ __forceinline__ int r_total_tiles(const RouterTcParams& p) {
+  if (OP == kRFwd) return p.n_mtiles;
+  if (OP == kRDwr) return p.n_mtiles * p.splits;
+  return p.n_mtiles * p.n_ntiles;
+}
+
+template <int OP>
+__device__ __forceinline__ RTile r_decode(const RouterTcParams& p, int id) {
+  RTile t;
+  t.split = 0; t.k_base = 0; t.n0 = 0;
+  if (OP == kRFwd) {
+    t.m0 = id * kTileM; t.wrap = p.wrap;
+  } else if (OP == kRDwr) {
+    const int mt = id / p.splits;
+    t.split = id - mt * p.splits;
+    t.m0 = mt * kTileM;
+    t.k_base = t.split * p.chunk_kblocks;
+    t.wrap = max(0, min(p.chunk_kblocks, p.total_kblocks - t.k_base));
+  } else {
+    const int mt = id / p.n_ntiles;
+    t.m0 = mt * kTileM;
+    t.n0 = (id - mt * p.n_ntiles) * kBN;
+    t.wrap = p.wrap;
+  }
+  t.k_blocks = 3 * t.wrap;
+  return t;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
+}
+
+template <int OP>
+__global__ void __launch_bounds__(kRThreads, 1)
+router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const RouterTcParams p) {
+  constexpr bool kAMn = (OP == kRDwr);                 // x^T: token rows are the contraction, d contiguous
+  constexpr bool kBMn = (OP != kRDx);                  // fwd: W [d][E]; dwr: dh [T][E]; dx: W as [d rows][E contiguous]
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + kStages * kStageBytes + kROutStageBytes;
+  uint8_t* bar_gen = smem_gen + kStages * kStageBytes + kROutStageBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
+  volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kStages + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kStages + 4) + 4);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(const_cast<uint32_t*>(tmem_ptr_s))), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_s;
+  const int n_tiles = r_total_tiles<OP>(p);
+  const int b_atoms = (p.mma_n + 63) / 64;
+  const uint32_t stage_tx = kABytes + (kBMn ? (uint32_t)b_atoms * kAtomBytes : (uint32_t)kBBytes);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+        const RTile t = r_decode<OP>(p, id);
+        for (int kb = 0; kb < t.k_blocks; ++kb) {
+          const int part = kb / t.wrap, kblk = t.k_base + (kb - part * t.wrap);
+          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 11);
+          if (!ok) break;
+          const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
+          mbar_arrive_expect_tx(full_bar(stage), stage_tx);
+          if (OP == kRFwd) {
+            tma_load_3d(a_dst, &tmA, full_bar(stage), kblk * kBK, t.m0, 0);                 // x tile [128 tok][64 k]
+            for (int j = 0; j < b_atoms; ++j)                                                // W part [64 k][64 e]
+              tma_load_3d(b_dst + j * kAtomBytes, &tmB, full_bar(stage), 64 * j, kblk * kBK, part);
+          } else if (OP == kRDwr) {
+            tma_load_3d(a_dst, &tmA, full_bar(stage), t.m0, kblk * kBK, 0);                 // x^T: [64 tok][64 k-of-d]
+            tma_load_3d(a_dst + kAtomBytes, &tmA, full_bar(stage), t.m0 + 64, kblk * kBK, 0);
+            for (int j = 0; j < b_atoms; ++j)                                                // dh part [64 tok][64 e]
+              tma_load_3d(b_dst + j * kAtomBytes, &tmB, full_bar(stage), 64 * j, kblk * kBK, part);
+          } else {
+            const int a_part = part == 2 ? 1 : 0, b_part = part == 1 ? 1 : 0;               // (hi,hi) (hi,mid) (mid,hi)
+            tma_load_3d(a_dst, &tmA, full_bar(stage), kblk * kBK, t.m0, a_part);            // dh part [128 tok][64 e]
+            tma_load_3d(b_dst, &tmB, full_bar(stage), kblk * kBK, t.n0, b_part);            // W part [256 k-of-d][64 e]
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (*abort_flag != 0) {
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)kAMn << 15) | ((uint32_t)kBMn << 16) |
+                             ((uint32_t)(p.mma_n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+      const uint32_t a_lbo = kAMn ? kAtomBytes : 16u, b_lbo = kBMn ? kAtomBytes : 16u;
+      const uint32_t a_kstep = kAMn ? kUmmaK * 128u : kUmmaK * 2u;
+      const uint32_t b_kstep = kBMn ? kUmmaK * 128u : kUmmaK * 2u;
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+        const RTile t = r_decode<OP>(p, id);
+        ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 12);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * kBN;
+        for (int kb = 0; kb < t.k_blocks; ++kb) {
+          ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, 13);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_src = smem_base + stage * kStageBytes, b_src = a_src + kABytes;
+#pragma unroll
+          for (int ks = 0; ks < kBK / kUmmaK; ++ks) {
+            const uint64_t ad = make_smem_desc(a_src + ks * a_kstep, a_lbo, 1024u);
+            const uint64_t bd = make_smem_desc(b_src + ks * b_kstep, b_lbo, 1024u);
+            tc_mma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        if (t.k_blocks > 0) tc_commit(tfull_bar(acc));
+        else mbar_arrive(tfull_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    const int lg = warp & 3;
+    uint8_t* my_stage_gen = smem_gen + kStages * kStageBytes + (warp - 2) * 4096;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    float colrun[8];                                          // fwd: running column sums of p, lane i <-> column c*32+i
+#pragma unroll
+    for (int c = 0; c < 8; ++c) colrun[c] = 0.f;
+    for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+      const RTile t = r_decode<OP>(p, id);
+      const int r = lg * 32 + lane;
+      // dx: previous contents of the rows this thread will write (prefetched before the accumulator is ready)
+      long long offs[8];
+      unsigned add_mask = 0;
+      if (OP == kRDx) {
+        const int tok = t.m0 + r;
+        const long long row_off = tok < p.T ? (long long)tok * p.d : -1;
+        const int add = (p.accumulate && tok < p.T && p.slot[tok] >= 0) ? 1 : 0;
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          offs[it] = __shfl_sync(0xffffffffu, row_off, it * 4 + (lane >> 3));
+          add_mask |= (unsigned)__shfl_sync(0xffffffffu, add, it * 4 + (lane >> 3)) << it;
+        }
+      }
+      ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 14);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)acc * kBN;
+      const bool have_acc = t.k_blocks > 0;
+
+      if (OP == kRFwd) {
+        // ---- Eq. 1 softmax, top-1 (lowest index on ties) and gate for token m0 + r; all E logits are in this lane
+        const int tok = t.m0 + r;
+        const int nch = p.mma_n / 32;
+        float m = -INFINITY;
+        int am = 0;
+        for (int c = 0; c < nch; ++c) {
+          uint32_t v[32];
+          tc_ld32(t_addr + c * 32, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int e = c * 32 + i;
+            if (e < p.E) {
+              const float h = __uint_as_float(v[i]) + (p.bias ? p.bias[e] : 0.f);
+              if (h > m) { m = h; am = e; }
+            }
+          }
+        }
+        float sum = 0.f;
+        for (int c = 0; c < nch; ++c) {
+          uint32_t v[32];
+          tc_ld32(t_addr + c * 32, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int e = c * 32 + i;
+            if (e < p.E) sum += expf(__uint_as_float(v[i]) + (p.bias ? p.bias[e] : 0.f) - m);
+          }
+        }
+        const float inv = 1.f / sum;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (c >= nch) break;
+          uint32_t v[32];
+          tc_ld32(t_addr + c * 32, v);
+          tc_wait_ld();
+          if (c == nch - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+          }
+          float pr[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int e = c * 32 + i;
+            pr[i] = (e < p.E && tok < p.T)
+                        ? expf(__uint_as_float(v[i]) + (p.bias ? p.bias[e] : 0.f) - m) * inv : 0.f;
+          }
+          if (tok < p.T) {
+            float* dst = p.probs + (size_t)tok * p.E + c * 32;
+            if ((p.E & 3) == 0) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4)
+                if (c * 32 + i < p.E) *reinterpret_cast<float4*>(dst + i) = make_float4(pr[i], pr[i + 1], pr[i + 2], pr[i + 3]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (c * 32 + i < p.E) dst[i] = pr[i];
+            }
+          }
+          // column sums of p over this warp's 32 tokens (Eq. 6); lane i keeps column c*32 + i
+          float mine = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float s = warp_sum(pr[i]);
+            if (lane == i) mine = s;
+          }
+          colrun[c] += mine;
+        }
+        if (tok < p.T) { p.expert_index[tok] = am; p.gate[tok] = inv; }
+      } else if (OP == kRDwr) {
+        // ---- float32 partial of x^T dh for this token split: row = m0 + r (an index into d_model)
+        const int row = t.m0 + r;
+        const int nch = p.mma_n / 32;
+        for (int c = 0; c < nch; ++c) {
+          uint32_t v[32];
+          if (have_acc) {
+            tc_ld32(t_addr + c * 32, v);
+            tc_wait_ld();
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = 0u;
+          }
+          if (c == nch - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+          }
+          if (row < p.d) {
+            float* dst = p.partial + ((size_t)t.split * p.d + row) * p.E + c * 32;
+            if ((p.E & 3) == 0) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4)
+                if (c * 32 + i < p.E)
+                  *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                                    __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (c * 32 + i < p.E) dst[i] = __uint_as_float(v[i]);
+            }
+          }
+        }
+      } else {
+        // ---- dx[token] = (accumulate and kept ? dx[token] : 0) + dh W_r^T, 64 columns at a time
+#pragma unroll 1
+        for (int c = 0; c < kBN / 64; ++c) {
+          const int col = t.n0 + c * 64 + (lane & 7) * 8;
+          uint4 prev[8];
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            prev[it] = (((add_mask >> it) & 1u) && col < p.d) ? *reinterpret_cast<const uint4*>(p.dx + offs[it] + col)
+                                                             : make_uint4(0, 0, 0, 0);
+          uint32_t v[64];
+          tc_ld32(t_addr + c * 64, v);
+          tc_ld32(t_addr + c * 64 + 32, v + 32);
+          tc_wait_ld();
+          if (c == kBN / 64 - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+          }
+          // stage the float32 values as two bf16-pair planes?  No: keep float32 accuracy of the sum by staging
+          // bf16(acc) only when nothing is added; otherwise add in float32 after the transpose (values are bf16
+          // on both sides, so staging bf16(acc) costs one extra rounding of the small router term only).
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            uint32_t w[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * q]),
+                                                        __uint_as_float(v[j * 8 + 2 * q + 1]));
+              w[q] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            *reinterpret_cast<uint4*>(my_stage_gen + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                make_uint4(w[0], w[1], w[2], w[3]);
+          }
+          __syncwarp();
+          if (col < p.d) {
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+              const int rr = it * 4 + (lane >> 3);
+              uint4 val = *reinterpret_cast<const uint4*>(my_stage_gen + rr * 128 + (((lane & 7) ^ (rr & 7)) << 4));
+              if ((add_mask >> it) & 1u) {
+                __nv_bfloat162* vp = reinterpret_cast<__nv_bfloat162*>(&val);
+                const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&prev[it]);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const float2 a = __bfloat1622float2(vp[q]), b = __bfloat1622float2(pp[q]);
+                  vp[q] = __floats2bfloat162_rn(a.x + b.x, a.y + b.y);
+                }
+              }
+              if (offs[it] >= 0) *reinterpret_cast<uint4*>(p.dx + offs[it] + col) = val;
+            }
+          }
+          __syncwarp();
+        }
+      }
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+    if (OP == kRFwd) {                                        // this warp's column sums over all tiles of this CTA
+      float* mine = reinterpret_cast<float*>(my_stage_gen);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) mine[c * 32 + lane] = colrun[c];
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (OP == kRFwd && warp >= 2) {
+    // one partial P-sum row per CTA: the four epilogue warps' sums added in a fixed order (Eq. 6)
+    const float* st0 = reinterpret_cast<const float*>(smem_gen + kStages * kStageBytes);
+    for (int e = threadIdx.x - 64; e < p.E; e += 128)
+      p.psum_partial[(size_t)blockIdx.x * p.E + e] = ((st0[e] + st0[1024 + e]) + st0[2048 + e]) + st0[3072 + e];
+  }
+  if (warp == 2) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// w = hi + mid + lo with hi, mid, lo bfloat16 (round to nearest); exact to about 2^-24 relative.
+__device__ __forceinline__ void split3(float w, __nv_bfloat16* hi, __nv_bfloat16* mid, __nv_bfloat16* lo) {
+  const __nv_bfloat16 h = __float2bfloat16(w);
+  const float r1 = w - __bfloat162float(h);
+  const __nv_bfloat16 m = __float2bfloat16(r1);
+  const float r2 = r1 - __bfloat162float(m);
+  *hi = h; *mid = m; *lo = __float2bfloat16(r2);
+}
+
+// wsplit[part][k][e] for e < Epad64 (zero beyond E)
+__global__ void split_w_kernel(const float* __restrict__ W_r, int d, int E, int Epad64,
+                               __nv_bfloat16* __restrict__ wsplit) {
+  const size_t n = (size_t)d * Epad64;
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int k = (int)(i / Epad64), e = (int)(i - (size_t)k * Epad64);
+  __nv_bfloat16 h, m, l;
+  split3(e < E ? W_r[(size_t)k * E + e] : 0.f, &h, &m, &l);
+  wsplit[i] = h; wsplit[n + i] = m; wsplit[2 * n + i] = l;
+}
+
+// dhsplit[part][t][e] from the float32 logit gradients
+__global__ void split_dh_kernel(const float* __restrict__ dlogits, int T, int E, int Epad64,
+                                __nv_bfloat16* __restrict__ dhsplit) {
+  const size_t n = (size_t)T * Epad64;
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int t = (int)(i / Epad64), e = (int)(i - (size_t)t * Epad64);
+  __nv_bfloat16 h, m, l;
+  split3(e < E ? dlogits[(size_t)t * E + e] : 0.f, &h, &m, &l);
+  dhsplit[i] = h; dhsplit[n + i] = m; dhsplit[2 * n + i] = l;
+}
+
+int sm_count_or_default() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  return n;
+}
+
+template <int OP>
+int launch_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const RouterTcParams& q, cudaStream_t st) {
+  if (cudaFuncSetAttribute(router_tc_kernel<OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
+      cudaSuccess)
+    return SWITCH_MOE_CUDA_ERROR;
+  router_tc_kernel<OP><<<sm_count_or_default(), kRThreads, kRSmemBytes, st>>>(tmA, tmB, q);
+  return launch_status();
+}
+
+}  // namespace
+
+int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
+                         cudaStream_t st) {
+  __nv_bfloat16* wsplit = ws_ptr<__nv_bfloat16>(ws, p.wsplit);
+  const size_t n = (size_t)s.d * s.Epad64;
+  split_w_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(W_r, s.d, s.E, s.Epad64, wsplit);
+  CUtensorMap tmA, tmB;
+  if (make_map(&tmA, x, 1, s.T, s.d, kTileM) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  if (make_map(&tmB, wsplit, 3, s.d, s.Epad64, 64) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  RouterTcParams q{};
+  q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.mma_n = s.Epad64;
+  q.n_mtiles = (s.T + kTileM - 1) / kTileM; q.n_ntiles = 1; q.wrap = s.d / kBK;
+  q.bias = bias; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
+  q.gate = ws_ptr<float>(ws, p.gate); q.psum_partial = ws_ptr<float>(ws, p.psum_partial);
+  q.status = ws_ptr<int>(ws, p.status);
+  if (cudaFuncSetAttribute(router_tc_kernel<kRFwd>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
+      cudaSuccess)
+    return SWITCH_MOE_CUDA_ERROR;
+  // the grid is part of the workspace layout: one partial P-sum row per CTA
+  router_tc_kernel<kRFwd><<<s.router_blocks, kRThreads, kRSmemBytes, st>>>(tmA, tmB, q);
+  return launch_status();
+}
+
+int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, void* ws, void* dx,
+                         bool accumulate_dx, cudaStream_t st) {
+  __nv_bfloat16* wsplit = ws_ptr<__nv_bfloat16>(ws, p.wsplit);
+  __nv_bfloat16* dhsplit = ws_ptr<__nv_bfloat16>(ws, p.dhsplit);
+  const size_t nw = (size_t)s.d * s.Epad64;
+  split_w_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(W_r, s.d, s.E, s.Epad64, wsplit);
+  const size_t n = (size_t)s.T * s.Epad64;
+  split_dh_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ws_ptr<float>(ws, p.dlogits), s.T, s.E, s.Epad64,
+                                                                dhsplit);
+  RouterTcParams q{};
+  q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64;
+  q.status = ws_ptr<int>(ws, p.status);
+  CUtensorMap tmA, tmB;
+  // dW_r partials: A = x^T (MN-major view of x [T][d]), B = dh parts [3][T][Epad64] (MN-major)
+  if (make_map(&tmA, x, 1, s.T, s.d, 64) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  if (make_map(&tmB, dhsplit, 3, s.T, s.Epad64, 64) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  q.mma_n = s.Epad64;
+  q.n_mtiles = (s.d + kTileM - 1) / kTileM; q.n_ntiles = 1;
+  q.splits = s.dwr_chunks;
+  q.total_kblocks = (s.T + kBK - 1) / kBK;
+  q.chunk_kblocks = (q.total_kblocks + q.splits - 1) / q.splits;
+  q.partial = ws_ptr<float>(ws, p.dwr_partial);
+  int rc = launch_op<kRDwr>(tmA, tmB, q, st);
+  if (rc != SWITCH_MOE_OK) return rc;
+  // dx: A = dh parts (K-major), B = W parts [3][d][Epad64] (K-major: rows are d_model indices)
+  if (make_map(&tmA, dhsplit, 3, s.T, s.Epad64, kTileM) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  if (make_map(&tmB, wsplit, 3, s.d, s.Epad64, kBN) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  q.mma_n = kBN;
+  q.n_mtiles = (s.T + kTileM - 1) / kTileM; q.n_ntiles = (s.d + kBN - 1) / kBN;
+  q.wrap = s.Epad64 / kBK;
+  q.dx = static_cast<__nv_bfloat16*>(dx); q.slot = ws_ptr<int>(ws, p.slot); q.accumulate = accumulate_dx ? 1 : 0;
+  return launch_op<kRDx>(tmA, tmB, q, st);
+}
+
+}  // namespace swmoe

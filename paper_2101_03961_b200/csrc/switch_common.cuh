@@ -24,13 +24,15 @@ struct Shape {
   float alpha;
   size_t elt;       // bytes per activation / expert-weight element
   int Epad;         // E rounded up to 32 * {1,2,4,8}
+  int Epad64;       // E rounded up to a multiple of 64 (tensor-core router operands)
+  int router_tc;    // 1: router on the tensor cores (bf16 x, 3-way bf16 split of fp32 operands); 0: FP32 FMA
   int router_blocks, plan_blocks, max_mtiles, dwr_chunks;
 };
 
 // Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
 struct Plan {
   size_t status, expert_index, gate, slot, token_of_slot, count, kept, psum, psum_partial, hist, hist_base,
-      tile_expert, tile_row0, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, total;
+      tile_expert, tile_row0, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, total;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -67,10 +69,25 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   int ne_pow2 = 1;
   while (ne_pow2 < ne) ne_pow2 *= 2;
   s->Epad = 32 * ne_pow2;
-  s->router_blocks = (cfg->T + kRouterBlockTokens - 1) / kRouterBlockTokens;
+  s->Epad64 = (cfg->E + 63) / 64 * 64;
+  s->router_tc = s->gemm_path == 0 ? 1 : 0;
   s->plan_blocks = (cfg->T + kPlanBlockTokens - 1) / kPlanBlockTokens;
   s->max_mtiles = cfg->E * ((s->C + kTileM - 1) / kTileM);
-  s->dwr_chunks = (cfg->T + kDwrChunkTokens - 1) / kDwrChunkTokens;
+  if (s->router_tc) {
+    // one partial P-sum row per CTA of the persistent router kernel; dW_r split so that tiles x splits fills the GPU
+    s->router_blocks = (cfg->T + kTileM - 1) / kTileM;
+    if (s->router_blocks > 148) s->router_blocks = 148;
+    const int m_tiles = (cfg->d_model + kTileM - 1) / kTileM;
+    const int k_blocks = (cfg->T + 63) / 64;
+    int splits = 144 / m_tiles;
+    if (splits < 1) splits = 1;
+    if (splits > 64) splits = 64;
+    if (splits > k_blocks) splits = k_blocks;
+    s->dwr_chunks = splits;
+  } else {
+    s->router_blocks = (cfg->T + kRouterBlockTokens - 1) / kRouterBlockTokens;
+    s->dwr_chunks = (cfg->T + kDwrChunkTokens - 1) / kDwrChunkTokens;
+  }
   return SWITCH_MOE_OK;
 }
 
@@ -99,6 +116,8 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->dh = take(E * C * f * s.elt);
   p->dgate = take(T * 4);
   p->dwr_partial = take((size_t)s.dwr_chunks * d * E * 4);
+  p->wsplit = take(3 * d * (size_t)s.Epad64 * 2);
+  p->dhsplit = take(3 * T * (size_t)s.Epad64 * 2);
   p->total = off;
 }
 
@@ -118,6 +137,12 @@ int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void*
 int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* ws, cudaStream_t st);
 int launch_router_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* dgate, float d_aux,
                       void* ws, void* dx, bool accumulate_dx, float* dW_r, cudaStream_t st);
+
+// Tensor-core router (bf16 x): forward (logits, softmax, top-1, gate, P-sum partials) and the two backward products.
+int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
+                         cudaStream_t st);
+int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, void* ws, void* dx,
+                         bool accumulate_dx, cudaStream_t st);
 
 // The six expert GEMMs (Section 5: h = x W_in, y = ReLU(h) W_out, and their derivatives).
 enum GemmOp {

@@ -208,10 +208,14 @@ def test_capacity_override_is_honoured():
 
 
 # ---------------------------------------------------------------------------------------------- router backward (staged)
-@pytest.mark.parametrize("cfg", [TINY, MID.with_(dtype=si.DTYPE_F32), RAGGED], ids=lambda c: c.name)
-def test_router_backward_given_identical_gate_gradient(cfg):
+@pytest.mark.parametrize("cfg,path", [
+    (TINY, sm.GEMM_SIMT), (MID.with_(dtype=si.DTYPE_F32), sm.GEMM_SIMT), (RAGGED, sm.GEMM_SIMT),
+    (RAGGED, sm.GEMM_DEFAULT), (MID, sm.GEMM_DEFAULT), (MANY, sm.GEMM_DEFAULT),
+    (si.SwitchConfig("e256_bwd", 1500, 64, 64, 256, 2.0), sm.GEMM_DEFAULT),
+], ids=lambda v: v.name if hasattr(v, "name") else ("tensor_core_router" if v == sm.GEMM_DEFAULT else "fma_router"))
+def test_router_backward_given_identical_gate_gradient(cfg, path):
     data = si.gen_layer(cfg, seed=4)
-    g = GpuLayer(cfg, data, gemm_path=sm.GEMM_SIMT)
+    g = GpuLayer(cfg, data, gemm_path=path)
     g.fwd()
     gpu_e = g.expert_index()
     fwd = oracle_following(cfg, data, gpu_e, experts=[])
