@@ -239,9 +239,11 @@ def run_ours(args, cfg):
     barrier()
     sampler.start()
     t_start.record(stream)
+    host_t0 = time.perf_counter()
     for k in range(args.steps):
         sm.set_stage_events(mcfg, events[k])
         step()
+    host_enqueue_ms = (time.perf_counter() - host_t0) * 1e3 / args.steps
     t_end.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -338,7 +340,7 @@ def run_ours(args, cfg):
                    "l2": "inputs larger than L2 (weights 2 x %.0f MB per pass), no flush" %
                          (cfg.E * cfg.d_model * cfg.d_ff * elt / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": sm.switch_moe_launches_per_step(mcfg) * args.steps,
-        "roofline": roofline, "cpu_baseline": cpu, "stages": stages,
+        "roofline": roofline, "cpu_baseline": cpu, "stages": stages, "host_enqueue_ms_per_step": host_enqueue_ms,
         "aux_loss": float(aux.item()),
     }
     print(json.dumps(line), flush=True)

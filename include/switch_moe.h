@@ -37,8 +37,10 @@ extern "C" {
 enum switch_moe_dtype { SWITCH_MOE_BF16 = 0, SWITCH_MOE_F32 = 1 };
 
 enum switch_moe_gemm_path {
-  SWITCH_MOE_GEMM_DEFAULT = 0, /* bf16: tcgen05 tensor-core grouped GEMM; f32: plain FP32 FMA grouped GEMM */
-  SWITCH_MOE_GEMM_SIMT = 1     /* validation only: FP32-FMA grouped GEMM for either dtype */
+  SWITCH_MOE_GEMM_DEFAULT = 0, /* bf16: tcgen05 grouped GEMM on CTA pairs (tokens on the MMA N side) and tensor-core
+                                  router; f32: plain FP32 FMA grouped GEMM and router */
+  SWITCH_MOE_GEMM_SIMT = 1,    /* validation only: FP32-FMA grouped GEMM and router for either dtype */
+  SWITCH_MOE_GEMM_TC_1CTA = 2  /* validation only: single-CTA tcgen05 grouped GEMM with 128-token tiles (bf16) */
 };
 
 typedef enum switch_moe_status {

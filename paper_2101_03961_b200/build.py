@@ -12,7 +12,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libswitch_moe.so")
-SOURCES = ["api.cu", "router.cu", "dispatch.cu", "simt_gemm.cu", "grouped_gemm_sm100.cu", "router_sm100.cu",
+SOURCES = ["api.cu", "router.cu", "dispatch.cu", "simt_gemm.cu", "grouped_gemm_sm100.cu", "expert_gemm_pair_sm100.cu", "router_sm100.cu",
            "dispatch_static.cu"]
 
 

@@ -26,7 +26,9 @@ int prepare(const switch_moe_config* cfg, const void* workspace, size_t workspac
 }
 
 int run_gemm(GemmOp op, const Ctx& c, const GemmArgs& a, void* ws, cudaStream_t st) {
-  return c.s.gemm_path == 0 ? launch_tc_gemm(op, c.s, c.p, a, ws, st) : launch_simt_gemm(op, c.s, c.p, a, ws, st);
+  if (c.s.gemm_path == 0) return launch_pair_gemm(op, c.s, c.p, a, ws, st);
+  if (c.s.gemm_path == 2) return launch_tc_gemm(op, c.s, c.p, a, ws, st);
+  return launch_simt_gemm(op, c.s, c.p, a, ws, st);
 }
 
 // Optional per-stage timing: records the caller's event `i` on the stream (see switch_moe_config::stage_events).

@@ -30,7 +30,8 @@ __global__ void __launch_bounds__(kScanGroups * kMaxExperts)
 plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __restrict__ psum_partial,
                  int router_blocks, int T, int E, int C, float alpha, int* __restrict__ hist_base,
                  int* __restrict__ count, int* __restrict__ kept, float* __restrict__ psum,
-                 float* __restrict__ aux_loss, int* __restrict__ tile_expert, int* __restrict__ tile_row0) {
+                 float* __restrict__ aux_loss, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
+                 int4* __restrict__ ntile) {
   __shared__ int qsum[kScanGroups][kMaxExperts];
   __shared__ float qps[kScanGroups][kMaxExperts];
   __shared__ float term[kMaxExperts];
@@ -83,19 +84,35 @@ plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __r
     }
   }
   __syncthreads();
+  // Tile lists.  128-row token tiles (single-CTA GEMM) and, for the paired-CTA GEMM, each expert's kept rows cut
+  // into the fewest pieces of at most 256 rows, equal up to rounding each piece to a multiple of 16 (the MMA's N
+  // granularity).  Thread 0 adds the loss terms and scans the per-expert tile counts; experts write their entries.
+  __shared__ int start128[kMaxExperts + 1], startn[kMaxExperts + 1];
   if (threadIdx.x == 0) {
     float s = 0.f;
     for (int i = 0; i < E; ++i) s += term[i];
     if (aux_loss != nullptr) *aux_loss = alpha * (float)E * s;                        // Eq. 4
-    int n = 0;
-    for (int i = 0; i < E; ++i)
-      for (int r = 0; r < kept_s[i]; r += kTileM) {
-        tile_expert[1 + n] = i;
-        tile_row0[1 + n] = r;
-        ++n;
-      }
+    int n = 0, m = 0;
+    for (int i = 0; i < E; ++i) {
+      start128[i] = n; startn[i] = m;
+      n += (kept_s[i] + kTileM - 1) / kTileM;
+      m += (kept_s[i] + 255) / 256;
+    }
     tile_expert[0] = n;
     tile_row0[0] = n;
+    ntile[0] = make_int4(m, 0, 0, 0);
+  }
+  __syncthreads();
+  if (g == 0 && e < E) {
+    const int k = kept_s[e];
+    int n = start128[e];
+    for (int r = 0; r < k; r += kTileM, ++n) { tile_expert[1 + n] = e; tile_row0[1 + n] = r; }
+    if (k > 0) {
+      const int pieces = (k + 255) / 256;
+      const int rows = ((k + pieces - 1) / pieces + 15) / 16 * 16;
+      int m = startn[e];
+      for (int r = 0; r < k; r += rows, ++m) ntile[1 + m] = make_int4(e, r, min(rows, (k - r + 15) / 16 * 16), 0);
+    }
   }
 }
 
@@ -227,7 +244,8 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
                                               ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, s.C,
                                               s.alpha, ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count),
                                               ws_ptr<int>(ws, p.kept), ws_ptr<float>(ws, p.psum), aux_loss,
-                                              ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0));
+                                              ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0),
+                                              ws_ptr<int4>(ws, p.ntile));
   plan_assign_kernel<<<s.plan_blocks, kPlanBlockTokens, 0, st>>>(ei, ws_ptr<int>(ws, p.hist_base),
                                                                  ws_ptr<int>(ws, p.kept), s.T, s.E, s.C,
                                                                  ws_ptr<int>(ws, p.slot),

@@ -1,0 +1,526 @@
+// Grouped expert GEMMs on pairs of SMs (tcgen05 cta_group::2, M = 256), bfloat16 in, float32 accumulate, bfloat16
+// out: the expert FFN h = x W_in, y = ReLU(h) W_out (Section 5, FFN review) and its derivatives, with the layer's
+// element-wise steps fused into the epilogues (ReLU, the gate of Eq. 2 with the scatter back to token order, the
+// ReLU mask of the backward pass).
+//
+// Orientation.  An expert has about 256 tokens but thousands of weight rows, so the weight matrix sits on the MMA's
+// M side (256 rows per CTA pair, 128 per CTA) and the expert's tokens on the N side, whose granularity is 16:
+//   H^T  [f, tok] = W_in^T  [f, d] . X_d^T  [d, tok]      y^T  [d, tok] = W_out^T [d, f] . H^T  [f, tok]
+//   dH^T [f, tok] = W_out   [f, d] . dY_d^T [d, tok]      dx^T [d, tok] = W_in    [d, f] . dH^T [f, tok]
+// so no 128-row token tile is padded, every weight element enters shared memory exactly once, and the epilogue
+// transposes 32x32 blocks through shared memory to write token-major rows.  The weight gradients keep the natural
+// orientation (dW_out = H^T dY_d, dW_in = X_d^T dH: M = weight rows, N = weight columns, contraction over tokens).
+//
+// A CTA pair shares the B operand: each CTA stages its own 128 A rows and half of B (32 KB per 64-deep k-block, six
+// stages), the leader CTA's single MMA thread issues M=256 instructions that read both CTAs' shared memory, and
+// tcgen05.commit with a cluster mask releases stages and publishes accumulators in both CTAs.  TMA loads carry no
+// multicast.  Each CTA drains its own 128 TMEM lanes with 8 epilogue warps while the next tile's MMAs run into the
+// second accumulator.
+//
+// Every mbarrier wait is bounded in time (status word + abort flag); both CTAs always reach the final cluster
+// barrier, so tensor memory is freed and no CTA exits while its peer can still address its shared memory.
+#include "tc_common.cuh"
+
+namespace swmoe {
+using namespace tc;
+namespace {
+
+constexpr int kPStages = 6;
+constexpr int kPHalfBytes = 16384;                     // A tile (128 x 64) and B half tile (<= 128 x 64)
+constexpr int kPStageBytes = 2 * kPHalfBytes;
+constexpr int kPTransBytes = 8 * 2048;                 // 8 epilogue warps x (32 x 64 B)
+constexpr int kPAuxBytes = 8 * 128;                    // 8 epilogue warps x 32 gates
+constexpr int kPSmemBytes = 1024 + kPStages * kPStageBytes + kPTransBytes + kPAuxBytes + 256;
+constexpr int kPThreads = 320;
+constexpr uint32_t kPeerMask = 0xFEFFFFFFu;            // clears the CTA-rank bit of a shared::cluster address
+
+struct PairParams {
+  int op;                  // GemmOp
+  int token_op;            // 1: tokens on N (transposed epilogue); 0: weight gradient (contraction over tokens)
+  int a_mn_major;
+  int Mw;                  // rows of the M-side operand per expert (d_ff or d_model)
+  int Nfix;                // weight gradients: output columns
+  int k_blocks_fixed;      // token ops: K / 64
+  int n_mpairs, n_ntiles_fixed;
+  int C, E;
+  const int4* ntile;       // [0].x = number of token tiles; then {expert, first slot row, rows (multiple of 16)}
+  const int* kept;
+  const int* token_of_slot;
+  const float* gate;
+  __nv_bfloat16* out;
+  const __nv_bfloat16* mask_src;
+  long long ld_out;
+  int* status;
+};
+
+struct PTile {
+  int e, m0, n0, row0, n, k_blocks, last_mmas;
+};
+
+__device__ __forceinline__ int p_total_tiles(const PairParams& p) {
+  return p.token_op ? p.ntile[0].x * p.n_mpairs : p.E * p.n_mpairs * p.n_ntiles_fixed;
+}
+
+__device__ __forceinline__ PTile p_decode(const PairParams& p, int id) {
+  PTile t;
+  if (p.token_op) {
+    const int nt = id / p.n_mpairs;
+    const int4 q = p.ntile[1 + nt];
+    t.e = q.x; t.row0 = q.y; t.n = q.z; t.n0 = 0;
+    t.m0 = (id - nt * p.n_mpairs) * 256;
+    t.k_blocks = p.k_blocks_fixed;
+    t.last_mmas = kBK / kUmmaK;
+  } else {
+    const int per_e = p.n_mpairs * p.n_ntiles_fixed;
+    t.e = id / per_e;
+    const int rem = id - t.e * per_e;
+    const int mp = rem / p.n_ntiles_fixed;
+    t.m0 = mp * 256;
+    t.n0 = (rem - mp * p.n_ntiles_fixed) * 256;
+    t.row0 = 0; t.n = 256;
+    const int k = p.kept[t.e];
+    t.k_blocks = (k + kBK - 1) / kBK;
+    const int rem_rows = k - (t.k_blocks - 1) * kBK;          // rows of the last k-block that hold tokens
+    t.last_mmas = (rem_rows + kUmmaK - 1) / kUmmaK;            // rows beyond them are never multiplied
+  }
+  return t;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t cta) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+      "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
+      ::"r"(local_bar), "r"(cta)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t leader_bar, int c0,
+                                                 int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(leader_bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// One instantiation per product (OP is a GemmOp): each kernel carries only its own epilogue, and the operand
+// orientations are compile-time constants, which keeps the code footprint of every role small.
+template <int OP>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                        const PairParams p) {
+  constexpr bool kTok = OP <= kDgrad1Scatter;                 // tokens on N, transposed epilogue
+  constexpr bool kAMn = (OP == kGemm1Relu || OP == kGemm2Combine || OP == kWgrad2 || OP == kWgrad1);
+  constexpr bool kBMn = !kTok;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  uint8_t* trans_gen = smem_gen + kPStages * kPStageBytes;
+  uint8_t* aux_gen = trans_gen + kPTransBytes;
+  uint8_t* bar_gen = aux_gen + kPAuxBytes;
+  const uint32_t bar_base = smem_base + kPStages * kPStageBytes + kPTransBytes + kPAuxBytes;
+  // barrier block: full[S] | empty[S] | tmem_full[2] | tmem_empty[2] | tmem_ptr | abort
+  const uint32_t full0 = bar_base, empty0 = bar_base + 8u * kPStages;
+  const uint32_t tfull0 = bar_base + 16u * kPStages, tempty0 = tfull0 + 16u;
+  volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kPStages + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kPStages + 4) + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();                   // 0 = leader (issues the MMAs)
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPStages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 16); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(const_cast<uint32_t*>(tmem_ptr_s))), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_s;
+  const int n_tiles = p_total_tiles(p);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int id = pair; id < n_tiles && ok; id += n_pairs) {
+        const PTile t = p_decode(p, id);
+        // coordinates of this CTA's boxes; only the contraction coordinate moves inside the tile
+        const int a_m = t.m0 + 128 * (int)rank;
+        const int b_r = kTok ? t.row0 + (int)rank * (t.n >> 1) : t.n0 + 128 * (int)rank;
+        const int e = t.e, kbs = t.k_blocks;
+#pragma unroll 1
+        for (int kb = 0; kb < kbs; ++kb) {
+          const uint32_t eb = empty0 + 8u * stage;
+          ok = mbar_wait(eb, phase ^ 1u, abort_flag, p.status, 21);
+          if (!ok) break;
+          const uint32_t a_dst = smem_base + stage * kPStageBytes, b_dst = a_dst + kPHalfBytes;
+          const uint32_t fb = full0 + 8u * stage;
+          const uint32_t lead_full = fb & kPeerMask;
+          const int k0 = kb * kBK;
+          if (rank == 0) mbar_arrive_expect_tx(fb, 2 * kPStageBytes);     // both CTAs' bytes land on the leader
+          if (kAMn) {
+            tma_load_3d_pair(a_dst, &tmA, lead_full, a_m, k0, e);
+            tma_load_3d_pair(a_dst + kAtomBytes, &tmA, lead_full, a_m + 64, k0, e);
+          } else {
+            tma_load_3d_pair(a_dst, &tmA, lead_full, k0, a_m, e);
+          }
+          if (kBMn) {                                         // this CTA's 128 of the 256 output columns
+            tma_load_3d_pair(b_dst, &tmB, lead_full, b_r, k0, e);
+            tma_load_3d_pair(b_dst + kAtomBytes, &tmB, lead_full, b_r + 64, k0, e);
+          } else {                                            // this CTA's half of the expert's token rows
+            tma_load_3d_pair(b_dst, &tmB, lead_full, k0, b_r, e);
+          }
+          if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (*abort_flag != 0) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 4000000ll) __nanosleep(1000);  // let copies in flight land (about 2 ms)
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------------------------------ MMA issuer (leader CTA)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)kAMn << 15) |
+                                      ((uint32_t)kBMn << 16) | ((uint32_t)(256 >> 4) << 24);
+      // descriptors differ between stages and k-steps only in the start-address field (units of 16 bytes)
+      constexpr uint32_t a_kstep = (kAMn ? kUmmaK * 128u : kUmmaK * 2u) >> 4;
+      constexpr uint32_t b_kstep = (kBMn ? kUmmaK * 128u : kUmmaK * 2u) >> 4;
+      const uint64_t a_desc0 = make_smem_desc(smem_base, kAMn ? kAtomBytes : 16u, 1024u);
+      const uint64_t b_desc0 = make_smem_desc(smem_base + kPHalfBytes, kBMn ? kAtomBytes : 16u, 1024u);
+      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+      bool ok = true;
+      for (int id = pair; id < n_tiles && ok; id += n_pairs) {
+        const PTile t = p_decode(p, id);
+        const uint32_t idesc = idesc_base | ((uint32_t)(t.n >> 3) << 17);
+        const int kbs = t.k_blocks, last_mmas = t.last_mmas;
+        ok = mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag, p.status, 22);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * 256u;
+#pragma unroll 1
+        for (int kb = 0; kb < kbs; ++kb) {
+          ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 23);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t ad = a_desc0 + (uint64_t)(stage * (kPStageBytes >> 4));
+          const uint64_t bd = b_desc0 + (uint64_t)(stage * (kPStageBytes >> 4));
+          const int n_mma = (!kTok && kb == kbs - 1) ? last_mmas : kBK / kUmmaK;
+          tc_mma_bf16_pair(d_tmem, ad, bd, idesc, kb > 0 ? 1u : 0u);
+          if (n_mma > 1) tc_mma_bf16_pair(d_tmem, ad + a_kstep, bd + b_kstep, idesc, 1u);
+          if (n_mma > 2) tc_mma_bf16_pair(d_tmem, ad + 2 * a_kstep, bd + 2 * b_kstep, idesc, 1u);
+          if (n_mma > 3) tc_mma_bf16_pair(d_tmem, ad + 3 * a_kstep, bd + 3 * b_kstep, idesc, 1u);
+          tc_commit_pair(empty0 + 8u * stage);                // frees this stage in both CTAs
+          if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        if (kbs > 0) {
+          tc_commit_pair(tfull0 + 8u * acc);                  // accumulator complete, in both CTAs
+        } else {                                              // nothing to contract: epilogues write zeros
+          mbar_arrive(tfull0 + 8u * acc);
+          mbar_arrive_remote(tfull0 + 8u * acc, 1);
+        }
+        acc ^= 1u;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------------------------------ epilogue warps (both CTAs)
+    const int lg = warp & 3;
+    const int half = (warp - 2) >> 2;
+    uint8_t* tr = trans_gen + (warp - 2) * 2048;              // this warp's 32 x 64 B transpose tile
+    float* gate_s = reinterpret_cast<float*>(aux_gen + (warp - 2) * 128);
+    uint32_t acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (int id = pair; id < n_tiles && ok; id += n_pairs) {
+      const PTile t = p_decode(p, id);
+      const int m_warp = t.m0 + 128 * (int)rank + 32 * lg;    // first M row (weight row) this warp holds
+      const int n_chunks = kTok ? (t.n + 31) >> 5 : 8;
+      const bool have_acc = t.k_blocks > 0;
+      // Token products: lane i describes token column c*32 + i of the chunk being processed: the element offset of
+      // its output row (or -1) and its gate.  The first chunk's description (and ReLU mask) is fetched before the
+      // accumulator is awaited, each later one while the previous chunk is being written.
+      constexpr bool kSlotRows = (OP == kGemm1Relu || OP == kDgrad2Mask);
+      int row_limit = 0;
+      long long cur_off = -1;
+      float cur_gate = 1.f;
+      uint4 hm[4];
+      const int mcol = m_warp + (lane & 3) * 8;               // store `it` writes weight rows mcol .. mcol + 7
+      auto describe = [&](int c, long long* off, float* g) {
+        const int col = c * 32 + lane, slot_row = t.row0 + col;
+        *off = -1;
+        *g = 1.f;
+        if (c < n_chunks && col < t.n && slot_row < row_limit) {
+          if (kSlotRows) {
+            *off = ((long long)t.e * p.C + slot_row) * p.ld_out;
+          } else {
+            const int tok = p.token_of_slot[(long long)t.e * p.C + slot_row];
+            *off = (long long)tok * p.ld_out;
+            if (OP == kGemm2Combine) *g = p.gate[tok];        // Eq. 2: y = p_i(x) E_i(x)
+          }
+        }
+      };
+      auto fetch_mask = [&](long long off_lane, uint4* m4) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+          const long long o = __shfl_sync(0xffffffffu, off_lane, it * 8 + (lane >> 2));
+          m4[it] = (o >= 0 && mcol < p.Mw) ? *reinterpret_cast<const uint4*>(p.mask_src + o + mcol)
+                                           : make_uint4(0, 0, 0, 0);
+        }
+      };
+      if (kTok) {
+        const int kept_e = p.kept[t.e];
+        row_limit = kSlotRows ? min(p.C, (kept_e + 15) / 16 * 16) : kept_e;
+        describe(half, &cur_off, &cur_gate);
+        if (OP == kDgrad2Mask) fetch_mask(cur_off, hm);
+      }
+      ok = mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag, p.status, 24);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * 256u;
+      bool released = false;
+
+#pragma unroll 1
+      for (int c = half; c < n_chunks; c += 2) {
+        uint32_t v[32];
+        if (have_acc) {
+          tc_ld32(t_addr + c * 32, v);
+          tc_wait_ld();
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = 0u;
+        }
+        if (c + 2 >= n_chunks) {                              // last chunk of this warp: accumulator read out
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
+          released = true;
+        }
+        if (kTok) {
+          long long offs[4];
+#pragma unroll
+          for (int it = 0; it < 4; ++it) offs[it] = __shfl_sync(0xffffffffu, cur_off, it * 8 + (lane >> 2));
+          if (OP == kGemm2Combine) gate_s[lane] = cur_gate;
+          long long next_off;
+          float next_gate;
+          describe(c + 2, &next_off, &next_gate);             // next chunk's description, in flight behind this one
+          uint4 hm_next[4];
+          if (OP == kDgrad2Mask) fetch_mask(next_off, hm_next);
+          __syncwarp();
+          // transpose: this lane holds weight row m_warp + lane for 32 tokens -> tr[token][lane]
+#pragma unroll
+          for (int i4 = 0; i4 < 32; i4 += 4) {
+            float g[4] = {1.f, 1.f, 1.f, 1.f};
+            if (OP == kGemm2Combine) {
+              const float4 g4 = *reinterpret_cast<const float4*>(gate_s + i4);
+              g[0] = g4.x; g[1] = g4.y; g[2] = g4.z; g[3] = g4.w;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              float a = __uint_as_float(v[i4 + u]);
+              if (OP == kGemm2Combine) a *= g[u];
+              if (OP == kGemm1Relu) a = fmaxf(a, 0.f);
+              *reinterpret_cast<__nv_bfloat16*>(tr + (i4 + u) * 64 + lane * 2) = __float2bfloat16(a);
+            }
+          }
+          __syncwarp();
+#pragma unroll
+          for (int it = 0; it < 4; ++it) {
+            const int rr = it * 8 + (lane >> 2);
+            uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (lane & 3) * 16);
+            if (OP == kDgrad2Mask) {                          // ReLU'(u) = [u > 0], from the saved activation
+              const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hm[it]);
+              __nv_bfloat162* vp = reinterpret_cast<__nv_bfloat162*>(&val);
+              const __nv_bfloat16 zero = __float2bfloat16(0.f);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                if (!(__low2float(hp[q]) > 0.f)) vp[q].x = zero;
+                if (!(__high2float(hp[q]) > 0.f)) vp[q].y = zero;
+              }
+            }
+            if (offs[it] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[it] + mcol) = val;
+          }
+          cur_off = next_off;
+          cur_gate = next_gate;
+          if (OP == kDgrad2Mask) {
+#pragma unroll
+            for (int it = 0; it < 4; ++it) hm[it] = hm_next[it];
+          }
+          __syncwarp();
+        } else {
+          // weight gradient: row = weight row, 32 output columns per chunk
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + 2 * h]),
+                                                        __uint_as_float(v[q * 8 + 2 * h + 1]));
+              w[h] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            *reinterpret_cast<uint4*>(tr + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
+                make_uint4(w[0], w[1], w[2], w[3]);
+          }
+          __syncwarp();
+          const int col = t.n0 + c * 32 + (lane & 3) * 8;
+#pragma unroll
+          for (int it = 0; it < 4; ++it) {
+            const int rr = it * 8 + (lane >> 2);
+            const uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (((lane & 3) ^ ((rr >> 1) & 3)) << 4));
+            const int orow = m_warp + rr;
+            if (orow < p.Mw && col < p.Nfix)
+              *reinterpret_cast<uint4*>(p.out + ((long long)t.e * p.Mw + orow) * p.ld_out + col) = val;
+          }
+          __syncwarp();
+        }
+      }
+      if (!released) {                                        // this warp had no chunk in this tile
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
+      }
+      acc ^= 1u;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  // ---------------------------------------------------------------------------------------------- teardown
+  __syncwarp();                                               // single-lane roles rejoin their warps
+  tc_fence_before();
+  cluster_sync_all();
+  if (warp == 2) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+template <int OP>
+int launch_pair_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairParams& q, int dev, int sm_count,
+                   cudaStream_t st) {
+  if (cudaFuncSetAttribute(expert_gemm_pair_kernel<OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmemBytes) !=
+      cudaSuccess)
+    return SWITCH_MOE_CUDA_ERROR;
+  // persistent grid: as many CTA pairs as can be resident at once (at most one CTA per SM).  The occupancy query
+  // costs tens of microseconds of host time, so its answer is kept per device.
+  static int cached_grid[64] = {0};
+  int grid = (dev >= 0 && dev < 64) ? cached_grid[dev] : 0;
+  if (grid == 0) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)(sm_count & ~1), 1, 1);
+    lc.blockDim = dim3(kPThreads, 1, 1);
+    lc.dynamicSmemBytes = kPSmemBytes;
+    lc.stream = st;
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, expert_gemm_pair_kernel<OP>, &lc) != cudaSuccess ||
+        max_clusters < 1) {
+      (void)cudaGetLastError();
+      max_clusters = sm_count / 2;
+    }
+    grid = 2 * (max_clusters < sm_count / 2 ? max_clusters : sm_count / 2);
+    if (grid < 2) return SWITCH_MOE_CUDA_ERROR;
+    if (dev >= 0 && dev < 64) cached_grid[dev] = grid;
+  }
+  expert_gemm_pair_kernel<OP><<<grid, kPThreads, kPSmemBytes, st>>>(tmA, tmB, q);
+  return launch_status();
+}
+
+}  // namespace
+
+int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st) {
+  int dev = 0, sm_count = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SWITCH_MOE_CUDA_ERROR;
+  const void* xd = ws_ptr<char>(ws, p.xd);
+  const void* h = ws_ptr<char>(ws, p.h);
+  const void* dyd = ws_ptr<char>(ws, p.dyd);
+  const void* dh = ws_ptr<char>(ws, p.dh);
+
+  PairParams q{};
+  q.op = (int)op;
+  q.C = s.C; q.E = s.E;
+  q.ntile = ws_ptr<int4>(ws, p.ntile);
+  q.kept = ws_ptr<int>(ws, p.kept);
+  q.token_of_slot = ws_ptr<int>(ws, p.token_of_slot);
+  q.gate = ws_ptr<float>(ws, p.gate);
+  q.status = ws_ptr<int>(ws, p.status);
+  CUtensorMap tmA, tmB;
+  int rc = SWITCH_MOE_OK, rc2 = SWITCH_MOE_OK;
+  int K = 0;
+  switch (op) {
+    case kGemm1Relu:       // A = W_in [E][d (k)][f (m)]: m contiguous -> MN-major; B = X_d [E][C][d] K-major
+      q.token_op = 1; q.a_mn_major = 1; q.Mw = s.f; K = s.d;
+      rc = make_map(&tmA, a.W_in, s.E, s.d, s.f, 64); rc2 = make_map(&tmB, xd, s.E, s.C, s.d, 128);
+      q.out = ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = s.f; break;
+    case kGemm2Combine:    // A = W_out [E][f (k)][d (m)] MN-major; B = H [E][C][f] K-major
+      q.token_op = 1; q.a_mn_major = 1; q.Mw = s.d; K = s.f;
+      rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 64); rc2 = make_map(&tmB, h, s.E, s.C, s.f, 128);
+      q.out = static_cast<__nv_bfloat16*>(a.y); q.ld_out = s.d; break;
+    case kDgrad2Mask:      // A = W_out [E][f (m)][d (k)] K-major; B = dY_d [E][C][d] K-major
+      q.token_op = 1; q.a_mn_major = 0; q.Mw = s.f; K = s.d;
+      rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 128); rc2 = make_map(&tmB, dyd, s.E, s.C, s.d, 128);
+      q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.mask_src = ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = s.f; break;
+    case kDgrad1Scatter:   // A = W_in [E][d (m)][f (k)] K-major; B = dH [E][C][f] K-major
+      q.token_op = 1; q.a_mn_major = 0; q.Mw = s.d; K = s.f;
+      rc = make_map(&tmA, a.W_in, s.E, s.d, s.f, 128); rc2 = make_map(&tmB, dh, s.E, s.C, s.f, 128);
+      q.out = static_cast<__nv_bfloat16*>(a.dx); q.ld_out = s.d; break;
+    case kWgrad2:          // dW_out [f][d] = H^T dY_d: A = H [E][C (k)][f (m)] MN-major; B = dY_d [E][C (k)][d (n)]
+      q.token_op = 0; q.a_mn_major = 1; q.Mw = s.f; q.Nfix = s.d;
+      rc = make_map(&tmA, h, s.E, s.C, s.f, 64); rc2 = make_map(&tmB, dyd, s.E, s.C, s.d, 64);
+      q.out = static_cast<__nv_bfloat16*>(a.dW_out); q.ld_out = s.d; break;
+    case kWgrad1:          // dW_in [d][f] = X_d^T dH
+      q.token_op = 0; q.a_mn_major = 1; q.Mw = s.d; q.Nfix = s.f;
+      rc = make_map(&tmA, xd, s.E, s.C, s.d, 64); rc2 = make_map(&tmB, dh, s.E, s.C, s.f, 64);
+      q.out = static_cast<__nv_bfloat16*>(a.dW_in); q.ld_out = s.f; break;
+    default: return SWITCH_MOE_INVALID_ARGUMENT;
+  }
+  if (rc != SWITCH_MOE_OK || rc2 != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  q.n_mpairs = (q.Mw + 255) / 256;
+  q.n_ntiles_fixed = q.token_op ? 0 : (q.Nfix + 255) / 256;
+  q.k_blocks_fixed = q.token_op ? K / kBK : 0;
+  switch (op) {
+    case kGemm1Relu: return launch_pair_op<kGemm1Relu>(tmA, tmB, q, dev, sm_count, st);
+    case kGemm2Combine: return launch_pair_op<kGemm2Combine>(tmA, tmB, q, dev, sm_count, st);
+    case kDgrad2Mask: return launch_pair_op<kDgrad2Mask>(tmA, tmB, q, dev, sm_count, st);
+    case kDgrad1Scatter: return launch_pair_op<kDgrad1Scatter>(tmA, tmB, q, dev, sm_count, st);
+    case kWgrad2: return launch_pair_op<kWgrad2>(tmA, tmB, q, dev, sm_count, st);
+    default: return launch_pair_op<kWgrad1>(tmA, tmB, q, dev, sm_count, st);
+  }
+}
+
+}  // namespace swmoe

@@ -20,7 +20,7 @@ constexpr int kDwrChunkTokens = 512;    // tokens per split of the dW_r reductio
 struct Shape {
   int T, d, f, E, C;
   int dtype;        // switch_moe_dtype
-  int gemm_path;    // resolved: 0 = tcgen05, 1 = SIMT
+  int gemm_path;    // resolved: 0 = tcgen05 on CTA pairs, 1 = SIMT, 2 = single-CTA tcgen05
   float alpha;
   size_t elt;       // bytes per activation / expert-weight element
   int Epad;         // E rounded up to 32 * {1,2,4,8}
@@ -32,7 +32,7 @@ struct Shape {
 // Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
 struct Plan {
   size_t status, expert_index, gate, slot, token_of_slot, count, kept, psum, psum_partial, hist, hist_base,
-      tile_expert, tile_row0, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, total;
+      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, total;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -43,7 +43,8 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (cfg->capacity_override < 0) return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->capacity_override == 0 && !(cfg->capacity_factor > 0.f)) return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->dtype != SWITCH_MOE_BF16 && cfg->dtype != SWITCH_MOE_F32) return SWITCH_MOE_INVALID_ARGUMENT;
-  if (cfg->gemm_path != SWITCH_MOE_GEMM_DEFAULT && cfg->gemm_path != SWITCH_MOE_GEMM_SIMT)
+  if (cfg->gemm_path != SWITCH_MOE_GEMM_DEFAULT && cfg->gemm_path != SWITCH_MOE_GEMM_SIMT &&
+      cfg->gemm_path != SWITCH_MOE_GEMM_TC_1CTA)
     return SWITCH_MOE_INVALID_ARGUMENT;
   for (int i = 0; i < 5; ++i)
     if (cfg->reserved[i] != 0) return SWITCH_MOE_INVALID_ARGUMENT;
@@ -63,14 +64,14 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if ((long long)cfg->E * C > 0x7fffffffLL) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   s->C = (int)C;
   s->elt = cfg->dtype == SWITCH_MOE_BF16 ? 2 : 4;
-  s->gemm_path = (cfg->dtype == SWITCH_MOE_F32 || cfg->gemm_path == SWITCH_MOE_GEMM_SIMT) ? 1 : 0;
-  if (s->gemm_path == 0 && (cfg->d_model % 64 != 0 || cfg->d_ff % 64 != 0)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->gemm_path = (cfg->dtype == SWITCH_MOE_F32 || cfg->gemm_path == SWITCH_MOE_GEMM_SIMT) ? 1 : cfg->gemm_path;
+  if (s->gemm_path != 1 && (cfg->d_model % 64 != 0 || cfg->d_ff % 64 != 0)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   int ne = (cfg->E + 31) / 32;
   int ne_pow2 = 1;
   while (ne_pow2 < ne) ne_pow2 *= 2;
   s->Epad = 32 * ne_pow2;
   s->Epad64 = (cfg->E + 63) / 64 * 64;
-  s->router_tc = s->gemm_path == 0 ? 1 : 0;
+  s->router_tc = s->gemm_path != 1 ? 1 : 0;
   s->plan_blocks = (cfg->T + kPlanBlockTokens - 1) / kPlanBlockTokens;
   s->max_mtiles = cfg->E * ((s->C + kTileM - 1) / kTileM);
   if (s->router_tc) {
@@ -108,6 +109,7 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->hist_base = take((size_t)s.plan_blocks * E * 4);
   p->tile_expert = take(((size_t)s.max_mtiles + 4) * 4);   // [0] = number of token tiles, then one entry per tile
   p->tile_row0 = take(((size_t)s.max_mtiles + 4) * 4);
+  p->ntile = take(((size_t)s.max_mtiles + 4) * 16);        // int4 {expert, first row, rows}; [0].x = count
   p->probs = take(T * E * 4);
   p->dlogits = take(T * E * 4);
   p->xd = take(E * C * d * s.elt);
@@ -159,5 +161,6 @@ struct GemmArgs {
 };
 int launch_simt_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
 int launch_tc_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
+int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
 
 }  // namespace swmoe

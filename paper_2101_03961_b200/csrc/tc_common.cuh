@@ -16,7 +16,7 @@ constexpr int kBBytes = kBN * kBK * 2;               // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;       // 48 KB
 constexpr int kAtomBytes = 64 * kBK * 2;             // one 64(MN) x 64(K) MN-major box: 8 KB
 constexpr int kTmemCols = 512;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+constexpr long long kWaitLimitCycles = 4000000000ll;          // about 2 s of SM clock per wait
 
 // ---------------------------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -48,15 +48,17 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // Bounded wait.  Returns false (after recording `code`) if the barrier did not flip within the limit or another
-// thread of the CTA already gave up.
-static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
+// thread of the CTA already gave up.  The common case -- the phase is complete, or completes within a few polls --
+// is inline: the single-thread producer and MMA loops must stay small and call-free, because a lone warp that
+// jumps to far code pays an instruction-cache miss per iteration while the epilogue warps stream through the cache.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                   int code) {
+  const long long t0 = clock64();
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 63u) == 0) {
+    if ((spin & 255u) == 0) {
       if (*abort_flag != 0) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (clock64() - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
         if (atomicCAS(status, 0, code) == 0) {
           status[1] = (int)blockIdx.x;
@@ -67,6 +69,13 @@ static __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, vol
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int code) {
+#pragma unroll 1
+  for (int i = 0; i < 32; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {

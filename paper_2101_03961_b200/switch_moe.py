@@ -17,7 +17,7 @@ BF16, F32 = 0, 1
 STAGE_EVENTS = 13
 STAGE_NAMES = ["router_fwd", "dispatch_plan", "gather_x", "gemm1_relu", "gemm2_combine", None,
                "gather_dy", "dgrad2_mask", "wgrad2", "dgrad1_scatter", "wgrad1", "router_bwd"]
-GEMM_DEFAULT, GEMM_SIMT = 0, 1
+GEMM_DEFAULT, GEMM_SIMT, GEMM_TC_1CTA = 0, 1, 2
 
 OK = 0
 INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, CUDA_ERROR, DEVICE_TIMEOUT = -1, -2, -3, -4, -5
@@ -59,10 +59,11 @@ def load_library() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
+    path = os.environ.get("SWITCH_MOE_LIBRARY", LIB_PATH)      # override: another build of the same library
+    if not os.path.exists(path):
         raise FileNotFoundError(
-            f"{LIB_PATH} not found: build it with `python -m paper_2101_03961_b200.build` (there is no fallback path)")
-    lib = ctypes.CDLL(LIB_PATH)
+            f"{path} not found: build it with `python -m paper_2101_03961_b200.build` (there is no fallback path)")
+    lib = ctypes.CDLL(path)
     vp, cp = ctypes.c_void_p, ctypes.POINTER(SwitchMoeConfig)
     i32p, szp = ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_size_t)
     lib.switch_moe_capacity.argtypes = [cp, i32p]

@@ -185,6 +185,17 @@ def test_bf16_layer_on_tensor_cores_matches_oracle(cfg):
     _check_layer(cfg, sm.GEMM_DEFAULT, TOL_BF16, d_aux=0.5)
 
 
+@pytest.mark.parametrize("cfg", [MID, RAGGED], ids=lambda c: c.name)
+def test_bf16_layer_on_single_cta_tensor_core_path_matches_oracle(cfg):
+    _check_layer(cfg, sm.GEMM_TC_1CTA, TOL_BF16, d_aux=0.5)
+
+
+def test_tensor_core_layer_with_two_token_tiles_per_expert():
+    # capacity 600 > 256: experts' tokens are cut into several N tiles of the paired-CTA GEMM
+    cfg = si.SwitchConfig("big_capacity", 2400, 128, 320, 4, 1.0, bias_std=0.5)
+    _check_layer(cfg, sm.GEMM_DEFAULT, TOL_BF16, seed=5)
+
+
 def test_tensor_core_layer_with_empty_and_overflowing_experts():
     # a strong bias leaves some experts empty and overflows others; capacity not a multiple of any tile
     cfg = si.SwitchConfig("skewed", 3000, 128, 192, 12, 1.0, bias_std=2.0)
