@@ -48,7 +48,8 @@ struct PairParams {
   const int* token_of_slot;
   const float* gate;
   __nv_bfloat16* out;
-  const __nv_bfloat16* mask_src;
+  uint32_t* hmask;          // [E*C][d_ff/32] bit i of word w: H[row][32w + i] > 0 (written by GEMM1, read by dgrad2)
+  int hmask_ld;
   long long ld_out;
   int* status;
 };
@@ -276,9 +277,9 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       // accumulator is awaited, each later one while the previous chunk is being written.
       constexpr bool kSlotRows = (OP == kGemm1Relu || OP == kDgrad2Mask);
       int row_limit = 0;
-      long long cur_off = -1;
-      float cur_gate = 1.f;
-      uint4 hm[4];
+      long long q_off[4] = {-1, -1, -1, -1};                   // this warp's (up to) four chunks, head = next to process
+      float q_gate[4] = {1.f, 1.f, 1.f, 1.f};
+      uint32_t q_mw[4] = {0u, 0u, 0u, 0u};                      // dgrad2: ReLU mask bits of weight rows m_warp..+31 per token
       const int mcol = m_warp + (lane & 3) * 8;               // store `it` writes weight rows mcol .. mcol + 7
       auto describe = [&](int c, long long* off, float* g) {
         const int col = c * 32 + lane, slot_row = t.row0 + col;
@@ -294,19 +295,18 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
           }
         }
       };
-      auto fetch_mask = [&](long long off_lane, uint4* m4) {
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-          const long long o = __shfl_sync(0xffffffffu, off_lane, it * 8 + (lane >> 2));
-          m4[it] = (o >= 0 && mcol < p.Mw) ? *reinterpret_cast<const uint4*>(p.mask_src + o + mcol)
-                                           : make_uint4(0, 0, 0, 0);
-        }
-      };
       if (kTok) {
         const int kept_e = p.kept[t.e];
         row_limit = kSlotRows ? min(p.C, (kept_e + 15) / 16 * 16) : kept_e;
-        describe(half, &cur_off, &cur_gate);
-        if (OP == kDgrad2Mask) fetch_mask(cur_off, hm);
+        // everything the epilogue needs from global memory is requested here, before the accumulator is awaited
+#pragma unroll
+        for (int k = 0; k < 4; ++k) describe(half + 2 * k, &q_off[k], &q_gate[k]);
+        if (OP == kDgrad2Mask && m_warp < p.Mw) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (q_off[k] >= 0)
+              q_mw[k] = p.hmask[((long long)t.e * p.C + t.row0 + (half + 2 * k) * 32 + lane) * p.hmask_ld + (m_warp >> 5)];
+        }
       }
       ok = mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag, p.status, 24);
       ok = __all_sync(0xffffffffu, ok);
@@ -334,13 +334,8 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         if (kTok) {
           long long offs[4];
 #pragma unroll
-          for (int it = 0; it < 4; ++it) offs[it] = __shfl_sync(0xffffffffu, cur_off, it * 8 + (lane >> 2));
-          if (OP == kGemm2Combine) gate_s[lane] = cur_gate;
-          long long next_off;
-          float next_gate;
-          describe(c + 2, &next_off, &next_gate);             // next chunk's description, in flight behind this one
-          uint4 hm_next[4];
-          if (OP == kDgrad2Mask) fetch_mask(next_off, hm_next);
+          for (int it = 0; it < 4; ++it) offs[it] = __shfl_sync(0xffffffffu, q_off[0], it * 8 + (lane >> 2));
+          if (OP == kGemm2Combine) gate_s[lane] = q_gate[0];
           __syncwarp();
           // transpose: this lane holds weight row m_warp + lane for 32 tokens -> tr[token][lane]
 #pragma unroll
@@ -363,23 +358,32 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
           for (int it = 0; it < 4; ++it) {
             const int rr = it * 8 + (lane >> 2);
             uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (lane & 3) * 16);
-            if (OP == kDgrad2Mask) {                          // ReLU'(u) = [u > 0], from the saved activation
-              const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hm[it]);
-              __nv_bfloat162* vp = reinterpret_cast<__nv_bfloat162*>(&val);
-              const __nv_bfloat16 zero = __float2bfloat16(0.f);
+            if (OP == kDgrad2Mask) {                          // ReLU'(u) = [u > 0]: bits saved by the forward GEMM
+              const uint32_t bits = __shfl_sync(0xffffffffu, q_mw[0], rr) >> ((lane & 3) * 8);
+              uint32_t* w = reinterpret_cast<uint32_t*>(&val);
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                if (!(__low2float(hp[q]) > 0.f)) vp[q].x = zero;
-                if (!(__high2float(hp[q]) > 0.f)) vp[q].y = zero;
-              }
+              for (int q = 0; q < 4; ++q)
+                w[q] &= ((bits >> (2 * q)) & 1u ? 0x0000FFFFu : 0u) | ((bits >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u);
+            }
+            if (OP == kGemm1Relu) {                           // save [H > 0] as one bit per element for the backward pass
+              const uint32_t* w = reinterpret_cast<const uint32_t*>(&val);
+              uint32_t m8 = 0;
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                m8 |= ((w[q] & 0x00007FFFu) ? 1u << (2 * q) : 0u) | ((w[q] & 0x7FFF0000u) ? 1u << (2 * q + 1) : 0u);
+              uint32_t word = m8 << ((lane & 3) * 8);
+              word |= __shfl_xor_sync(0xffffffffu, word, 1);
+              word |= __shfl_xor_sync(0xffffffffu, word, 2);
+              if ((lane & 3) == 0 && offs[it] >= 0 && m_warp < p.Mw)
+                p.hmask[((long long)t.e * p.C + t.row0 + c * 32 + rr) * p.hmask_ld + (m_warp >> 5)] = word;
             }
             if (offs[it] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[it] + mcol) = val;
           }
-          cur_off = next_off;
-          cur_gate = next_gate;
-          if (OP == kDgrad2Mask) {
 #pragma unroll
-            for (int it = 0; it < 4; ++it) hm[it] = hm_next[it];
+          for (int k = 0; k < 3; ++k) {                       // advance the queue
+            q_off[k] = q_off[k + 1];
+            q_gate[k] = q_gate[k + 1];
+            q_mw[k] = q_mw[k + 1];
           }
           __syncwarp();
         } else {
@@ -479,6 +483,8 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   q.token_of_slot = ws_ptr<int>(ws, p.token_of_slot);
   q.gate = ws_ptr<float>(ws, p.gate);
   q.status = ws_ptr<int>(ws, p.status);
+  q.hmask = ws_ptr<uint32_t>(ws, p.hmask);
+  q.hmask_ld = s.f / 32;
   CUtensorMap tmA, tmB;
   int rc = SWITCH_MOE_OK, rc2 = SWITCH_MOE_OK;
   int K = 0;
@@ -494,7 +500,7 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
     case kDgrad2Mask:      // A = W_out [E][f (m)][d (k)] K-major; B = dY_d [E][C][d] K-major
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.f; K = s.d;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 128); rc2 = make_map(&tmB, dyd, s.E, s.C, s.d, 128);
-      q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.mask_src = ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = s.f; break;
+      q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.ld_out = s.f; break;
     case kDgrad1Scatter:   // A = W_in [E][d (m)][f (k)] K-major; B = dH [E][C][f] K-major
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.d; K = s.f;
       rc = make_map(&tmA, a.W_in, s.E, s.d, s.f, 128); rc2 = make_map(&tmB, dh, s.E, s.C, s.f, 128);

@@ -32,7 +32,7 @@ struct Shape {
 // Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
 struct Plan {
   size_t status, expert_index, gate, slot, token_of_slot, count, kept, psum, psum_partial, hist, hist_base,
-      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, total;
+      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, total;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -120,6 +120,7 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->dwr_partial = take((size_t)s.dwr_chunks * d * E * 4);
   p->wsplit = take(3 * d * (size_t)s.Epad64 * 2);
   p->dhsplit = take(3 * T * (size_t)s.Epad64 * 2);
+  p->hmask = take(E * C * ((f + 31) / 32) * 4);            // one bit per element of H: [H > 0]
   p->total = off;
 }
 
