@@ -164,12 +164,19 @@ router_fwd_kernel(const XT* __restrict__ x, const float* __restrict__ W_r, const
 }
 
 // ------------------------------------------------------------------------------------------------ backward
+template <int N> struct BfVec;                               // N consecutive bfloat16 as one store
+template <> struct BfVec<1> { using type = unsigned short; };
+template <> struct BfVec<2> { using type = unsigned int; };
+template <> struct BfVec<4> { using type = uint2; };
+template <> struct BfVec<8> { using type = uint4; };
+
 // dh[t,i] = p[t,i] (G[t,i] - sum_j p[t,j] G[t,j]),  G[t,i] = cG.count_i + [i = e_t and t kept].dgate_t
 template <int NE>
 __global__ void __launch_bounds__(256)
 router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ expert_index,
                       const int* __restrict__ slot, const int* __restrict__ count, const float* __restrict__ dgate,
-                      float cG, int T, int E, float* __restrict__ dlogits) {
+                      float cG, int T, int E, float* __restrict__ dlogits, __nv_bfloat16* __restrict__ dhsplit,
+                      int Epad64) {
   const int lane = threadIdx.x & 31;
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (t >= T) return;
@@ -188,7 +195,27 @@ router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ e
 #pragma unroll
   for (int n = 0; n < NE; ++n) {
     const int e = lane * NE + n;
-    if (e < E) dlogits[(size_t)t * E + e] = p[n] * (G[n] - s);
+    const float dh = p[n] * (G[n] - s);
+    if (e < E) dlogits[(size_t)t * E + e] = dh;
+    G[n] = e < E ? dh : 0.f;
+  }
+  if (dhsplit != nullptr && lane * NE < Epad64) {             // bf16 hi/mid/lo parts for the tensor-core products
+    __align__(16) __nv_bfloat16 hi[NE], mid[NE], lo[NE];
+#pragma unroll
+    for (int n = 0; n < NE; ++n) split3(G[n], &hi[n], &mid[n], &lo[n]);
+    const size_t plane = (size_t)T * Epad64, at = (size_t)t * Epad64 + lane * NE;    // NE consecutive experts per lane
+    using Vec = typename BfVec<NE>::type;
+    *reinterpret_cast<Vec*>(dhsplit + at) = *reinterpret_cast<const Vec*>(hi);
+    *reinterpret_cast<Vec*>(dhsplit + plane + at) = *reinterpret_cast<const Vec*>(mid);
+    *reinterpret_cast<Vec*>(dhsplit + 2 * plane + at) = *reinterpret_cast<const Vec*>(lo);
+  }
+  if (dhsplit != nullptr) {                                   // padding columns beyond the lanes' experts
+    const __nv_bfloat16 z = __float2bfloat16(0.f);
+    const size_t plane = (size_t)T * Epad64;
+    for (int e = 32 * NE + lane; e < Epad64; e += 32) {
+      const size_t at = (size_t)t * Epad64 + e;
+      dhsplit[at] = z; dhsplit[plane + at] = z; dhsplit[2 * plane + at] = z;
+    }
   }
 }
 
@@ -350,7 +377,10 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
   float* dlogits = ws_ptr<float>(ws, p.dlogits);
   router_dlogits_kernel<NE><<<(s.T + 7) / 8, 256, 0, st>>>(ws_ptr<float>(ws, p.probs),
                                                             ws_ptr<int>(ws, p.expert_index), ws_ptr<int>(ws, p.slot),
-                                                            ws_ptr<int>(ws, p.count), dgate, cG, s.T, s.E, dlogits);
+                                                            ws_ptr<int>(ws, p.count), dgate, cG, s.T, s.E, dlogits,
+                                                            (s.router_tc && sizeof(XT) == 2)
+                                                                ? ws_ptr<__nv_bfloat16>(ws, p.dhsplit) : nullptr,
+                                                            s.Epad64);
   float* partial = ws_ptr<float>(ws, p.dwr_partial);
   const size_t n = (size_t)s.d * s.E;
   if constexpr (sizeof(XT) == 2) {

@@ -30,7 +30,7 @@ struct RouterTcParams {
   int n_mtiles, n_ntiles;
   int splits, chunk_kblocks, total_kblocks;   // dwr: split of the token contraction
   int wrap;                  // k-blocks per part: d/64 (fwd), Epad64/64 (dx); dwr derives it per tile
-  const float* bias; float* probs; int* expert_index; float* gate; float* psum_partial;   // fwd
+  const float* bias; float* probs; int* expert_index; float* gate;   // fwd
   float* partial;                                                                         // dwr
   __nv_bfloat16* dx; const int* slot; int accumulate;                                     // dx
   int* status;
@@ -67,12 +67,6 @@ __device__ __forceinline__ RTile r_decode(const RouterTcParams& p, int id) {
   }
   t.k_blocks = 3 * t.wrap;
   return t;
-}
-
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-  return v;
 }
 
 template <int OP>
@@ -191,9 +185,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    float colrun[8];                                          // fwd: running column sums of p, lane i <-> column c*32+i
-#pragma unroll
-    for (int c = 0; c < 8; ++c) colrun[c] = 0.f;
     for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
       const RTile t = r_decode<OP>(p, id);
       const int r = lg * 32 + lane;
@@ -278,14 +269,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (c * 32 + i < p.E) dst[i] = pr[i];
             }
           }
-          // column sums of p over this warp's 32 tokens (Eq. 6); lane i keeps column c*32 + i
-          float mine = 0.f;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float s = warp_sum(pr[i]);
-            if (lane == i) mine = s;
-          }
-          colrun[c] += mine;
         }
         if (tok < p.T) { p.expert_index[tok] = am; p.gate[tok] = inv; }
       } else if (OP == kRDwr) {
@@ -378,34 +361,214 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
-    if (OP == kRFwd) {                                        // this warp's column sums over all tiles of this CTA
-      float* mine = reinterpret_cast<float*>(my_stage_gen);
-#pragma unroll
-      for (int c = 0; c < 8; ++c) mine[c * 32 + lane] = colrun[c];
-    }
   }
 
   tc_fence_before();
   __syncthreads();
-  if (OP == kRFwd && warp >= 2) {
-    // one partial P-sum row per CTA: the four epilogue warps' sums added in a fixed order (Eq. 6)
-    const float* st0 = reinterpret_cast<const float*>(smem_gen + kStages * kStageBytes);
-    for (int e = threadIdx.x - 64; e < p.E; e += 128)
-      p.psum_partial[(size_t)blockIdx.x * p.E + e] = ((st0[e] + st0[1024 + e]) + st0[2048 + e]) + st0[3072 + e];
-  }
   if (warp == 2) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
-// w = hi + mid + lo with hi, mid, lo bfloat16 (round to nearest); exact to about 2^-24 relative.
-__device__ __forceinline__ void split3(float w, __nv_bfloat16* hi, __nv_bfloat16* mid, __nv_bfloat16* lo) {
-  const __nv_bfloat16 h = __float2bfloat16(w);
-  const float r1 = w - __bfloat162float(h);
-  const __nv_bfloat16 m = __float2bfloat16(r1);
-  const float r2 = r1 - __bfloat162float(m);
-  *hi = h; *mid = m; *lo = __float2bfloat16(r2);
+// ------------------------------------------------------------------------------------------------------------------
+// Forward router for E <= 128: the x tile of a k-block is staged once and multiplied with all three parts of W_r;
+// the epilogue keeps a token's logits in registers (one TMEM pass, one expf per logit) and writes the probabilities
+// through a 32x32 shared-memory transpose so that global stores are 128-byte rows.
+struct RouterFwdParams {
+  int T, d, E, Epad64, n_mtiles, k_blocks, b_atoms, stages, stage_bytes;
+  const float* bias; float* probs; int* expert_index; float* gate;
+  int* status;
+};
+constexpr int kRFRingBytes = kStages * kStageBytes;            // 192 KB of operand stages
+
+template <int NCH>                                             // 32-logit chunks per token: 2 (E <= 64) or 4 (E <= 128)
+__global__ void __launch_bounds__(kRThreads, 1)
+router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const RouterFwdParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + kRFRingBytes + kROutStageBytes;
+  uint8_t* bar_gen = smem_gen + kRFRingBytes + kROutStageBytes;
+  const uint32_t full0 = bar_base, empty0 = bar_base + 8u * kStages;
+  const uint32_t tfull0 = bar_base + 16u * kStages, tempty0 = tfull0 + 16u;
+  volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kStages + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kStages + 4) + 4);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(const_cast<uint32_t*>(tmem_ptr_s))), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_s;
+  const int n_tiles = p.n_mtiles, kbs = p.k_blocks, b_atoms = p.b_atoms;
+  const uint32_t n_stages = (uint32_t)p.stages, stage_bytes = (uint32_t)p.stage_bytes;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+        const int m0 = id * kTileM;
+#pragma unroll 1
+        for (int kb = 0; kb < kbs; ++kb) {
+          ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag, p.status, 31);
+          if (!ok) break;
+          const uint32_t a_dst = smem_base + stage * stage_bytes, fb = full0 + 8u * stage;
+          mbar_arrive_expect_tx(fb, stage_bytes);
+          tma_load_3d(a_dst, &tmA, fb, kb * kBK, m0, 0);                              // x tile [128 tok][64 k]
+          uint32_t b_dst = a_dst + kABytes;
+          for (int part = 0; part < 3; ++part)
+            for (int j = 0; j < b_atoms; ++j, b_dst += kAtomBytes)                     // W part [64 k][64 e]
+              tma_load_3d(b_dst, &tmB, fb, 64 * j, kb * kBK, part);
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (*abort_flag != 0) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 4000000ll) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(p.Epad64 >> 3) << 17) |
+                             ((uint32_t)(kTileM >> 4) << 24);
+      const uint64_t a_desc0 = make_smem_desc(smem_base, 16u, 1024u);
+      const uint64_t b_desc0 = make_smem_desc(smem_base + kABytes, kAtomBytes, 1024u);
+      const uint32_t part_step = (uint32_t)(b_atoms * kAtomBytes) >> 4;
+      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+      bool ok = true;
+      for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+        ok = mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag, p.status, 32);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * (uint32_t)kBN;
+#pragma unroll 1
+        for (int kb = 0; kb < kbs; ++kb) {
+          ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 33);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t ad = a_desc0 + (uint64_t)(stage * (stage_bytes >> 4));
+          uint64_t bd = b_desc0 + (uint64_t)(stage * (stage_bytes >> 4));
+#pragma unroll
+          for (int part = 0; part < 3; ++part, bd += part_step) {
+#pragma unroll
+            for (int ks = 0; ks < kBK / kUmmaK; ++ks)
+              tc_mma_bf16(d_tmem, ad + (uint64_t)(ks * ((kUmmaK * 2) >> 4)), bd + (uint64_t)(ks * ((kUmmaK * 128) >> 4)),
+                          idesc, (kb > 0 || part > 0 || ks > 0) ? 1u : 0u);
+          }
+          tc_commit(empty0 + 8u * stage);
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull0 + 8u * acc);
+        acc ^= 1u;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    const int lg = warp & 3;
+    float* tile = reinterpret_cast<float*>(smem_gen + kRFRingBytes + (warp - 2) * 4096);   // 32 x 32 floats
+    uint32_t acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+      const int tok = id * kTileM + lg * 32 + lane;           // the token whose logits this lane holds
+      ok = mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag, p.status, 34);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * (uint32_t)kBN;
+      float h[NCH * 32];
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        uint32_t v[32];
+        tc_ld32(t_addr + c * 32, v);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) h[c * 32 + i] = __uint_as_float(v[i]);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8u * acc);         // logits are in registers: the accumulator is free
+      // Eq. 1 and top-1 (first maximum wins), all within this lane
+      float m = -INFINITY;
+      int am = 0;
+#pragma unroll
+      for (int e = 0; e < NCH * 32; ++e) {
+        if (e < p.E) {
+          h[e] += p.bias ? p.bias[e] : 0.f;
+          if (h[e] > m) { m = h[e]; am = e; }
+        }
+      }
+      float sum = 0.f;
+#pragma unroll
+      for (int e = 0; e < NCH * 32; ++e) {
+        h[e] = e < p.E ? expf(h[e] - m) : 0.f;
+        sum += h[e];
+      }
+      const float inv = 1.f / sum;
+      if (tok < p.T) { p.expert_index[tok] = am; p.gate[tok] = inv; }
+      // probabilities: 32 tokens x 32 experts at a time through shared memory, stored as 128-byte rows
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) tile[lane * 32 + (i ^ lane)] = h[c * 32 + i] * inv;
+        __syncwarp();
+        const int e = c * 32 + lane;
+#pragma unroll 8
+        for (int rr = 0; rr < 32; ++rr) {
+          const int t2 = id * kTileM + lg * 32 + rr;
+          const float pv = tile[rr * 32 + (lane ^ rr)];
+          if (t2 < p.T && e < p.E) p.probs[(size_t)t2 * p.E + e] = pv;
+        }
+        __syncwarp();
+      }
+      acc ^= 1u;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// partial[b][e] = sum of p[t][e] over the rows of block b (Eq. 6), in a fixed order: 4 row groups per column, each
+// summed sequentially, then added in order.
+__global__ void __launch_bounds__(1024)
+probs_colsum_kernel(const float* __restrict__ probs, int T, int E, int rows_per_block, float* __restrict__ partial) {
+  __shared__ float part[4][kMaxExperts];
+  const int e = threadIdx.x % kMaxExperts, g = threadIdx.x / kMaxExperts;
+  const int r0 = blockIdx.x * rows_per_block, r1 = min(T, r0 + rows_per_block);
+  const int q = (r1 - r0 + 3) / 4, a = r0 + g * q, b = min(r1, a + q);
+  if (e < E) {
+    float s = 0.f;
+    for (int t0 = a; t0 < b; t0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = t0 + j < b ? probs[(size_t)(t0 + j) * E + e] : 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) s += v[j];
+    }
+    part[g][e] = s;
+  }
+  __syncthreads();
+  if (g == 0 && e < E) partial[(size_t)blockIdx.x * E + e] = ((part[0][e] + part[1][e]) + part[2][e]) + part[3][e];
 }
 
 // wsplit[part][k][e] for e < Epad64 (zero beyond E)
@@ -418,18 +581,6 @@ __global__ void split_w_kernel(const float* __restrict__ W_r, int d, int E, int 
   __nv_bfloat16 h, m, l;
   split3(e < E ? W_r[(size_t)k * E + e] : 0.f, &h, &m, &l);
   wsplit[i] = h; wsplit[n + i] = m; wsplit[2 * n + i] = l;
-}
-
-// dhsplit[part][t][e] from the float32 logit gradients
-__global__ void split_dh_kernel(const float* __restrict__ dlogits, int T, int E, int Epad64,
-                                __nv_bfloat16* __restrict__ dhsplit) {
-  const size_t n = (size_t)T * Epad64;
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const int t = (int)(i / Epad64), e = (int)(i - (size_t)t * Epad64);
-  __nv_bfloat16 h, m, l;
-  split3(e < E ? dlogits[(size_t)t * E + e] : 0.f, &h, &m, &l);
-  dhsplit[i] = h; dhsplit[n + i] = m; dhsplit[2 * n + i] = l;
 }
 
 int sm_count_or_default() {
@@ -458,17 +609,42 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
   CUtensorMap tmA, tmB;
   if (make_map(&tmA, x, 1, s.T, s.d, kTileM) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
   if (make_map(&tmB, wsplit, 3, s.d, s.Epad64, 64) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
-  RouterTcParams q{};
-  q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.mma_n = s.Epad64;
-  q.n_mtiles = (s.T + kTileM - 1) / kTileM; q.n_ntiles = 1; q.wrap = s.d / kBK;
-  q.bias = bias; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
-  q.gate = ws_ptr<float>(ws, p.gate); q.psum_partial = ws_ptr<float>(ws, p.psum_partial);
-  q.status = ws_ptr<int>(ws, p.status);
-  if (cudaFuncSetAttribute(router_tc_kernel<kRFwd>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
-      cudaSuccess)
-    return SWITCH_MOE_CUDA_ERROR;
-  // the grid is part of the workspace layout: one partial P-sum row per CTA
-  router_tc_kernel<kRFwd><<<s.router_blocks, kRThreads, kRSmemBytes, st>>>(tmA, tmB, q);
+  const int n_mtiles = (s.T + kTileM - 1) / kTileM;
+  const int grid = n_mtiles < sm_count_or_default() ? n_mtiles : sm_count_or_default();
+  int rc;
+  if (s.Epad64 <= 128) {
+    RouterFwdParams q{};
+    q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.n_mtiles = n_mtiles; q.k_blocks = s.d / kBK;
+    q.b_atoms = s.Epad64 / 64;
+    q.stage_bytes = kABytes + 3 * q.b_atoms * kAtomBytes;
+    q.stages = kRFRingBytes / q.stage_bytes < kStages ? kRFRingBytes / q.stage_bytes : kStages;
+    q.bias = bias; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
+    q.gate = ws_ptr<float>(ws, p.gate); q.status = ws_ptr<int>(ws, p.status);
+    if (s.Epad64 == 64) {
+      if (cudaFuncSetAttribute(router_fwd_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
+          cudaSuccess)
+        return SWITCH_MOE_CUDA_ERROR;
+      router_fwd_tc_kernel<2><<<grid, kRThreads, kRSmemBytes, st>>>(tmA, tmB, q);
+    } else {
+      if (cudaFuncSetAttribute(router_fwd_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
+          cudaSuccess)
+        return SWITCH_MOE_CUDA_ERROR;
+      router_fwd_tc_kernel<4><<<grid, kRThreads, kRSmemBytes, st>>>(tmA, tmB, q);
+    }
+    rc = launch_status();
+  } else {
+    RouterTcParams q{};
+    q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.mma_n = s.Epad64;
+    q.n_mtiles = n_mtiles; q.n_ntiles = 1; q.wrap = s.d / kBK;
+    q.bias = bias; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
+    q.gate = ws_ptr<float>(ws, p.gate); q.status = ws_ptr<int>(ws, p.status);
+    rc = launch_op<kRFwd>(tmA, tmB, q, st);
+  }
+  if (rc != SWITCH_MOE_OK) return rc;
+  // Eq. 6 partial sums: one row per block of tokens, reduced in a fixed order by the dispatch plan
+  const int rows = (s.T + s.router_blocks - 1) / s.router_blocks;
+  probs_colsum_kernel<<<s.router_blocks, 1024, 0, st>>>(ws_ptr<float>(ws, p.probs), s.T, s.E, rows,
+                                                        ws_ptr<float>(ws, p.psum_partial));
   return launch_status();
 }
 
@@ -478,9 +654,6 @@ int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const flo
   __nv_bfloat16* dhsplit = ws_ptr<__nv_bfloat16>(ws, p.dhsplit);
   const size_t nw = (size_t)s.d * s.Epad64;
   split_w_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(W_r, s.d, s.E, s.Epad64, wsplit);
-  const size_t n = (size_t)s.T * s.Epad64;
-  split_dh_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ws_ptr<float>(ws, p.dlogits), s.T, s.E, s.Epad64,
-                                                                dhsplit);
   RouterTcParams q{};
   q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64;
   q.status = ws_ptr<int>(ws, p.status);

@@ -75,9 +75,9 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   s->plan_blocks = (cfg->T + kPlanBlockTokens - 1) / kPlanBlockTokens;
   s->max_mtiles = cfg->E * ((s->C + kTileM - 1) / kTileM);
   if (s->router_tc) {
-    // one partial P-sum row per CTA of the persistent router kernel; dW_r split so that tiles x splits fills the GPU
-    s->router_blocks = (cfg->T + kTileM - 1) / kTileM;
-    if (s->router_blocks > 148) s->router_blocks = 148;
+    // dW_r split so that tiles x splits fills the GPU
+    s->router_blocks = (cfg->T + 255) / 256;                 // one partial P-sum row per 256 tokens, at most 256 rows
+    if (s->router_blocks > 256) s->router_blocks = 256;
     const int m_tiles = (cfg->d_model + kTileM - 1) / kTileM;
     const int k_blocks = (cfg->T + 63) / 64;
     int splits = 144 / m_tiles;
@@ -122,6 +122,15 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->dhsplit = take(3 * T * (size_t)s.Epad64 * 2);
   p->hmask = take(E * C * ((f + 31) / 32) * 4);            // one bit per element of H: [H > 0]
   p->total = off;
+}
+
+// w = hi + mid + lo with hi, mid, lo bfloat16 (round to nearest); exact to about 2^-24 relative.
+__device__ __forceinline__ void split3(float w, __nv_bfloat16* hi, __nv_bfloat16* mid, __nv_bfloat16* lo) {
+  const __nv_bfloat16 h = __float2bfloat16(w);
+  const float r1 = w - __bfloat162float(h);
+  const __nv_bfloat16 m = __float2bfloat16(r1);
+  const float r2 = r1 - __bfloat162float(m);
+  *hi = h; *mid = m; *lo = __float2bfloat16(r2);
 }
 
 template <typename T>
