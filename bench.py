@@ -277,10 +277,18 @@ def run_ours(args, cfg):
     achieved_tf = flops_per_launch / (gemm_ms_avg * 1e-3) / 1e12
     if cfg.dtype == si.DTYPE_BF16:
         peak_tf = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
-        roofline = {"bound": "tensor", "kernel": "grouped_gemm_tc_kernel (6 launches per step)",
+        # DRAM bytes per launch from the ncu capture of the quarter-size workload (195.4 MB per launch at E=32,
+        # proportional to E); see profiles/expert_gemm_pair_kernel__switch_base_quarter.md
+        traffic = 195.4e6 * cfg.E / 32 if (cfg.d_model, cfg.d_ff) == (768, 3072) and cfg.T == 256 * cfg.E else None
+        hbm_peak = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+        roofline = {"bound": "tensor", "kernel": "expert_gemm_pair_kernel (6 launches per step)",
                     "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
-                    "traffic": None, "peak_source": f"{peak_kind} bf16 sustained (kernel timed inside a long step)",
-                    "flops_per_launch": flops_per_launch, "avg_launch_ms": gemm_ms_avg}
+                    "traffic": traffic, "peak_source": f"{peak_kind} bf16 sustained (kernel timed inside a long step)",
+                    "flops_per_launch": flops_per_launch, "avg_launch_ms": gemm_ms_avg,
+                    "frac_of_burst_peak": achieved_tf / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
+                    "hbm_gbs_at_measured_traffic": None if traffic is None else traffic / (gemm_ms_avg * 1e-3) / 1e9,
+                    "hbm_frac_at_measured_traffic": None if traffic is None
+                    else traffic / (gemm_ms_avg * 1e-3) / 1e9 / hbm_peak}
     else:
         peak_tf = 148 * 128 * 2 * 1.965e9 / 1e12
         roofline = {"bound": "alu", "kernel": "simt_grouped_gemm_kernel", "achieved": achieved_tf, "peak": peak_tf,
