@@ -30,7 +30,10 @@ constexpr int kPHalfBytes = 16384;                     // A tile (128 x 64) and 
 constexpr int kPStageBytes = 2 * kPHalfBytes;
 constexpr int kPTransBytes = 8 * 2048;                 // 8 epilogue warps x (32 x 64 B)
 constexpr int kPAuxBytes = 8 * 128;                    // 8 epilogue warps x 32 gates
-constexpr int kPSmemBytes = 1024 + kPStages * kPStageBytes + kPTransBytes + kPAuxBytes + 256;
+constexpr int kPKeptCache = kMaxExperts;                 // kept[e] for every expert
+constexpr int kPTileCache = 448;                        // first token tiles of the list ({expert, row, rows})
+constexpr int kPCacheBytes = kPKeptCache * 4 + kPTileCache * 16;
+constexpr int kPSmemBytes = 1024 + kPStages * kPStageBytes + kPTransBytes + kPAuxBytes + 256 + kPCacheBytes;
 constexpr int kPThreads = 320;
 constexpr uint32_t kPeerMask = 0xFEFFFFFFu;            // clears the CTA-rank bit of a shared::cluster address
 
@@ -58,15 +61,13 @@ struct PTile {
   int e, m0, n0, row0, n, k_blocks, last_mmas;
 };
 
-__device__ __forceinline__ int p_total_tiles(const PairParams& p) {
-  return p.token_op ? p.ntile[0].x * p.n_mpairs : p.E * p.n_mpairs * p.n_ntiles_fixed;
-}
-
-__device__ __forceinline__ PTile p_decode(const PairParams& p, int id) {
+// Tile decode reads the plan through shared-memory copies made at kernel start: a dependent global load per tile
+// would stall the single-thread producer for longer than a short tile's whole k-loop.
+__device__ __forceinline__ PTile p_decode(const PairParams& p, int id, const int* kept_s, const int4* tile_s) {
   PTile t;
   if (p.token_op) {
     const int nt = id / p.n_mpairs;
-    const int4 q = p.ntile[1 + nt];
+    const int4 q = nt < kPTileCache ? tile_s[nt] : p.ntile[1 + nt];
     t.e = q.x; t.row0 = q.y; t.n = q.z; t.n0 = 0;
     t.m0 = (id - nt * p.n_mpairs) * 256;
     t.k_blocks = p.k_blocks_fixed;
@@ -79,7 +80,7 @@ __device__ __forceinline__ PTile p_decode(const PairParams& p, int id) {
     t.m0 = mp * 256;
     t.n0 = (rem - mp * p.n_ntiles_fixed) * 256;
     t.row0 = 0; t.n = 256;
-    const int k = p.kept[t.e];
+    const int k = kept_s[t.e];
     t.k_blocks = (k + kBK - 1) / kBK;
     const int rem_rows = k - (t.k_blocks - 1) * kBK;          // rows of the last k-block that hold tokens
     t.last_mmas = (rem_rows + kUmmaK - 1) / kUmmaK;            // rows beyond them are never multiplied
@@ -149,9 +150,14 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   const uint32_t tfull0 = bar_base + 16u * kPStages, tempty0 = tfull0 + 16u;
   volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kPStages + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kPStages + 4) + 4);
+  int* kept_s = reinterpret_cast<int*>(bar_gen + 256);
+  int4* tile_s = reinterpret_cast<int4*>(bar_gen + 256 + kPKeptCache * 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();                   // 0 = leader (issues the MMAs)
+  const int n_ntiles_listed = kTok ? p.ntile[0].x : 0;
+  for (int i = threadIdx.x; i < p.E; i += kPThreads) kept_s[i] = p.kept[i];
+  for (int i = threadIdx.x; i < min(n_ntiles_listed, kPTileCache); i += kPThreads) tile_s[i] = p.ntile[1 + i];
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
@@ -170,7 +176,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_s;
-  const int n_tiles = p_total_tiles(p);
+  const int n_tiles = kTok ? n_ntiles_listed * p.n_mpairs : p.E * p.n_mpairs * p.n_ntiles_fixed;
 
   if (warp == 0) {
     // ------------------------------------------------------------------------------------------ TMA producer (both CTAs)
@@ -178,7 +184,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int id = pair; id < n_tiles && ok; id += n_pairs) {
-        const PTile t = p_decode(p, id);
+        const PTile t = p_decode(p, id, kept_s, tile_s);
         // coordinates of this CTA's boxes; only the contraction coordinate moves inside the tile
         const int a_m = t.m0 + 128 * (int)rank;
         const int b_r = kTok ? t.row0 + (int)rank * (t.n >> 1) : t.n0 + 128 * (int)rank;
@@ -226,7 +232,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
       for (int id = pair; id < n_tiles && ok; id += n_pairs) {
-        const PTile t = p_decode(p, id);
+        const PTile t = p_decode(p, id, kept_s, tile_s);
         const uint32_t idesc = idesc_base | ((uint32_t)(t.n >> 3) << 17);
         const int kbs = t.k_blocks, last_mmas = t.last_mmas;
         ok = mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag, p.status, 22);
@@ -268,7 +274,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int id = pair; id < n_tiles && ok; id += n_pairs) {
-      const PTile t = p_decode(p, id);
+      const PTile t = p_decode(p, id, kept_s, tile_s);
       const int m_warp = t.m0 + 128 * (int)rank + 32 * lg;    // first M row (weight row) this warp holds
       const int n_chunks = kTok ? (t.n + 31) >> 5 : 8;
       const bool have_acc = t.k_blocks > 0;
@@ -296,7 +302,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
       };
       if (kTok) {
-        const int kept_e = p.kept[t.e];
+        const int kept_e = kept_s[t.e];
         row_limit = kSlotRows ? min(p.C, (kept_e + 15) / 16 * 16) : kept_e;
         // everything the epilogue needs from global memory is requested here, before the accumulator is awaited
 #pragma unroll
