@@ -223,8 +223,8 @@ int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches
   Shape s;
   SWMOE_TRY(resolve_shape(cfg, &s));
   // fwd: router, 3 plan kernels, gather, 2 GEMMs; bwd: gather, 4 GEMMs, 4 router-backward kernels.
-  // The tensor-core router adds an operand-split kernel in forward and two in backward.
-  *launches_out = s.router_tc ? (8 + 11) : (7 + 9);
+  // Tensor-core router: forward = operand split, router, column sums; backward = logit gradients, two products, reduce.
+  *launches_out = s.router_tc ? (9 + 9) : (7 + 9);
   return SWITCH_MOE_OK;
 }
 

@@ -18,7 +18,10 @@ namespace swmoe {
 using namespace tc;
 namespace {
 
-constexpr int kRThreads = 192;                       // TMA warp, MMA warp, 4 epilogue warps
+constexpr int kRThreads = 192;                       // forward kernel: TMA warp, MMA warp, 4 epilogue warps
+constexpr int kRTcThreads = 320;                     // generic kernel: TMA warp, MMA warp, 8 epilogue warps
+constexpr int kRTcOutStageBytes = 8 * 32 * 128;
+constexpr int kRTcSmemBytes = 1024 + kStages * kStageBytes + kRTcOutStageBytes + 128;
 constexpr int kROutStageBytes = 4 * 32 * 128;
 constexpr int kRSmemBytes = 1024 + kStages * kStageBytes + kROutStageBytes + 128;
 
@@ -70,7 +73,7 @@ __device__ __forceinline__ RTile r_decode(const RouterTcParams& p, int id) {
 }
 
 template <int OP>
-__global__ void __launch_bounds__(kRThreads, 1)
+__global__ void __launch_bounds__(kRTcThreads, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const RouterTcParams p) {
   constexpr bool kAMn = (OP == kRDwr);                 // x^T: token rows are the contraction, d contiguous
@@ -78,8 +81,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + kStages * kStageBytes + kROutStageBytes;
-  uint8_t* bar_gen = smem_gen + kStages * kStageBytes + kROutStageBytes;
+  const uint32_t bar_base = smem_base + kStages * kStageBytes + kRTcOutStageBytes;
+  uint8_t* bar_gen = smem_gen + kStages * kStageBytes + kRTcOutStageBytes;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
@@ -90,7 +93,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -181,6 +184,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
   } else {
     const int lg = warp & 3;
+    const int half = (warp - 2) >> 2;                         // second warp of the lane group: other half of the columns
     uint8_t* my_stage_gen = smem_gen + kStages * kStageBytes + (warp - 2) * 4096;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -208,7 +212,11 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)acc * kBN;
       const bool have_acc = t.k_blocks > 0;
 
-      if (OP == kRFwd) {
+      if (OP == kRFwd && half == 1) {                         // one token per thread needs all columns: first warp only
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+      } else if (OP == kRFwd) {
         // ---- Eq. 1 softmax, top-1 (lowest index on ties) and gate for token m0 + r; all E logits are in this lane
         const int tok = t.m0 + r;
         const int nch = p.mma_n / 32;
@@ -275,7 +283,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ---- float32 partial of x^T dh for this token split: row = m0 + r (an index into d_model)
         const int row = t.m0 + r;
         const int nch = p.mma_n / 32;
-        for (int c = 0; c < nch; ++c) {
+        bool released = false;
+        for (int c = half; c < nch; c += 2) {
           uint32_t v[32];
           if (have_acc) {
             tc_ld32(t_addr + c * 32, v);
@@ -284,10 +293,11 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0u;
           }
-          if (c == nch - 1) {
+          if (c + 2 >= nch) {
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
+            released = true;
           }
           if (row < p.d) {
             float* dst = p.partial + ((size_t)t.split * p.d + row) * p.E + c * 32;
@@ -304,10 +314,15 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           }
         }
+        if (!released) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(tempty_bar(acc));
+        }
       } else {
         // ---- dx[token] = (accumulate and kept ? dx[token] : 0) + dh W_r^T, 64 columns at a time
 #pragma unroll 1
-        for (int c = 0; c < kBN / 64; ++c) {
+        for (int c = 2 * half; c < 2 * half + 2; ++c) {
           const int col = t.n0 + c * 64 + (lane & 7) * 8;
           uint4 prev[8];
 #pragma unroll
@@ -318,7 +333,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           tc_ld32(t_addr + c * 64, v);
           tc_ld32(t_addr + c * 64 + 32, v + 32);
           tc_wait_ld();
-          if (c == kBN / 64 - 1) {
+          if (c == 2 * half + 1) {
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -619,10 +634,10 @@ int sm_count_or_default() {
 
 template <int OP>
 int launch_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const RouterTcParams& q, cudaStream_t st) {
-  if (cudaFuncSetAttribute(router_tc_kernel<OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
+  if (cudaFuncSetAttribute(router_tc_kernel<OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRTcSmemBytes) !=
       cudaSuccess)
     return SWITCH_MOE_CUDA_ERROR;
-  router_tc_kernel<OP><<<sm_count_or_default(), kRThreads, kRSmemBytes, st>>>(tmA, tmB, q);
+  router_tc_kernel<OP><<<sm_count_or_default(), kRTcThreads, kRTcSmemBytes, st>>>(tmA, tmB, q);
   return launch_status();
 }
 
@@ -679,8 +694,12 @@ int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const flo
                          bool accumulate_dx, cudaStream_t st) {
   __nv_bfloat16* wsplit = ws_ptr<__nv_bfloat16>(ws, p.wsplit);
   __nv_bfloat16* dhsplit = ws_ptr<__nv_bfloat16>(ws, p.dhsplit);
-  const size_t nw = (size_t)s.d * s.Epad64;
-  split_w_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(W_r, s.d, s.E, s.Epad64, wsplit);
+  if (!accumulate_dx) {
+    // staged call: split W_r here.  The whole-layer backward (accumulate_dx) reuses the parts its forward pass left
+    // in the workspace: W_r must be unchanged between the two calls anyway.
+    const size_t nw = (size_t)s.d * s.Epad64;
+    split_w_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(W_r, s.d, s.E, s.Epad64, wsplit);
+  }
   RouterTcParams q{};
   q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64;
   q.status = ws_ptr<int>(ws, p.status);

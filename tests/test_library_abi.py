@@ -80,4 +80,4 @@ def test_status_strings(lib):
 
 def test_launch_count_is_reported(lib):
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, dtype=sm.F32)) == 16
-    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 19
+    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 18
