@@ -14,6 +14,8 @@ namespace {
 // hist[b][e] = number of tokens of block b routed to expert e
 __global__ void __launch_bounds__(kPlanBlockTokens)
 plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int* __restrict__ hist) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int h[kMaxExperts];
   for (int e = threadIdx.x; e < E; e += blockDim.x) h[e] = 0;
   __syncthreads();
@@ -32,6 +34,8 @@ plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __r
                  int* __restrict__ count, int* __restrict__ kept, float* __restrict__ psum,
                  float* __restrict__ aux_loss, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
                  int4* __restrict__ ntile) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int qsum[kScanGroups][kMaxExperts];
   __shared__ float qps[kScanGroups][kMaxExperts];
   __shared__ float term[kMaxExperts];
@@ -121,6 +125,8 @@ __global__ void __launch_bounds__(kPlanBlockTokens)
 plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__ hist_base,
                    const int* __restrict__ kept, int T, int E, int C, int* __restrict__ slot,
                    int* __restrict__ token_of_slot) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int warp_cnt[kPlanBlockTokens / 32][kMaxExperts];
   constexpr int kWarps = kPlanBlockTokens / 32;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -155,6 +161,8 @@ __global__ void __launch_bounds__(256)
 gather_x_kernel(const uint4* __restrict__ x, const int* __restrict__ token_of_slot, const int* __restrict__ kept,
                 const int* __restrict__ slot, int T, int E, int C, int row_vec, int slot_blocks,
                 uint4* __restrict__ xd, uint4* __restrict__ y) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   if ((int)blockIdx.x < slot_blocks) {
     const int s = blockIdx.x * 8 + wib;
@@ -206,6 +214,8 @@ __global__ void __launch_bounds__(256)
 gather_dy_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ y, const float* __restrict__ gate,
                  const int* __restrict__ token_of_slot, const int* __restrict__ kept, int E, int C, int row_vec,
                  uint4* __restrict__ dyd, float* __restrict__ dgate) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int s = blockIdx.x * 8 + wib;
   if (s >= E * C) return;
@@ -239,14 +249,14 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
     if (cudaMemcpyAsync(ei, expert_index, (size_t)s.T * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return SWITCH_MOE_CUDA_ERROR;
   }
-  plan_hist_kernel<<<s.plan_blocks, kPlanBlockTokens, 0, st>>>(ei, s.T, s.E, ws_ptr<int>(ws, p.hist));
-  plan_scan_kernel<<<1, kScanGroups * kMaxExperts, 0, st>>>(ws_ptr<int>(ws, p.hist), s.plan_blocks,
+  launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, s.T, s.E, ws_ptr<int>(ws, p.hist));
+  launch_k(plan_scan_kernel, dim3(1), dim3(kScanGroups * kMaxExperts), 0, st, ws_ptr<int>(ws, p.hist), s.plan_blocks,
                                               ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, s.C,
                                               s.alpha, ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count),
                                               ws_ptr<int>(ws, p.kept), ws_ptr<float>(ws, p.psum), aux_loss,
                                               ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0),
                                               ws_ptr<int4>(ws, p.ntile));
-  plan_assign_kernel<<<s.plan_blocks, kPlanBlockTokens, 0, st>>>(ei, ws_ptr<int>(ws, p.hist_base),
+  launch_k(plan_assign_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, ws_ptr<int>(ws, p.hist_base),
                                                                  ws_ptr<int>(ws, p.kept), s.T, s.E, s.C,
                                                                  ws_ptr<int>(ws, p.slot),
                                                                  ws_ptr<int>(ws, p.token_of_slot));
@@ -256,7 +266,7 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
 int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void* ws, cudaStream_t st) {
   const int row_vec = (int)((size_t)s.d * s.elt / 16);
   const int slot_blocks = (s.E * s.C + 7) / 8, tok_blocks = (s.T + 7) / 8;
-  gather_x_kernel<<<slot_blocks + tok_blocks, 256, 0, st>>>(
+  launch_k(gather_x_kernel, dim3(slot_blocks + tok_blocks), dim3(256), 0, st, 
       static_cast<const uint4*>(x), ws_ptr<int>(ws, p.token_of_slot), ws_ptr<int>(ws, p.kept),
       ws_ptr<int>(ws, p.slot), s.T, s.E, s.C, row_vec, slot_blocks, ws_ptr<uint4>(ws, p.xd), static_cast<uint4*>(y));
   return launch_status();
@@ -266,12 +276,12 @@ int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* 
   const int row_vec = (int)((size_t)s.d * s.elt / 16);
   const int blocks = (s.E * s.C + 7) / 8;
   if (s.dtype == SWITCH_MOE_BF16)
-    gather_dy_kernel<true><<<blocks, 256, 0, st>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(y),
+    launch_k(gather_dy_kernel<true>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(dy), static_cast<const uint4*>(y),
                                                    ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
                                                    ws_ptr<int>(ws, p.kept), s.E, s.C, row_vec,
                                                    ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate));
   else
-    gather_dy_kernel<false><<<blocks, 256, 0, st>>>(static_cast<const uint4*>(dy), static_cast<const uint4*>(y),
+    launch_k(gather_dy_kernel<false>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(dy), static_cast<const uint4*>(y),
                                                     ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
                                                     ws_ptr<int>(ws, p.kept), s.E, s.C, row_vec,
                                                     ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate));

@@ -138,6 +138,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   constexpr bool kTok = OP <= kDgrad1Scatter;                 // tokens on N, transposed epilogue
   constexpr bool kAMn = (OP == kGemm1Relu || OP == kGemm2Combine || OP == kWgrad2 || OP == kWgrad1);
   constexpr bool kBMn = !kTok;
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -155,9 +156,6 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();                   // 0 = leader (issues the MMAs)
-  const int n_ntiles_listed = kTok ? p.ntile[0].x : 0;
-  for (int i = threadIdx.x; i < p.E; i += kPThreads) kept_s[i] = p.kept[i];
-  for (int i = threadIdx.x; i < min(n_ntiles_listed, kPTileCache); i += kPThreads) tile_s[i] = p.ntile[1 + i];
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
@@ -172,6 +170,10 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                      smem_u32(const_cast<uint32_t*>(tmem_ptr_s))), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
+  pdl_wait();                                                 // the previous kernel's results are needed from here on
+  const int n_ntiles_listed = kTok ? p.ntile[0].x : 0;
+  for (int i = threadIdx.x; i < p.E; i += kPThreads) kept_s[i] = p.kept[i];
+  for (int i = threadIdx.x; i < min(n_ntiles_listed, kPTileCache); i += kPThreads) tile_s[i] = p.ntile[1 + i];
   tc_fence_before();
   cluster_sync_all();
   tc_fence_after();
@@ -465,7 +467,7 @@ int launch_pair_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairPar
     if (grid < 2) return SWITCH_MOE_CUDA_ERROR;
     if (dev >= 0 && dev < 64) cached_grid[dev] = grid;
   }
-  expert_gemm_pair_kernel<OP><<<grid, kPThreads, kPSmemBytes, st>>>(tmA, tmB, q);
+  launch_k(expert_gemm_pair_kernel<OP>, dim3(grid), dim3(kPThreads), kPSmemBytes, st, tmA, tmB, q);
   return launch_status();
 }
 

@@ -75,6 +75,7 @@ __device__ __forceinline__ TileCoord decode_tile(const TcParams& p, int id) {
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                        const TcParams p) {
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -107,6 +108,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_s;
+  pdl_wait();                                                 // the previous kernel's results are needed from here on
 
   const int n_tiles = total_tiles(p);
 
@@ -400,7 +402,7 @@ int launch_tc_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, 
   q.n_mtiles_fixed = q.token_m ? 0 : (q.M + kTileM - 1) / kTileM;
   q.k_blocks_fixed = q.token_m ? K / kBK : 0;
   const int grid = sm_count > 0 ? sm_count : 148;
-  grouped_gemm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tmA, tmB, q);
+  launch_k(grouped_gemm_tc_kernel, dim3(grid), dim3(kThreads), kSmemBytes, st, tmA, tmB, q);
   return launch_status();
 }
 

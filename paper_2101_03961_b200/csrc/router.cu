@@ -42,6 +42,8 @@ __global__ void __launch_bounds__(kFwdThreads)
 router_fwd_kernel(const XT* __restrict__ x, const float* __restrict__ W_r, const float* __restrict__ bias, int T, int d,
                   int E, float* __restrict__ probs, int* __restrict__ expert_index, float* __restrict__ gate,
                   float* __restrict__ psum_partial) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int EP = 32 * NE;
   constexpr int XS = kKC + 4;                               // padded row of the x tile (floats)
   constexpr int VEC = Vec16<XT>::n;
@@ -177,6 +179,8 @@ router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ e
                       const int* __restrict__ slot, const int* __restrict__ count, const float* __restrict__ dgate,
                       float cG, int T, int E, float* __restrict__ dlogits, __nv_bfloat16* __restrict__ dhsplit,
                       int Epad64) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (t >= T) return;
@@ -225,6 +229,8 @@ template <typename XT, int NE>
 __global__ void __launch_bounds__(256)
 router_dwr_partial_kernel(const XT* __restrict__ x, const float* __restrict__ dlogits, int T, int d, int E,
                           float* __restrict__ partial) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int EP = 32 * NE;
   constexpr int VEC = Vec16<XT>::n;
   __shared__ __align__(16) float xs[kDwrTok * kDwrK];
@@ -289,6 +295,8 @@ router_dwr_partial_kernel(const XT* __restrict__ x, const float* __restrict__ dl
 
 __global__ void router_dwr_reduce_kernel(const float* __restrict__ partial, int chunks, size_t n,
                                          float* __restrict__ dW_r) {
+  pdl_launch_dependents();
+  pdl_wait();
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   float s = 0.f;
@@ -301,6 +309,8 @@ template <typename XT, int NE>
 __global__ void __launch_bounds__(256)
 router_dx_kernel(const float* __restrict__ dlogits, const float* __restrict__ W_r, const int* __restrict__ slot,
                  int T, int d, int E, int accumulate, XT* __restrict__ dx) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int EP = 32 * NE;
   constexpr int ES = EP + 4;
   extern __shared__ __align__(16) float smem[];
@@ -363,7 +373,7 @@ router_dx_kernel(const float* __restrict__ dlogits, const float* __restrict__ W_
 template <typename XT, int NE>
 int router_fwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
                  cudaStream_t st) {
-  router_fwd_kernel<XT, NE><<<s.router_blocks, kFwdThreads, 0, st>>>(
+  launch_k(router_fwd_kernel<XT, NE>, dim3(s.router_blocks), dim3(kFwdThreads), 0, st, 
       static_cast<const XT*>(x), W_r, bias, s.T, s.d, s.E, ws_ptr<float>(ws, p.probs),
       ws_ptr<int>(ws, p.expert_index), ws_ptr<float>(ws, p.gate), ws_ptr<float>(ws, p.psum_partial));
   return launch_status();
@@ -375,7 +385,7 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
   // G's auxiliary-loss term: d_aux . alpha . E . f_i / T with f_i = count_i / T  (Eq. 4-6; f is a constant)
   const float cG = (float)((double)d_aux * (double)s.alpha * (double)s.E / ((double)s.T * (double)s.T));
   float* dlogits = ws_ptr<float>(ws, p.dlogits);
-  router_dlogits_kernel<NE><<<(s.T + 7) / 8, 256, 0, st>>>(ws_ptr<float>(ws, p.probs),
+  launch_k(router_dlogits_kernel<NE>, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs),
                                                             ws_ptr<int>(ws, p.expert_index), ws_ptr<int>(ws, p.slot),
                                                             ws_ptr<int>(ws, p.count), dgate, cG, s.T, s.E, dlogits,
                                                             (s.router_tc && sizeof(XT) == 2)
@@ -388,19 +398,19 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
       // tensor-core products (bf16-split operands), then the same fixed-order reduction of the token splits
       int rc = launch_router_tc_bwd(s, p, x, W_r, ws, dx, accumulate_dx, st);
       if (rc != SWITCH_MOE_OK) return rc;
-      router_dwr_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partial, s.dwr_chunks, n, dW_r);
+      launch_k(router_dwr_reduce_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, partial, s.dwr_chunks, n, dW_r);
       return launch_status();
     }
   }
   dim3 grid((s.d + kDwrK - 1) / kDwrK, s.dwr_chunks);
-  router_dwr_partial_kernel<XT, NE><<<grid, 256, 0, st>>>(static_cast<const XT*>(x), dlogits, s.T, s.d, s.E, partial);
-  router_dwr_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partial, s.dwr_chunks, n, dW_r);
+  launch_k(router_dwr_partial_kernel<XT, NE>, dim3(grid), dim3(256), 0, st, static_cast<const XT*>(x), dlogits, s.T, s.d, s.E, partial);
+  launch_k(router_dwr_reduce_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, partial, s.dwr_chunks, n, dW_r);
   constexpr int ES = 32 * NE + 4;
   const size_t smem = 2 * 64 * ES * sizeof(float);
   if (cudaFuncSetAttribute(router_dx_kernel<XT, NE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return SWITCH_MOE_CUDA_ERROR;
-  router_dx_kernel<XT, NE><<<(s.T + 63) / 64, 256, smem, st>>>(dlogits, W_r, ws_ptr<int>(ws, p.slot), s.T, s.d, s.E,
+  launch_k(router_dx_kernel<XT, NE>, dim3((s.T + 63) / 64), dim3(256), smem, st, dlogits, W_r, ws_ptr<int>(ws, p.slot), s.T, s.d, s.E,
                                                               accumulate_dx ? 1 : 0, static_cast<XT*>(dx));
   return launch_status();
 }

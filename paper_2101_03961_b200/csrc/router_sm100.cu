@@ -78,6 +78,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const RouterTcParams p) {
   constexpr bool kAMn = (OP == kRDwr);                 // x^T: token rows are the contraction, d contiguous
   constexpr bool kBMn = (OP != kRDx);                  // fwd: W [d][E]; dwr: dh [T][E]; dx: W as [d rows][E contiguous]
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -107,6 +108,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_s;
+  pdl_wait();                                                 // the previous kernel's results are needed from here on
   const int n_tiles = r_total_tiles<OP>(p);
   const int b_atoms = (p.mma_n + 63) / 64;
   const uint32_t stage_tx = kABytes + (kBMn ? (uint32_t)b_atoms * kAtomBytes : (uint32_t)kBBytes);
@@ -401,6 +403,7 @@ template <int NCH>                                             // 32-logit chunk
 __global__ void __launch_bounds__(kRThreads, 1)
 router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const RouterFwdParams p) {
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -428,6 +431,7 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_s;
+  pdl_wait();                                                 // the previous kernel's results are needed from here on
   const int n_tiles = p.n_mtiles, kbs = p.k_blocks, b_atoms = p.b_atoms;
   const uint32_t n_stages = (uint32_t)p.stages, stage_bytes = (uint32_t)p.stage_bytes;
 
@@ -594,6 +598,8 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 // summed sequentially, then added in order.
 __global__ void __launch_bounds__(1024)
 probs_colsum_kernel(const float* __restrict__ probs, int T, int E, int rows_per_block, float* __restrict__ partial) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float part[4][kMaxExperts];
   const int e = threadIdx.x % kMaxExperts, g = threadIdx.x / kMaxExperts;
   const int r0 = blockIdx.x * rows_per_block, r1 = min(T, r0 + rows_per_block);
@@ -616,6 +622,8 @@ probs_colsum_kernel(const float* __restrict__ probs, int T, int E, int rows_per_
 // wsplit[part][k][e] for e < Epad64 (zero beyond E)
 __global__ void split_w_kernel(const float* __restrict__ W_r, int d, int E, int Epad64,
                                __nv_bfloat16* __restrict__ wsplit) {
+  pdl_launch_dependents();
+  pdl_wait();
   const size_t n = (size_t)d * Epad64;
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
@@ -637,7 +645,7 @@ int launch_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const RouterTcPara
   if (cudaFuncSetAttribute(router_tc_kernel<OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRTcSmemBytes) !=
       cudaSuccess)
     return SWITCH_MOE_CUDA_ERROR;
-  router_tc_kernel<OP><<<sm_count_or_default(), kRTcThreads, kRTcSmemBytes, st>>>(tmA, tmB, q);
+  launch_k(router_tc_kernel<OP>, dim3(sm_count_or_default()), dim3(kRTcThreads), kRTcSmemBytes, st, tmA, tmB, q);
   return launch_status();
 }
 
@@ -647,7 +655,7 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
                          cudaStream_t st) {
   __nv_bfloat16* wsplit = ws_ptr<__nv_bfloat16>(ws, p.wsplit);
   const size_t n = (size_t)s.d * s.Epad64;
-  split_w_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(W_r, s.d, s.E, s.Epad64, wsplit);
+  launch_k(split_w_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, W_r, s.d, s.E, s.Epad64, wsplit);
   CUtensorMap tmA, tmB;
   if (make_map(&tmA, x, 1, s.T, s.d, kTileM) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
   if (make_map(&tmB, wsplit, 3, s.d, s.Epad64, 64) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
@@ -666,12 +674,12 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
       if (cudaFuncSetAttribute(router_fwd_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
           cudaSuccess)
         return SWITCH_MOE_CUDA_ERROR;
-      router_fwd_tc_kernel<2><<<grid, kRThreads, kRSmemBytes, st>>>(tmA, tmB, q);
+      launch_k(router_fwd_tc_kernel<2>, dim3(grid), dim3(kRThreads), kRSmemBytes, st, tmA, tmB, q);
     } else {
       if (cudaFuncSetAttribute(router_fwd_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
           cudaSuccess)
         return SWITCH_MOE_CUDA_ERROR;
-      router_fwd_tc_kernel<4><<<grid, kRThreads, kRSmemBytes, st>>>(tmA, tmB, q);
+      launch_k(router_fwd_tc_kernel<4>, dim3(grid), dim3(kRThreads), kRSmemBytes, st, tmA, tmB, q);
     }
     rc = launch_status();
   } else {
@@ -685,7 +693,7 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
   if (rc != SWITCH_MOE_OK) return rc;
   // Eq. 6 partial sums: one row per block of tokens, reduced in a fixed order by the dispatch plan
   const int rows = (s.T + s.router_blocks - 1) / s.router_blocks;
-  probs_colsum_kernel<<<s.router_blocks, 1024, 0, st>>>(ws_ptr<float>(ws, p.probs), s.T, s.E, rows,
+  launch_k(probs_colsum_kernel, dim3(s.router_blocks), dim3(1024), 0, st, ws_ptr<float>(ws, p.probs), s.T, s.E, rows,
                                                         ws_ptr<float>(ws, p.psum_partial));
   return launch_status();
 }
@@ -698,7 +706,7 @@ int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const flo
     // staged call: split W_r here.  The whole-layer backward (accumulate_dx) reuses the parts its forward pass left
     // in the workspace: W_r must be unchanged between the two calls anyway.
     const size_t nw = (size_t)s.d * s.Epad64;
-    split_w_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(W_r, s.d, s.E, s.Epad64, wsplit);
+    launch_k(split_w_kernel, dim3((unsigned)((nw + 255) / 256)), dim3(256), 0, st, W_r, s.d, s.E, s.Epad64, wsplit);
   }
   RouterTcParams q{};
   q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64;

@@ -136,7 +136,34 @@ __device__ __forceinline__ void split3(float w, __nv_bfloat16* hi, __nv_bfloat16
 template <typename T>
 inline T* ws_ptr(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
 
-inline int launch_status() { return cudaGetLastError() == cudaSuccess ? SWITCH_MOE_OK : SWITCH_MOE_CUDA_ERROR; }
+// ---- programmatic dependent launch --------------------------------------------------------------------------
+// Every kernel of the layer is launched with programmatic stream serialization: it may be scheduled (and run its
+// prologue: barrier init, tensor-memory allocation) while the previous kernel of the stream is still draining.
+// The contract inside the kernels: call pdl_launch_dependents() first, and pdl_wait() before the first access to
+// global memory; pdl_wait() returns once the previous kernel has completed and its writes are visible.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
+inline bool& launch_failed_flag() { static thread_local bool failed = false; return failed; }
+
+template <typename Kern, typename... Args>
+inline void launch_k(Kern kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kernel, args...) != cudaSuccess) launch_failed_flag() = true;
+}
+
+inline int launch_status() {
+  const bool failed = launch_failed_flag();
+  launch_failed_flag() = false;
+  return (cudaGetLastError() == cudaSuccess && !failed) ? SWITCH_MOE_OK : SWITCH_MOE_CUDA_ERROR;
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
