@@ -324,9 +324,11 @@ def run_ours(args, cfg):
     auxh = torch.zeros(1).pin_memory()
     e2e_steps = max(2, min(args.steps, 10))
 
+    up_stream, down_stream = torch.cuda.Stream(), torch.cuda.Stream()
+
     def host_step():
         sm.switch_moe_step_host(mcfg, xh, dyh, 1.0, W_r, bias, W_in, W_out, x, dy, y, dx, aux, dW_r, dW_in, dW_out,
-                                yh, dxh, auxh, ws, stream)
+                                yh, dxh, auxh, ws, stream, up_stream, down_stream)
 
     host_step()
     torch.cuda.synchronize()
@@ -337,7 +339,8 @@ def run_ours(args, cfg):
     act_bytes = cfg.T * row_bytes
     e2e = {"value": world * cfg.T / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 2 * act_bytes,
            "d2h_bytes_per_step": 2 * act_bytes + 4, "ms_per_step": e2e_s * 1e3,
-           "note": "x, dy copied from pinned host memory; y, dx, aux copied back; weights and weight gradients resident"}
+           "note": "x, dy copied from pinned host memory; y, dx, aux copied back (dy upload overlaps forward, y "
+                   "download overlaps backward); weights and weight gradients resident"}
 
     # ---- CPU baseline: the oracle on a bounded sample, this machine's host cores
     cpu = None

@@ -164,13 +164,16 @@ int switch_moe_dispatch_plan_static(const switch_moe_config* cfg, const int32_t*
 
 /* One training step with HOST activations: copies x_host and dy_host (pinned host memory, [T,d_model]) to the
  * device buffers x_dev / dy_dev, runs switch_moe_fwd and switch_moe_bwd, and copies y, dx and the auxiliary loss
- * back to y_host, dx_host, aux_host.  Weights and weight gradients stay on the device.  Synchronises the stream
- * before returning.  x_dev, dy_dev, y_dev, dx_dev, aux_dev are caller-owned device staging buffers. */
+ * back to y_host, dx_host, aux_host.  Weights and weight gradients stay on the device.  x_dev, dy_dev, y_dev, dx_dev,
+ * aux_dev are caller-owned device staging buffers.  h2d_stream / d2h_stream (cudaStream_t, may be NULL) are
+ * optional extra streams: with them dy is uploaded during the forward pass and y downloaded during the backward
+ * pass; with NULL every copy runs on `stream`.  The call creates and destroys a few CUDA events (no device
+ * memory) and synchronises all the streams it used before returning. */
 int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const void* dy_host, float d_aux,
                          const float* W_r, const float* router_bias, const void* W_in, const void* W_out,
                          void* x_dev, void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r,
                          void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host, void* workspace,
-                         size_t workspace_bytes, void* stream);
+                         size_t workspace_bytes, void* stream, void* h2d_stream, void* d2h_stream);
 
 /* Synchronises `stream`, reads the workspace's status word and returns SWITCH_MOE_DEVICE_TIMEOUT if a kernel
  * gave up on a bounded wait (its results are then invalid), SWITCH_MOE_CUDA_ERROR if the stream reports an

@@ -184,25 +184,54 @@ int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const
                          const float* W_r, const float* router_bias, const void* W_in, const void* W_out,
                          void* x_dev, void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r,
                          void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host, void* workspace,
-                         size_t workspace_bytes, void* stream) {
+                         size_t workspace_bytes, void* stream, void* h2d_stream, void* d2h_stream) {
   Ctx c;
   SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
   if (!x_host || !dy_host || !x_dev || !dy_dev || !y_dev || !dx_dev || !aux_dev || !y_host || !dx_host || !aux_host)
     return SWITCH_MOE_INVALID_ARGUMENT;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // Optional copy streams let dy travel to the device during the forward pass and y travel back during the
+  // backward pass.  Without them (NULL) every copy is ordered on `stream`.
+  cudaStream_t up = h2d_stream ? static_cast<cudaStream_t>(h2d_stream) : st;
+  cudaStream_t down = d2h_stream ? static_cast<cudaStream_t>(d2h_stream) : st;
   const size_t act = (size_t)c.s.T * c.s.d * c.s.elt;
-  if (cudaMemcpyAsync(x_dev, x_host, act, cudaMemcpyHostToDevice, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
-  if (cudaMemcpyAsync(dy_dev, dy_host, act, cudaMemcpyHostToDevice, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
-  SWMOE_TRY(switch_moe_fwd(cfg, x_dev, W_r, router_bias, W_in, W_out, y_dev, aux_dev, workspace, workspace_bytes,
-                           stream));
-  if (cudaMemcpyAsync(y_host, y_dev, act, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
-  if (cudaMemcpyAsync(aux_host, aux_dev, sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return SWITCH_MOE_CUDA_ERROR;
-  SWMOE_TRY(switch_moe_bwd(cfg, dy_dev, d_aux, x_dev, W_r, W_in, W_out, y_dev, workspace, workspace_bytes, dx_dev, dW_r,
-                           dW_in, dW_out, stream));
-  if (cudaMemcpyAsync(dx_host, dx_dev, act, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
-  return SWITCH_MOE_OK;
+  cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // start, x up, dy up, fwd done, bwd done
+  int rc = SWITCH_MOE_OK;
+  auto ck = [&](cudaError_t e) { if (e != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR; };
+  for (int i = 0; i < 5; ++i) ck(cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming));
+  if (rc == SWITCH_MOE_OK) {
+    ck(cudaEventRecord(ev[0], st));                            // copies start after earlier work on `stream`
+    if (up != st) ck(cudaStreamWaitEvent(up, ev[0], 0));
+    ck(cudaMemcpyAsync(x_dev, x_host, act, cudaMemcpyHostToDevice, up));
+    ck(cudaEventRecord(ev[1], up));
+    ck(cudaMemcpyAsync(dy_dev, dy_host, act, cudaMemcpyHostToDevice, up));
+    ck(cudaEventRecord(ev[2], up));
+    if (up != st) ck(cudaStreamWaitEvent(st, ev[1], 0));
+  }
+  if (rc == SWITCH_MOE_OK)
+    rc = switch_moe_fwd(cfg, x_dev, W_r, router_bias, W_in, W_out, y_dev, aux_dev, workspace, workspace_bytes, stream);
+  if (rc == SWITCH_MOE_OK) {
+    ck(cudaEventRecord(ev[3], st));
+    if (down != st) ck(cudaStreamWaitEvent(down, ev[3], 0));
+    ck(cudaMemcpyAsync(y_host, y_dev, act, cudaMemcpyDeviceToHost, down));
+    ck(cudaMemcpyAsync(aux_host, aux_dev, sizeof(float), cudaMemcpyDeviceToHost, down));
+    if (up != st) ck(cudaStreamWaitEvent(st, ev[2], 0));
+  }
+  if (rc == SWITCH_MOE_OK)
+    rc = switch_moe_bwd(cfg, dy_dev, d_aux, x_dev, W_r, W_in, W_out, y_dev, workspace, workspace_bytes, dx_dev, dW_r,
+                        dW_in, dW_out, stream);
+  if (rc == SWITCH_MOE_OK) {
+    ck(cudaEventRecord(ev[4], st));
+    if (down != st) ck(cudaStreamWaitEvent(down, ev[4], 0));
+    ck(cudaMemcpyAsync(dx_host, dx_dev, act, cudaMemcpyDeviceToHost, down));
+  }
+  // always drain what was enqueued, also after an error, before the events go away
+  if (cudaStreamSynchronize(up) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
+  if (cudaStreamSynchronize(st) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
+  if (cudaStreamSynchronize(down) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
+  for (int i = 0; i < 5; ++i)
+    if (ev[i] != nullptr) cudaEventDestroy(ev[i]);
+  return rc;
 }
 
 int switch_moe_check_device_status(const switch_moe_config* cfg, void* workspace, int32_t* info_out, void* stream) {

@@ -75,7 +75,7 @@ def load_library() -> ctypes.CDLL:
     lib.switch_moe_dispatch_plan.argtypes = [cp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.switch_moe_dispatch_plan_static.argtypes = [cp, vp, vp, vp, vp, vp, vp]
     lib.switch_moe_router_bwd.argtypes = [cp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp, vp, vp]
-    lib.switch_moe_step_host.argtypes = [cp, vp, vp, ctypes.c_float] + [vp] * 15 + [vp, ctypes.c_size_t, vp]
+    lib.switch_moe_step_host.argtypes = [cp, vp, vp, ctypes.c_float] + [vp] * 15 + [vp, ctypes.c_size_t, vp, vp, vp]
     lib.switch_moe_check_device_status.argtypes = [cp, vp, i32p, vp]
     lib.switch_moe_launches_per_step.argtypes = [cp, i32p]
     lib.switch_moe_status_string.argtypes = [ctypes.c_int]
@@ -210,12 +210,14 @@ def switch_moe_router_bwd(cfg, x, W_r, dgate, d_aux, workspace, dx_router, dW_r,
 
 
 def switch_moe_step_host(cfg, x_host, dy_host, d_aux, W_r, router_bias, W_in, W_out, x_dev, dy_dev, y_dev, dx_dev,
-                         aux_dev, dW_r, dW_in, dW_out, y_host, dx_host, aux_host, workspace, stream=None) -> None:
+                         aux_dev, dW_r, dW_in, dW_out, y_host, dx_host, aux_host, workspace, stream=None,
+                         h2d_stream=None, d2h_stream=None) -> None:
     _check(load_library().switch_moe_step_host(
         ctypes.byref(cfg), _ptr(x_host), _ptr(dy_host), float(d_aux), _ptr(W_r), _ptr(router_bias), _ptr(W_in),
         _ptr(W_out), _ptr(x_dev), _ptr(dy_dev), _ptr(y_dev), _ptr(dx_dev), _ptr(aux_dev), _ptr(dW_r), _ptr(dW_in),
         _ptr(dW_out), _ptr(y_host), _ptr(dx_host), _ptr(aux_host), _ptr(workspace), workspace.numel(),
-        _stream(stream)), "switch_moe_step_host")
+        _stream(stream), None if h2d_stream is None else _stream(h2d_stream),
+        None if d2h_stream is None else _stream(d2h_stream)), "switch_moe_step_host")
 
 
 def switch_moe_check_device_status(cfg, workspace, stream=None) -> list:

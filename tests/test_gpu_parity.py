@@ -261,3 +261,27 @@ def test_undersized_workspace_and_misaligned_pointers_are_rejected():
     rc = lib.switch_moe_router_fwd(ctypes.byref(cfg), x.data_ptr(), W_r.data_ptr(), None, ws.data_ptr() + 16,
                                    ws.numel(), None)
     assert rc == sm.UNSUPPORTED_SHAPE
+
+
+# ---------------------------------------------------------------------------------------------- host-buffer step
+@pytest.mark.parametrize("extra_streams", [False, True], ids=["one_stream", "copy_streams"])
+def test_step_with_host_activations_equals_device_calls(extra_streams):
+    cfg = MID
+    data = si.gen_layer(cfg, seed=6)
+    g = GpuLayer(cfg, data)
+    g.fwd()
+    g.bwd()
+    y_ref, dx_ref, aux_ref = g.y.clone(), g.dx.clone(), float(g.aux.item())
+    dW_in_ref = g.dW_in.clone()
+    xh, dyh = g.x.cpu().pin_memory(), g.dy.cpu().pin_memory()
+    yh, dxh = torch.empty_like(xh).pin_memory(), torch.empty_like(xh).pin_memory()
+    auxh = torch.zeros(1).pin_memory()
+    x_dev, dy_dev = torch.zeros_like(g.x), torch.zeros_like(g.x)
+    g.y.fill_(float("nan")); g.dx.fill_(float("nan")); g.dW_in.fill_(float("nan"))
+    up, down = (torch.cuda.Stream(), torch.cuda.Stream()) if extra_streams else (None, None)
+    for _ in range(2):                                       # twice: the call must leave nothing pending behind it
+        sm.switch_moe_step_host(g.cfg, xh, dyh, 1.0, g.W_r, g.bias, g.W_in, g.W_out, x_dev, dy_dev, g.y, g.dx, g.aux,
+                                g.dW_r, g.dW_in, g.dW_out, yh, dxh, auxh, g.ws, None, up, down)
+    assert torch.equal(yh.cuda(), y_ref) and torch.equal(dxh.cuda(), dx_ref)
+    assert float(auxh.item()) == aux_ref
+    assert torch.equal(g.dW_in, dW_in_ref)
