@@ -173,18 +173,16 @@ class ClockSampler:
 # ----------------------------------------------------------------------------------------------- GPU arm
 def run_ours(args, cfg):
     import torch
-    import torch.distributed as dist
     from paper_2101_03961_b200 import build as sbuild
     from paper_2101_03961_b200 import switch_moe as sm
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2101_03961_b200.replicas import Replicas
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the layer has no CPU fallback")
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    reps = Replicas("nccl", torch.device("cuda", local_rank))
+    rank, world = reps.rank, reps.world
     sbuild.build()
     sm.load_library()
 
@@ -221,8 +219,7 @@ def run_ours(args, cfg):
         sm.switch_moe_bwd(mcfg, dy, 1.0, x, W_r, W_in, W_out, y, ws, dx, dW_r, dW_in, dW_out, stream)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        reps.barrier()
         torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
@@ -260,12 +257,9 @@ def run_ours(args, cfg):
     sm.switch_moe_check_device_status(mcfg, ws, stream)
     elapsed_ms = t_start.elapsed_time(t_end)
     staged_ms_per_step = ts_start.elapsed_time(ts_end) / args.steps
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = reps.max_over_ranks(elapsed_ms)
     ms_per_step = elapsed_ms / args.steps
-    value = world * cfg.T / (ms_per_step * 1e-3)
+    value = reps.tokens_per_second(cfg.T, ms_per_step)
 
     stage_ms = {}
     for i, name in enumerate(sm.STAGE_NAMES):
@@ -273,10 +267,8 @@ def run_ours(args, cfg):
             continue
         stage_ms[name] = statistics.mean(events[k][i].elapsed_time(events[k][i + 1]) for k in range(args.steps))
 
-    if rank != 0:
-        if world > 1:
-            dist.barrier()
-            dist.destroy_process_group()
+    if not reps.is_reporting_rank:
+        reps.close()
         return
 
     kept = int(sm.switch_moe_workspace_view(mcfg, ws, sm.WS_KEPT).sum().item())
@@ -366,9 +358,7 @@ def run_ours(args, cfg):
         "aux_loss": float(aux.item()),
     }
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    reps.close()
 
 
 def main():
