@@ -21,7 +21,8 @@ Readings taken where the paper is silent or its listing is garbled (each is chec
     would keep C - 1, whereas Fig. 3 gives every expert a batch of exactly the capacity of Eq. 3);
   * f_i counts the argmax before the capacity cut (Eq. 5 is the argmax indicator);
   * argmax ties go to the lowest expert index;
-  * a dropped token's output row is 0 (its gate is masked to 0; the residual add belongs to the caller);
+  * a dropped token's output row is 0 (its gate is masked to 0); with `residual` the layer adds its own
+    input, so a dropped token's row is exactly its input row;
   * the gate multiplies in full precision (no bfloat16 rounding of the combine weights);
   * one call is one routing group; the row order of x is the token order;
   * ReLU'(0) = 0;
@@ -101,7 +102,7 @@ def dispatch_plan(e, E: int, C: int):
 
 
 def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None,
-                   capacity: int | None = None, expert_index=None, experts=None):
+                   capacity: int | None = None, expert_index=None, experts=None, residual: bool = False):
     """Forward of the Switch FFN layer for one routing group.
 
     x [T, d]; W_r [d, E]; W_in [E, d, f]; W_out [E, f, d].  `capacity` overrides Eq. 3 when given.
@@ -109,6 +110,9 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     device router); the gate is then p[t, expert_index[t]].  `experts`, when given, restricts the
     expert FFN work to that subset (rows of y for other experts' tokens stay 0): the router, plan and
     loss are always computed for every token.  W_in / W_out may be any object indexable by expert.
+    `residual` adds the layer's input to its output, y_t = x_t + g_t . E_{e_t}(x_t): the residual connection
+    around the Switch FFN layer (Fig. 2), through which a dropped token's representation reaches the next
+    layer unchanged (Section 2.2).  "layer_y" always holds the output without it.
     Returns a dict with every intermediate the staged comparisons need.
     """
     x64 = np.asarray(x, dtype=F64)
@@ -140,8 +144,8 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
         u[i] = u_i
         o[tok] = o_i
         y[tok] = g[tok, None] * o_i                              # Eq. 2 with one selected expert
-    out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "y": y, "o": o, "u": u,
-           "T": T, "E": E, "alpha": alpha}
+    out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "layer_y": y,
+           "y": x64 + y if residual else y, "o": o, "u": u, "T": T, "E": E, "alpha": alpha, "residual": bool(residual)}
     out.update(plan)
     return out
 
@@ -193,6 +197,8 @@ def switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=No
     db = dh.sum(axis=0)
     dx_router = dh @ W_r64.T
     dx = dx + dx_router
+    if fwd.get("residual", False):
+        dx = dx + dy64                                   # y = x + layer(x): the skip path carries dy to x unchanged
     return {"dx": dx, "dW_r": dW_r, "db": db, "dW_in": dW_in, "dW_out": dW_out, "dgate": dgate, "dh": dh,
             "dx_router": dx_router, "G": G}
 

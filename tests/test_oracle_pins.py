@@ -345,3 +345,49 @@ def test_router_backward_helper_agrees_with_full_backward():
                                         0.02, d_aux=0.5)
     np.testing.assert_allclose(rb["dW_r"], bwd["dW_r"], rtol=1e-13, atol=1e-15)
     np.testing.assert_allclose(rb["dx_router"], bwd["dx_router"], rtol=1e-13, atol=1e-15)
+
+
+# ------------------------------------------------------------------ residual connection around the layer (Fig. 2, Section 2.2)
+def test_residual_output_is_input_plus_layer_and_dropped_rows_pass_through():
+    T, d, f, E = 40, 6, 8, 4
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=21, scale=2.0)
+    plain = so.switch_forward(x, W_r, W_in, W_out, 0.5, 0.01)
+    res = so.switch_forward(x, W_r, W_in, W_out, 0.5, 0.01, residual=True)
+    dropped = ~res["keep"]
+    assert dropped.sum() >= 3
+    assert np.array_equal(res["y"][dropped], x[dropped])                    # a dropped token leaves the layer unchanged
+    assert np.array_equal(res["layer_y"], plain["y"])
+    np.testing.assert_allclose(res["y"] - x, plain["y"], rtol=0, atol=1e-15)
+    assert res["aux"] == plain["aux"] and res["slot"].tolist() == plain["slot"].tolist()
+
+
+def test_residual_backward_adds_dy_and_matches_finite_differences():
+    T, d, f, E, cf, alpha, d_aux = 14, 5, 9, 3, 0.75, 0.03, 0.9
+    rng = np.random.default_rng(22)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=22, scale=2.0)
+    R = rng.standard_normal((T, d))
+    fwd = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, residual=True)
+    srt = np.sort(fwd["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-3 and (~fwd["keep"]).any()
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    plain_fwd = so.switch_forward(x, W_r, W_in, W_out, cf, alpha)
+    plain = so.switch_backward(plain_fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    np.testing.assert_allclose(bwd["dx"], plain["dx"] + R, rtol=0, atol=1e-14)   # the skip path carries dy unchanged
+    for k in ("dW_r", "dgate"):
+        assert np.array_equal(bwd[k], plain[k])                              # no other gradient sees the skip path
+    e_frozen, eps = fwd["e"], 1e-6
+
+    def loss():
+        out = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, expert_index=e_frozen, residual=True)
+        return float(np.sum(out["y"] * R) + d_aux * out["aux"])
+
+    num = np.zeros_like(x)
+    for idx in np.ndindex(x.shape):
+        old = x[idx]
+        x[idx] = old + eps
+        lp = loss()
+        x[idx] = old - eps
+        lm = loss()
+        x[idx] = old
+        num[idx] = (lp - lm) / (2 * eps)
+    assert np.linalg.norm(num - bwd["dx"]) / np.linalg.norm(bwd["dx"]) < 1e-7
