@@ -207,7 +207,8 @@ def run_ours(args, cfg):
     b_np = si.gen_router_bias(cfg, args.seed)
     bias = None if b_np is None else torch.from_numpy(b_np).cuda()
 
-    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype)
+    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype,
+                          residual=args.residual)
     ws = sm.allocate_workspace(mcfg)
     y, dx = torch.empty_like(x), torch.empty_like(x)
     dW_in, dW_out, dW_r = torch.empty_like(W_in), torch.empty_like(W_out), torch.empty_like(W_r)
@@ -350,6 +351,7 @@ def run_ours(args, cfg):
         "config": {"workload": cfg.name, "T": cfg.T, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "E": cfg.E,
                    "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha, "capacity": sm.switch_moe_capacity(mcfg),
                    "kept_tokens": kept, "parallelism": "replicas" if world > 1 else "single",
+                   "skip_path_inside_layer": bool(args.residual),
                    "l2": "inputs larger than L2 (weights 2 x %.0f MB per pass), no flush" %
                          (cfg.E * cfg.d_model * cfg.d_ff * elt / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": sm.switch_moe_launches_per_step(mcfg) * args.steps,
@@ -372,6 +374,9 @@ def main():
     ap.add_argument("--oracle-experts", type=int, default=None,
                     help="experts whose FFN the CPU oracle runs in its bounded sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--residual", action="store_true",
+                    help="time the variant that adds the layer's input to its output inside the combine step "
+                         "(y = x + layer(x), dx = dy + ...); not the headline configuration")
     args = ap.parse_args()
     cfg = si.CONFIGS[args.workload]
     if args.oracle_experts is None:

@@ -43,6 +43,14 @@ enum switch_moe_gemm_path {
   SWITCH_MOE_GEMM_TC_1CTA = 2  /* validation only: single-CTA tcgen05 grouped GEMM with 128-token tiles (bf16) */
 };
 
+/* SWITCH_MOE_FLAG_RESIDUAL: the layer adds its own input to its output, y_t = x_t + g_t E_{e_t}(x_t): the residual
+   connection around the Switch FFN layer (Fig. 2), fused into the combine step.  A dropped token's row is then its
+   input row (Section 2.2: it reaches the next layer through the residual connection).  The backward pass adds dy to
+   dx accordingly.  bf16: the expert term is rounded to bf16 before the addition and the sum is rounded again.  The
+   forward pass also keeps the output without the skip path in the workspace (SWITCH_MOE_WS_LAYER_Y): the gate's
+   gradient <dy_t, E(x_t)> cannot be recovered from a bf16 y_t - x_t.  Not available on SWITCH_MOE_GEMM_TC_1CTA. */
+enum switch_moe_flags { SWITCH_MOE_FLAG_RESIDUAL = 1 };
+
 typedef enum switch_moe_status {
   SWITCH_MOE_OK = 0,
   SWITCH_MOE_INVALID_ARGUMENT = -1,    /* null pointer, non-positive size, capacity 0 */
@@ -62,7 +70,8 @@ typedef struct switch_moe_config {
   int32_t capacity_override; /* 0: use Eq. 3; > 0: use this expert capacity instead */
   int32_t dtype;             /* switch_moe_dtype */
   int32_t gemm_path;         /* switch_moe_gemm_path */
-  int32_t reserved[5];       /* must be 0 */
+  int32_t flags;             /* bitwise OR of switch_moe_flags */
+  int32_t reserved[4];       /* must be 0 */
   void* const* stage_events; /* HOST array of SWITCH_MOE_STAGE_EVENTS cudaEvent_t handles, or NULL (default).
                                 When set, fwd records event i on the stream before its stage i (0 router, 1 dispatch
                                 plan, 2 gather, 3 GEMM1+ReLU, 4 GEMM2+combine) and event 5 after the last one; bwd
@@ -89,7 +98,9 @@ enum switch_moe_ws_region {
   SWITCH_MOE_WS_DH = 12,            /* [E,C,d_ff]    gradient of the pre-activation per slot (backward) */
   SWITCH_MOE_WS_DGATE = 13,         /* float[T]   <dy_t, o_t> for kept tokens (backward) */
   SWITCH_MOE_WS_DLOGITS = 14,       /* float[T,E] gradient of the router logits (backward) */
-  SWITCH_MOE_WS_REGION_COUNT = 15
+  SWITCH_MOE_WS_LAYER_Y = 15,       /* [T,d_model] g_t E(x_t) without the skip path (only with SWITCH_MOE_FLAG_RESIDUAL;
+                                       rows of dropped tokens are not written) */
+  SWITCH_MOE_WS_REGION_COUNT = 16
 };
 
 /* Eq. 3.  HOST call.  *C_out = capacity_override if > 0, else floor(T * capacity_factor / E) capped at T.

@@ -89,6 +89,9 @@ int switch_moe_workspace_view(const switch_moe_config* cfg, void* workspace, int
     case SWITCH_MOE_WS_DH: off = p.dh; bytes = E * C * s.f * s.elt; break;
     case SWITCH_MOE_WS_DGATE: off = p.dgate; bytes = T * 4; break;
     case SWITCH_MOE_WS_DLOGITS: off = p.dlogits; bytes = T * E * 4; break;
+    case SWITCH_MOE_WS_LAYER_Y:
+      if (!s.residual) return SWITCH_MOE_INVALID_ARGUMENT;
+      off = p.layer_y; bytes = T * s.d * s.elt; break;
     default: return SWITCH_MOE_INVALID_ARGUMENT;
   }
   *ptr_out = static_cast<char*>(workspace) + off;
@@ -129,7 +132,7 @@ int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r
   SWMOE_TRY(mark(cfg, 2, st));
   SWMOE_TRY(launch_gather_x(c.s, c.p, x, y, workspace, st));
   GemmArgs a{};
-  a.W_in = W_in; a.W_out = W_out; a.y = y;
+  a.W_in = W_in; a.W_out = W_out; a.y = y; a.x = x;
   SWMOE_TRY(mark(cfg, 3, st));
   SWMOE_TRY(run_gemm(kGemm1Relu, c, a, workspace, st));
   SWMOE_TRY(mark(cfg, 4, st));
@@ -150,9 +153,9 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   GemmArgs a{};
-  a.W_in = W_in; a.W_out = W_out; a.dx = dx; a.dW_in = dW_in; a.dW_out = dW_out;
+  a.W_in = W_in; a.W_out = W_out; a.dx = dx; a.dW_in = dW_in; a.dW_out = dW_out; a.dy = dy;
   SWMOE_TRY(mark(cfg, 6, st));
-  SWMOE_TRY(launch_gather_dy(c.s, c.p, dy, y, workspace, st));
+  SWMOE_TRY(launch_gather_dy(c.s, c.p, dy, y, dx, workspace, st));
   SWMOE_TRY(mark(cfg, 7, st));
   SWMOE_TRY(run_gemm(kDgrad2Mask, c, a, workspace, st));
   SWMOE_TRY(mark(cfg, 8, st));

@@ -156,10 +156,11 @@ plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__
 // Forward gather.  Part 1 (blockIdx.x < slot_blocks): one warp per slot row; kept slots copy the token's row
 // with 128-bit loads and stores, slots in [kept_i, roundup(kept_i, kTileM)) are zero-filled so that tensor-core
 // tiles never read stale rows.  Part 2: one warp per token; dropped tokens get a zero output row (their
-// representation reaches the next layer only through the caller's residual connection, Section 2.2).
+// representation reaches the next layer only through the residual connection, Section 2.2), or, when the layer
+// itself adds the skip path (`residual`), their input row.
 __global__ void __launch_bounds__(256)
 gather_x_kernel(const uint4* __restrict__ x, const int* __restrict__ token_of_slot, const int* __restrict__ kept,
-                const int* __restrict__ slot, int T, int E, int C, int row_vec, int slot_blocks,
+                const int* __restrict__ slot, int T, int E, int C, int row_vec, int slot_blocks, int residual,
                 uint4* __restrict__ xd, uint4* __restrict__ y) {
   pdl_launch_dependents();
   pdl_wait();
@@ -179,7 +180,8 @@ gather_x_kernel(const uint4* __restrict__ x, const int* __restrict__ token_of_sl
     const int t = (blockIdx.x - slot_blocks) * 8 + wib;
     if (t >= T || slot[t] >= 0) return;
     uint4* dst = y + (size_t)t * row_vec;
-    for (int v = lane; v < row_vec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+    const uint4* src = x + (size_t)t * row_vec;
+    for (int v = lane; v < row_vec; v += 32) dst[v] = residual ? src[v] : make_uint4(0, 0, 0, 0);
   }
 }
 
@@ -209,14 +211,25 @@ __device__ __forceinline__ float dot_scale4(const uint4& a, const uint4& b, floa
 
 // Backward gather: dY_d[slot] = g . dy[token] (derivative of Eq. 2 w.r.t. the expert output) and
 // dgate[token] = <dy, o> with o = y / g (derivative w.r.t. the gate).  Tail rows are zero-filled as in forward.
+// With the skip path inside the layer, blocks past `slot_blocks` (one warp per token) start the dropped tokens'
+// dx rows at dy: the router's gradient is added to them later, and no expert ever writes them.
 template <bool kBf16>
 __global__ void __launch_bounds__(256)
 gather_dy_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ y, const float* __restrict__ gate,
-                 const int* __restrict__ token_of_slot, const int* __restrict__ kept, int E, int C, int row_vec,
-                 uint4* __restrict__ dyd, float* __restrict__ dgate) {
+                 const int* __restrict__ token_of_slot, const int* __restrict__ kept, const int* __restrict__ slot,
+                 int T, int E, int C, int row_vec, int slot_blocks, uint4* __restrict__ dyd,
+                 float* __restrict__ dgate, uint4* __restrict__ dx) {
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  if ((int)blockIdx.x >= slot_blocks) {
+    const int t = (blockIdx.x - slot_blocks) * 8 + wib;
+    if (t >= T || slot[t] >= 0) return;
+    const uint4* src = dy + (size_t)t * row_vec;
+    uint4* dst = dx + (size_t)t * row_vec;
+    for (int v = lane; v < row_vec; v += 32) dst[v] = src[v];
+    return;
+  }
   const int s = blockIdx.x * 8 + wib;
   if (s >= E * C) return;
   const int ex = s / C, pos = s - ex * C, k = kept[ex];
@@ -268,23 +281,27 @@ int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void*
   const int slot_blocks = (s.E * s.C + 7) / 8, tok_blocks = (s.T + 7) / 8;
   launch_k(gather_x_kernel, dim3(slot_blocks + tok_blocks), dim3(256), 0, st, 
       static_cast<const uint4*>(x), ws_ptr<int>(ws, p.token_of_slot), ws_ptr<int>(ws, p.kept),
-      ws_ptr<int>(ws, p.slot), s.T, s.E, s.C, row_vec, slot_blocks, ws_ptr<uint4>(ws, p.xd), static_cast<uint4*>(y));
+      ws_ptr<int>(ws, p.slot), s.T, s.E, s.C, row_vec, slot_blocks, s.residual, ws_ptr<uint4>(ws, p.xd),
+      static_cast<uint4*>(y));
   return launch_status();
 }
 
-int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* ws, cudaStream_t st) {
+int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* dx, void* ws, cudaStream_t st) {
   const int row_vec = (int)((size_t)s.d * s.elt / 16);
-  const int blocks = (s.E * s.C + 7) / 8;
+  const int slot_blocks = (s.E * s.C + 7) / 8;
+  const int blocks = slot_blocks + (s.residual ? (s.T + 7) / 8 : 0);
+  // with the skip path inside the layer, y holds x + g . E(x): the gate's gradient needs the copy without x
+  const void* ysrc = s.residual ? ws_ptr<char>(ws, p.layer_y) : y;
   if (s.dtype == SWITCH_MOE_BF16)
-    launch_k(gather_dy_kernel<true>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(dy), static_cast<const uint4*>(y),
-                                                   ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
-                                                   ws_ptr<int>(ws, p.kept), s.E, s.C, row_vec,
-                                                   ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate));
+    launch_k(gather_dy_kernel<true>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(dy),
+             static_cast<const uint4*>(ysrc), ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
+             ws_ptr<int>(ws, p.kept), ws_ptr<int>(ws, p.slot), s.T, s.E, s.C, row_vec, slot_blocks,
+             ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate), static_cast<uint4*>(dx));
   else
-    launch_k(gather_dy_kernel<false>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(dy), static_cast<const uint4*>(y),
-                                                    ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
-                                                    ws_ptr<int>(ws, p.kept), s.E, s.C, row_vec,
-                                                    ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate));
+    launch_k(gather_dy_kernel<false>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(dy),
+             static_cast<const uint4*>(ysrc), ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
+             ws_ptr<int>(ws, p.kept), ws_ptr<int>(ws, p.slot), s.T, s.E, s.C, row_vec, slot_blocks,
+             ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate), static_cast<uint4*>(dx));
   return launch_status();
 }
 

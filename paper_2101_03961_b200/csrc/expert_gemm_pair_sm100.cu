@@ -55,6 +55,8 @@ struct PairParams {
   int hmask_ld;
   long long ld_out;
   int* status;
+  const __nv_bfloat16* res;   // combine / scatter with the skip path inside the layer: rows added to the output (x or dy)
+  __nv_bfloat16* out2;        // combine with the skip path: second copy of the output without it
 };
 
 struct PTile {
@@ -385,6 +387,18 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
               if ((lane & 3) == 0 && offs[it] >= 0 && m_warp < p.Mw)
                 p.hmask[((long long)t.e * p.C + t.row0 + c * 32 + rr) * p.hmask_ld + (m_warp >> 5)] = word;
             }
+            if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[it] >= 0 && mcol < p.Mw) {
+              // skip path inside the layer: y = x + g E(x), dx = dy + dH W_in^T (the expert term is already bf16)
+              if (OP == kGemm2Combine) *reinterpret_cast<uint4*>(p.out2 + offs[it] + mcol) = val;
+              const uint4 r = *reinterpret_cast<const uint4*>(p.res + offs[it] + mcol);
+              const __nv_bfloat162* rv = reinterpret_cast<const __nv_bfloat162*>(&r);
+              __nv_bfloat162* vv = reinterpret_cast<__nv_bfloat162*>(&val);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float2 a2 = __bfloat1622float2(vv[q]), b2 = __bfloat1622float2(rv[q]);
+                vv[q] = __floats2bfloat162_rn(a2.x + b2.x, a2.y + b2.y);
+              }
+            }
             if (offs[it] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[it] + mcol) = val;
           }
 #pragma unroll
@@ -504,7 +518,9 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
     case kGemm2Combine:    // A = W_out [E][f (k)][d (m)] MN-major; B = H [E][C][f] K-major
       q.token_op = 1; q.a_mn_major = 1; q.Mw = s.d; K = s.f;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 64); rc2 = make_map(&tmB, h, s.E, s.C, s.f, 128);
-      q.out = static_cast<__nv_bfloat16*>(a.y); q.ld_out = s.d; break;
+      q.out = static_cast<__nv_bfloat16*>(a.y); q.ld_out = s.d;
+      if (s.residual) { q.res = static_cast<const __nv_bfloat16*>(a.x); q.out2 = ws_ptr<__nv_bfloat16>(ws, p.layer_y); }
+      break;
     case kDgrad2Mask:      // A = W_out [E][f (m)][d (k)] K-major; B = dY_d [E][C][d] K-major
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.f; K = s.d;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 128); rc2 = make_map(&tmB, dyd, s.E, s.C, s.d, 128);
@@ -512,7 +528,9 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
     case kDgrad1Scatter:   // A = W_in [E][d (m)][f (k)] K-major; B = dH [E][C][f] K-major
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.d; K = s.f;
       rc = make_map(&tmA, a.W_in, s.E, s.d, s.f, 128); rc2 = make_map(&tmB, dh, s.E, s.C, s.f, 128);
-      q.out = static_cast<__nv_bfloat16*>(a.dx); q.ld_out = s.d; break;
+      q.out = static_cast<__nv_bfloat16*>(a.dx); q.ld_out = s.d;
+      if (s.residual) q.res = static_cast<const __nv_bfloat16*>(a.dy);
+      break;
     case kWgrad2:          // dW_out [f][d] = H^T dY_d: A = H [E][C (k)][f (m)] MN-major; B = dY_d [E][C (k)][d (n)]
       q.token_op = 0; q.a_mn_major = 1; q.Mw = s.f; q.Nfix = s.d;
       rc = make_map(&tmA, h, s.E, s.C, s.f, 64); rc2 = make_map(&tmB, dyd, s.E, s.C, s.d, 64);

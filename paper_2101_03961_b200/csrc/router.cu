@@ -305,6 +305,7 @@ __global__ void router_dwr_reduce_kernel(const float* __restrict__ partial, int 
 }
 
 // dx[t,k] = (accumulate and t kept ? dx[t,k] : 0) + sum_i dh[t,i] W_r[k,i]; block = 64 tokens x 64 k per step.
+// accumulate = 2 adds to every token's row (the layer's own skip path has already put dy into the dropped ones).
 template <typename XT, int NE>
 __global__ void __launch_bounds__(256)
 router_dx_kernel(const float* __restrict__ dlogits, const float* __restrict__ W_r, const int* __restrict__ slot,
@@ -356,7 +357,7 @@ router_dx_kernel(const float* __restrict__ dlogits, const float* __restrict__ W_
     for (int a = 0; a < 4; ++a) {
       const int t = tok0 + ty * 4 + a;
       if (t >= T) continue;
-      const bool add = accumulate && slot[t] >= 0;
+      const bool add = accumulate == 2 || (accumulate && slot[t] >= 0);
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
         const int k = k0 + tx + 16 * b;
@@ -411,7 +412,7 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
       cudaSuccess)
     return SWITCH_MOE_CUDA_ERROR;
   launch_k(router_dx_kernel<XT, NE>, dim3((s.T + 63) / 64), dim3(256), smem, st, dlogits, W_r, ws_ptr<int>(ws, p.slot), s.T, s.d, s.E,
-                                                              accumulate_dx ? 1 : 0, static_cast<XT*>(dx));
+                                                              accumulate_dx ? (s.residual ? 2 : 1) : 0, static_cast<XT*>(dx));
   return launch_status();
 }
 

@@ -200,7 +200,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (OP == kRDx) {
         const int tok = t.m0 + r;
         const long long row_off = tok < p.T ? (long long)tok * p.d : -1;
-        const int add = (p.accumulate && tok < p.T && p.slot[tok] >= 0) ? 1 : 0;
+        const int add = (p.accumulate && tok < p.T && (p.accumulate == 2 || p.slot[tok] >= 0)) ? 1 : 0;
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
           offs[it] = __shfl_sync(0xffffffffu, row_off, it * 4 + (lane >> 3));
@@ -729,7 +729,7 @@ int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const flo
   q.mma_n = kBN;
   q.n_mtiles = (s.T + kTileM - 1) / kTileM; q.n_ntiles = (s.d + kBN - 1) / kBN;
   q.wrap = s.Epad64 / kBK;
-  q.dx = static_cast<__nv_bfloat16*>(dx); q.slot = ws_ptr<int>(ws, p.slot); q.accumulate = accumulate_dx ? 1 : 0;
+  q.dx = static_cast<__nv_bfloat16*>(dx); q.slot = ws_ptr<int>(ws, p.slot); q.accumulate = accumulate_dx ? (s.residual ? 2 : 1) : 0;   // 2: every row (skip path inside the layer)
   return launch_op<kRDx>(tmA, tmB, q, st);
 }
 

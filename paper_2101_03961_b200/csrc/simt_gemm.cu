@@ -16,12 +16,16 @@ struct SimtProblem {
   int C;                                        // expert capacity (rows per expert of the slot buffers)
   const int* kept; const int* token_of_slot; const float* gate;
   void* out; const void* mask_src; int ld_out;
+  const void* res;   // combine / scatter with the skip path inside the layer: row added to the output (x or dy)
+  void* out2;        // combine with the skip path: second copy of the output without it
 };
 
 __device__ __forceinline__ float ldf(const float* p) { return *p; }
 __device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 __device__ __forceinline__ void stf(float* p, float v) { *p = v; }
 __device__ __forceinline__ void stf(__nv_bfloat16* p, float v) { *p = __float2bfloat16(v); }
+__device__ __forceinline__ float rnd(const float*, float v) { return v; }
+__device__ __forceinline__ float rnd(const __nv_bfloat16*, float v) { return __bfloat162float(__float2bfloat16(v)); }
 
 template <typename ET, int OP>
 __global__ void __launch_bounds__(256) simt_grouped_gemm_kernel(SimtProblem pr) {
@@ -91,6 +95,9 @@ __global__ void __launch_bounds__(256) simt_grouped_gemm_kernel(SimtProblem pr) 
       float v = acc[i][j] * scale;
       if (OP == kGemm1Relu) v = fmaxf(v, 0.f);
       if (OP == kDgrad2Mask) v = ldf(static_cast<const ET*>(pr.mask_src) + row + n) > 0.f ? v : 0.f;
+      if (OP == kGemm2Combine && pr.out2 != nullptr) stf(static_cast<ET*>(pr.out2) + row + n, v);
+      if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && pr.res != nullptr)   // the expert term is rounded first
+        v = rnd(static_cast<const ET*>(nullptr), v) + ldf(static_cast<const ET*>(pr.res) + row + n);
       stf(static_cast<ET*>(pr.out) + row + n, v);
     }
   }
@@ -134,6 +141,8 @@ int launch_t(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* 
       max_m = s.d; break;
     default: return SWITCH_MOE_INVALID_ARGUMENT;
   }
+  if (s.residual && op == kGemm2Combine) { pr.res = a.x; pr.out2 = ws_ptr<char>(ws, p.layer_y); }
+  if (s.residual && op == kDgrad1Scatter) pr.res = a.dy;
   dim3 grid((pr.N + kBN - 1) / kBN, (max_m + kBM - 1) / kBM, s.E);
   switch (op) {
     case kGemm1Relu: simt_grouped_gemm_kernel<ET, kGemm1Relu><<<grid, 256, 0, st>>>(pr); break;

@@ -27,12 +27,13 @@ struct Shape {
   int Epad64;       // E rounded up to a multiple of 64 (tensor-core router operands)
   int router_tc;    // 1: router on the tensor cores (bf16 x, 3-way bf16 split of fp32 operands); 0: FP32 FMA
   int router_blocks, plan_blocks, max_mtiles, dwr_chunks;
+  int residual;     // 1: y = x + layer(x), dx = dy + d layer / dx (SWITCH_MOE_FLAG_RESIDUAL)
 };
 
 // Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
 struct Plan {
   size_t status, expert_index, gate, slot, token_of_slot, count, kept, psum, psum_partial, hist, hist_base,
-      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, total;
+      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, layer_y, total;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -46,8 +47,9 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (cfg->gemm_path != SWITCH_MOE_GEMM_DEFAULT && cfg->gemm_path != SWITCH_MOE_GEMM_SIMT &&
       cfg->gemm_path != SWITCH_MOE_GEMM_TC_1CTA)
     return SWITCH_MOE_INVALID_ARGUMENT;
-  for (int i = 0; i < 5; ++i)
+  for (int i = 0; i < 4; ++i)
     if (cfg->reserved[i] != 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if ((cfg->flags & ~SWITCH_MOE_FLAG_RESIDUAL) != 0) return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->E > kMaxExperts) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if (cfg->d_model % 8 != 0 || cfg->d_ff % 8 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   s->T = cfg->T; s->d = cfg->d_model; s->f = cfg->d_ff; s->E = cfg->E;
@@ -66,6 +68,8 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   s->elt = cfg->dtype == SWITCH_MOE_BF16 ? 2 : 4;
   s->gemm_path = (cfg->dtype == SWITCH_MOE_F32 || cfg->gemm_path == SWITCH_MOE_GEMM_SIMT) ? 1 : cfg->gemm_path;
   if (s->gemm_path != 1 && (cfg->d_model % 64 != 0 || cfg->d_ff % 64 != 0)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->residual = (cfg->flags & SWITCH_MOE_FLAG_RESIDUAL) ? 1 : 0;
+  if (s->residual && s->gemm_path == SWITCH_MOE_GEMM_TC_1CTA) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   int ne = (cfg->E + 31) / 32;
   int ne_pow2 = 1;
   while (ne_pow2 < ne) ne_pow2 *= 2;
@@ -121,6 +125,7 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->wsplit = take(3 * d * (size_t)s.Epad64 * 2);
   p->dhsplit = take(3 * T * (size_t)s.Epad64 * 2);
   p->hmask = take(E * C * ((f + 31) / 32) * 4);            // one bit per element of H: [H > 0]
+  p->layer_y = s.residual ? take(T * d * s.elt) : 0;       // g . E(x) without the skip path (for the gate's gradient)
   p->total = off;
 }
 
@@ -173,7 +178,7 @@ int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float*
 int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_index, float* aux_loss, void* ws,
                          cudaStream_t st);
 int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void* ws, cudaStream_t st);
-int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* ws, cudaStream_t st);
+int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* dx, void* ws, cudaStream_t st);
 int launch_router_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* dgate, float d_aux,
                       void* ws, void* dx, bool accumulate_dx, float* dW_r, cudaStream_t st);
 
@@ -195,6 +200,7 @@ enum GemmOp {
 struct GemmArgs {
   const void* W_in; const void* W_out;   // expert weights
   void* y; void* dx; void* dW_in; void* dW_out;
+  const void* x; const void* dy;         // skip-path sources (residual configuration only): y += x, dx += dy
 };
 int launch_simt_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
 int launch_tc_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);

@@ -23,7 +23,8 @@ OK = 0
 INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, CUDA_ERROR, DEVICE_TIMEOUT = -1, -2, -3, -4, -5
 
 WS_STATUS, WS_EXPERT_INDEX, WS_GATE, WS_SLOT, WS_TOKEN_OF_SLOT, WS_COUNT, WS_KEPT, WS_PSUM, WS_PROBS, WS_XD, WS_H, \
-    WS_DYD, WS_DH, WS_DGATE, WS_DLOGITS = range(15)
+    WS_DYD, WS_DH, WS_DGATE, WS_DLOGITS, WS_LAYER_Y = range(16)
+FLAG_RESIDUAL = 1
 
 EXPORTED_SYMBOLS = [
     "switch_moe_capacity", "switch_moe_workspace_bytes", "switch_moe_workspace_view", "switch_moe_fwd",
@@ -40,7 +41,7 @@ class SwitchMoeConfig(ctypes.Structure):
         ("T", ctypes.c_int32), ("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("E", ctypes.c_int32),
         ("capacity_factor", ctypes.c_float), ("alpha", ctypes.c_float),
         ("capacity_override", ctypes.c_int32), ("dtype", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
-        ("reserved", ctypes.c_int32 * 5),
+        ("flags", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4),
         ("stage_events", ctypes.POINTER(ctypes.c_void_p)),
     ]
 
@@ -88,11 +89,12 @@ def load_library() -> ctypes.CDLL:
 
 
 def make_config(T, d_model, d_ff, E, capacity_factor, alpha=0.01, dtype=BF16, capacity_override=0,
-                gemm_path=GEMM_DEFAULT) -> SwitchMoeConfig:
+                gemm_path=GEMM_DEFAULT, residual=False) -> SwitchMoeConfig:
     cfg = SwitchMoeConfig()
     cfg.T, cfg.d_model, cfg.d_ff, cfg.E = int(T), int(d_model), int(d_ff), int(E)
     cfg.capacity_factor, cfg.alpha = float(capacity_factor), float(alpha)
     cfg.capacity_override, cfg.dtype, cfg.gemm_path = int(capacity_override), int(dtype), int(gemm_path)
+    cfg.flags = FLAG_RESIDUAL if residual else 0
     return cfg
 
 

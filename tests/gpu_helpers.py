@@ -41,11 +41,13 @@ def to_np(t: torch.Tensor) -> np.ndarray:
 class GpuLayer:
     """Device buffers of one layer call plus the library calls on them."""
 
-    def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0):
+    def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0,
+                 residual=False):
         sbuild.build()
         self.scfg = cfg
         self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
-                                  dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path)
+                                  dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path,
+                                  residual=residual)
         dt = cfg.dtype
         self.x = to_dev(data["x"], dt)
         self.dy = to_dev(data["dy"], dt)
@@ -96,13 +98,24 @@ def check_flips(gpu_e: np.ndarray, ora: dict) -> int:
     return int(diff.size)
 
 
-def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capacity=None, experts=None):
+def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capacity=None, experts=None,
+                     residual=False):
     """Oracle forward with the device's expert choice (identical unless a near-tie flipped), after checking flips."""
     first = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                               router_bias=data.get("router_bias"), capacity=capacity, experts=[])
     flips = check_flips(gpu_e, first)
     fwd = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                             router_bias=data.get("router_bias"), capacity=capacity, expert_index=gpu_e,
-                            experts=experts)
+                            experts=experts, residual=residual)
     fwd["flips"] = flips
     return fwd
+
+
+def skip_path_ok(got, want_sum, want_layer, tol, dtype) -> bool:
+    """Bound for an output that carries the skip path (y = x + layer, dx = dy + layer gradient): the layer term is
+    held to `tol` as everywhere else, and the stored sum may be off by two roundings of the storage type (the term is
+    rounded, then the sum): 2 x 2^-9 for bfloat16, 2 x 2^-24 for float32, relative to the sum."""
+    ulp2 = 2.0 ** -8 if dtype == sm.BF16 else 2.0 ** -23
+    got = np.asarray(got, dtype=np.float64)
+    err = np.linalg.norm(got - want_sum)
+    return bool(err <= ulp2 * np.linalg.norm(want_sum) + tol * np.linalg.norm(want_layer))

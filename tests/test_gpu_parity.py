@@ -12,7 +12,8 @@ import torch
 from oracle import switch_oracle as so
 from paper_2101_03961_b200 import inputs as si
 from paper_2101_03961_b200 import switch_moe as sm
-from tests.gpu_helpers import (TOL_BF16, TOL_F32, TOL_ROUTER, GpuLayer, check_flips, oracle_following, rel_err, to_np)
+from tests.gpu_helpers import (TOL_BF16, TOL_F32, TOL_ROUTER, GpuLayer, check_flips, oracle_following, rel_err,
+                               skip_path_ok, to_np)
 
 pytestmark = pytest.mark.gpu
 
@@ -118,13 +119,13 @@ def test_dispatch_plan_is_deterministic():
 
 
 # ---------------------------------------------------------------------------------------------- whole layer
-def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0):
+def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False):
     data = si.gen_layer(cfg, seed=seed)
-    g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override)
+    g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual)
     g.fwd()
     gpu_e = g.expert_index()
     cap = capacity_override if capacity_override else None
-    fwd = oracle_following(cfg, data, gpu_e, capacity=cap)
+    fwd = oracle_following(cfg, data, gpu_e, capacity=cap, residual=residual)
     E, C = cfg.E, g.C
     assert C == fwd["C"]
     # integer state: bit exact
@@ -150,14 +151,25 @@ def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0):
         errs[f"H[{i}]"] = rel_err(hid[i, :k], np.maximum(fwd["u"][i], 0.0))
     y = to_np(g.y)
     assert np.isfinite(y).all()
-    assert np.all(y[~fwd["keep"]] == 0.0)                      # dropped tokens: zero rows
-    errs["y"] = rel_err(y, fwd["y"])
+    if residual:
+        # dropped tokens leave the layer unchanged, bit for bit; kept ones: the layer term (kept in the workspace
+        # without the skip path) is held to the usual tolerance, the sum to the rounding of its storage type
+        np.testing.assert_array_equal(y[~fwd["keep"]], to_np(g.x)[~fwd["keep"]])
+        layer_y = to_np(g.view(sm.WS_LAYER_Y)).reshape(cfg.T, cfg.d_model)
+        errs["layer_y"] = rel_err(layer_y[fwd["keep"]], fwd["layer_y"][fwd["keep"]])
+        assert skip_path_ok(y, fwd["y"], fwd["layer_y"], tol, cfg.dtype)
+    else:
+        assert np.all(y[~fwd["keep"]] == 0.0)                  # dropped tokens: zero rows
+        errs["y"] = rel_err(y, fwd["y"])
 
     g.bwd(d_aux=d_aux)
     bwd = so.switch_backward(fwd, data["x"], data["W_r"], data["W_in"], data["W_out"], data["dy"], d_aux=d_aux)
     kept_tok = np.flatnonzero(fwd["keep"])
     errs["dgate"] = rel_err(to_np(g.view(sm.WS_DGATE))[kept_tok], bwd["dgate"][kept_tok])
-    errs["dx"] = rel_err(to_np(g.dx), bwd["dx"])
+    if residual:
+        assert skip_path_ok(to_np(g.dx), bwd["dx"], bwd["dx"] - np.asarray(data["dy"], dtype=np.float64), tol, cfg.dtype)
+    else:
+        errs["dx"] = rel_err(to_np(g.dx), bwd["dx"])
     errs["dW_r"] = rel_err(to_np(g.dW_r), bwd["dW_r"])
     dW_in, dW_out = to_np(g.dW_in), to_np(g.dW_out)
     assert np.isfinite(dW_in).all() and np.isfinite(dW_out).all() and np.isfinite(to_np(g.dx)).all()
@@ -188,6 +200,22 @@ def test_bf16_layer_on_tensor_cores_matches_oracle(cfg):
 @pytest.mark.parametrize("cfg", [MID, RAGGED], ids=lambda c: c.name)
 def test_bf16_layer_on_single_cta_tensor_core_path_matches_oracle(cfg):
     _check_layer(cfg, sm.GEMM_TC_1CTA, TOL_BF16, d_aux=0.5)
+
+
+@pytest.mark.parametrize("cfg,path,tol", [(TINY, sm.GEMM_DEFAULT, TOL_F32), (MID, sm.GEMM_SIMT, TOL_BF16),
+                                          (MID, sm.GEMM_DEFAULT, TOL_BF16), (RAGGED, sm.GEMM_DEFAULT, TOL_BF16),
+                                          (MANY, sm.GEMM_DEFAULT, TOL_BF16)],
+                         ids=["tiny_f32", "mid_fma", "mid_tc", "ragged_tc", "many_tc"])
+def test_layer_with_the_skip_path_inside_matches_oracle(cfg, path, tol):
+    """y = x + g E(x) fused into the combine step, dx = dy + ... fused into the scatter step (Fig. 2, Section 2.2)."""
+    _check_layer(cfg, path, tol, residual=True)
+
+
+def test_skip_path_is_refused_on_the_single_cta_validation_path():
+    cfg = sm.make_config(MID.T, MID.d_model, MID.d_ff, MID.E, MID.capacity_factor, gemm_path=sm.GEMM_TC_1CTA,
+                         residual=True)
+    with pytest.raises(sm.SwitchMoeError):
+        sm.switch_moe_workspace_bytes(cfg)
 
 
 def test_tensor_core_layer_with_two_token_tiles_per_expert():
