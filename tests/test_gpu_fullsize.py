@@ -12,7 +12,7 @@ from oracle import switch_oracle as so
 from paper_2101_03961_b200 import build as sbuild
 from paper_2101_03961_b200 import inputs as si
 from paper_2101_03961_b200 import switch_moe as sm
-from tests.gpu_helpers import TOL_BF16, TOL_ROUTER, check_flips, rel_err, to_np
+from tests.gpu_helpers import TOL_BF16, TOL_ROUTER, check_flips, rel_err, skip_path_ok, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -21,7 +21,7 @@ def _bits_to_dev(bits: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def _run_fullsize(name, seed=0, n_extra=2):
+def _run_fullsize(name, seed=0, n_extra=2, residual=False):
     sbuild.build()
     cfg = si.CONFIGS[name]
     assert cfg.dtype == si.DTYPE_BF16
@@ -32,7 +32,7 @@ def _run_fullsize(name, seed=0, n_extra=2):
     W_out = _bits_to_dev(si.gen_W_out(cfg, seed, as_bits=True, threads=16))
     W_r = torch.from_numpy(W_r_np).cuda()
     bias = None if b_np is None else torch.from_numpy(b_np).cuda()
-    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha)
+    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, residual=residual)
     ws = sm.allocate_workspace(mcfg)
     ws.fill_(0xFF)
     y, dx = torch.full_like(x, float("nan")), torch.full_like(x, float("nan"))
@@ -72,7 +72,7 @@ def _run_fullsize(name, seed=0, n_extra=2):
     W_in_s = {i: si.gen_W_in_expert(cfg, i, seed) for i in sample}
     W_out_s = {i: si.gen_W_out_expert(cfg, i, seed) for i in sample}
     fwd = so.switch_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, router_bias=b_np,
-                            expert_index=gpu_e, experts=sample)
+                            expert_index=gpu_e, experts=sample, residual=residual)
     bwd = so.switch_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
     keep = plan["keep"]
     hid = view(sm.WS_H).view(E, C, cfg.d_ff)
@@ -83,8 +83,15 @@ def _run_fullsize(name, seed=0, n_extra=2):
         assert k == plan["kept"][i]
         tt = torch.from_numpy(tok).cuda()
         errs[f"H[{i}]"] = rel_err(to_np(hid[i, :k]), np.maximum(fwd["u"][i], 0.0))
-        errs[f"y[{i}]"] = rel_err(to_np(y[tt]), fwd["y"][tok])
-        errs[f"dx[{i}]"] = rel_err(to_np(dx[tt]), bwd["dx"][tok])
+        if residual:
+            layer_y = view(sm.WS_LAYER_Y).view(T, cfg.d_model)
+            errs[f"layer_y[{i}]"] = rel_err(to_np(layer_y[tt]), fwd["layer_y"][tok])
+            assert skip_path_ok(to_np(y[tt]), fwd["y"][tok], fwd["layer_y"][tok], TOL_BF16, sm.BF16)
+            assert skip_path_ok(to_np(dx[tt]), bwd["dx"][tok], bwd["dx"][tok] - dy_np[tok].astype(np.float64),
+                                TOL_BF16, sm.BF16)
+        else:
+            errs[f"y[{i}]"] = rel_err(to_np(y[tt]), fwd["y"][tok])
+            errs[f"dx[{i}]"] = rel_err(to_np(dx[tt]), bwd["dx"][tok])
         errs[f"dW_in[{i}]"] = rel_err(to_np(dW_in[i]), bwd["dW_in"][i])
         errs[f"dW_out[{i}]"] = rel_err(to_np(dW_out[i]), bwd["dW_out"][i])
         errs[f"dgate[{i}]"] = rel_err(to_np(view(sm.WS_DGATE)[tt]), bwd["dgate"][tok])
@@ -94,7 +101,15 @@ def _run_fullsize(name, seed=0, n_extra=2):
     # properties that hold at any size
     dropped = torch.from_numpy(np.flatnonzero(~keep)).cuda()
     if dropped.numel():
-        assert bool((y[dropped] == 0).all())
+        assert bool((y[dropped] == (x[dropped] if residual else 0)).all())   # skip path: the input row, bit for bit
+    if residual and dropped.numel():
+        # a dropped token's dx is dy plus the router's gradient only (checked exactly against the oracle's router)
+        some = np.flatnonzero(~keep)[:64]
+        G = np.broadcast_to((cfg.alpha * E / T) * fwd["f"][None, :], (some.size, E))
+        dh = p[some] * (G - np.sum(p[some] * G, axis=1, keepdims=True))
+        want = dy_np[some].astype(np.float64) + dh @ W_r_np.astype(np.float64).T
+        assert skip_path_ok(to_np(dx[torch.from_numpy(some).cuda()]), want, dh @ W_r_np.astype(np.float64).T, 1e-3,
+                            sm.BF16)
     assert bool(torch.isfinite(y).all()) and bool(torch.isfinite(dx).all()) and bool(torch.isfinite(dW_r).all())
     assert bool(torch.isfinite(dW_in).all()) and bool(torch.isfinite(dW_out).all())
     for i in np.flatnonzero(count == 0):
@@ -124,3 +139,8 @@ def test_switch_large_full_size():
 
 def test_wide_expert_full_size():
     _run_fullsize("wide", n_extra=1)
+
+
+def test_overflow_stress_with_the_skip_path_inside_full_size():
+    out = _run_fullsize("stress_calibrated", residual=True)
+    assert out["dropped"] > 0.15 * 32768
