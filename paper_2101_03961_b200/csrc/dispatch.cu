@@ -25,60 +25,58 @@ plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int* __rest
   for (int e = threadIdx.x; e < E; e += blockDim.x) hist[(size_t)blockIdx.x * E + e] = h[e];
 }
 
-// One block of 4 x 256 threads: thread (g, e) owns quarter g of the rows of column e.  Column scan of the
-// histograms, counts, kept, P-sums (all in a fixed order), the auxiliary loss and the token-tile list.
-constexpr int kScanGroups = 4;
-__global__ void __launch_bounds__(kScanGroups * kMaxExperts)
+// One block of 1024 threads = G groups x Ew columns (Ew = E rounded up to a power of two, at least 32; G = 1024 / Ew):
+// thread (g, e) owns slice g of the rows of column e.  Column scan of the histograms, counts, kept, P-sums (all in a
+// fixed order), the auxiliary loss and the token-tile list.  A thread's rows are loaded once, all loads in flight
+// together, and kept in registers for the scan (up to kScanRows rows per thread; longer slices are re-read).
+constexpr int kScanThreads = 1024;
+constexpr int kScanRows = 16;
+__global__ void __launch_bounds__(kScanThreads)
 plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __restrict__ psum_partial,
-                 int router_blocks, int T, int E, int C, float alpha, int* __restrict__ hist_base,
+                 int router_blocks, int T, int E, int Ew, int C, float alpha, int* __restrict__ hist_base,
                  int* __restrict__ count, int* __restrict__ kept, float* __restrict__ psum,
                  float* __restrict__ aux_loss, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
                  int4* __restrict__ ntile) {
   pdl_launch_dependents();
   pdl_wait();
-  __shared__ int qsum[kScanGroups][kMaxExperts];
-  __shared__ float qps[kScanGroups][kMaxExperts];
+  __shared__ int qsum[kScanThreads];                         // [g][e], Ew columns per row
+  __shared__ float qps[kScanThreads];
   __shared__ float term[kMaxExperts];
   __shared__ int kept_s[kMaxExperts];
-  const int e = threadIdx.x % kMaxExperts, g = threadIdx.x / kMaxExperts;
-  const int hq = (plan_blocks + kScanGroups - 1) / kScanGroups, h0 = g * hq, h1 = min(plan_blocks, h0 + hq);
-  const int rq = (router_blocks + kScanGroups - 1) / kScanGroups, r0 = g * rq, r1 = min(router_blocks, r0 + rq);
+  const int G = kScanThreads / Ew;
+  const int e = threadIdx.x % Ew, g = threadIdx.x / Ew;
+  const int hq = (plan_blocks + G - 1) / G, h0 = g * hq, h1 = min(plan_blocks, h0 + hq);
+  const int rq = (router_blocks + G - 1) / G, r0 = g * rq, r1 = min(router_blocks, r0 + rq);
+  int hv[kScanRows];
   if (e < E) {
+#pragma unroll
+    for (int j = 0; j < kScanRows; ++j) hv[j] = h0 + j < h1 ? hist[(size_t)(h0 + j) * E + e] : 0;
+    float pv[kScanRows];
+#pragma unroll
+    for (int j = 0; j < kScanRows; ++j) pv[j] = r0 + j < r1 ? psum_partial[(size_t)(r0 + j) * E + e] : 0.f;
     int sum = 0;
-    for (int b0 = h0; b0 < h1; b0 += 8) {
-      int v[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = b0 + j < h1 ? hist[(size_t)(b0 + j) * E + e] : 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) sum += v[j];
-    }
-    qsum[g][e] = sum;
+    for (int j = 0; j < kScanRows; ++j) sum += hv[j];
+    for (int b = h0 + kScanRows; b < h1; ++b) sum += hist[(size_t)b * E + e];
     float ps = 0.f;
-    for (int b0 = r0; b0 < r1; b0 += 8) {
-      float v[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = b0 + j < r1 ? psum_partial[(size_t)(b0 + j) * E + e] : 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) ps += v[j];                                          // fixed order
-    }
-    qps[g][e] = ps;
+    for (int j = 0; j < kScanRows; ++j) ps += pv[j];                                   // fixed order
+    for (int b = r0 + kScanRows; b < r1; ++b) ps += psum_partial[(size_t)b * E + e];
+    qsum[g * Ew + e] = sum;
+    qps[g * Ew + e] = ps;
   }
   __syncthreads();
   if (e < E) {
     int run = 0;
-    for (int q = 0; q < g; ++q) run += qsum[q][e];
-    for (int b0 = h0; b0 < h1; b0 += 8) {
-      int v[8];
+    for (int q = 0; q < g; ++q) run += qsum[q * Ew + e];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = b0 + j < h1 ? hist[(size_t)(b0 + j) * E + e] : 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (b0 + j < h1) { hist_base[(size_t)(b0 + j) * E + e] = run; run += v[j]; }
-    }
+    for (int j = 0; j < kScanRows; ++j)
+      if (h0 + j < h1) { hist_base[(size_t)(h0 + j) * E + e] = run; run += hv[j]; }
+    for (int b = h0 + kScanRows; b < h1; ++b) { hist_base[(size_t)b * E + e] = run; run += hist[(size_t)b * E + e]; }
     if (g == 0) {
       int total = 0;
       float ps = 0.f;
-      for (int q = 0; q < kScanGroups; ++q) { total += qsum[q][e]; ps += qps[q][e]; }
+      for (int q = 0; q < G; ++q) { total += qsum[q * Ew + e]; ps += qps[q * Ew + e]; }
       count[e] = total;
       const int k = min(total, C);
       kept[e] = k;
@@ -263,8 +261,10 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
       return SWITCH_MOE_CUDA_ERROR;
   }
   launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, s.T, s.E, ws_ptr<int>(ws, p.hist));
-  launch_k(plan_scan_kernel, dim3(1), dim3(kScanGroups * kMaxExperts), 0, st, ws_ptr<int>(ws, p.hist), s.plan_blocks,
-                                              ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, s.C,
+  int Ew = 32;
+  while (Ew < s.E) Ew *= 2;
+  launch_k(plan_scan_kernel, dim3(1), dim3(kScanThreads), 0, st, ws_ptr<int>(ws, p.hist), s.plan_blocks,
+                                              ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, Ew, s.C,
                                               s.alpha, ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count),
                                               ws_ptr<int>(ws, p.kept), ws_ptr<float>(ws, p.psum), aux_loss,
                                               ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0),
