@@ -214,3 +214,67 @@ def router_backward_given_dgate(p, e, keep, count, dgate, x, W_r, alpha: float, 
     dh = p * (G - np.sum(p * G, axis=1, keepdims=True))
     x64 = np.asarray(x, dtype=F64)
     return {"dh": dh, "dW_r": x64.T @ dh, "dx_router": dh @ np.asarray(W_r, dtype=F64).T}
+
+
+# ------------------------------------------------------------------------------------------------------------
+# Several routing groups in one call.  The appendix pseudo-code carries a leading [num_cores] dimension on every
+# router tensor: each core routes its own tokens_per_core tokens (own capacity from Eq. 3, own f and P in Eq. 5-6),
+# the experts are shared, and the loss is the mean over cores and experts times num_experts^2, i.e. the mean of the
+# groups' losses.  Here a group is T / G consecutive rows of x.
+def switch_forward_groups(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, groups: int, router_bias=None,
+                          expert_index=None, experts=None, residual: bool = False):
+    """Forward for G routing groups: switch_forward on each group, results concatenated in token order.
+
+    The merged plan numbers an expert's rows group by group (group 0's kept tokens in token order, then group 1's,
+    ...): slot[t] = e_t * (G * C) + (kept tokens of expert e_t in earlier groups) + pos_t, with pos_t and the
+    capacity cut taken inside the token's own group.  "aux" is the mean of the groups' losses.
+    """
+    x64 = np.asarray(x, dtype=F64)
+    T = x64.shape[0]
+    G = int(groups)
+    assert G >= 1 and T % G == 0
+    Tg = T // G
+    E = np.asarray(W_r).shape[1]
+    parts = []
+    for g in range(G):
+        rows = slice(g * Tg, (g + 1) * Tg)
+        ei = None if expert_index is None else np.asarray(expert_index)[rows]
+        parts.append(switch_forward(x64[rows], W_r, W_in, W_out, capacity_factor, alpha, router_bias=router_bias,
+                                    expert_index=ei, experts=experts, residual=residual))
+    C = parts[0]["C"]
+    cat = lambda k: np.concatenate([q[k] for q in parts], axis=0)
+    kept_g = np.stack([q["kept"] for q in parts])                       # [G, E]
+    count_g = np.stack([q["count"] for q in parts])
+    base_g = np.cumsum(kept_g, axis=0) - kept_g                        # kept tokens of the expert in earlier groups
+    e, pos, keep = cat("e"), cat("pos"), cat("keep")
+    grp = np.repeat(np.arange(G), Tg)
+    slot = np.where(keep, e * (G * C) + base_g[grp, e] + pos, -1)
+    token_of_slot = np.full(E * G * C, -1, dtype=np.int64)
+    token_of_slot[slot[keep]] = np.flatnonzero(keep)
+    out = {"parts": parts, "G": G, "Tg": Tg, "C": C, "E": E, "T": T, "alpha": alpha, "residual": bool(residual),
+           "aux": float(np.mean([q["aux"] for q in parts])),
+           "y": cat("y"), "layer_y": cat("layer_y"), "o": cat("o"), "p": cat("p"), "h": cat("h"), "g": cat("g"),
+           "e": e, "pos": pos, "keep": keep, "slot": slot, "token_of_slot": token_of_slot,
+           "count": count_g.sum(axis=0), "kept": kept_g.sum(axis=0), "count_g": count_g, "kept_g": kept_g}
+    return out
+
+
+def switch_backward_groups(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=None, want_weight_grads=True):
+    """Backward of switch_forward_groups: each group's backward with d_aux / G (the loss is the groups' mean);
+    dx, dgate and dh are concatenated, the weight gradients are summed over the groups."""
+    x64 = np.asarray(x, dtype=F64)
+    dy64 = np.asarray(dy, dtype=F64)
+    G, Tg = fwd["G"], fwd["Tg"]
+    outs = []
+    for g in range(G):
+        rows = slice(g * Tg, (g + 1) * Tg)
+        outs.append(switch_backward(fwd["parts"][g], x64[rows], W_r, W_in, W_out, dy64[rows], d_aux=d_aux / G,
+                                    experts=experts, want_weight_grads=want_weight_grads))
+    cat = lambda k: np.concatenate([q[k] for q in outs], axis=0)
+    res = {"dx": cat("dx"), "dgate": cat("dgate"), "dh": cat("dh"), "dx_router": cat("dx_router"),
+           "dW_r": sum(q["dW_r"] for q in outs), "db": sum(q["db"] for q in outs), "dW_in": {}, "dW_out": {}}
+    if want_weight_grads:
+        for i in outs[0]["dW_in"]:
+            res["dW_in"][i] = sum(q["dW_in"][i] for q in outs)
+            res["dW_out"][i] = sum(q["dW_out"][i] for q in outs)
+    return res

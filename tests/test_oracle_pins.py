@@ -391,3 +391,107 @@ def test_residual_backward_adds_dy_and_matches_finite_differences():
         x[idx] = old
         num[idx] = (lp - lm) / (2 * eps)
     assert np.linalg.norm(num - bwd["dx"]) / np.linalg.norm(bwd["dx"]) < 1e-7
+
+
+# ------------------------------------------------------------------ several routing groups (the pseudo-code's [num_cores] dimension)
+def _literal_grouped_layer(x, W_r, W_in, W_out, cf, alpha, G):
+    """The appendix formulation with its leading group dimension: tensors [G, T/G, ...], one-hot dispatch and
+    combine tensors [G, T/G, E, C], experts shared; loss = mean(density . density_proxy) . E^2."""
+    T, d = x.shape
+    n = T // G
+    E = W_r.shape[1]
+    C = int(math.floor(n * cf / E))
+    xg = x.reshape(G, n, d)
+    logits = np.einsum("gtd,de->gte", xg, W_r)
+    probs = np.exp(logits - logits.max(2, keepdims=True))
+    probs /= probs.sum(2, keepdims=True)
+    index = probs.argmax(2)
+    gate = probs.max(2)
+    mask = np.eye(E)[index]                                            # [G, n, E]
+    aux = alpha * np.mean(mask.mean(1) * probs.mean(1)) * E * E
+    position = (np.cumsum(mask, axis=1) - 1.0) * mask
+    mask = mask * (position < C)
+    gate = gate * mask.sum(2)
+    pos_index = position.sum(2).astype(int)
+    pos_one_hot = (np.arange(C)[None, None, :] == pos_index[:, :, None]).astype(float)
+    combine = gate[..., None, None] * mask[..., None] * pos_one_hot[:, :, None, :]   # [G, n, E, C]
+    dispatch = (combine != 0).astype(float)
+    expert_inputs = np.einsum("gtd,gtec->egcd", xg, dispatch)
+    hidden = np.maximum(np.einsum("egcd,edf->egcf", expert_inputs, W_in), 0.0)
+    expert_outputs = np.einsum("egcf,efd->egcd", hidden, W_out)
+    y = np.einsum("egcd,gtec->gtd", expert_outputs, combine)
+    return y.reshape(T, d), aux, dispatch
+
+
+@pytest.mark.parametrize("T,d,f,E,cf,G,seed", [(48, 6, 10, 4, 1.0, 3, 0), (64, 8, 12, 8, 1.25, 2, 1), (60, 5, 7, 5, 0.5, 4, 2)])
+def test_grouped_layer_equals_literal_formulation_with_group_dimension(T, d, f, E, cf, G, seed):
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=seed, scale=2.0)
+    out = so.switch_forward_groups(x, W_r, W_in, W_out, cf, 0.01, G)
+    y, aux, dispatch = _literal_grouped_layer(x, W_r, W_in, W_out, cf, 0.01, G)
+    np.testing.assert_allclose(out["y"], y, rtol=1e-12, atol=1e-13)
+    assert abs(out["aux"] - aux) < 1e-15
+    n, C = T // G, out["C"]
+    mine = np.zeros((G, n, E, C))
+    for t in range(T):
+        if out["keep"][t]:
+            mine[t // n, t % n, out["e"][t], out["pos"][t]] = 1.0
+    np.testing.assert_array_equal(mine, dispatch)
+    # merged plan: a permutation of the kept tokens, expert-major, groups in order, token order inside a group
+    kept_tok = np.flatnonzero(out["keep"])
+    order = sorted(kept_tok, key=lambda t: (out["e"][t], t))
+    rows = [s for s in out["token_of_slot"] if s >= 0]
+    assert rows == order
+    for i in range(E):
+        seg = out["token_of_slot"][i * G * C:(i + 1) * G * C]
+        k = int(out["kept"][i])
+        assert np.all(seg[:k] >= 0) and np.all(seg[k:] == -1)           # an expert's rows are dense from its first row
+    assert np.array_equal(out["slot"][kept_tok], [int(np.flatnonzero(out["token_of_slot"] == t)[0]) for t in kept_tok])
+
+
+def test_one_group_is_the_plain_layer_and_groups_do_not_share_capacity():
+    T, d, f, E = 64, 6, 8, 4
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=31, scale=2.0)
+    one = so.switch_forward_groups(x, W_r, W_in, W_out, 0.75, 0.02, 1)
+    plain = so.switch_forward(x, W_r, W_in, W_out, 0.75, 0.02)
+    assert np.array_equal(one["y"], plain["y"]) and one["aux"] == plain["aux"]
+    assert np.array_equal(one["slot"], plain["slot"])
+    two = so.switch_forward_groups(x, W_r, W_in, W_out, 0.75, 0.02, 2)
+    assert two["C"] == plain["C"] // 2
+    # an expert that overflows in group 0 drops tokens there even if group 1 leaves room
+    assert np.all(two["kept_g"] <= two["C"]) and (two["count_g"] > two["C"]).any()
+
+
+def test_grouped_backward_matches_finite_differences():
+    T, d, f, E, cf, alpha, d_aux, G = 16, 5, 7, 3, 0.75, 0.04, 1.3, 2
+    rng = np.random.default_rng(32)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=32, scale=2.0)
+    R = rng.standard_normal((T, d))
+    fwd = so.switch_forward_groups(x, W_r, W_in, W_out, cf, alpha, G)
+    srt = np.sort(fwd["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-3 and (~fwd["keep"]).any()
+    bwd = so.switch_backward_groups(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    e_frozen, eps = fwd["e"], 1e-6
+
+    def loss():
+        out = so.switch_forward_groups(x, W_r, W_in, W_out, cf, alpha, G, expert_index=e_frozen)
+        return float(np.sum(out["y"] * R) + d_aux * out["aux"])
+
+    def fd(arr, idx):
+        old = arr[idx]
+        arr[idx] = old + eps
+        lp = loss()
+        arr[idx] = old - eps
+        lm = loss()
+        arr[idx] = old
+        return (lp - lm) / (2 * eps)
+
+    dW_in = np.stack([bwd["dW_in"][i] for i in range(E)])
+    dW_out = np.stack([bwd["dW_out"][i] for i in range(E)])
+    for name, arr, grad in [("dx", x, bwd["dx"]), ("dW_r", W_r, bwd["dW_r"]), ("dW_in", W_in, dW_in),
+                            ("dW_out", W_out, dW_out)]:
+        idxs = list(np.ndindex(arr.shape))
+        if len(idxs) > 200:
+            idxs = [idxs[i] for i in rng.choice(len(idxs), 200, replace=False)]
+        num = np.array([fd(arr, i) for i in idxs])
+        ana = np.array([grad[i] for i in idxs])
+        assert np.linalg.norm(num - ana) / np.linalg.norm(ana) < 1e-7, name
