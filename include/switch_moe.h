@@ -71,7 +71,14 @@ typedef struct switch_moe_config {
   int32_t dtype;             /* switch_moe_dtype */
   int32_t gemm_path;         /* switch_moe_gemm_path */
   int32_t flags;             /* bitwise OR of switch_moe_flags */
-  int32_t reserved[4];       /* must be 0 */
+  int32_t groups;            /* routing groups G in this call (0 or 1: one group).  The pseudo-code's leading cores
+                                dimension: group g is rows [g T/G, (g+1) T/G) of x and is routed on its own -- own
+                                capacity floor((T/G) capacity_factor / E) by Eq. 3, own f and P in Eq. 5-6 -- while
+                                the experts are shared; the auxiliary loss is the mean of the groups' losses.  An
+                                expert's rows in the slot buffers are numbered group by group, each group's kept
+                                tokens in token order, G x capacity rows per expert.  G > 1 needs T / G to be a
+                                multiple of 256, T <= 65536 and G <= 64. */
+  int32_t reserved[3];       /* must be 0 */
   void* const* stage_events; /* HOST array of SWITCH_MOE_STAGE_EVENTS cudaEvent_t handles, or NULL (default).
                                 When set, fwd records event i on the stream before its stage i (0 router, 1 dispatch
                                 plan, 2 gather, 3 GEMM1+ReLU, 4 GEMM2+combine) and event 5 after the last one; bwd
@@ -86,13 +93,14 @@ enum switch_moe_ws_region {
   SWITCH_MOE_WS_STATUS = 0,         /* int32[16]; [0] != 0 after a device-side timeout */
   SWITCH_MOE_WS_EXPERT_INDEX = 1,   /* int32[T]   e_t */
   SWITCH_MOE_WS_GATE = 2,           /* float[T]   g_t (the un-masked top-1 probability, also for dropped tokens) */
-  SWITCH_MOE_WS_SLOT = 3,           /* int32[T]   e_t * C + pos_t, or -1 if dropped */
-  SWITCH_MOE_WS_TOKEN_OF_SLOT = 4,  /* int32[E*C] token stored in each slot, or -1 */
+  SWITCH_MOE_WS_SLOT = 3,           /* int32[T]   row of the token in the slot buffers: e_t * (G C) + (kept tokens of
+                                       e_t in earlier groups) + pos_t, or -1 if dropped */
+  SWITCH_MOE_WS_TOKEN_OF_SLOT = 4,  /* int32[E*G*C] token stored in each slot, or -1 */
   SWITCH_MOE_WS_COUNT = 5,          /* int32[E]   tokens whose argmax is expert i, before the capacity cut */
-  SWITCH_MOE_WS_KEPT = 6,           /* int32[E]   min(count, C) */
+  SWITCH_MOE_WS_KEPT = 6,           /* int32[E]   kept tokens: sum over groups of min(count in the group, C) */
   SWITCH_MOE_WS_PSUM = 7,           /* float[E]   sum_t p[t,i] */
   SWITCH_MOE_WS_PROBS = 8,          /* float[T,E] router probabilities */
-  SWITCH_MOE_WS_XD = 9,             /* [E,C,d_model] dispatched tokens (dtype of x) */
+  SWITCH_MOE_WS_XD = 9,             /* [E,G*C,d_model] dispatched tokens (dtype of x); likewise the next three */
   SWITCH_MOE_WS_H = 10,             /* [E,C,d_ff]    ReLU(x W_in) per slot */
   SWITCH_MOE_WS_DYD = 11,           /* [E,C,d_model] g . dy per slot (backward) */
   SWITCH_MOE_WS_DH = 12,            /* [E,C,d_ff]    gradient of the pre-activation per slot (backward) */
@@ -103,7 +111,8 @@ enum switch_moe_ws_region {
   SWITCH_MOE_WS_REGION_COUNT = 16
 };
 
-/* Eq. 3.  HOST call.  *C_out = capacity_override if > 0, else floor(T * capacity_factor / E) capped at T.
+/* Eq. 3.  HOST call.  *C_out = capacity_override if > 0, else floor((T / G) * capacity_factor / E) capped at T / G:
+   the capacity of one expert for one routing group (the slot buffers hold G * C rows per expert).
  * Errors: INVALID_ARGUMENT for null pointers, non-positive sizes or a resulting capacity of 0. */
 int switch_moe_capacity(const switch_moe_config* cfg, int32_t* C_out);
 

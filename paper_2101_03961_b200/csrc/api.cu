@@ -52,7 +52,7 @@ int switch_moe_capacity(const switch_moe_config* cfg, int32_t* C_out) {
   if (C_out == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
   Shape s;
   SWMOE_TRY(resolve_shape(cfg, &s));
-  *C_out = s.C;
+  *C_out = s.Cg;
   return SWITCH_MOE_OK;
 }
 

@@ -25,6 +25,44 @@ plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int* __rest
   for (int e = threadIdx.x; e < E; e += blockDim.x) hist[(size_t)blockIdx.x * E + e] = h[e];
 }
 
+// Tile lists, shared by both scan kernels: 128-row token tiles (single-CTA GEMM) and, for the paired-CTA GEMM, each
+// expert's kept rows cut into the fewest pieces of at most 256 rows, equal up to rounding each piece to a multiple of
+// 16 (the MMA's N granularity).  Thread 0 adds the loss terms and scans the per-expert tile counts; the first E
+// threads write their expert's entries.  `term` and `kept_s` are shared-memory arrays filled before the call.
+__device__ __forceinline__ void write_tile_lists(const float* term, const int* kept_s, int E, float loss_scale,
+                                                 float* __restrict__ aux_loss, int* __restrict__ tile_expert,
+                                                 int* __restrict__ tile_row0, int4* __restrict__ ntile) {
+  __shared__ int start128[kMaxExperts + 1], startn[kMaxExperts + 1];
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float s = 0.f;
+    for (int i = 0; i < E; ++i) s += term[i];
+    if (aux_loss != nullptr) *aux_loss = loss_scale * s;                              // Eq. 4
+    int n = 0, m = 0;
+    for (int i = 0; i < E; ++i) {
+      start128[i] = n; startn[i] = m;
+      n += (kept_s[i] + kTileM - 1) / kTileM;
+      m += (kept_s[i] + 255) / 256;
+    }
+    tile_expert[0] = n;
+    tile_row0[0] = n;
+    ntile[0] = make_int4(m, 0, 0, 0);
+  }
+  __syncthreads();
+  const int e = threadIdx.x;
+  if (e < E) {
+    const int k = kept_s[e];
+    int n = start128[e];
+    for (int r = 0; r < k; r += kTileM, ++n) { tile_expert[1 + n] = e; tile_row0[1 + n] = r; }
+    if (k > 0) {
+      const int pieces = (k + 255) / 256;
+      const int rows = ((k + pieces - 1) / pieces + 15) / 16 * 16;
+      int m = startn[e];
+      for (int r = 0; r < k; r += rows, ++m) ntile[1 + m] = make_int4(e, r, min(rows, (k - r + 15) / 16 * 16), 0);
+    }
+  }
+}
+
 // One block of 1024 threads = G groups x Ew columns (Ew = E rounded up to a power of two, at least 32; G = 1024 / Ew):
 // thread (g, e) owns slice g of the rows of column e.  Column scan of the histograms, counts, kept, P-sums (all in a
 // fixed order), the auxiliary loss and the token-tile list.  A thread's rows are loaded once, all loads in flight
@@ -36,7 +74,7 @@ plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __r
                  int router_blocks, int T, int E, int Ew, int C, float alpha, int* __restrict__ hist_base,
                  int* __restrict__ count, int* __restrict__ kept, float* __restrict__ psum,
                  float* __restrict__ aux_loss, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
-                 int4* __restrict__ ntile) {
+                 int4* __restrict__ ntile, int* __restrict__ count_g, int* __restrict__ group_base) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ int qsum[kScanThreads];                         // [g][e], Ew columns per row
@@ -78,6 +116,8 @@ plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __r
       float ps = 0.f;
       for (int q = 0; q < G; ++q) { total += qsum[q * Ew + e]; ps += qps[q * Ew + e]; }
       count[e] = total;
+      count_g[e] = total;                                                              // one routing group
+      group_base[e] = 0;
       const int k = min(total, C);
       kept[e] = k;
       kept_s[e] = k;
@@ -85,44 +125,73 @@ plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __r
       term[e] = ((float)total / (float)T) * (ps / (float)T);                           // f_i . P_i  (Eq. 5, 6)
     }
   }
-  __syncthreads();
-  // Tile lists.  128-row token tiles (single-CTA GEMM) and, for the paired-CTA GEMM, each expert's kept rows cut
-  // into the fewest pieces of at most 256 rows, equal up to rounding each piece to a multiple of 16 (the MMA's N
-  // granularity).  Thread 0 adds the loss terms and scans the per-expert tile counts; experts write their entries.
-  __shared__ int start128[kMaxExperts + 1], startn[kMaxExperts + 1];
-  if (threadIdx.x == 0) {
-    float s = 0.f;
-    for (int i = 0; i < E; ++i) s += term[i];
-    if (aux_loss != nullptr) *aux_loss = alpha * (float)E * s;                        // Eq. 4
-    int n = 0, m = 0;
-    for (int i = 0; i < E; ++i) {
-      start128[i] = n; startn[i] = m;
-      n += (kept_s[i] + kTileM - 1) / kTileM;
-      m += (kept_s[i] + 255) / 256;
+  write_tile_lists(term, kept_s, E, alpha * (float)E, aux_loss, tile_expert, tile_row0, ntile);
+}
+
+// Several routing groups (the pseudo-code's leading cores dimension): every group has its own counts, its own
+// capacity cut and its own f and P; an expert's rows are numbered group by group.  One block of 1024 threads;
+// thread (q, e) handles groups q, q + Q, ... of column e (Q = 1024 / Ew).  hist_base[b][e] is the position base of
+// block b inside its own group; group_base[g][e] = kept tokens of expert e in groups before g; the loss is the mean
+// of the groups' losses: (alpha E / G) sum_g sum_i (count_gi / Tg)(Psum_gi / Tg).
+constexpr int kScanGroupCells = 8192;                        // G x Ew counters kept in shared memory
+__global__ void __launch_bounds__(kScanThreads)
+plan_scan_groups_kernel(const int* __restrict__ hist, int blocks_per_group, const float* __restrict__ psum_partial,
+                        int rows_per_group, int NG, int Tg, int E, int Ew, int Cg, float alpha,
+                        int* __restrict__ hist_base, int* __restrict__ count, int* __restrict__ kept,
+                        float* __restrict__ psum, float* __restrict__ aux_loss, int* __restrict__ tile_expert,
+                        int* __restrict__ tile_row0, int4* __restrict__ ntile, int* __restrict__ count_g,
+                        int* __restrict__ group_base) {
+  pdl_launch_dependents();
+  pdl_wait();
+  __shared__ int cnt_s[kScanGroupCells];                     // [g][e], Ew columns per row
+  __shared__ float qps[kScanThreads], qterm[kScanThreads];   // [q][e]
+  __shared__ float term[kMaxExperts];
+  __shared__ int kept_s[kMaxExperts];
+  const int Q = kScanThreads / Ew;
+  const int e = threadIdx.x % Ew, q = threadIdx.x / Ew;
+  float ps_tot = 0.f, t_tot = 0.f;
+  if (e < E) {
+    for (int g = q; g < NG; g += Q) {
+      int run = 0;
+      for (int b = g * blocks_per_group; b < (g + 1) * blocks_per_group; ++b) {
+        hist_base[(size_t)b * E + e] = run;
+        run += hist[(size_t)b * E + e];
+      }
+      float ps = 0.f;
+      for (int r = g * rows_per_group; r < (g + 1) * rows_per_group; ++r) ps += psum_partial[(size_t)r * E + e];
+      cnt_s[g * Ew + e] = run;
+      count_g[(size_t)g * E + e] = run;
+      ps_tot += ps;                                                                    // fixed order
+      t_tot += ((float)run / (float)Tg) * (ps / (float)Tg);                            // f_gi . P_gi  (Eq. 5, 6)
     }
-    tile_expert[0] = n;
-    tile_row0[0] = n;
-    ntile[0] = make_int4(m, 0, 0, 0);
   }
+  qps[threadIdx.x] = ps_tot;
+  qterm[threadIdx.x] = t_tot;
   __syncthreads();
-  if (g == 0 && e < E) {
-    const int k = kept_s[e];
-    int n = start128[e];
-    for (int r = 0; r < k; r += kTileM, ++n) { tile_expert[1 + n] = e; tile_row0[1 + n] = r; }
-    if (k > 0) {
-      const int pieces = (k + 255) / 256;
-      const int rows = ((k + pieces - 1) / pieces + 15) / 16 * 16;
-      int m = startn[e];
-      for (int r = 0; r < k; r += rows, ++m) ntile[1 + m] = make_int4(e, r, min(rows, (k - r + 15) / 16 * 16), 0);
+  if (q == 0 && e < E) {
+    int base = 0, total = 0;
+    for (int g = 0; g < NG; ++g) {
+      const int c = cnt_s[g * Ew + e];
+      group_base[(size_t)g * E + e] = base;
+      base += min(c, Cg);
+      total += c;
     }
+    float ps = 0.f, tm = 0.f;
+    for (int k = 0; k < Q; ++k) { ps += qps[k * Ew + e]; tm += qterm[k * Ew + e]; }
+    count[e] = total;
+    kept[e] = base;
+    kept_s[e] = base;
+    psum[e] = ps;
+    term[e] = tm;
   }
+  write_tile_lists(term, kept_s, E, alpha * (float)E / (float)NG, aux_loss, tile_expert, tile_row0, ntile);
 }
 
 // pos_t = base[block][e] + (tokens of earlier warps with e) + (earlier lanes with e); slot, token_of_slot.
 __global__ void __launch_bounds__(kPlanBlockTokens)
 plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__ hist_base,
-                   const int* __restrict__ kept, int T, int E, int C, int* __restrict__ slot,
-                   int* __restrict__ token_of_slot) {
+                   const int* __restrict__ kept, const int* __restrict__ group_base, int blocks_per_group, int T,
+                   int E, int C, int Cg, int* __restrict__ slot, int* __restrict__ token_of_slot) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ int warp_cnt[kPlanBlockTokens / 32][kMaxExperts];
@@ -137,9 +206,10 @@ plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__
   if (t < T && rank == 0) warp_cnt[warp][e] = __popc(same);
   __syncthreads();
   if (t < T) {
-    int pos = hist_base[(size_t)blockIdx.x * E + e] + rank;
+    int pos = hist_base[(size_t)blockIdx.x * E + e] + rank;                  // position inside the token's own group
     for (int w = 0; w < warp; ++w) pos += warp_cnt[w][e];
-    const int s = pos < C ? e * C + pos : -1;
+    const int grp = blockIdx.x / blocks_per_group;
+    const int s = pos < Cg ? e * C + group_base[(size_t)grp * E + e] + pos : -1;
     slot[t] = s;
     if (s >= 0) token_of_slot[s] = t;
   }
@@ -263,16 +333,26 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
   launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, s.T, s.E, ws_ptr<int>(ws, p.hist));
   int Ew = 32;
   while (Ew < s.E) Ew *= 2;
-  launch_k(plan_scan_kernel, dim3(1), dim3(kScanThreads), 0, st, ws_ptr<int>(ws, p.hist), s.plan_blocks,
-                                              ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, Ew, s.C,
-                                              s.alpha, ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count),
-                                              ws_ptr<int>(ws, p.kept), ws_ptr<float>(ws, p.psum), aux_loss,
-                                              ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0),
-                                              ws_ptr<int4>(ws, p.ntile));
+  const int blocks_per_group = s.plan_blocks / s.G;
+  int* count_g = ws_ptr<int>(ws, p.count_g);
+  int* group_base = ws_ptr<int>(ws, p.group_base);
+  if (s.G == 1) {
+    launch_k(plan_scan_kernel, dim3(1), dim3(kScanThreads), 0, st, ws_ptr<int>(ws, p.hist), s.plan_blocks,
+             ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, Ew, s.Cg, s.alpha,
+             ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count), ws_ptr<int>(ws, p.kept),
+             ws_ptr<float>(ws, p.psum), aux_loss, ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0),
+             ws_ptr<int4>(ws, p.ntile), count_g, group_base);
+  } else {
+    if (s.G * Ew > kScanGroupCells || s.router_blocks % s.G != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+    launch_k(plan_scan_groups_kernel, dim3(1), dim3(kScanThreads), 0, st, ws_ptr<int>(ws, p.hist), blocks_per_group,
+             ws_ptr<float>(ws, p.psum_partial), s.router_blocks / s.G, s.G, s.Tg, s.E, Ew, s.Cg, s.alpha,
+             ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count), ws_ptr<int>(ws, p.kept),
+             ws_ptr<float>(ws, p.psum), aux_loss, ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0),
+             ws_ptr<int4>(ws, p.ntile), count_g, group_base);
+  }
   launch_k(plan_assign_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, ws_ptr<int>(ws, p.hist_base),
-                                                                 ws_ptr<int>(ws, p.kept), s.T, s.E, s.C,
-                                                                 ws_ptr<int>(ws, p.slot),
-                                                                 ws_ptr<int>(ws, p.token_of_slot));
+           ws_ptr<int>(ws, p.kept), group_base, blocks_per_group, s.T, s.E, s.C, s.Cg, ws_ptr<int>(ws, p.slot),
+           ws_ptr<int>(ws, p.token_of_slot));
   return launch_status();
 }
 

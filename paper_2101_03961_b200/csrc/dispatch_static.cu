@@ -109,7 +109,7 @@ extern "C" int switch_moe_dispatch_plan_static(const switch_moe_config* cfg, con
   int rc = resolve_shape(cfg, &s);
   if (rc != SWITCH_MOE_OK) return rc;
   if (!expert_index || !count || !kept || !slot || !token_of_slot) return SWITCH_MOE_INVALID_ARGUMENT;
-  if (s.T > kStaticMaxTokens) return SWITCH_MOE_UNSUPPORTED_SHAPE;      // the static scratch holds 256 x 256 counters twice
+  if (s.T > kStaticMaxTokens || s.G != 1) return SWITCH_MOE_UNSUPPORTED_SHAPE;      // the static scratch holds 256 x 256 counters twice
   int32_t* scratch = nullptr;
   rc = scratch_for_current_device(&scratch);
   if (rc != SWITCH_MOE_OK) return rc;

@@ -172,13 +172,14 @@ template <> struct BfVec<2> { using type = unsigned int; };
 template <> struct BfVec<4> { using type = uint2; };
 template <> struct BfVec<8> { using type = uint4; };
 
-// dh[t,i] = p[t,i] (G[t,i] - sum_j p[t,j] G[t,j]),  G[t,i] = cG.count_i + [i = e_t and t kept].dgate_t
+// dh[t,i] = p[t,i] (G[t,i] - sum_j p[t,j] G[t,j]),  G[t,i] = cG.count_gi + [i = e_t and t kept].dgate_t,
+// count_gi counted inside the token's own routing group g = t / Tg
 template <int NE>
 __global__ void __launch_bounds__(256)
 router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ expert_index,
                       const int* __restrict__ slot, const int* __restrict__ count, const float* __restrict__ dgate,
-                      float cG, int T, int E, float* __restrict__ dlogits, __nv_bfloat16* __restrict__ dhsplit,
-                      int Epad64) {
+                      float cG, int T, int Tg, int E, float* __restrict__ dlogits,
+                      __nv_bfloat16* __restrict__ dhsplit, int Epad64) {
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -186,6 +187,7 @@ router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ e
   if (t >= T) return;
   const int et = expert_index[t];
   const float dg = slot[t] >= 0 ? dgate[t] : 0.f;
+  count += (size_t)(t / Tg) * E;
   float p[NE], G[NE], s = 0.f;
 #pragma unroll
   for (int n = 0; n < NE; ++n) {
@@ -383,12 +385,13 @@ int router_fwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
 template <typename XT, int NE>
 int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* dgate, float d_aux,
                  void* ws, void* dx, bool accumulate_dx, float* dW_r, cudaStream_t st) {
-  // G's auxiliary-loss term: d_aux . alpha . E . f_i / T with f_i = count_i / T  (Eq. 4-6; f is a constant)
-  const float cG = (float)((double)d_aux * (double)s.alpha * (double)s.E / ((double)s.T * (double)s.T));
+  // G's auxiliary-loss term: d_aux . alpha . E . f_gi / T with f_gi = count_gi / Tg  (Eq. 4-6; f is a constant;
+  // the loss is the mean over the routing groups, and T = G . Tg)
+  const float cG = (float)((double)d_aux * (double)s.alpha * (double)s.E / ((double)s.T * (double)s.Tg));
   float* dlogits = ws_ptr<float>(ws, p.dlogits);
   launch_k(router_dlogits_kernel<NE>, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs),
                                                             ws_ptr<int>(ws, p.expert_index), ws_ptr<int>(ws, p.slot),
-                                                            ws_ptr<int>(ws, p.count), dgate, cG, s.T, s.E, dlogits,
+                                                            ws_ptr<int>(ws, p.count_g), dgate, cG, s.T, s.Tg, s.E, dlogits,
                                                             (s.router_tc && sizeof(XT) == 2)
                                                                 ? ws_ptr<__nv_bfloat16>(ws, p.dhsplit) : nullptr,
                                                             s.Epad64);

@@ -16,9 +16,12 @@ constexpr int kRouterBlockTokens = 64;  // tokens per router-forward block (one 
 constexpr int kPlanBlockTokens = 256;   // tokens per dispatch-plan block (one histogram row each)
 constexpr int kTileM = 128;             // token rows per tensor-core tile; tails are zero-filled to this
 constexpr int kDwrChunkTokens = 512;    // tokens per split of the dW_r reduction
+constexpr int kMaxGroups = 64;          // routing groups per call
 
 struct Shape {
-  int T, d, f, E, C;
+  int T, d, f, E;
+  int C;            // rows per expert in the slot buffers: groups x capacity
+  int G, Tg, Cg;    // routing groups, tokens per group, capacity of one expert for one group (Eq. 3)
   int dtype;        // switch_moe_dtype
   int gemm_path;    // resolved: 0 = tcgen05 on CTA pairs, 1 = SIMT, 2 = single-CTA tcgen05
   float alpha;
@@ -32,7 +35,7 @@ struct Shape {
 
 // Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
 struct Plan {
-  size_t status, expert_index, gate, slot, token_of_slot, count, kept, psum, psum_partial, hist, hist_base,
+  size_t status, expert_index, gate, slot, token_of_slot, count, kept, count_g, group_base, psum, psum_partial, hist, hist_base,
       tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, layer_y, total;
 };
 
@@ -47,8 +50,13 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (cfg->gemm_path != SWITCH_MOE_GEMM_DEFAULT && cfg->gemm_path != SWITCH_MOE_GEMM_SIMT &&
       cfg->gemm_path != SWITCH_MOE_GEMM_TC_1CTA)
     return SWITCH_MOE_INVALID_ARGUMENT;
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 3; ++i)
     if (cfg->reserved[i] != 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (cfg->groups < 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  const int G = cfg->groups > 1 ? cfg->groups : 1;
+  if (cfg->T % G != 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (G > 1 && ((cfg->T / G) % kPlanBlockTokens != 0 || cfg->T > 65536 || G > kMaxGroups))
+    return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if ((cfg->flags & ~SWITCH_MOE_FLAG_RESIDUAL) != 0) return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->E > kMaxExperts) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if (cfg->d_model % 8 != 0 || cfg->d_ff % 8 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
@@ -58,13 +66,14 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (cfg->capacity_override > 0) {
     C = cfg->capacity_override;
   } else {
-    double c = (double)cfg->T * (double)cfg->capacity_factor / (double)cfg->E;   // Eq. 3, floored
+    double c = (double)(cfg->T / G) * (double)cfg->capacity_factor / (double)cfg->E;   // Eq. 3, floored
     C = (long long)c;
   }
-  if (C > cfg->T) C = cfg->T;
+  if (C > cfg->T / G) C = cfg->T / G;
   if (C <= 0) return SWITCH_MOE_INVALID_ARGUMENT;
-  if ((long long)cfg->E * C > 0x7fffffffLL) return SWITCH_MOE_UNSUPPORTED_SHAPE;
-  s->C = (int)C;
+  if ((long long)cfg->E * C * G > 0x7fffffffLL) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->G = G; s->Tg = cfg->T / G; s->Cg = (int)C;
+  s->C = (int)C * G;
   s->elt = cfg->dtype == SWITCH_MOE_BF16 ? 2 : 4;
   s->gemm_path = (cfg->dtype == SWITCH_MOE_F32 || cfg->gemm_path == SWITCH_MOE_GEMM_SIMT) ? 1 : cfg->gemm_path;
   if (s->gemm_path != 1 && (cfg->d_model % 64 != 0 || cfg->d_ff % 64 != 0)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
@@ -107,6 +116,8 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->token_of_slot = take(E * C * 4);
   p->count = take(E * 4);
   p->kept = take(E * 4);
+  p->count_g = take((size_t)s.G * E * 4);                  // per group: tokens whose argmax is expert i
+  p->group_base = take((size_t)s.G * E * 4);               // per group: kept tokens of expert i in earlier groups
   p->psum = take(E * 4);
   p->psum_partial = take((size_t)s.router_blocks * E * 4);
   p->hist = take((size_t)s.plan_blocks * E * 4);

@@ -41,7 +41,7 @@ class SwitchMoeConfig(ctypes.Structure):
         ("T", ctypes.c_int32), ("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("E", ctypes.c_int32),
         ("capacity_factor", ctypes.c_float), ("alpha", ctypes.c_float),
         ("capacity_override", ctypes.c_int32), ("dtype", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
-        ("flags", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4),
+        ("flags", ctypes.c_int32), ("groups", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
         ("stage_events", ctypes.POINTER(ctypes.c_void_p)),
     ]
 
@@ -89,12 +89,13 @@ def load_library() -> ctypes.CDLL:
 
 
 def make_config(T, d_model, d_ff, E, capacity_factor, alpha=0.01, dtype=BF16, capacity_override=0,
-                gemm_path=GEMM_DEFAULT, residual=False) -> SwitchMoeConfig:
+                gemm_path=GEMM_DEFAULT, residual=False, groups=1) -> SwitchMoeConfig:
     cfg = SwitchMoeConfig()
     cfg.T, cfg.d_model, cfg.d_ff, cfg.E = int(T), int(d_model), int(d_ff), int(E)
     cfg.capacity_factor, cfg.alpha = float(capacity_factor), float(alpha)
     cfg.capacity_override, cfg.dtype, cfg.gemm_path = int(capacity_override), int(dtype), int(gemm_path)
     cfg.flags = FLAG_RESIDUAL if residual else 0
+    cfg.groups = int(groups)
     return cfg
 
 

@@ -42,12 +42,12 @@ class GpuLayer:
     """Device buffers of one layer call plus the library calls on them."""
 
     def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0,
-                 residual=False):
+                 residual=False, groups=1):
         sbuild.build()
         self.scfg = cfg
         self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
                                   dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path,
-                                  residual=residual)
+                                  residual=residual, groups=groups)
         dt = cfg.dtype
         self.x = to_dev(data["x"], dt)
         self.dy = to_dev(data["dy"], dt)
@@ -99,8 +99,18 @@ def check_flips(gpu_e: np.ndarray, ora: dict) -> int:
 
 
 def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capacity=None, experts=None,
-                     residual=False):
+                     residual=False, groups=1):
     """Oracle forward with the device's expert choice (identical unless a near-tie flipped), after checking flips."""
+    if groups > 1:
+        assert capacity is None
+        first = so.switch_forward_groups(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
+                                         cfg.alpha, groups, router_bias=data.get("router_bias"), experts=[])
+        flips = check_flips(gpu_e, first)
+        fwd = so.switch_forward_groups(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
+                                       cfg.alpha, groups, router_bias=data.get("router_bias"), expert_index=gpu_e,
+                                       experts=experts, residual=residual)
+        fwd["flips"] = flips
+        return fwd
     first = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                               router_bias=data.get("router_bias"), capacity=capacity, experts=[])
     flips = check_flips(gpu_e, first)
@@ -119,3 +129,11 @@ def skip_path_ok(got, want_sum, want_layer, tol, dtype) -> bool:
     got = np.asarray(got, dtype=np.float64)
     err = np.linalg.norm(got - want_sum)
     return bool(err <= ulp2 * np.linalg.norm(want_sum) + tol * np.linalg.norm(want_layer))
+
+
+def expert_preactivation(fwd: dict, i: int):
+    """Rows of u = x W_in for expert i in slot order (group by group when the call had several routing groups)."""
+    if "parts" not in fwd:
+        return fwd["u"].get(i)
+    rows = [q["u"][i] for q in fwd["parts"] if i in q["u"]]
+    return np.concatenate(rows, axis=0) if rows else None

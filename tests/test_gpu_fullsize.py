@@ -12,7 +12,7 @@ from oracle import switch_oracle as so
 from paper_2101_03961_b200 import build as sbuild
 from paper_2101_03961_b200 import inputs as si
 from paper_2101_03961_b200 import switch_moe as sm
-from tests.gpu_helpers import TOL_BF16, TOL_ROUTER, check_flips, rel_err, skip_path_ok, to_np
+from tests.gpu_helpers import TOL_BF16, TOL_ROUTER, check_flips, expert_preactivation, rel_err, skip_path_ok, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -21,7 +21,7 @@ def _bits_to_dev(bits: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def _run_fullsize(name, seed=0, n_extra=2, residual=False):
+def _run_fullsize(name, seed=0, n_extra=2, residual=False, groups=1):
     sbuild.build()
     cfg = si.CONFIGS[name]
     assert cfg.dtype == si.DTYPE_BF16
@@ -32,7 +32,8 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False):
     W_out = _bits_to_dev(si.gen_W_out(cfg, seed, as_bits=True, threads=16))
     W_r = torch.from_numpy(W_r_np).cuda()
     bias = None if b_np is None else torch.from_numpy(b_np).cuda()
-    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, residual=residual)
+    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, residual=residual,
+                          groups=groups)
     ws = sm.allocate_workspace(mcfg)
     ws.fill_(0xFF)
     y, dx = torch.full_like(x, float("nan")), torch.full_like(x, float("nan"))
@@ -43,7 +44,7 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False):
     sm.switch_moe_bwd(mcfg, dy, 1.0, x, W_r, W_in, W_out, y, ws, dx, dW_r, dW_in, dW_out)
     sm.switch_moe_check_device_status(mcfg, ws)
     view = lambda r: sm.switch_moe_workspace_view(mcfg, ws, r)
-    T, E, C = cfg.T, cfg.E, sm.switch_moe_capacity(mcfg)
+    T, E, C = cfg.T, cfg.E, sm.switch_moe_capacity(mcfg) * groups      # C: rows per expert in the slot buffers
 
     # router for all tokens; flips only inside the allowed gap; then the oracle follows the device's choice
     gpu_e = view(sm.WS_EXPERT_INDEX).cpu().numpy().astype(np.int64)
@@ -53,13 +54,18 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False):
     flips = check_flips(gpu_e, {"e": e0, "p": p})
     assert flips <= 8
     assert np.abs(to_np(view(sm.WS_PROBS)).reshape(T, E) - p).max() <= TOL_ROUTER
-    plan = so.dispatch_plan(gpu_e, E, so.expert_capacity(T, E, cfg.capacity_factor))
-    assert C == so.expert_capacity(T, E, cfg.capacity_factor)
+    if groups == 1:
+        plan = so.dispatch_plan(gpu_e, E, so.expert_capacity(T, E, cfg.capacity_factor))
+        aux_ref, _, _ = so.load_balance_loss(p, gpu_e, cfg.alpha)
+    else:                                                    # every group on its own; no expert FFN work here
+        plan = so.switch_forward_groups(x_np, W_r_np, {}, {}, cfg.capacity_factor, cfg.alpha, groups,
+                                        router_bias=b_np, expert_index=gpu_e, experts=[])
+        aux_ref = plan["aux"]
+    assert C == groups * so.expert_capacity(T // groups, E, cfg.capacity_factor)
     np.testing.assert_array_equal(view(sm.WS_SLOT).cpu().numpy(), plan["slot"])
     np.testing.assert_array_equal(view(sm.WS_TOKEN_OF_SLOT).cpu().numpy(), plan["token_of_slot"])
     np.testing.assert_array_equal(view(sm.WS_COUNT).cpu().numpy(), plan["count"])
     np.testing.assert_array_equal(view(sm.WS_KEPT).cpu().numpy(), plan["kept"])
-    aux_ref, _, _ = so.load_balance_loss(p, gpu_e, cfg.alpha)
     assert abs(float(aux.item()) - aux_ref) <= TOL_ROUTER * aux_ref
 
     # sampled experts: fullest, emptiest non-empty, and a few fixed ones
@@ -71,9 +77,14 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False):
     sample = sorted(sample)
     W_in_s = {i: si.gen_W_in_expert(cfg, i, seed) for i in sample}
     W_out_s = {i: si.gen_W_out_expert(cfg, i, seed) for i in sample}
-    fwd = so.switch_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, router_bias=b_np,
-                            expert_index=gpu_e, experts=sample, residual=residual)
-    bwd = so.switch_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
+    if groups == 1:
+        fwd = so.switch_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, router_bias=b_np,
+                                expert_index=gpu_e, experts=sample, residual=residual)
+        bwd = so.switch_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
+    else:
+        fwd = so.switch_forward_groups(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, groups,
+                                       router_bias=b_np, expert_index=gpu_e, experts=sample, residual=residual)
+        bwd = so.switch_backward_groups(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
     keep = plan["keep"]
     hid = view(sm.WS_H).view(E, C, cfg.d_ff)
     errs = {}
@@ -82,7 +93,7 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False):
         k = tok.size
         assert k == plan["kept"][i]
         tt = torch.from_numpy(tok).cuda()
-        errs[f"H[{i}]"] = rel_err(to_np(hid[i, :k]), np.maximum(fwd["u"][i], 0.0))
+        errs[f"H[{i}]"] = rel_err(to_np(hid[i, :k]), np.maximum(expert_preactivation(fwd, i), 0.0))
         if residual:
             layer_y = view(sm.WS_LAYER_Y).view(T, cfg.d_model)
             errs[f"layer_y[{i}]"] = rel_err(to_np(layer_y[tt]), fwd["layer_y"][tok])
@@ -105,6 +116,7 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False):
     if residual and dropped.numel():
         # a dropped token's dx is dy plus the router's gradient only (checked exactly against the oracle's router)
         some = np.flatnonzero(~keep)[:64]
+        assert groups == 1
         G = np.broadcast_to((cfg.alpha * E / T) * fwd["f"][None, :], (some.size, E))
         dh = p[some] * (G - np.sum(p[some] * G, axis=1, keepdims=True))
         want = dy_np[some].astype(np.float64) + dh @ W_r_np.astype(np.float64).T
@@ -144,3 +156,8 @@ def test_wide_expert_full_size():
 def test_overflow_stress_with_the_skip_path_inside_full_size():
     out = _run_fullsize("stress_calibrated", residual=True)
     assert out["dropped"] > 0.15 * 32768
+
+
+def test_switch_base_in_eight_routing_groups_full_size():
+    out = _run_fullsize("switch_base", groups=8)
+    assert 0.01 * 32768 < out["dropped"] < 0.2 * 32768        # 40 slots per expert and group: overflow is common

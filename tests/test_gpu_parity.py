@@ -12,8 +12,8 @@ import torch
 from oracle import switch_oracle as so
 from paper_2101_03961_b200 import inputs as si
 from paper_2101_03961_b200 import switch_moe as sm
-from tests.gpu_helpers import (TOL_BF16, TOL_F32, TOL_ROUTER, GpuLayer, check_flips, oracle_following, rel_err,
-                               skip_path_ok, to_np)
+from tests.gpu_helpers import (TOL_BF16, TOL_F32, TOL_ROUTER, GpuLayer, check_flips, expert_preactivation,
+                               oracle_following, rel_err, skip_path_ok, to_np)
 
 pytestmark = pytest.mark.gpu
 
@@ -119,15 +119,16 @@ def test_dispatch_plan_is_deterministic():
 
 
 # ---------------------------------------------------------------------------------------------- whole layer
-def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False):
+def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False, groups=1):
     data = si.gen_layer(cfg, seed=seed)
-    g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual)
+    g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual,
+                 groups=groups)
     g.fwd()
     gpu_e = g.expert_index()
     cap = capacity_override if capacity_override else None
-    fwd = oracle_following(cfg, data, gpu_e, capacity=cap, residual=residual)
-    E, C = cfg.E, g.C
-    assert C == fwd["C"]
+    fwd = oracle_following(cfg, data, gpu_e, capacity=cap, residual=residual, groups=groups)
+    assert g.C == fwd["C"]                                     # Eq. 3 for one routing group
+    E, C = cfg.E, g.C * groups                                 # rows per expert in the slot buffers
     # integer state: bit exact
     np.testing.assert_array_equal(g.view(sm.WS_SLOT).cpu().numpy(), fwd["slot"])
     np.testing.assert_array_equal(g.view(sm.WS_COUNT).cpu().numpy(), fwd["count"])
@@ -148,7 +149,7 @@ def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, re
             continue
         tok = fwd["token_of_slot"][i * C:i * C + k]
         np.testing.assert_array_equal(xd[i, :k], x64[tok])
-        errs[f"H[{i}]"] = rel_err(hid[i, :k], np.maximum(fwd["u"][i], 0.0))
+        errs[f"H[{i}]"] = rel_err(hid[i, :k], np.maximum(expert_preactivation(fwd, i), 0.0))
     y = to_np(g.y)
     assert np.isfinite(y).all()
     if residual:
@@ -163,7 +164,8 @@ def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, re
         errs["y"] = rel_err(y, fwd["y"])
 
     g.bwd(d_aux=d_aux)
-    bwd = so.switch_backward(fwd, data["x"], data["W_r"], data["W_in"], data["W_out"], data["dy"], d_aux=d_aux)
+    backward = so.switch_backward_groups if groups > 1 else so.switch_backward
+    bwd = backward(fwd, data["x"], data["W_r"], data["W_in"], data["W_out"], data["dy"], d_aux=d_aux)
     kept_tok = np.flatnonzero(fwd["keep"])
     errs["dgate"] = rel_err(to_np(g.view(sm.WS_DGATE))[kept_tok], bwd["dgate"][kept_tok])
     if residual:
@@ -209,6 +211,29 @@ def test_bf16_layer_on_single_cta_tensor_core_path_matches_oracle(cfg):
 def test_layer_with_the_skip_path_inside_matches_oracle(cfg, path, tol):
     """y = x + g E(x) fused into the combine step, dx = dy + ... fused into the scatter step (Fig. 2, Section 2.2)."""
     _check_layer(cfg, path, tol, residual=True)
+
+
+GROUPED = si.SwitchConfig("grouped", 2048, 128, 256, 8, 1.0, bias_std=0.3)
+GROUPED_F32 = si.SwitchConfig("grouped_f32", 512, 64, 128, 4, 0.75, dtype=si.DTYPE_F32)
+
+
+@pytest.mark.parametrize("cfg,path,tol,groups,residual", [
+    (GROUPED_F32, sm.GEMM_DEFAULT, TOL_F32, 2, False), (GROUPED, sm.GEMM_SIMT, TOL_BF16, 4, False),
+    (GROUPED, sm.GEMM_DEFAULT, TOL_BF16, 2, False), (GROUPED, sm.GEMM_DEFAULT, TOL_BF16, 8, False),
+    (GROUPED, sm.GEMM_TC_1CTA, TOL_BF16, 4, False), (GROUPED, sm.GEMM_DEFAULT, TOL_BF16, 4, True)],
+    ids=["f32_g2", "fma_g4", "tc_g2", "tc_g8", "tc1_g4", "tc_g4_skip"])
+def test_several_routing_groups_in_one_call_match_oracle(cfg, path, tol, groups, residual):
+    """Each group of T / G rows is routed on its own (capacity, f, P), experts shared, loss = mean over groups."""
+    errs = _check_layer(cfg, path, tol, groups=groups, residual=residual, d_aux=0.7)
+    assert errs
+
+
+def test_group_count_limits_are_enforced():
+    for kw in (dict(T=2048, groups=3), dict(T=2048 + 256, groups=2), dict(T=1000, groups=2)):
+        base = dict(T=2048, d_model=128, d_ff=256, E=8, capacity_factor=1.0)
+        base.update(kw)
+        with pytest.raises(sm.SwitchMoeError):
+            sm.switch_moe_workspace_bytes(sm.make_config(**base))
 
 
 def test_skip_path_is_refused_on_the_single_cta_validation_path():

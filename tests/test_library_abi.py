@@ -36,6 +36,9 @@ def test_capacity_follows_eq3(lib):
                         (10, 4, 1.25, 3), (8, 1, 2.0, 8)]:
         assert sm.switch_moe_capacity(sm.make_config(T, 64, 64, E, cf)) == C
     assert sm.switch_moe_capacity(sm.make_config(512, 64, 64, 8, 1.0, capacity_override=17)) == 17
+    # several routing groups: Eq. 3 on the tokens of one group
+    assert sm.switch_moe_capacity(sm.make_config(32768, 768, 3072, 128, 1.25, groups=8)) == 40
+    assert sm.switch_moe_capacity(sm.make_config(2048, 64, 64, 8, 1.0, groups=2)) == 128
 
 
 def test_workspace_size_is_positive_and_grows(lib):
@@ -51,6 +54,10 @@ def test_workspace_size_is_positive_and_grows(lib):
     (dict(E=257), sm.UNSUPPORTED_SHAPE), (dict(d_model=100), sm.UNSUPPORTED_SHAPE),
     (dict(T=4, E=8, capacity_factor=1.0), sm.INVALID_ARGUMENT),          # capacity would be 0
     (dict(dtype=7), sm.INVALID_ARGUMENT),
+    (dict(T=2048, groups=3), sm.INVALID_ARGUMENT),                       # T not a multiple of the group count
+    (dict(T=1000, groups=2), sm.UNSUPPORTED_SHAPE),                      # groups of 500 tokens: not a multiple of 256
+    (dict(T=131072, groups=2), sm.UNSUPPORTED_SHAPE),
+    (dict(T=2048, groups=-1), sm.INVALID_ARGUMENT),
 ])
 def test_bad_configs_are_rejected(lib, kw, status):
     base = dict(T=512, d_model=64, d_ff=256, E=8, capacity_factor=1.0)
