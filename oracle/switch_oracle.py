@@ -101,8 +101,42 @@ def dispatch_plan(e, E: int, C: int):
     return {"pos": pos, "keep": keep, "slot": slot, "token_of_slot": token_of_slot, "count": count, "kept": kept}
 
 
+def second_choice(p, e):
+    """The expert with the second-highest probability of each token: the argmax over the experts other than e_t
+    (lowest index on ties)."""
+    q = np.array(p, dtype=F64, copy=True)
+    q[np.arange(q.shape[0]), e] = -np.inf
+    return np.argmax(q, axis=1).astype(np.int64)
+
+
+def reroute_overflow(plan, e, alt, E: int, C: int):
+    """Stage 2 of No-Token-Left-Behind routing (Appendix B, its figure): every token that overflowed its first
+    expert is offered, in token order, to its second-choice expert `alt[t]` and takes that expert's next free slot
+    if it still has one; tokens kept in stage 1 keep their slots.  Returns the updated plan plus "e_proc", the
+    expert that processes each token (its first choice unless it was rerouted)."""
+    e = np.asarray(e, dtype=np.int64)
+    alt = np.asarray(alt, dtype=np.int64)
+    keep, pos, kept = plan["keep"].copy(), plan["pos"].copy(), plan["kept"].copy()
+    e_proc = e.copy()
+    for t in np.flatnonzero(~plan["keep"]):
+        i = alt[t]
+        if kept[i] < C:
+            pos[t] = kept[i]
+            kept[i] += 1
+            keep[t] = True
+            e_proc[t] = i
+    slot = np.where(keep, e_proc * C + pos, -1)
+    token_of_slot = np.full(E * C, -1, dtype=np.int64)
+    token_of_slot[slot[keep]] = np.flatnonzero(keep)
+    out = dict(plan)
+    out.update({"pos": pos, "keep": keep, "slot": slot, "token_of_slot": token_of_slot, "kept": kept,
+                "e_proc": e_proc, "rerouted": keep & ~plan["keep"]})
+    return out
+
+
 def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None,
-                   capacity: int | None = None, expert_index=None, experts=None, residual: bool = False):
+                   capacity: int | None = None, expert_index=None, experts=None, residual: bool = False,
+                   reroute: bool = False, alt_index=None):
     """Forward of the Switch FFN layer for one routing group.
 
     x [T, d]; W_r [d, E]; W_in [E, d, f]; W_out [E, f, d].  `capacity` overrides Eq. 3 when given.
@@ -113,6 +147,10 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     `residual` adds the layer's input to its output, y_t = x_t + g_t . E_{e_t}(x_t): the residual connection
     around the Switch FFN layer (Fig. 2), through which a dropped token's representation reaches the next
     layer unchanged (Section 2.2).  "layer_y" always holds the output without it.
+    `reroute` adds stage 2 of No-Token-Left-Behind routing (Appendix B): overflowed tokens go to their second-choice
+    expert where it has room, and their gate is that expert's probability (Eq. 2 with the expert that processes the
+    token); f in the auxiliary loss still counts the argmax (Eq. 5).  `alt_index`, when given, replaces the second
+    choice (to follow a legitimate near-tie flip of the device).
     Returns a dict with every intermediate the staged comparisons need.
     """
     x64 = np.asarray(x, dtype=F64)
@@ -128,6 +166,13 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     aux, f, P = load_balance_loss(p, e, alpha)
     C = expert_capacity(T, E, capacity_factor) if capacity is None else int(capacity)
     plan = dispatch_plan(e, E, C)
+    e_proc = e
+    if reroute:
+        alt = second_choice(p, e) if alt_index is None else np.asarray(alt_index, dtype=np.int64)
+        plan = reroute_overflow(plan, e, alt, E, C)
+        e_proc = plan["e_proc"]
+        g = p[np.arange(T), e_proc]
+        plan["alt"] = alt
     keep = plan["keep"]
 
     y = np.zeros((T, d), dtype=F64)
@@ -135,7 +180,7 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     o = np.zeros((T, d), dtype=F64)          # un-gated expert output E_i(x_t); 0 for dropped tokens
     todo = range(E) if experts is None else experts
     for i in todo:
-        tok = np.flatnonzero(keep & (e == i))            # kept tokens of expert i, in token order
+        tok = plan["token_of_slot"][i * C:i * C + int(plan["kept"][i])]   # kept tokens of expert i, in slot order
         if tok.size == 0:
             continue
         u_i = x64[tok] @ np.asarray(W_in[i], dtype=F64)          # h = x W_in
@@ -145,7 +190,8 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
         o[tok] = o_i
         y[tok] = g[tok, None] * o_i                              # Eq. 2 with one selected expert
     out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "layer_y": y,
-           "y": x64 + y if residual else y, "o": o, "u": u, "T": T, "E": E, "alpha": alpha, "residual": bool(residual)}
+           "y": x64 + y if residual else y, "o": o, "u": u, "T": T, "E": E, "alpha": alpha, "residual": bool(residual),
+           "e_proc": e_proc}
     out.update(plan)
     return out
 
@@ -167,8 +213,10 @@ def switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=No
     dgate = np.zeros(T, dtype=F64)
     dW_in, dW_out = {}, {}
     todo = range(E) if experts is None else experts
+    C = fwd["C"]
+    e_proc = fwd["e_proc"]
     for i in todo:
-        tok = np.flatnonzero(keep & (e == i))
+        tok = fwd["token_of_slot"][i * C:i * C + int(fwd["kept"][i])]      # the expert's tokens in slot order
         W_in_i = np.asarray(W_in[i], dtype=F64)
         W_out_i = np.asarray(W_out[i], dtype=F64)
         if tok.size == 0:
@@ -191,7 +239,7 @@ def switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=No
     # (f is piecewise constant, hence no gradient).  aux = alpha . E . sum_i f_i . (1/T) sum_t p[t, i].
     G = np.broadcast_to((d_aux * alpha * E / T) * fwd["f"][None, :], (T, E)).copy()
     kept_tok = np.flatnonzero(keep)
-    G[kept_tok, e[kept_tok]] += dgate[kept_tok]
+    G[kept_tok, e_proc[kept_tok]] += dgate[kept_tok]        # the gate is the probability of the expert that processes the token
     dh = p * (G - np.sum(p * G, axis=1, keepdims=True))     # softmax Jacobian applied to G
     dW_r = x64.T @ dh
     db = dh.sum(axis=0)

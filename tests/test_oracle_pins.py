@@ -495,3 +495,97 @@ def test_grouped_backward_matches_finite_differences():
         num = np.array([fd(arr, i) for i in idxs])
         ana = np.array([grad[i] for i in idxs])
         assert np.linalg.norm(num - ana) / np.linalg.norm(ana) < 1e-7, name
+
+
+# ------------------------------------------------------------------ No-Token-Left-Behind, stage 2 (Appendix B)
+def test_reroute_hand_example():
+    # 6 tokens, 3 experts, capacity 2.  First choices 0 0 0 0 1 2 -> tokens 2, 3 overflow expert 0.  Second choices of
+    # tokens 2 and 3 are experts 1 and 1: expert 1 has one slot left after its own token 4, so token 2 gets it
+    # (token order) and token 3 stays dropped.
+    p = np.array([[.7, .2, .1], [.6, .3, .1], [.5, .3, .2], [.5, .4, .1], [.1, .8, .1], [.2, .1, .7]])
+    e, _ = so.top1(p)
+    plan = so.dispatch_plan(e, 3, 2)
+    alt = so.second_choice(p, e)
+    assert alt.tolist() == [1, 1, 1, 1, 0, 0]
+    out = so.reroute_overflow(plan, e, alt, 3, 2)
+    assert out["keep"].tolist() == [True, True, True, False, True, True]
+    assert out["e_proc"].tolist() == [0, 0, 1, 0, 1, 2]
+    assert out["slot"].tolist() == [0, 1, 3, -1, 2, 4]
+    assert out["kept"].tolist() == [2, 2, 1]
+    assert out["token_of_slot"].tolist() == [0, 1, 4, 2, 5, -1]
+    ties = np.array([[.4, .4, .2], [.2, .4, .4], [.5, .25, .25]])
+    assert so.second_choice(ties, np.array([0, 1, 0])).tolist() == [1, 2, 1]     # ties: lowest index among the others
+
+
+def _reroute_brute_force(p, E, C):
+    """The figure's description, one token at a time: stage 1 for everybody, then stage 2 for the overflowed."""
+    T = p.shape[0]
+    order = np.argsort(-p, axis=1, kind="stable")
+    load = [[] for _ in range(E)]
+    dropped = []
+    for t in range(T):
+        (load[order[t, 0]].append(t) if len(load[order[t, 0]]) < C else dropped.append(t))
+    for t in dropped:
+        if len(load[order[t, 1]]) < C:
+            load[order[t, 1]].append(t)
+    return load
+
+
+@pytest.mark.parametrize("T,E,cf,seed", [(60, 4, 0.75, 0), (80, 8, 1.0, 1), (33, 3, 0.5, 2), (64, 4, 4.0, 3)])
+def test_reroute_matches_brute_force_and_keeps_stage_one(T, E, cf, seed):
+    rng = np.random.default_rng(seed)
+    p = so.router_probs(rng.standard_normal((T, E)) * 2.0 + np.linspace(1.5, 0.0, E))
+    e, _ = so.top1(p)
+    C = so.expert_capacity(T, E, cf)
+    plan = so.dispatch_plan(e, E, C)
+    out = so.reroute_overflow(plan, e, so.second_choice(p, e), E, C)
+    load = _reroute_brute_force(p, E, C)
+    for i in range(E):
+        assert out["token_of_slot"][i * C:i * C + len(load[i])].tolist() == load[i]
+        assert out["kept"][i] == len(load[i]) <= C
+    assert np.array_equal(out["slot"][plan["keep"]], plan["slot"][plan["keep"]])       # stage 1 is untouched
+    assert out["keep"].sum() >= plan["keep"].sum()
+    if cf >= 4.0:
+        assert np.array_equal(out["slot"], plan["slot"])                                # nothing overflowed
+
+
+def test_reroute_layer_gate_and_gradient():
+    T, d, f, E, cf, alpha, d_aux = 18, 5, 8, 3, 0.67, 0.03, 1.1
+    rng = np.random.default_rng(41)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=41, scale=2.0)
+    b = np.array([1.0, 0.0, -0.5])                                       # expert 0 overflows
+    R = rng.standard_normal((T, d))
+    fwd = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_bias=b, reroute=True)
+    plain = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_bias=b)
+    moved = fwd["rerouted"]
+    assert moved.sum() >= 2 and (~fwd["keep"]).sum() < (~plain["keep"]).sum()
+    assert fwd["aux"] == plain["aux"]                                    # f still counts the argmax (Eq. 5)
+    for t in np.flatnonzero(moved):                                      # Eq. 2 with the expert that processes the token
+        i = fwd["e_proc"][t]
+        want = fwd["p"][t, i] * (np.maximum(x[t] @ W_in[i], 0.0) @ W_out[i])
+        np.testing.assert_allclose(fwd["y"][t], want, rtol=1e-12, atol=1e-14)
+        assert i != fwd["e"][t] and fwd["p"][t, i] == np.sort(fwd["p"][t])[-2]
+    stay = plain["keep"]
+    np.testing.assert_array_equal(fwd["y"][stay], plain["y"][stay])
+    # gradients against central differences with the routing frozen
+    srt = np.sort(fwd["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-3 and (srt[:, -2] - srt[:, -3]).min() > 1e-3
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    e_frozen, alt_frozen, eps = fwd["e"], fwd["alt"], 1e-6
+
+    def loss():
+        out = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_bias=b, expert_index=e_frozen, reroute=True,
+                                alt_index=alt_frozen)
+        return float(np.sum(out["y"] * R) + d_aux * out["aux"])
+
+    for name, arr, grad in [("dx", x, bwd["dx"]), ("dW_r", W_r, bwd["dW_r"])]:
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            old = arr[idx]
+            arr[idx] = old + eps
+            lp = loss()
+            arr[idx] = old - eps
+            lm = loss()
+            arr[idx] = old
+            num[idx] = (lp - lm) / (2 * eps)
+        assert np.linalg.norm(num - grad) / np.linalg.norm(grad) < 1e-7, name
