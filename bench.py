@@ -208,7 +208,7 @@ def run_ours(args, cfg):
     bias = None if b_np is None else torch.from_numpy(b_np).cuda()
 
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype,
-                          residual=args.residual, groups=args.groups)
+                          residual=args.residual, groups=args.groups, reroute=args.reroute)
     ws = sm.allocate_workspace(mcfg)
     y, dx = torch.empty_like(x), torch.empty_like(x)
     dW_in, dW_out, dW_r = torch.empty_like(W_in), torch.empty_like(W_out), torch.empty_like(W_r)
@@ -351,7 +351,7 @@ def run_ours(args, cfg):
         "config": {"workload": cfg.name, "T": cfg.T, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "E": cfg.E,
                    "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha, "capacity": sm.switch_moe_capacity(mcfg),
                    "kept_tokens": kept, "parallelism": "replicas" if world > 1 else "single",
-                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups,
+                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute),
                    "l2": "inputs larger than L2 (weights 2 x %.0f MB per pass), no flush" %
                          (cfg.E * cfg.d_model * cfg.d_ff * elt / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": sm.switch_moe_launches_per_step(mcfg) * args.steps,
@@ -377,6 +377,9 @@ def main():
     ap.add_argument("--groups", type=int, default=1,
                     help="route the batch as this many independent groups of T / groups tokens (own capacity and "
                          "loss each, experts shared); the headline configuration is one group")
+    ap.add_argument("--reroute", action="store_true",
+                    help="offer tokens that overflow their expert to their second choice (stage 2 of "
+                         "No-Token-Left-Behind routing); not the headline configuration")
     ap.add_argument("--residual", action="store_true",
                     help="time the variant that adds the layer's input to its output inside the combine step "
                          "(y = x + layer(x), dx = dy + ...); not the headline configuration")

@@ -48,8 +48,13 @@ enum switch_moe_gemm_path {
    input row (Section 2.2: it reaches the next layer through the residual connection).  The backward pass adds dy to
    dx accordingly.  bf16: the expert term is rounded to bf16 before the addition and the sum is rounded again.  The
    forward pass also keeps the output without the skip path in the workspace (SWITCH_MOE_WS_LAYER_Y): the gate's
-   gradient <dy_t, E(x_t)> cannot be recovered from a bf16 y_t - x_t.  Not available on SWITCH_MOE_GEMM_TC_1CTA. */
-enum switch_moe_flags { SWITCH_MOE_FLAG_RESIDUAL = 1 };
+   gradient <dy_t, E(x_t)> cannot be recovered from a bf16 y_t - x_t.  Not available on SWITCH_MOE_GEMM_TC_1CTA.
+   SWITCH_MOE_FLAG_REROUTE: stage 2 of No-Token-Left-Behind routing (Appendix B): after the Switch routing of
+   Section 2.2, every token that overflowed its expert is offered, in token order, to the expert with its
+   second-highest probability and takes that expert's next free slot if one is left; its gate is that expert's
+   probability.  Tokens kept by the first stage keep their slots, and f in the auxiliary loss still counts the
+   argmax.  One routing group only. */
+enum switch_moe_flags { SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2 };
 
 typedef enum switch_moe_status {
   SWITCH_MOE_OK = 0,
@@ -108,7 +113,11 @@ enum switch_moe_ws_region {
   SWITCH_MOE_WS_DLOGITS = 14,       /* float[T,E] gradient of the router logits (backward) */
   SWITCH_MOE_WS_LAYER_Y = 15,       /* [T,d_model] g_t E(x_t) without the skip path (only with SWITCH_MOE_FLAG_RESIDUAL;
                                        rows of dropped tokens are not written) */
-  SWITCH_MOE_WS_REGION_COUNT = 16
+  SWITCH_MOE_WS_EXPERT_PROC = 16,   /* int32[T] the expert that processes the token: e_t unless stage 2 rerouted it
+                                       (only with SWITCH_MOE_FLAG_REROUTE) */
+  SWITCH_MOE_WS_SECOND_CHOICE = 17, /* int32[T] second-choice expert of a token that overflowed in stage 1, -1 for the
+                                       others (only with SWITCH_MOE_FLAG_REROUTE) */
+  SWITCH_MOE_WS_REGION_COUNT = 18
 };
 
 /* Eq. 3.  HOST call.  *C_out = capacity_override if > 0, else floor((T / G) * capacity_factor / E) capped at T / G:

@@ -89,6 +89,12 @@ int switch_moe_workspace_view(const switch_moe_config* cfg, void* workspace, int
     case SWITCH_MOE_WS_DH: off = p.dh; bytes = E * C * s.f * s.elt; break;
     case SWITCH_MOE_WS_DGATE: off = p.dgate; bytes = T * 4; break;
     case SWITCH_MOE_WS_DLOGITS: off = p.dlogits; bytes = T * E * 4; break;
+    case SWITCH_MOE_WS_EXPERT_PROC:
+      if (!s.reroute) return SWITCH_MOE_INVALID_ARGUMENT;
+      off = p.expert_proc; bytes = T * 4; break;
+    case SWITCH_MOE_WS_SECOND_CHOICE:
+      if (!s.reroute) return SWITCH_MOE_INVALID_ARGUMENT;
+      off = p.alt; bytes = T * 4; break;
     case SWITCH_MOE_WS_LAYER_Y:
       if (!s.residual) return SWITCH_MOE_INVALID_ARGUMENT;
       off = p.layer_y; bytes = T * s.d * s.elt; break;
@@ -256,7 +262,8 @@ int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches
   SWMOE_TRY(resolve_shape(cfg, &s));
   // fwd: router, 3 plan kernels, gather, 2 GEMMs; bwd: gather, 4 GEMMs, 4 router-backward kernels.
   // Tensor-core router: forward = operand split, router, column sums; backward = logit gradients, two products, reduce.
-  *launches_out = s.router_tc ? (9 + 9) : (7 + 9);
+  // Rerouting of overflowed tokens adds four plan kernels to the forward pass.
+  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0);
   return SWITCH_MOE_OK;
 }
 

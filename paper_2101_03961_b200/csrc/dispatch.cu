@@ -20,7 +20,8 @@ plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int* __rest
   for (int e = threadIdx.x; e < E; e += blockDim.x) h[e] = 0;
   __syncthreads();
   const int t = blockIdx.x * kPlanBlockTokens + threadIdx.x;
-  if (t < T) atomicAdd(&h[expert_index[t]], 1);              // integer counts: order-independent
+  const int e = t < T ? expert_index[t] : -1;
+  if (e >= 0) atomicAdd(&h[e], 1);                           // integer counts: order-independent; negative = no vote
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) hist[(size_t)blockIdx.x * E + e] = h[e];
 }
@@ -221,6 +222,104 @@ plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__
   }
 }
 
+// ---- stage 2 of No-Token-Left-Behind routing (Appendix B) ----------------------------------------------------
+// alt[t] = the expert with the second-highest probability of an overflowed token (lowest index on ties), -1 for a
+// token that kept its slot.  One warp per token.
+__global__ void __launch_bounds__(256)
+reroute_choice_kernel(const float* __restrict__ probs, const int* __restrict__ expert_index,
+                      const int* __restrict__ slot, int T, int E, int* __restrict__ alt) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= T) return;
+  if (slot[t] >= 0) {
+    if (lane == 0) alt[t] = -1;
+    return;
+  }
+  const int e1 = expert_index[t];
+  float best = -1.f;
+  int arg = 0x7fffffff;
+  for (int e = lane; e < E; e += 32) {
+    const float v = probs[(size_t)t * E + e];
+    if (e != e1 && v > best) { best = v; arg = e; }          // ascending e: the first maximum wins
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+    const int oa = __shfl_xor_sync(0xffffffffu, arg, off);
+    if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+  }
+  if (lane == 0) alt[t] = arg < E ? arg : -1;                  // E == 1: there is no second choice
+}
+
+// Position bases of the second stage: the rerouted tokens of expert e queue up behind its kept[e] first-stage tokens.
+// One thread per expert; also rewrites kept[] and the tile lists for the grown experts.
+__global__ void __launch_bounds__(kMaxExperts)
+reroute_scan_kernel(const int* __restrict__ hist, int plan_blocks, int E, int C, int* __restrict__ hist_base,
+                    int* __restrict__ kept, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
+                    int4* __restrict__ ntile) {
+  pdl_launch_dependents();
+  pdl_wait();
+  __shared__ float term[kMaxExperts];
+  __shared__ int kept_s[kMaxExperts];
+  const int e = threadIdx.x;
+  if (e < E) {
+    int run = kept[e];
+    for (int b0 = 0; b0 < plan_blocks; b0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = b0 + j < plan_blocks ? hist[(size_t)(b0 + j) * E + e] : 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (b0 + j < plan_blocks) { hist_base[(size_t)(b0 + j) * E + e] = run; run += v[j]; }
+    }
+    const int k = min(run, C);
+    kept[e] = k;
+    kept_s[e] = k;
+    term[e] = 0.f;
+  }
+  write_tile_lists(term, kept_s, E, 0.f, nullptr, tile_expert, tile_row0, ntile);
+}
+
+// Slots of the rerouted tokens (same stable in-block rank as the first stage), their gate (the probability of the
+// expert that now processes them, Eq. 2) and, for every token, the expert that processes it.
+__global__ void __launch_bounds__(kPlanBlockTokens)
+reroute_assign_kernel(const int* __restrict__ alt, const int* __restrict__ expert_index,
+                      const int* __restrict__ hist_base, const float* __restrict__ probs, int T, int E, int C,
+                      int* __restrict__ slot, int* __restrict__ token_of_slot, float* __restrict__ gate,
+                      int* __restrict__ expert_proc) {
+  pdl_launch_dependents();
+  pdl_wait();
+  __shared__ int warp_cnt[kPlanBlockTokens / 32][kMaxExperts];
+  constexpr int kWarps = kPlanBlockTokens / 32;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  for (int i = tid; i < kWarps * kMaxExperts; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
+  __syncthreads();
+  const int t = blockIdx.x * kPlanBlockTokens + tid;
+  const int a = t < T ? alt[t] : -1;
+  const int key = a >= 0 ? a : -1 - lane;                     // distinct dummies for tokens that do not move
+  const unsigned same = __match_any_sync(0xffffffffu, key);
+  const int rank = __popc(same & ((1u << lane) - 1u));
+  if (a >= 0 && rank == 0) warp_cnt[warp][a] = __popc(same);
+  __syncthreads();
+  if (t < T) {
+    int proc = expert_index[t];
+    if (a >= 0) {
+      int pos = hist_base[(size_t)blockIdx.x * E + a] + rank;
+      for (int w = 0; w < warp; ++w) pos += warp_cnt[w][a];
+      if (pos < C) {
+        const int s = a * C + pos;
+        slot[t] = s;
+        token_of_slot[s] = t;
+        gate[t] = probs[(size_t)t * E + a];
+        proc = a;
+      }
+    }
+    expert_proc[t] = proc;
+  }
+}
+
 // Forward gather.  Part 1 (blockIdx.x < slot_blocks): one warp per slot row; kept slots copy the token's row
 // with 128-bit loads and stores, slots in [kept_i, roundup(kept_i, kTileM)) are zero-filled so that tensor-core
 // tiles never read stale rows.  Part 2: one warp per token; dropped tokens get a zero output row (their
@@ -353,6 +452,19 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
   launch_k(plan_assign_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, ws_ptr<int>(ws, p.hist_base),
            ws_ptr<int>(ws, p.kept), group_base, blocks_per_group, s.T, s.E, s.C, s.Cg, ws_ptr<int>(ws, p.slot),
            ws_ptr<int>(ws, p.token_of_slot));
+  if (s.reroute) {
+    int* alt = ws_ptr<int>(ws, p.alt);
+    launch_k(reroute_choice_kernel, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs), ei,
+             ws_ptr<int>(ws, p.slot), s.T, s.E, alt);
+    launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, alt, s.T, s.E,
+             ws_ptr<int>(ws, p.hist));
+    launch_k(reroute_scan_kernel, dim3(1), dim3(kMaxExperts), 0, st, ws_ptr<int>(ws, p.hist), s.plan_blocks, s.E, s.C,
+             ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.kept), ws_ptr<int>(ws, p.tile_expert),
+             ws_ptr<int>(ws, p.tile_row0), ws_ptr<int4>(ws, p.ntile));
+    launch_k(reroute_assign_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, alt, ei,
+             ws_ptr<int>(ws, p.hist_base), ws_ptr<float>(ws, p.probs), s.T, s.E, s.C, ws_ptr<int>(ws, p.slot),
+             ws_ptr<int>(ws, p.token_of_slot), ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.expert_proc));
+  }
   return launch_status();
 }
 

@@ -390,7 +390,7 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
   const float cG = (float)((double)d_aux * (double)s.alpha * (double)s.E / ((double)s.T * (double)s.Tg));
   float* dlogits = ws_ptr<float>(ws, p.dlogits);
   launch_k(router_dlogits_kernel<NE>, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs),
-                                                            ws_ptr<int>(ws, p.expert_index), ws_ptr<int>(ws, p.slot),
+                                                            ws_ptr<int>(ws, p.expert_proc), ws_ptr<int>(ws, p.slot),
                                                             ws_ptr<int>(ws, p.count_g), dgate, cG, s.T, s.Tg, s.E, dlogits,
                                                             (s.router_tc && sizeof(XT) == 2)
                                                                 ? ws_ptr<__nv_bfloat16>(ws, p.dhsplit) : nullptr,

@@ -31,12 +31,13 @@ struct Shape {
   int router_tc;    // 1: router on the tensor cores (bf16 x, 3-way bf16 split of fp32 operands); 0: FP32 FMA
   int router_blocks, plan_blocks, max_mtiles, dwr_chunks;
   int residual;     // 1: y = x + layer(x), dx = dy + d layer / dx (SWITCH_MOE_FLAG_RESIDUAL)
+  int reroute;      // 1: overflowed tokens are offered to their second-choice expert (SWITCH_MOE_FLAG_REROUTE)
 };
 
 // Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
 struct Plan {
   size_t status, expert_index, gate, slot, token_of_slot, count, kept, count_g, group_base, psum, psum_partial, hist, hist_base,
-      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, layer_y, total;
+      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, layer_y, alt, expert_proc, total;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -57,7 +58,7 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (cfg->T % G != 0) return SWITCH_MOE_INVALID_ARGUMENT;
   if (G > 1 && ((cfg->T / G) % kPlanBlockTokens != 0 || cfg->T > 65536 || G > kMaxGroups))
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
-  if ((cfg->flags & ~SWITCH_MOE_FLAG_RESIDUAL) != 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if ((cfg->flags & ~(SWITCH_MOE_FLAG_RESIDUAL | SWITCH_MOE_FLAG_REROUTE)) != 0) return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->E > kMaxExperts) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if (cfg->d_model % 8 != 0 || cfg->d_ff % 8 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   s->T = cfg->T; s->d = cfg->d_model; s->f = cfg->d_ff; s->E = cfg->E;
@@ -79,6 +80,8 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (s->gemm_path != 1 && (cfg->d_model % 64 != 0 || cfg->d_ff % 64 != 0)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   s->residual = (cfg->flags & SWITCH_MOE_FLAG_RESIDUAL) ? 1 : 0;
   if (s->residual && s->gemm_path == SWITCH_MOE_GEMM_TC_1CTA) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->reroute = (cfg->flags & SWITCH_MOE_FLAG_REROUTE) ? 1 : 0;
+  if (s->reroute && G > 1) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   int ne = (cfg->E + 31) / 32;
   int ne_pow2 = 1;
   while (ne_pow2 < ne) ne_pow2 *= 2;
@@ -137,6 +140,8 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->dhsplit = take(3 * T * (size_t)s.Epad64 * 2);
   p->hmask = take(E * C * ((f + 31) / 32) * 4);            // one bit per element of H: [H > 0]
   p->layer_y = s.residual ? take(T * d * s.elt) : 0;       // g . E(x) without the skip path (for the gate's gradient)
+  p->alt = s.reroute ? take(T * 4) : 0;                     // second choice of overflowed tokens, -1 for the others
+  p->expert_proc = s.reroute ? take(T * 4) : p->expert_index;   // the expert that processes each token
   p->total = off;
 }
 

@@ -23,8 +23,8 @@ OK = 0
 INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, CUDA_ERROR, DEVICE_TIMEOUT = -1, -2, -3, -4, -5
 
 WS_STATUS, WS_EXPERT_INDEX, WS_GATE, WS_SLOT, WS_TOKEN_OF_SLOT, WS_COUNT, WS_KEPT, WS_PSUM, WS_PROBS, WS_XD, WS_H, \
-    WS_DYD, WS_DH, WS_DGATE, WS_DLOGITS, WS_LAYER_Y = range(16)
-FLAG_RESIDUAL = 1
+    WS_DYD, WS_DH, WS_DGATE, WS_DLOGITS, WS_LAYER_Y, WS_EXPERT_PROC, WS_SECOND_CHOICE = range(18)
+FLAG_RESIDUAL, FLAG_REROUTE = 1, 2
 
 EXPORTED_SYMBOLS = [
     "switch_moe_capacity", "switch_moe_workspace_bytes", "switch_moe_workspace_view", "switch_moe_fwd",
@@ -89,12 +89,12 @@ def load_library() -> ctypes.CDLL:
 
 
 def make_config(T, d_model, d_ff, E, capacity_factor, alpha=0.01, dtype=BF16, capacity_override=0,
-                gemm_path=GEMM_DEFAULT, residual=False, groups=1) -> SwitchMoeConfig:
+                gemm_path=GEMM_DEFAULT, residual=False, groups=1, reroute=False) -> SwitchMoeConfig:
     cfg = SwitchMoeConfig()
     cfg.T, cfg.d_model, cfg.d_ff, cfg.E = int(T), int(d_model), int(d_ff), int(E)
     cfg.capacity_factor, cfg.alpha = float(capacity_factor), float(alpha)
     cfg.capacity_override, cfg.dtype, cfg.gemm_path = int(capacity_override), int(dtype), int(gemm_path)
-    cfg.flags = FLAG_RESIDUAL if residual else 0
+    cfg.flags = (FLAG_RESIDUAL if residual else 0) | (FLAG_REROUTE if reroute else 0)
     cfg.groups = int(groups)
     return cfg
 
@@ -158,7 +158,8 @@ def allocate_workspace(cfg: SwitchMoeConfig, device="cuda") -> torch.Tensor:
 _REGION_DTYPES = {
     WS_STATUS: torch.int32, WS_EXPERT_INDEX: torch.int32, WS_GATE: torch.float32, WS_SLOT: torch.int32,
     WS_TOKEN_OF_SLOT: torch.int32, WS_COUNT: torch.int32, WS_KEPT: torch.int32, WS_PSUM: torch.float32,
-    WS_PROBS: torch.float32, WS_DGATE: torch.float32, WS_DLOGITS: torch.float32,
+    WS_PROBS: torch.float32, WS_DGATE: torch.float32, WS_DLOGITS: torch.float32, WS_EXPERT_PROC: torch.int32,
+    WS_SECOND_CHOICE: torch.int32,
 }
 
 

@@ -42,12 +42,12 @@ class GpuLayer:
     """Device buffers of one layer call plus the library calls on them."""
 
     def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0,
-                 residual=False, groups=1):
+                 residual=False, groups=1, reroute=False):
         sbuild.build()
         self.scfg = cfg
         self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
                                   dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path,
-                                  residual=residual, groups=groups)
+                                  residual=residual, groups=groups, reroute=reroute)
         dt = cfg.dtype
         self.x = to_dev(data["x"], dt)
         self.dy = to_dev(data["dy"], dt)
@@ -98,8 +98,21 @@ def check_flips(gpu_e: np.ndarray, ora: dict) -> int:
     return int(diff.size)
 
 
+def check_second_choice(gpu_alt: np.ndarray, p: np.ndarray, e: np.ndarray, overflowed: np.ndarray) -> np.ndarray:
+    """The device's second choice of every overflowed token must be the oracle's, except where the second and third
+    probabilities are closer than FLIP_GAP; tokens that kept their slot carry -1.  Returns the choices to follow."""
+    want = so.second_choice(p, e)
+    assert np.all(gpu_alt[~overflowed] == -1)
+    diff = np.flatnonzero(overflowed & (gpu_alt != want))
+    if diff.size:
+        assert np.all(gpu_alt[diff] != e[diff]) and np.all(gpu_alt[diff] >= 0)
+        gap = p[diff, want[diff]] - p[diff, gpu_alt[diff]]
+        assert np.all(np.abs(gap) < FLIP_GAP), f"{diff.size} second-choice flips, largest gap {np.abs(gap).max():.3e}"
+    return np.where(overflowed, gpu_alt, want)
+
+
 def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capacity=None, experts=None,
-                     residual=False, groups=1):
+                     residual=False, groups=1, gpu_alt=None):
     """Oracle forward with the device's expert choice (identical unless a near-tie flipped), after checking flips."""
     if groups > 1:
         assert capacity is None
@@ -114,9 +127,15 @@ def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capaci
     first = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                               router_bias=data.get("router_bias"), capacity=capacity, experts=[])
     flips = check_flips(gpu_e, first)
+    alt = None
+    if gpu_alt is not None:                                   # stage 2 of No-Token-Left-Behind routing
+        stage1 = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
+                                   cfg.alpha, router_bias=data.get("router_bias"), capacity=capacity,
+                                   expert_index=gpu_e, experts=[])
+        alt = check_second_choice(gpu_alt, stage1["p"], gpu_e, ~stage1["keep"])
     fwd = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                             router_bias=data.get("router_bias"), capacity=capacity, expert_index=gpu_e,
-                            experts=experts, residual=residual)
+                            experts=experts, residual=residual, reroute=gpu_alt is not None, alt_index=alt)
     fwd["flips"] = flips
     return fwd
 

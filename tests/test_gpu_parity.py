@@ -119,14 +119,19 @@ def test_dispatch_plan_is_deterministic():
 
 
 # ---------------------------------------------------------------------------------------------- whole layer
-def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False, groups=1):
+def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False, groups=1,
+                 reroute=False):
     data = si.gen_layer(cfg, seed=seed)
     g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual,
-                 groups=groups)
+                 groups=groups, reroute=reroute)
     g.fwd()
     gpu_e = g.expert_index()
     cap = capacity_override if capacity_override else None
-    fwd = oracle_following(cfg, data, gpu_e, capacity=cap, residual=residual, groups=groups)
+    gpu_alt = g.view(sm.WS_SECOND_CHOICE).cpu().numpy().astype(np.int64) if reroute else None
+    fwd = oracle_following(cfg, data, gpu_e, capacity=cap, residual=residual, groups=groups, gpu_alt=gpu_alt)
+    if reroute:
+        np.testing.assert_array_equal(g.view(sm.WS_EXPERT_PROC).cpu().numpy(), fwd["e_proc"])
+        np.testing.assert_allclose(to_np(g.view(sm.WS_GATE))[fwd["keep"]], fwd["g"][fwd["keep"]], rtol=2e-5)
     assert g.C == fwd["C"]                                     # Eq. 3 for one routing group
     E, C = cfg.E, g.C * groups                                 # rows per expert in the slot buffers
     # integer state: bit exact
@@ -234,6 +239,29 @@ def test_group_count_limits_are_enforced():
         base.update(kw)
         with pytest.raises(sm.SwitchMoeError):
             sm.switch_moe_workspace_bytes(sm.make_config(**base))
+
+
+OVERFLOW = si.SwitchConfig("overflow", 2048, 128, 256, 8, 1.0, bias_std=0.5)
+OVERFLOW_F32 = si.SwitchConfig("overflow_f32", 512, 64, 128, 4, 0.75, dtype=si.DTYPE_F32, bias_std=0.5)
+
+
+@pytest.mark.parametrize("cfg,path,tol,residual", [
+    (OVERFLOW_F32, sm.GEMM_DEFAULT, TOL_F32, False), (OVERFLOW, sm.GEMM_SIMT, TOL_BF16, False),
+    (OVERFLOW, sm.GEMM_DEFAULT, TOL_BF16, False), (MANY, sm.GEMM_DEFAULT, TOL_BF16, False),
+    (RAGGED, sm.GEMM_TC_1CTA, TOL_BF16, False), (OVERFLOW, sm.GEMM_DEFAULT, TOL_BF16, True)],
+    ids=["f32", "fma", "tc", "many_tc", "ragged_tc1", "tc_skip"])
+def test_rerouting_of_overflowed_tokens_matches_oracle(cfg, path, tol, residual):
+    """Stage 2 of No-Token-Left-Behind routing (Appendix B): overflow goes to the second choice where it has room."""
+    data = si.gen_layer(cfg, seed=0)
+    plain = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
+                              router_bias=data.get("router_bias"), experts=[])
+    assert (~plain["keep"]).sum() > 0.03 * cfg.T               # the case does overflow
+    _check_layer(cfg, path, tol, reroute=True, residual=residual, d_aux=0.7)
+
+
+def test_rerouting_is_refused_with_several_routing_groups():
+    with pytest.raises(sm.SwitchMoeError):
+        sm.switch_moe_workspace_bytes(sm.make_config(2048, 128, 256, 8, 1.0, groups=2, reroute=True))
 
 
 def test_skip_path_is_refused_on_the_single_cta_validation_path():
