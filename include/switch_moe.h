@@ -89,6 +89,11 @@ typedef struct switch_moe_config {
                                 plan, 2 gather, 3 GEMM1+ReLU, 4 GEMM2+combine) and event 5 after the last one; bwd
                                 records events 6..11 before (6 gather dy, 7 dgrad2, 8 wgrad2, 9 dgrad1, 10 wgrad1,
                                 11 router backward) and event 12 after.  For per-kernel timing only. */
+  const float* router_noise; /* DEVICE float[T, E] added to the router logits before the softmax, or NULL (default).
+                                The router pseudo-code of the appendix adds uniform(1 - eps, 1 + eps) noise to the
+                                logits in training (the text instead speaks of multiplicative jitter on the router's
+                                input; this field follows the pseudo-code).  The noise is an input, drawn by the
+                                caller; it is a constant of the backward pass. */
 } switch_moe_config;
 
 #define SWITCH_MOE_STAGE_EVENTS 13

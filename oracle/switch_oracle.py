@@ -27,7 +27,9 @@ Readings taken where the paper is silent or its listing is garbled (each is chec
   * one call is one routing group; the row order of x is the token order;
   * ReLU'(0) = 0;
   * an optional constant per-expert bias may be added to the logits (used by the overflow-stress
-    workload only; the paper's router has none).
+    workload only; the paper's router has none);
+  * exploration noise follows the router pseudo-code (added to the logits), not the text's multiplicative
+    jitter of the router input; it is passed in, never drawn here.
 
 All functions here are pinned by tests/test_oracle_pins.py: none is "parity unpinned".
 """
@@ -46,11 +48,17 @@ def expert_capacity(T: int, E: int, capacity_factor: float) -> int:
     return min(C, T)
 
 
-def router_logits(x, W_r, router_bias=None):
-    """Section 2.1: h(x) = W_r . x for every token; x [T, d], W_r [d, E] -> h [T, E] (float64)."""
+def router_logits(x, W_r, router_bias=None, router_noise=None):
+    """Section 2.1: h(x) = W_r . x for every token; x [T, d], W_r [d, E] -> h [T, E] (float64).
+
+    `router_noise` [T, E], when given, is added to the logits: the appendix's router pseudo-code adds
+    uniform(1 - eps, 1 + eps) noise to the logits in training "for exploration across experts".  It is an input
+    here (the caller draws it) and a constant of the backward pass."""
     h = np.asarray(x, dtype=F64) @ np.asarray(W_r, dtype=F64)
     if router_bias is not None:
         h = h + np.asarray(router_bias, dtype=F64)[None, :]
+    if router_noise is not None:
+        h = h + np.asarray(router_noise, dtype=F64)
     return h
 
 
@@ -136,7 +144,7 @@ def reroute_overflow(plan, e, alt, E: int, C: int):
 
 def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None,
                    capacity: int | None = None, expert_index=None, experts=None, residual: bool = False,
-                   reroute: bool = False, alt_index=None):
+                   reroute: bool = False, alt_index=None, router_noise=None):
     """Forward of the Switch FFN layer for one routing group.
 
     x [T, d]; W_r [d, E]; W_in [E, d, f]; W_out [E, f, d].  `capacity` overrides Eq. 3 when given.
@@ -156,7 +164,7 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     x64 = np.asarray(x, dtype=F64)
     T, d = x64.shape
     E = np.asarray(W_r).shape[1]
-    h = router_logits(x64, W_r, router_bias)
+    h = router_logits(x64, W_r, router_bias, router_noise)
     p = router_probs(h)
     if expert_index is None:
         e, g = top1(p)

@@ -111,7 +111,8 @@ int switch_moe_router_fwd(const switch_moe_config* cfg, const void* x, const flo
   SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
   if (x == nullptr || W_r == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
   if (!aligned16(x) || !aligned16(W_r)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
-  return launch_router_fwd(c.s, c.p, x, W_r, router_bias, workspace, static_cast<cudaStream_t>(stream));
+  return launch_router_fwd(c.s, c.p, x, W_r, router_bias, cfg->router_noise, workspace,
+                           static_cast<cudaStream_t>(stream));
 }
 
 int switch_moe_dispatch_plan(const switch_moe_config* cfg, const int32_t* expert_index, float* aux_loss,
@@ -132,7 +133,7 @@ int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ws_ptr<char>(workspace, c.p.status), 0, 16 * 4, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
   SWMOE_TRY(mark(cfg, 0, st));
-  SWMOE_TRY(launch_router_fwd(c.s, c.p, x, W_r, router_bias, workspace, st));
+  SWMOE_TRY(launch_router_fwd(c.s, c.p, x, W_r, router_bias, cfg->router_noise, workspace, st));
   SWMOE_TRY(mark(cfg, 1, st));
   SWMOE_TRY(launch_dispatch_plan(c.s, c.p, nullptr, aux_loss, workspace, st));
   SWMOE_TRY(mark(cfg, 2, st));

@@ -39,7 +39,8 @@ __device__ __forceinline__ void load16_as_f32(const XT* src, float* dst) {
 // ------------------------------------------------------------------------------------------------ forward
 template <typename XT, int NE>
 __global__ void __launch_bounds__(kFwdThreads)
-router_fwd_kernel(const XT* __restrict__ x, const float* __restrict__ W_r, const float* __restrict__ bias, int T, int d,
+router_fwd_kernel(const XT* __restrict__ x, const float* __restrict__ W_r, const float* __restrict__ bias,
+                  const float* __restrict__ noise, int T, int d,
                   int E, float* __restrict__ probs, int* __restrict__ expert_index, float* __restrict__ gate,
                   float* __restrict__ psum_partial) {
   pdl_launch_dependents();
@@ -120,7 +121,8 @@ router_fwd_kernel(const XT* __restrict__ x, const float* __restrict__ W_r, const
 #pragma unroll
     for (int n = 0; n < NE; ++n) {
       const int e = lane * NE + n;
-      const float h = e < E ? acc[j][n] + bv[n] : -INFINITY;
+      float h = e < E ? acc[j][n] + bv[n] : -INFINITY;
+      if (noise != nullptr && e < E && t < T) h += noise[(size_t)t * E + e];   // exploration noise on the logits
       acc[j][n] = h;
       if (h > m) { m = h; am = e; }                          // ascending e: first maximum wins
     }
@@ -374,10 +376,11 @@ router_dx_kernel(const float* __restrict__ dlogits, const float* __restrict__ W_
 }
 
 template <typename XT, int NE>
-int router_fwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
+int router_fwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias,
+                 const float* noise, void* ws,
                  cudaStream_t st) {
   launch_k(router_fwd_kernel<XT, NE>, dim3(s.router_blocks), dim3(kFwdThreads), 0, st, 
-      static_cast<const XT*>(x), W_r, bias, s.T, s.d, s.E, ws_ptr<float>(ws, p.probs),
+      static_cast<const XT*>(x), W_r, bias, noise, s.T, s.d, s.E, ws_ptr<float>(ws, p.probs),
       ws_ptr<int>(ws, p.expert_index), ws_ptr<float>(ws, p.gate), ws_ptr<float>(ws, p.psum_partial));
   return launch_status();
 }
@@ -430,10 +433,11 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
     default: return SWITCH_MOE_UNSUPPORTED_SHAPE;                                         \
   }
 
-int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
+int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias,
+                      const float* noise, void* ws,
                       cudaStream_t st) {
-  if (s.router_tc && s.dtype == SWITCH_MOE_BF16) return launch_router_tc_fwd(s, p, x, W_r, bias, ws, st);
-  SWMOE_DISPATCH_NE(router_fwd_t, s, p, x, W_r, bias, ws, st)
+  if (s.router_tc && s.dtype == SWITCH_MOE_BF16) return launch_router_tc_fwd(s, p, x, W_r, bias, noise, ws, st);
+  SWMOE_DISPATCH_NE(router_fwd_t, s, p, x, W_r, bias, noise, ws, st)
 }
 
 int launch_router_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* dgate, float d_aux,

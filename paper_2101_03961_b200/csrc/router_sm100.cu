@@ -33,7 +33,7 @@ struct RouterTcParams {
   int n_mtiles, n_ntiles;
   int splits, chunk_kblocks, total_kblocks;   // dwr: split of the token contraction
   int wrap;                  // k-blocks per part: d/64 (fwd), Epad64/64 (dx); dwr derives it per tile
-  const float* bias; float* probs; int* expert_index; float* gate;   // fwd
+  const float* bias; const float* noise; float* probs; int* expert_index; float* gate;   // fwd
   float* partial;                                                                         // dwr
   __nv_bfloat16* dx; const int* slot; int accumulate;                                     // dx
   int* status;
@@ -222,6 +222,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ---- Eq. 1 softmax, top-1 (lowest index on ties) and gate for token m0 + r; all E logits are in this lane
         const int tok = t.m0 + r;
         const int nch = p.mma_n / 32;
+        const float* nrow = (p.noise != nullptr && tok < p.T) ? p.noise + (size_t)tok * p.E : nullptr;
+        auto addend = [&](int e) { return (p.bias ? p.bias[e] : 0.f) + (nrow ? nrow[e] : 0.f); };
         float m = -INFINITY;
         int am = 0;
         for (int c = 0; c < nch; ++c) {
@@ -232,7 +234,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           for (int i = 0; i < 32; ++i) {
             const int e = c * 32 + i;
             if (e < p.E) {
-              const float h = __uint_as_float(v[i]) + (p.bias ? p.bias[e] : 0.f);
+              const float h = __uint_as_float(v[i]) + addend(e);
               if (h > m) { m = h; am = e; }
             }
           }
@@ -245,7 +247,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const int e = c * 32 + i;
-            if (e < p.E) sum += expf(__uint_as_float(v[i]) + (p.bias ? p.bias[e] : 0.f) - m);
+            if (e < p.E) sum += expf(__uint_as_float(v[i]) + addend(e) - m);
           }
         }
         const float inv = 1.f / sum;
@@ -265,7 +267,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           for (int i = 0; i < 32; ++i) {
             const int e = c * 32 + i;
             pr[i] = (e < p.E && tok < p.T)
-                        ? expf(__uint_as_float(v[i]) + (p.bias ? p.bias[e] : 0.f) - m) * inv : 0.f;
+                        ? expf(__uint_as_float(v[i]) + addend(e) - m) * inv : 0.f;
           }
           if (tok < p.T) {
             float* dst = p.probs + (size_t)tok * p.E + c * 32;
@@ -394,7 +396,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // through a 32x32 shared-memory transpose so that global stores are 128-byte rows.
 struct RouterFwdParams {
   int T, d, E, Epad64, n_mtiles, k_blocks, b_atoms, stages, stage_bytes;
-  const float* bias; float* probs; int* expert_index; float* gate;
+  const float* bias; const float* noise; float* probs; int* expert_index; float* gate;
   int* status;
 };
 constexpr int kRFRingBytes = kStages * kStageBytes;            // 192 KB of operand stages
@@ -534,6 +536,12 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         for (int e = 0; e < NCH * 32; ++e)
           if (e < p.E) h[e] += p.bias[e];
       }
+      if (p.noise != nullptr && tok < p.T) {                  // exploration noise on the logits (an input)
+        const float* nrow = p.noise + (size_t)tok * p.E;
+#pragma unroll
+        for (int e = 0; e < NCH * 32; ++e)
+          if (e < p.E) h[e] += nrow[e];
+      }
       float mq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       int aq[4] = {0, 1, 2, 3};
 #pragma unroll
@@ -651,7 +659,8 @@ int launch_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const RouterTcPara
 
 }  // namespace
 
-int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
+int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias,
+                         const float* noise, void* ws,
                          cudaStream_t st) {
   __nv_bfloat16* wsplit = ws_ptr<__nv_bfloat16>(ws, p.wsplit);
   const size_t n = (size_t)s.d * s.Epad64;
@@ -668,7 +677,7 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
     q.b_atoms = s.Epad64 / 64;
     q.stage_bytes = kABytes + 3 * q.b_atoms * kAtomBytes;
     q.stages = kRFRingBytes / q.stage_bytes < kStages ? kRFRingBytes / q.stage_bytes : kStages;
-    q.bias = bias; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
+    q.bias = bias; q.noise = noise; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
     q.gate = ws_ptr<float>(ws, p.gate); q.status = ws_ptr<int>(ws, p.status);
     if (s.Epad64 == 64) {
       if (cudaFuncSetAttribute(router_fwd_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
@@ -686,7 +695,7 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
     RouterTcParams q{};
     q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.mma_n = s.Epad64;
     q.n_mtiles = n_mtiles; q.n_ntiles = 1; q.wrap = s.d / kBK;
-    q.bias = bias; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
+    q.bias = bias; q.noise = noise; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
     q.gate = ws_ptr<float>(ws, p.gate); q.status = ws_ptr<int>(ws, p.status);
     rc = launch_op<kRFwd>(tmA, tmB, q, st);
   }

@@ -189,8 +189,8 @@ inline int launch_status() {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---- kernels' host launchers (each returns a switch_moe_status) ----------------------------------------
-int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
-                      cudaStream_t st);
+int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias,
+                      const float* noise, void* ws, cudaStream_t st);
 int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_index, float* aux_loss, void* ws,
                          cudaStream_t st);
 int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void* ws, cudaStream_t st);
@@ -199,8 +199,8 @@ int launch_router_bwd(const Shape& s, const Plan& p, const void* x, const float*
                       void* ws, void* dx, bool accumulate_dx, float* dW_r, cudaStream_t st);
 
 // Tensor-core router (bf16 x): forward (logits, softmax, top-1, gate, P-sum partials) and the two backward products.
-int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias, void* ws,
-                         cudaStream_t st);
+int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias,
+                         const float* noise, void* ws, cudaStream_t st);
 int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, void* ws, void* dx,
                          bool accumulate_dx, cudaStream_t st);
 

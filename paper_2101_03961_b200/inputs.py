@@ -24,7 +24,7 @@ import numpy as np
 DTYPE_BF16 = 0
 DTYPE_F32 = 1
 
-_TENSOR_X, _TENSOR_DY, _TENSOR_WR, _TENSOR_WIN, _TENSOR_WOUT, _TENSOR_BIAS = 1, 2, 3, 4, 5, 6
+_TENSOR_X, _TENSOR_DY, _TENSOR_WR, _TENSOR_WIN, _TENSOR_WOUT, _TENSOR_BIAS, _TENSOR_NOISE = 1, 2, 3, 4, 5, 6, 7
 
 
 @dataclass(frozen=True)
@@ -127,6 +127,13 @@ def gen_router_bias(cfg: SwitchConfig, seed: int = 0):
     if cfg.bias_std == 0.0:
         return None
     return (_normal(_rng(seed, _TENSOR_BIAS), (cfg.E,)) * np.float32(cfg.bias_std)).astype(np.float32)
+
+
+def gen_router_noise(cfg: SwitchConfig, eps: float, seed: int = 0) -> np.ndarray:
+    """Exploration noise for the router logits [T, E], uniform in [1 - eps, 1 + eps), float32 (an input of the
+    layer: the library and the oracle are both handed this array)."""
+    u = _rng(seed, _TENSOR_NOISE).random((cfg.T, cfg.E), dtype=np.float32)
+    return (np.float32(1.0 - eps) + np.float32(2.0 * eps) * u).astype(np.float32)
 
 
 def gen_W_in_expert(cfg: SwitchConfig, e: int, seed: int = 0) -> np.ndarray:

@@ -43,6 +43,7 @@ class SwitchMoeConfig(ctypes.Structure):
         ("capacity_override", ctypes.c_int32), ("dtype", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
         ("flags", ctypes.c_int32), ("groups", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
         ("stage_events", ctypes.POINTER(ctypes.c_void_p)),
+        ("router_noise", ctypes.c_void_p),
     ]
 
 

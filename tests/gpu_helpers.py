@@ -54,6 +54,10 @@ class GpuLayer:
         self.W_r = torch.from_numpy(np.ascontiguousarray(data["W_r"], dtype=np.float32)).cuda()
         b = data.get("router_bias")
         self.bias = None if b is None else torch.from_numpy(np.ascontiguousarray(b, dtype=np.float32)).cuda()
+        n = data.get("router_noise")
+        self.noise = None if n is None else torch.from_numpy(np.ascontiguousarray(n, dtype=np.float32)).cuda()
+        if self.noise is not None:
+            self.cfg.router_noise = self.noise.data_ptr()
         self.W_in = to_dev(data["W_in"], dt)
         self.W_out = to_dev(data["W_out"], dt)
         tdt = torch.bfloat16 if dt == sm.BF16 else torch.float32
@@ -125,17 +129,19 @@ def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capaci
         fwd["flips"] = flips
         return fwd
     first = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
-                              router_bias=data.get("router_bias"), capacity=capacity, experts=[])
+                              router_bias=data.get("router_bias"), capacity=capacity, experts=[],
+                              router_noise=data.get("router_noise"))
     flips = check_flips(gpu_e, first)
     alt = None
     if gpu_alt is not None:                                   # stage 2 of No-Token-Left-Behind routing
         stage1 = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
                                    cfg.alpha, router_bias=data.get("router_bias"), capacity=capacity,
-                                   expert_index=gpu_e, experts=[])
+                                   expert_index=gpu_e, experts=[], router_noise=data.get("router_noise"))
         alt = check_second_choice(gpu_alt, stage1["p"], gpu_e, ~stage1["keep"])
     fwd = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                             router_bias=data.get("router_bias"), capacity=capacity, expert_index=gpu_e,
-                            experts=experts, residual=residual, reroute=gpu_alt is not None, alt_index=alt)
+                            experts=experts, residual=residual, reroute=gpu_alt is not None, alt_index=alt,
+                            router_noise=data.get("router_noise"))
     fwd["flips"] = flips
     return fwd
 

@@ -120,8 +120,10 @@ def test_dispatch_plan_is_deterministic():
 
 # ---------------------------------------------------------------------------------------------- whole layer
 def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False, groups=1,
-                 reroute=False):
+                 reroute=False, noise_eps=0.0):
     data = si.gen_layer(cfg, seed=seed)
+    if noise_eps:
+        data["router_noise"] = si.gen_router_noise(cfg, noise_eps, seed)
     g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual,
                  groups=groups, reroute=reroute)
     g.fwd()
@@ -257,6 +259,22 @@ def test_rerouting_of_overflowed_tokens_matches_oracle(cfg, path, tol, residual)
                               router_bias=data.get("router_bias"), experts=[])
     assert (~plain["keep"]).sum() > 0.03 * cfg.T               # the case does overflow
     _check_layer(cfg, path, tol, reroute=True, residual=residual, d_aux=0.7)
+
+
+@pytest.mark.parametrize("cfg,path,tol", [(TINY, sm.GEMM_DEFAULT, TOL_F32), (MID, sm.GEMM_SIMT, TOL_BF16),
+                                          (MID, sm.GEMM_DEFAULT, TOL_BF16), (MANY, sm.GEMM_DEFAULT, TOL_BF16),
+                                          (si.SwitchConfig("e160", 1024, 128, 128, 160, 1.25), sm.GEMM_DEFAULT, TOL_BF16)],
+                         ids=["tiny_f32", "mid_fma", "mid_tc", "many_tc", "e160_tc_generic"])
+def test_exploration_noise_on_the_logits_matches_oracle(cfg, path, tol):
+    """uniform(1 - eps, 1 + eps) noise added to the router logits (router pseudo-code), passed in as an input."""
+    data = si.gen_layer(cfg, seed=0)
+    quiet = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
+                              router_bias=data.get("router_bias"), experts=[])
+    noisy = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
+                              router_bias=data.get("router_bias"), experts=[],
+                              router_noise=si.gen_router_noise(cfg, 0.5, 0))
+    assert (quiet["e"] != noisy["e"]).mean() > 0.05           # the noise does change the routing
+    _check_layer(cfg, path, tol, noise_eps=0.5)
 
 
 def test_rerouting_is_refused_with_several_routing_groups():

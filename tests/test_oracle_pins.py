@@ -589,3 +589,41 @@ def test_reroute_layer_gate_and_gradient():
             arr[idx] = old
             num[idx] = (lp - lm) / (2 * eps)
         assert np.linalg.norm(num - grad) / np.linalg.norm(grad) < 1e-7, name
+
+
+# ------------------------------------------------------------------ exploration noise on the router logits (appendix pseudo-code)
+def test_logit_noise_is_additive_and_its_mean_cancels_in_the_softmax():
+    T, d, f, E = 24, 6, 8, 5
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=51, scale=2.0)
+    rng = np.random.default_rng(51)
+    eps = 0.3
+    noise = rng.uniform(1 - eps, 1 + eps, size=(T, E))
+    h0 = so.router_logits(x, W_r)
+    np.testing.assert_allclose(so.router_logits(x, W_r, router_noise=noise), h0 + noise, rtol=0, atol=1e-15)
+    # uniform(1 - eps, 1 + eps) = 1 + uniform(-eps, eps): the common 1 is a shift the softmax does not see
+    p1 = so.router_probs(so.router_logits(x, W_r, router_noise=noise))
+    p2 = so.router_probs(so.router_logits(x, W_r, router_noise=noise - 1.0))
+    np.testing.assert_allclose(p1, p2, rtol=1e-13)
+    a = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01, router_noise=np.ones((T, E)))
+    b = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01)
+    np.testing.assert_allclose(a["p"], b["p"], rtol=1e-13)
+    assert np.array_equal(a["e"], b["e"]) and np.array_equal(a["slot"], b["slot"])
+    # noise that large does move tokens, and the gradient treats it as a constant
+    c = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01, router_noise=noise * 5.0)
+    assert (c["e"] != b["e"]).any()
+    R = rng.standard_normal((T, d))
+    bwd = so.switch_backward(c, x, W_r, W_in, W_out, R)
+    srt = np.sort(c["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-4
+    e_frozen, step = c["e"], 1e-6
+    num = np.zeros_like(W_r)
+    for idx in np.ndindex(W_r.shape):
+        old = W_r[idx]
+        vals = []
+        for sgn in (1.0, -1.0):
+            W_r[idx] = old + sgn * step
+            out = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01, router_noise=noise * 5.0, expert_index=e_frozen)
+            vals.append(float(np.sum(out["y"] * R) + out["aux"]))
+        W_r[idx] = old
+        num[idx] = (vals[0] - vals[1]) / (2 * step)
+    assert np.linalg.norm(num - bwd["dW_r"]) / np.linalg.norm(bwd["dW_r"]) < 1e-7
