@@ -144,7 +144,7 @@ def reroute_overflow(plan, e, alt, E: int, C: int):
 
 def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None,
                    capacity: int | None = None, expert_index=None, experts=None, residual: bool = False,
-                   reroute: bool = False, alt_index=None, router_noise=None):
+                   reroute: bool = False, alt_index=None, router_noise=None, router_jitter=None, storage_round=None):
     """Forward of the Switch FFN layer for one routing group.
 
     x [T, d]; W_r [d, E]; W_in [E, d, f]; W_out [E, f, d].  `capacity` overrides Eq. 3 when given.
@@ -159,12 +159,21 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     expert where it has room, and their gate is that expert's probability (Eq. 2 with the expert that processes the
     token); f in the auxiliary loss still counts the argmax (Eq. 5).  `alt_index`, when given, replaces the second
     choice (to follow a legitimate near-tie flip of the device).
+    `router_jitter` [T, d], when given, multiplies the router's input element by element (the text's "multiplicative
+    jitter noise on the incoming representation", Appendix C): the router sees x . u, the experts see x.  It is an
+    input (the caller draws it).  `storage_round`, when given, is applied to x . u: the router's input is a tensor
+    of the layer's activation type, so the product is rounded to that type before the router's float32 arithmetic.
     Returns a dict with every intermediate the staged comparisons need.
     """
     x64 = np.asarray(x, dtype=F64)
     T, d = x64.shape
     E = np.asarray(W_r).shape[1]
-    h = router_logits(x64, W_r, router_bias, router_noise)
+    x_router = x64
+    if router_jitter is not None:
+        x_router = x64 * np.asarray(router_jitter, dtype=F64)
+        if storage_round is not None:
+            x_router = np.asarray(storage_round(x_router), dtype=F64)
+    h = router_logits(x_router, W_r, router_bias, router_noise)
     p = router_probs(h)
     if expert_index is None:
         e, g = top1(p)
@@ -199,7 +208,8 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
         y[tok] = g[tok, None] * o_i                              # Eq. 2 with one selected expert
     out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "layer_y": y,
            "y": x64 + y if residual else y, "o": o, "u": u, "T": T, "E": E, "alpha": alpha, "residual": bool(residual),
-           "e_proc": e_proc}
+           "e_proc": e_proc, "x_router": x_router,
+           "router_jitter": None if router_jitter is None else np.asarray(router_jitter, dtype=F64)}
     out.update(plan)
     return out
 
@@ -249,9 +259,11 @@ def switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=No
     kept_tok = np.flatnonzero(keep)
     G[kept_tok, e_proc[kept_tok]] += dgate[kept_tok]        # the gate is the probability of the expert that processes the token
     dh = p * (G - np.sum(p * G, axis=1, keepdims=True))     # softmax Jacobian applied to G
-    dW_r = x64.T @ dh
+    dW_r = fwd.get("x_router", x64).T @ dh                 # the router's input (x, or x . u under input jitter)
     db = dh.sum(axis=0)
     dx_router = dh @ W_r64.T
+    if fwd.get("router_jitter") is not None:
+        dx_router = dx_router * fwd["router_jitter"]        # d(x . u)/dx = u; the storage rounding is passed straight through
     dx = dx + dx_router
     if fwd.get("residual", False):
         dx = dx + dy64                                   # y = x + layer(x): the skip path carries dy to x unchanged

@@ -627,3 +627,44 @@ def test_logit_noise_is_additive_and_its_mean_cancels_in_the_softmax():
         W_r[idx] = old
         num[idx] = (vals[0] - vals[1]) / (2 * step)
     assert np.linalg.norm(num - bwd["dW_r"]) / np.linalg.norm(bwd["dW_r"]) < 1e-7
+
+
+# ------------------------------------------------------------------ multiplicative jitter on the router's input (Appendix C, text)
+def test_input_jitter_reaches_only_the_router_and_its_gradient_is_scaled():
+    T, d, f, E, cf, alpha, d_aux = 14, 5, 7, 3, 1.0, 0.05, 0.8
+    rng = np.random.default_rng(61)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=61, scale=2.0)
+    u = rng.uniform(0.7, 1.3, size=(T, d))
+    fwd = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_jitter=u)
+    np.testing.assert_allclose(fwd["h"], (x * u) @ W_r, rtol=1e-13)               # the router sees x . u
+    for t in np.flatnonzero(fwd["keep"])[:5]:                                      # the experts see x
+        i = fwd["e"][t]
+        np.testing.assert_allclose(fwd["y"][t], fwd["g"][t] * (np.maximum(x[t] @ W_in[i], 0) @ W_out[i]), rtol=1e-12)
+    same = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_jitter=np.ones((T, d)))
+    plain = so.switch_forward(x, W_r, W_in, W_out, cf, alpha)
+    assert np.array_equal(same["y"], plain["y"]) and same["aux"] == plain["aux"]
+    # storage rounding is applied to the product only
+    coarse = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_jitter=u, storage_round=lambda a: np.round(a, 1))
+    np.testing.assert_allclose(coarse["h"], np.round(x * u, 1) @ W_r, rtol=1e-13)
+    # gradients against central differences (routing frozen)
+    R = rng.standard_normal((T, d))
+    srt = np.sort(fwd["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-3
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    e_frozen, eps = fwd["e"], 1e-6
+
+    def loss():
+        out = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_jitter=u, expert_index=e_frozen)
+        return float(np.sum(out["y"] * R) + d_aux * out["aux"])
+
+    for name, arr, grad in [("dx", x, bwd["dx"]), ("dW_r", W_r, bwd["dW_r"])]:
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            old = arr[idx]
+            arr[idx] = old + eps
+            lp = loss()
+            arr[idx] = old - eps
+            lm = loss()
+            arr[idx] = old
+            num[idx] = (lp - lm) / (2 * eps)
+        assert np.linalg.norm(num - grad) / np.linalg.norm(grad) < 1e-7, name
