@@ -208,11 +208,16 @@ def run_ours(args, cfg):
     bias = None if b_np is None else torch.from_numpy(b_np).cuda()
 
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype,
-                          residual=args.residual, groups=args.groups, reroute=args.reroute)
+                          residual=args.residual, groups=args.groups, reroute=args.reroute,
+                          input_jitter=args.input_jitter > 0.0)
     noise = None
     if args.router_noise > 0.0:                              # exploration noise on the logits: an input of the layer
         noise = torch.from_numpy(si.gen_router_noise(cfg, args.router_noise, seed)).cuda()
         mcfg.router_noise = noise.data_ptr()
+    jitter = None
+    if args.input_jitter > 0.0:                              # multiplicative jitter on the router's input: an input too
+        jitter = dev(si.gen_router_jitter(cfg, args.input_jitter, seed))
+        mcfg.router_jitter = jitter.data_ptr()
     ws = sm.allocate_workspace(mcfg)
     y, dx = torch.empty_like(x), torch.empty_like(x)
     dW_in, dW_out, dW_r = torch.empty_like(W_in), torch.empty_like(W_out), torch.empty_like(W_r)
@@ -355,7 +360,7 @@ def run_ours(args, cfg):
         "config": {"workload": cfg.name, "T": cfg.T, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "E": cfg.E,
                    "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha, "capacity": sm.switch_moe_capacity(mcfg),
                    "kept_tokens": kept, "parallelism": "replicas" if world > 1 else "single",
-                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "router_noise_eps": args.router_noise,
+                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "router_noise_eps": args.router_noise, "input_jitter_eps": args.input_jitter,
                    "l2": "inputs larger than L2 (weights 2 x %.0f MB per pass), no flush" %
                          (cfg.E * cfg.d_model * cfg.d_ff * elt / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": sm.switch_moe_launches_per_step(mcfg) * args.steps,
@@ -383,6 +388,9 @@ def main():
                          "loss each, experts shared); the headline configuration is one group")
     ap.add_argument("--router-noise", type=float, default=0.0,
                     help="add uniform(1 - eps, 1 + eps) noise (a seeded input tensor) to the router logits; "
+                         "the headline configuration has none")
+    ap.add_argument("--input-jitter", type=float, default=0.0,
+                    help="multiply the router's input by uniform(1 - eps, 1 + eps) factors (a seeded input tensor); "
                          "the headline configuration has none")
     ap.add_argument("--reroute", action="store_true",
                     help="offer tokens that overflow their expert to their second choice (stage 2 of "

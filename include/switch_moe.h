@@ -53,8 +53,12 @@ enum switch_moe_gemm_path {
    Section 2.2, every token that overflowed its expert is offered, in token order, to the expert with its
    second-highest probability and takes that expert's next free slot if one is left; its gate is that expert's
    probability.  Tokens kept by the first stage keep their slots, and f in the auxiliary loss still counts the
-   argmax.  One routing group only. */
-enum switch_moe_flags { SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2 };
+   argmax.  One routing group only.
+   SWITCH_MOE_FLAG_INPUT_JITTER: the router's input is x . u, element by element, with u = router_jitter (the text's
+   "multiplicative jitter noise on the incoming representation", Appendix C); the experts still see x.  The product
+   is rounded to the activation dtype (the router's input is a tensor of that type) and kept in the workspace for
+   the backward pass, where dW_r uses it and the router's part of dx is multiplied by u. */
+enum switch_moe_flags { SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2, SWITCH_MOE_FLAG_INPUT_JITTER = 4 };
 
 typedef enum switch_moe_status {
   SWITCH_MOE_OK = 0,
@@ -94,6 +98,10 @@ typedef struct switch_moe_config {
                                 logits in training (the text instead speaks of multiplicative jitter on the router's
                                 input; this field follows the pseudo-code).  The noise is an input, drawn by the
                                 caller; it is a constant of the backward pass. */
+  const void* router_jitter; /* DEVICE [T, d_model] in the activation dtype: the factors u of SWITCH_MOE_FLAG_INPUT_JITTER
+                                (e.g. uniform(1 - eps, 1 + eps), drawn by the caller); must be set, 16-byte aligned,
+                                when the flag is, and is ignored otherwise.  Needed by fwd, router_fwd, bwd and
+                                router_bwd alike. */
 } switch_moe_config;
 
 #define SWITCH_MOE_STAGE_EVENTS 13

@@ -264,7 +264,8 @@ int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches
   // fwd: router, 3 plan kernels, gather, 2 GEMMs; bwd: gather, 4 GEMMs, 4 router-backward kernels.
   // Tensor-core router: forward = operand split, router, column sums; backward = logit gradients, two products, reduce.
   // Rerouting of overflowed tokens adds four plan kernels to the forward pass.
-  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0);
+  // Input jitter adds the element-wise product kernel.
+  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0);
   return SWITCH_MOE_OK;
 }
 

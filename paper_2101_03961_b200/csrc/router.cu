@@ -174,6 +174,35 @@ template <> struct BfVec<2> { using type = unsigned int; };
 template <> struct BfVec<4> { using type = uint2; };
 template <> struct BfVec<8> { using type = uint4; };
 
+// Router input under multiplicative jitter (Appendix C): xr = x . u element by element, rounded to the activation type.
+template <typename XT>
+__global__ void __launch_bounds__(256)
+router_jitter_kernel(const uint4* __restrict__ x, const uint4* __restrict__ u, size_t n_vec, uint4* __restrict__ xr) {
+  pdl_launch_dependents();
+  pdl_wait();
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (size_t)gridDim.x * blockDim.x) {
+    const uint4 a = x[i], b = u[i];
+    uint4 o;
+    if constexpr (sizeof(XT) == 2) {
+      const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+      __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 fa = __bfloat1622float2(pa[q]), fb = __bfloat1622float2(pb[q]);
+        po[q] = __floats2bfloat162_rn(fa.x * fb.x, fa.y * fb.y);      // the float32 product of two bf16 is exact
+      }
+    } else {
+      const float* fa = reinterpret_cast<const float*>(&a);
+      const float* fb = reinterpret_cast<const float*>(&b);
+      float* fo = reinterpret_cast<float*>(&o);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) fo[q] = fa[q] * fb[q];
+    }
+    xr[i] = o;
+  }
+}
+
 // dh[t,i] = p[t,i] (G[t,i] - sum_j p[t,j] G[t,j]),  G[t,i] = cG.count_gi + [i = e_t and t kept].dgate_t,
 // count_gi counted inside the token's own routing group g = t / Tg
 template <int NE>
@@ -313,7 +342,7 @@ __global__ void router_dwr_reduce_kernel(const float* __restrict__ partial, int 
 template <typename XT, int NE>
 __global__ void __launch_bounds__(256)
 router_dx_kernel(const float* __restrict__ dlogits, const float* __restrict__ W_r, const int* __restrict__ slot,
-                 int T, int d, int E, int accumulate, XT* __restrict__ dx) {
+                 int T, int d, int E, int accumulate, const XT* __restrict__ jitter_u, XT* __restrict__ dx) {
   pdl_launch_dependents();
   pdl_wait();
   constexpr int EP = 32 * NE;
@@ -368,6 +397,7 @@ router_dx_kernel(const float* __restrict__ dlogits, const float* __restrict__ W_
         if (k >= d) continue;
         XT* o = dx + (size_t)t * d + k;
         float v = acc[a][b];
+        if (jitter_u != nullptr) v *= to_f32(jitter_u[(size_t)t * d + k]);     // d(x . u)/dx = u
         if (add) v += to_f32(*o);
         if constexpr (sizeof(XT) == 4) *o = v; else *o = __float2bfloat16(v);
       }
@@ -400,6 +430,10 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
                                                             s.Epad64);
   float* partial = ws_ptr<float>(ws, p.dwr_partial);
   const size_t n = (size_t)s.d * s.E;
+  if (s.jitter) {                                             // the router's input was x . u (left by the forward pass)
+    if (s.jitter_u == nullptr || !aligned16(s.jitter_u)) return SWITCH_MOE_INVALID_ARGUMENT;
+    x = ws_ptr<char>(ws, p.xr);
+  }
   if constexpr (sizeof(XT) == 2) {
     if (s.router_tc) {
       // tensor-core products (bf16-split operands), then the same fixed-order reduction of the token splits
@@ -418,7 +452,8 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
       cudaSuccess)
     return SWITCH_MOE_CUDA_ERROR;
   launch_k(router_dx_kernel<XT, NE>, dim3((s.T + 63) / 64), dim3(256), smem, st, dlogits, W_r, ws_ptr<int>(ws, p.slot), s.T, s.d, s.E,
-                                                              accumulate_dx ? (s.residual ? 2 : 1) : 0, static_cast<XT*>(dx));
+                                                              accumulate_dx ? (s.residual ? 2 : 1) : 0,
+                                                              static_cast<const XT*>(s.jitter_u), static_cast<XT*>(dx));
   return launch_status();
 }
 
@@ -436,6 +471,19 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
 int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* bias,
                       const float* noise, void* ws,
                       cudaStream_t st) {
+  if (s.jitter) {
+    if (s.jitter_u == nullptr || !aligned16(s.jitter_u)) return SWITCH_MOE_INVALID_ARGUMENT;
+    const size_t n_vec = (size_t)s.T * s.d * s.elt / 16;
+    uint4* xr = ws_ptr<uint4>(ws, p.xr);
+    const unsigned blocks = (unsigned)((n_vec + 255) / 256 < 148 * 16 ? (n_vec + 255) / 256 : 148 * 16);
+    if (s.dtype == SWITCH_MOE_BF16)
+      launch_k(router_jitter_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(x),
+               static_cast<const uint4*>(s.jitter_u), n_vec, xr);
+    else
+      launch_k(router_jitter_kernel<float>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(x),
+               static_cast<const uint4*>(s.jitter_u), n_vec, xr);
+    x = xr;
+  }
   if (s.router_tc && s.dtype == SWITCH_MOE_BF16) return launch_router_tc_fwd(s, p, x, W_r, bias, noise, ws, st);
   SWMOE_DISPATCH_NE(router_fwd_t, s, p, x, W_r, bias, noise, ws, st)
 }

@@ -35,7 +35,7 @@ struct RouterTcParams {
   int wrap;                  // k-blocks per part: d/64 (fwd), Epad64/64 (dx); dwr derives it per tile
   const float* bias; const float* noise; float* probs; int* expert_index; float* gate;   // fwd
   float* partial;                                                                         // dwr
-  __nv_bfloat16* dx; const int* slot; int accumulate;                                     // dx
+  __nv_bfloat16* dx; const int* slot; int accumulate; const __nv_bfloat16* jitter_u;      // dx
   int* status;
 };
 
@@ -363,7 +363,25 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int it = 0; it < 8; ++it) {
               const int rr = it * 4 + (lane >> 3);
               uint4 val = *reinterpret_cast<const uint4*>(my_stage_gen + rr * 128 + (((lane & 7) ^ (rr & 7)) << 4));
-              if ((add_mask >> it) & 1u) {
+              if (p.jitter_u != nullptr && offs[it] >= 0) {      // d(x . u)/dx = u
+                const uint4 uu = *reinterpret_cast<const uint4*>(p.jitter_u + offs[it] + col);
+                __nv_bfloat162* vp = reinterpret_cast<__nv_bfloat162*>(&val);
+                const __nv_bfloat162* up = reinterpret_cast<const __nv_bfloat162*>(&uu);
+                if ((add_mask >> it) & 1u) {                     // one rounding for (router term . u) + dx
+                  const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&prev[it]);
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const float2 a = __bfloat1622float2(vp[q]), b = __bfloat1622float2(pp[q]), c2 = __bfloat1622float2(up[q]);
+                    vp[q] = __floats2bfloat162_rn(fmaf(a.x, c2.x, b.x), fmaf(a.y, c2.y, b.y));
+                  }
+                } else {
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const float2 a = __bfloat1622float2(vp[q]), c2 = __bfloat1622float2(up[q]);
+                    vp[q] = __floats2bfloat162_rn(a.x * c2.x, a.y * c2.y);
+                  }
+                }
+              } else if ((add_mask >> it) & 1u) {
                 __nv_bfloat162* vp = reinterpret_cast<__nv_bfloat162*>(&val);
                 const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&prev[it]);
 #pragma unroll
@@ -739,6 +757,7 @@ int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const flo
   q.n_mtiles = (s.T + kTileM - 1) / kTileM; q.n_ntiles = (s.d + kBN - 1) / kBN;
   q.wrap = s.Epad64 / kBK;
   q.dx = static_cast<__nv_bfloat16*>(dx); q.slot = ws_ptr<int>(ws, p.slot); q.accumulate = accumulate_dx ? (s.residual ? 2 : 1) : 0;   // 2: every row (skip path inside the layer)
+  q.jitter_u = static_cast<const __nv_bfloat16*>(s.jitter_u);
   return launch_op<kRDx>(tmA, tmB, q, st);
 }
 

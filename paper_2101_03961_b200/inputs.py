@@ -24,7 +24,7 @@ import numpy as np
 DTYPE_BF16 = 0
 DTYPE_F32 = 1
 
-_TENSOR_X, _TENSOR_DY, _TENSOR_WR, _TENSOR_WIN, _TENSOR_WOUT, _TENSOR_BIAS, _TENSOR_NOISE = 1, 2, 3, 4, 5, 6, 7
+_TENSOR_X, _TENSOR_DY, _TENSOR_WR, _TENSOR_WIN, _TENSOR_WOUT, _TENSOR_BIAS, _TENSOR_NOISE, _TENSOR_JITTER = 1, 2, 3, 4, 5, 6, 7, 8
 
 
 @dataclass(frozen=True)
@@ -134,6 +134,20 @@ def gen_router_noise(cfg: SwitchConfig, eps: float, seed: int = 0) -> np.ndarray
     layer: the library and the oracle are both handed this array)."""
     u = _rng(seed, _TENSOR_NOISE).random((cfg.T, cfg.E), dtype=np.float32)
     return (np.float32(1.0 - eps) + np.float32(2.0 * eps) * u).astype(np.float32)
+
+
+def gen_router_jitter(cfg: SwitchConfig, eps: float, seed: int = 0) -> np.ndarray:
+    """Multiplicative jitter factors for the router's input [T, d_model], uniform in [1 - eps, 1 + eps), float32
+    (bf16-representable where cfg.dtype is bf16); an input of the layer like x."""
+    u = _rng(seed, _TENSOR_JITTER).random((cfg.T, cfg.d_model), dtype=np.float32)
+    return _finish(cfg, (np.float32(1.0 - eps) + np.float32(2.0 * eps) * u).astype(np.float32))
+
+
+def storage_round(cfg: SwitchConfig):
+    """Rounding of a float64 array to the layer's activation type (bfloat16 or float32), returned as float64."""
+    if cfg.dtype == DTYPE_BF16:
+        return lambda a: round_to_bf16(np.asarray(a, dtype=np.float32)).astype(np.float64)
+    return lambda a: np.asarray(a, dtype=np.float32).astype(np.float64)
 
 
 def gen_W_in_expert(cfg: SwitchConfig, e: int, seed: int = 0) -> np.ndarray:

@@ -44,10 +44,11 @@ class GpuLayer:
     def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0,
                  residual=False, groups=1, reroute=False):
         sbuild.build()
+        jit = data.get("router_jitter")
         self.scfg = cfg
         self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
                                   dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path,
-                                  residual=residual, groups=groups, reroute=reroute)
+                                  residual=residual, groups=groups, reroute=reroute, input_jitter=jit is not None)
         dt = cfg.dtype
         self.x = to_dev(data["x"], dt)
         self.dy = to_dev(data["dy"], dt)
@@ -58,6 +59,9 @@ class GpuLayer:
         self.noise = None if n is None else torch.from_numpy(np.ascontiguousarray(n, dtype=np.float32)).cuda()
         if self.noise is not None:
             self.cfg.router_noise = self.noise.data_ptr()
+        self.jitter = None if jit is None else to_dev(jit, dt)
+        if self.jitter is not None:
+            self.cfg.router_jitter = self.jitter.data_ptr()
         self.W_in = to_dev(data["W_in"], dt)
         self.W_out = to_dev(data["W_out"], dt)
         tdt = torch.bfloat16 if dt == sm.BF16 else torch.float32
@@ -118,6 +122,9 @@ def check_second_choice(gpu_alt: np.ndarray, p: np.ndarray, e: np.ndarray, overf
 def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capacity=None, experts=None,
                      residual=False, groups=1, gpu_alt=None):
     """Oracle forward with the device's expert choice (identical unless a near-tie flipped), after checking flips."""
+    jit_kw = {}
+    if data.get("router_jitter") is not None:                  # the router sees x . u rounded to the activation type
+        jit_kw = {"router_jitter": data["router_jitter"], "storage_round": si.storage_round(cfg)}
     if groups > 1:
         assert capacity is None
         first = so.switch_forward_groups(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
@@ -130,18 +137,18 @@ def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capaci
         return fwd
     first = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                               router_bias=data.get("router_bias"), capacity=capacity, experts=[],
-                              router_noise=data.get("router_noise"))
+                              router_noise=data.get("router_noise"), **jit_kw)
     flips = check_flips(gpu_e, first)
     alt = None
     if gpu_alt is not None:                                   # stage 2 of No-Token-Left-Behind routing
         stage1 = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
                                    cfg.alpha, router_bias=data.get("router_bias"), capacity=capacity,
-                                   expert_index=gpu_e, experts=[], router_noise=data.get("router_noise"))
+                                   expert_index=gpu_e, experts=[], router_noise=data.get("router_noise"), **jit_kw)
         alt = check_second_choice(gpu_alt, stage1["p"], gpu_e, ~stage1["keep"])
     fwd = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                             router_bias=data.get("router_bias"), capacity=capacity, expert_index=gpu_e,
                             experts=experts, residual=residual, reroute=gpu_alt is not None, alt_index=alt,
-                            router_noise=data.get("router_noise"))
+                            router_noise=data.get("router_noise"), **jit_kw)
     fwd["flips"] = flips
     return fwd
 

@@ -120,8 +120,10 @@ def test_dispatch_plan_is_deterministic():
 
 # ---------------------------------------------------------------------------------------------- whole layer
 def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False, groups=1,
-                 reroute=False, noise_eps=0.0):
+                 reroute=False, noise_eps=0.0, jitter_eps=0.0):
     data = si.gen_layer(cfg, seed=seed)
+    if jitter_eps:
+        data["router_jitter"] = si.gen_router_jitter(cfg, jitter_eps, seed)
     if noise_eps:
         data["router_noise"] = si.gen_router_noise(cfg, noise_eps, seed)
     g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual,
@@ -275,6 +277,24 @@ def test_exploration_noise_on_the_logits_matches_oracle(cfg, path, tol):
                               router_noise=si.gen_router_noise(cfg, 0.5, 0))
     assert (quiet["e"] != noisy["e"]).mean() > 0.05           # the noise does change the routing
     _check_layer(cfg, path, tol, noise_eps=0.5)
+
+
+@pytest.mark.parametrize("cfg,path,tol,residual", [
+    (TINY, sm.GEMM_DEFAULT, TOL_F32, False), (MID, sm.GEMM_SIMT, TOL_BF16, False), (MID, sm.GEMM_DEFAULT, TOL_BF16, False),
+    (RAGGED, sm.GEMM_DEFAULT, TOL_BF16, False), (MANY, sm.GEMM_DEFAULT, TOL_BF16, True)],
+    ids=["tiny_f32", "mid_fma", "mid_tc", "ragged_tc", "many_tc_skip"])
+def test_multiplicative_jitter_on_the_router_input_matches_oracle(cfg, path, tol, residual):
+    """The router sees x . u (Appendix C, text), the experts see x; dW_r uses x . u and the router's dx is scaled by u."""
+    _check_layer(cfg, path, tol, jitter_eps=0.25, residual=residual, d_aux=0.7)
+
+
+def test_jitter_flag_without_the_factors_is_refused():
+    cfg = sm.make_config(MID.T, MID.d_model, MID.d_ff, MID.E, MID.capacity_factor, input_jitter=True)
+    ws = sm.allocate_workspace(cfg)
+    x = torch.zeros(MID.T, MID.d_model, dtype=torch.bfloat16, device="cuda")
+    W_r = torch.zeros(MID.d_model, MID.E, device="cuda")
+    with pytest.raises(sm.SwitchMoeError):
+        sm.switch_moe_router_fwd(cfg, x, W_r, None, ws)
 
 
 def test_rerouting_is_refused_with_several_routing_groups():
