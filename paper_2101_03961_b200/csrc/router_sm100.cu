@@ -333,6 +333,13 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           for (int it = 0; it < 8; ++it)
             prev[it] = (((add_mask >> it) & 1u) && col < p.d) ? *reinterpret_cast<const uint4*>(p.dx + offs[it] + col)
                                                              : make_uint4(0, 0, 0, 0);
+          uint4 uu[8];                                        // jitter factors of the same elements, fetched early too
+          if (p.jitter_u != nullptr) {
+#pragma unroll
+            for (int it = 0; it < 8; ++it)
+              uu[it] = (offs[it] >= 0 && col < p.d) ? *reinterpret_cast<const uint4*>(p.jitter_u + offs[it] + col)
+                                                    : make_uint4(0, 0, 0, 0);
+          }
           uint32_t v[64];
           tc_ld32(t_addr + c * 64, v);
           tc_ld32(t_addr + c * 64 + 32, v + 32);
@@ -364,9 +371,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               const int rr = it * 4 + (lane >> 3);
               uint4 val = *reinterpret_cast<const uint4*>(my_stage_gen + rr * 128 + (((lane & 7) ^ (rr & 7)) << 4));
               if (p.jitter_u != nullptr && offs[it] >= 0) {      // d(x . u)/dx = u
-                const uint4 uu = *reinterpret_cast<const uint4*>(p.jitter_u + offs[it] + col);
                 __nv_bfloat162* vp = reinterpret_cast<__nv_bfloat162*>(&val);
-                const __nv_bfloat162* up = reinterpret_cast<const __nv_bfloat162*>(&uu);
+                const __nv_bfloat162* up = reinterpret_cast<const __nv_bfloat162*>(&uu[it]);
                 if ((add_mask >> it) & 1u) {                     // one rounding for (router term . u) + dx
                   const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&prev[it]);
 #pragma unroll
