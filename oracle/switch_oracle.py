@@ -109,6 +109,21 @@ def dispatch_plan(e, E: int, C: int):
     return {"pos": pos, "keep": keep, "slot": slot, "token_of_slot": token_of_slot, "count": count, "kept": kept}
 
 
+def gelu(z):
+    """GELU(z) = z . Phi(z) with Phi the standard normal distribution function (the exact form, not the tanh fit)."""
+    z = np.asarray(z, dtype=F64)
+    return z * 0.5 * (1.0 + _erf(z / math.sqrt(2.0)))
+
+
+def gelu_prime(z):
+    """d GELU / dz = Phi(z) + z . phi(z)."""
+    z = np.asarray(z, dtype=F64)
+    return 0.5 * (1.0 + _erf(z / math.sqrt(2.0))) + z * np.exp(-0.5 * z * z) / math.sqrt(2.0 * math.pi)
+
+
+_erf = np.vectorize(math.erf, otypes=[F64])
+
+
 def second_choice(p, e):
     """The expert with the second-highest probability of each token: the argmax over the experts other than e_t
     (lowest index on ties)."""
@@ -144,7 +159,8 @@ def reroute_overflow(plan, e, alt, E: int, C: int):
 
 def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None,
                    capacity: int | None = None, expert_index=None, experts=None, residual: bool = False,
-                   reroute: bool = False, alt_index=None, router_noise=None, router_jitter=None, storage_round=None):
+                   reroute: bool = False, alt_index=None, router_noise=None, router_jitter=None, storage_round=None,
+                   geglu: bool = False):
     """Forward of the Switch FFN layer for one routing group.
 
     x [T, d]; W_r [d, E]; W_in [E, d, f]; W_out [E, f, d].  `capacity` overrides Eq. 3 when given.
@@ -163,6 +179,9 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     jitter noise on the incoming representation", Appendix C): the router sees x . u, the experts see x.  It is an
     input (the caller draws it).  `storage_round`, when given, is applied to x . u: the router's input is a tensor
     of the layer's activation type, so the product is rounded to that type before the router's float32 arithmetic.
+    `geglu` replaces the expert's ReLU FFN by the GEGLU FFN of the paper's Table 9 ("the expansion matrix is
+    substituted with two sets of weights which are non-linearly combined"): W_in[i] is [d, 2 f] = [W_0 | W_1],
+    a = x W_0, b = x W_1, hidden = GELU(a) . b, output = hidden W_out.  "u" then holds the rows [a | b].
     Returns a dict with every intermediate the staged comparisons need.
     """
     x64 = np.asarray(x, dtype=F64)
@@ -200,15 +219,19 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
         tok = plan["token_of_slot"][i * C:i * C + int(plan["kept"][i])]   # kept tokens of expert i, in slot order
         if tok.size == 0:
             continue
-        u_i = x64[tok] @ np.asarray(W_in[i], dtype=F64)          # h = x W_in
-        a_i = np.maximum(u_i, 0.0)                               # ReLU(h)
+        u_i = x64[tok] @ np.asarray(W_in[i], dtype=F64)          # h = x W_in  (GEGLU: [a | b] = x [W_0 | W_1])
+        if geglu:
+            fh = u_i.shape[1] // 2
+            a_i = gelu(u_i[:, :fh]) * u_i[:, fh:]                # GELU(x W_0) . (x W_1)
+        else:
+            a_i = np.maximum(u_i, 0.0)                           # ReLU(h)
         o_i = a_i @ np.asarray(W_out[i], dtype=F64)              # y = ReLU(h) W_out
         u[i] = u_i
         o[tok] = o_i
         y[tok] = g[tok, None] * o_i                              # Eq. 2 with one selected expert
     out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "layer_y": y,
            "y": x64 + y if residual else y, "o": o, "u": u, "T": T, "E": E, "alpha": alpha, "residual": bool(residual),
-           "e_proc": e_proc, "x_router": x_router,
+           "e_proc": e_proc, "x_router": x_router, "geglu": bool(geglu),
            "router_jitter": None if router_jitter is None else np.asarray(router_jitter, dtype=F64)}
     out.update(plan)
     return out
@@ -243,11 +266,17 @@ def switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=No
                 dW_out[i] = np.zeros_like(W_out_i)
             continue
         u_i = fwd["u"][i]
-        a_i = np.maximum(u_i, 0.0)
         do_i = g[tok, None] * dy64[tok]                 # y = g . o        =>  do = g . dy
         dgate[tok] = np.sum(dy64[tok] * fwd["o"][tok], axis=1)   #          =>  dg = <dy, o>
         da_i = do_i @ W_out_i.T                         # o = a W_out
-        du_i = da_i * (u_i > 0.0)                       # a = ReLU(u), ReLU'(0) = 0
+        if fwd.get("geglu", False):
+            fh = u_i.shape[1] // 2
+            ua, ub = u_i[:, :fh], u_i[:, fh:]
+            a_i = gelu(ua) * ub                         # hidden = GELU(a) . b
+            du_i = np.concatenate([da_i * ub * gelu_prime(ua), da_i * gelu(ua)], axis=1)
+        else:
+            a_i = np.maximum(u_i, 0.0)
+            du_i = da_i * (u_i > 0.0)                   # a = ReLU(u), ReLU'(0) = 0
         dx[tok] = du_i @ W_in_i.T                       # u = x W_in
         if want_weight_grads:
             dW_out[i] = a_i.T @ do_i

@@ -668,3 +668,63 @@ def test_input_jitter_reaches_only_the_router_and_its_gradient_is_scaled():
             arr[idx] = old
             num[idx] = (lp - lm) / (2 * eps)
         assert np.linalg.norm(num - grad) / np.linalg.norm(grad) < 1e-7, name
+
+
+# ------------------------------------------------------------------ GEGLU experts (Table 9)
+def test_gelu_closed_forms():
+    from scipy.stats import norm
+    z = np.linspace(-6, 6, 241)
+    np.testing.assert_allclose(so.gelu(z), z * norm.cdf(z), rtol=1e-13, atol=1e-15)        # z . Phi(z)
+    np.testing.assert_allclose(so.gelu(z) - so.gelu(-z), z, rtol=1e-13, atol=1e-15)        # odd part is z / 2 + z / 2
+    assert so.gelu(0.0) == 0.0 and abs(so.gelu(10.0) - 10.0) < 1e-12 and abs(so.gelu(-10.0)) < 1e-12
+    np.testing.assert_allclose(so.gelu_prime(z), norm.cdf(z) + z * norm.pdf(z), rtol=1e-12, atol=1e-15)
+    h = 1e-6
+    np.testing.assert_allclose(so.gelu_prime(z), (so.gelu(z + h) - so.gelu(z - h)) / (2 * h), rtol=1e-7, atol=1e-9)
+
+
+def test_geglu_single_expert_is_the_dense_geglu_ffn_and_gradients_match_finite_differences():
+    from scipy.stats import norm
+    T, d, f = 10, 5, 6
+    rng = np.random.default_rng(71)
+    x = rng.standard_normal((T, d))
+    W_r = rng.standard_normal((d, 1))
+    W_in = rng.standard_normal((1, d, 2 * f)) * 0.7
+    W_out = rng.standard_normal((1, f, d)) * 0.7
+    out = so.switch_forward(x, W_r, W_in, W_out, 1.0, 0.01, geglu=True)
+    a, b = x @ W_in[0][:, :f], x @ W_in[0][:, f:]
+    np.testing.assert_allclose(out["y"], ((a * norm.cdf(a)) * b) @ W_out[0], rtol=1e-12)   # gate = 1 with one expert
+    # several experts, drops, frozen routing: all gradients against central differences
+    T, d, f, E, cf, alpha, d_aux = 16, 5, 6, 3, 0.75, 0.03, 1.2
+    x = rng.standard_normal((T, d)) * 2
+    W_r = rng.standard_normal((d, E))
+    W_in = rng.standard_normal((E, d, 2 * f)) * 0.6
+    W_out = rng.standard_normal((E, f, d)) * 0.6
+    R = rng.standard_normal((T, d))
+    fwd = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, geglu=True)
+    srt = np.sort(fwd["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-3 and (~fwd["keep"]).any()
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    e_frozen, eps = fwd["e"], 1e-6
+
+    def loss():
+        o = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, geglu=True, expert_index=e_frozen)
+        return float(np.sum(o["y"] * R) + d_aux * o["aux"])
+
+    dW_in = np.stack([bwd["dW_in"][i] for i in range(E)])
+    dW_out = np.stack([bwd["dW_out"][i] for i in range(E)])
+    for name, arr, grad in [("dx", x, bwd["dx"]), ("dW_r", W_r, bwd["dW_r"]), ("dW_in", W_in, dW_in),
+                            ("dW_out", W_out, dW_out)]:
+        idxs = list(np.ndindex(arr.shape))
+        if len(idxs) > 150:
+            idxs = [idxs[i] for i in rng.choice(len(idxs), 150, replace=False)]
+        num = []
+        for idx in idxs:
+            old = arr[idx]
+            arr[idx] = old + eps
+            lp = loss()
+            arr[idx] = old - eps
+            lm = loss()
+            arr[idx] = old
+            num.append((lp - lm) / (2 * eps))
+        ana = np.array([grad[i] for i in idxs])
+        assert np.linalg.norm(np.array(num) - ana) / np.linalg.norm(ana) < 1e-7, name
