@@ -62,7 +62,7 @@ class OracleSample:
         Each of the four passes is timed `reps` times and the minimum kept (host timing noise is large)."""
         from oracle import switch_oracle as so
         cfg, a = self.cfg, (self.x, self.W_r, self.W_in, self.W_out)
-        kw = dict(router_bias=self.b)
+        kw = dict(router_bias=self.b, geglu=cfg.geglu)
         t_rf, t_af, t_ab, t_rb = [], [], [], []
         for _ in range(reps):
             t0 = time.perf_counter()
@@ -209,7 +209,7 @@ def run_ours(args, cfg):
 
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype,
                           residual=args.residual, groups=args.groups, reroute=args.reroute,
-                          input_jitter=args.input_jitter > 0.0)
+                          input_jitter=args.input_jitter > 0.0, geglu=cfg.geglu)
     noise = None
     if args.router_noise > 0.0:                              # exploration noise on the logits: an input of the layer
         noise = torch.from_numpy(si.gen_router_noise(cfg, args.router_noise, seed)).cuda()
@@ -285,7 +285,13 @@ def run_ours(args, cfg):
     peaks, peak_kind = load_peaks()
     gemm_names = ["gemm1_relu", "gemm2_combine", "dgrad2_mask", "wgrad2", "dgrad1_scatter", "wgrad1"]
     gemm_ms_avg = statistics.mean(stage_ms[n] for n in gemm_names)
-    flops_per_launch = 2.0 * kept * cfg.d_model * cfg.d_ff           # useful flops of one expert GEMM (kept rows only)
+    # useful flops of one expert GEMM (kept rows only); with GEGLU experts the three GEMMs that touch W_in have twice
+    # the columns, and the figure is the mean over the six launches
+    gemm_weight = {n: 1.0 for n in gemm_names}
+    if cfg.geglu:
+        gemm_weight.update({"gemm1_relu": 2.0, "dgrad1_scatter": 2.0, "wgrad1": 2.0})
+    flops_unit = 2.0 * kept * cfg.d_model * cfg.d_ff
+    flops_per_launch = flops_unit * sum(gemm_weight.values()) / 6.0
     achieved_tf = flops_per_launch / (gemm_ms_avg * 1e-3) / 1e12
     if cfg.dtype == si.DTYPE_BF16:
         peak_tf = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
@@ -311,7 +317,7 @@ def run_ours(args, cfg):
     row_bytes = cfg.d_model * elt
     stages = {n: {"ms": stage_ms[n]} for n in stage_ms}
     for n in gemm_names:
-        stages[n]["tflops"] = flops_per_launch / (stage_ms[n] * 1e-3) / 1e12
+        stages[n]["tflops"] = flops_unit * gemm_weight[n] / (stage_ms[n] * 1e-3) / 1e12
     stages["gather_x"]["gbs"] = (2 * kept * row_bytes) / (stage_ms["gather_x"] * 1e-3) / 1e9
     stages["gather_dy"]["gbs"] = (3 * kept * row_bytes) / (stage_ms["gather_dy"] * 1e-3) / 1e9
     stages["router_fwd"]["gbs"] = (cfg.T * row_bytes + cfg.T * cfg.E * 4) / (stage_ms["router_fwd"] * 1e-3) / 1e9
@@ -358,6 +364,7 @@ def run_ours(args, cfg):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.dtype == si.DTYPE_BF16 else "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "T": cfg.T, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "E": cfg.E,
+                   "geglu_experts": cfg.geglu,
                    "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha, "capacity": sm.switch_moe_capacity(mcfg),
                    "kept_tokens": kept, "parallelism": "replicas" if world > 1 else "single",
                    "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "router_noise_eps": args.router_noise, "input_jitter_eps": args.input_jitter,

@@ -57,8 +57,15 @@ enum switch_moe_gemm_path {
    SWITCH_MOE_FLAG_INPUT_JITTER: the router's input is x . u, element by element, with u = router_jitter (the text's
    "multiplicative jitter noise on the incoming representation", Appendix C); the experts still see x.  The product
    is rounded to the activation dtype (the router's input is a tensor of that type) and kept in the workspace for
-   the backward pass, where dW_r uses it and the router's part of dx is multiplied by u. */
-enum switch_moe_flags { SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2, SWITCH_MOE_FLAG_INPUT_JITTER = 4 };
+   the backward pass, where dW_r uses it and the router's part of dx is multiplied by u.
+   SWITCH_MOE_FLAG_GEGLU: the experts are GEGLU FFNs (Table 9: "the expansion matrix is substituted with two sets of
+   weights which are non-linearly combined"): W_in is [E, d_model, 2 d_ff] = [W_0 | W_1] per expert (and dW_in
+   likewise), hidden = GELU(x W_0) . (x W_1) with the exact GELU z Phi(z), y = hidden W_out.  The two products are
+   one grouped GEMM with 2 d_ff output columns; the gating and its derivative are element-wise kernels over the
+   kept rows.  Not available on SWITCH_MOE_GEMM_TC_1CTA. */
+enum switch_moe_flags {
+  SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2, SWITCH_MOE_FLAG_INPUT_JITTER = 4, SWITCH_MOE_FLAG_GEGLU = 8
+};
 
 typedef enum switch_moe_status {
   SWITCH_MOE_OK = 0,

@@ -13,7 +13,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libswitch_moe.so")
 SOURCES = ["api.cu", "router.cu", "dispatch.cu", "simt_gemm.cu", "grouped_gemm_sm100.cu", "expert_gemm_pair_sm100.cu", "router_sm100.cu",
-           "dispatch_static.cu"]
+           "dispatch_static.cu", "geglu.cu"]
 
 
 def _nvcc() -> str:

@@ -142,6 +142,7 @@ int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r
   a.W_in = W_in; a.W_out = W_out; a.y = y; a.x = x;
   SWMOE_TRY(mark(cfg, 3, st));
   SWMOE_TRY(run_gemm(kGemm1Relu, c, a, workspace, st));
+  if (c.s.geglu) SWMOE_TRY(launch_geglu_fwd(c.s, c.p, workspace, st));     // hidden = GELU(a) . b
   SWMOE_TRY(mark(cfg, 4, st));
   SWMOE_TRY(run_gemm(kGemm2Combine, c, a, workspace, st));
   SWMOE_TRY(mark(cfg, 5, st));
@@ -165,6 +166,7 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
   SWMOE_TRY(launch_gather_dy(c.s, c.p, dy, y, dx, workspace, st));
   SWMOE_TRY(mark(cfg, 7, st));
   SWMOE_TRY(run_gemm(kDgrad2Mask, c, a, workspace, st));
+  if (c.s.geglu) SWMOE_TRY(launch_geglu_bwd(c.s, c.p, workspace, st));     // d[a | b] from dH
   SWMOE_TRY(mark(cfg, 8, st));
   SWMOE_TRY(run_gemm(kWgrad2, c, a, workspace, st));
   SWMOE_TRY(mark(cfg, 9, st));
@@ -265,7 +267,8 @@ int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches
   // Tensor-core router: forward = operand split, router, column sums; backward = logit gradients, two products, reduce.
   // Rerouting of overflowed tokens adds four plan kernels to the forward pass.
   // Input jitter adds the element-wise product kernel.
-  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0);
+  // GEGLU experts add the gating kernel to each pass.
+  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0) + (s.geglu ? 2 : 0);
   return SWITCH_MOE_OK;
 }
 

@@ -57,6 +57,7 @@ struct PairParams {
   int* status;
   const __nv_bfloat16* res;   // combine / scatter with the skip path inside the layer: rows added to the output (x or dy)
   __nv_bfloat16* out2;        // combine with the skip path: second copy of the output without it
+  int plain;                  // GEMM1 / dgrad2 without ReLU and without the ReLU mask (GEGLU experts gate elsewhere)
 };
 
 struct PTile {
@@ -311,7 +312,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         // everything the epilogue needs from global memory is requested here, before the accumulator is awaited
 #pragma unroll
         for (int k = 0; k < 4; ++k) describe(half + 2 * k, &q_off[k], &q_gate[k]);
-        if (OP == kDgrad2Mask && m_warp < p.Mw) {
+        if (OP == kDgrad2Mask && !p.plain && m_warp < p.Mw) {
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             if (q_off[k] >= 0)
@@ -359,7 +360,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             for (int u = 0; u < 4; ++u) {
               float a = __uint_as_float(v[i4 + u]);
               if (OP == kGemm2Combine) a *= g[u];
-              if (OP == kGemm1Relu) a = fmaxf(a, 0.f);
+              if (OP == kGemm1Relu && !p.plain) a = fmaxf(a, 0.f);
               *reinterpret_cast<__nv_bfloat16*>(tr + (i4 + u) * 64 + lane * 2) = __float2bfloat16(a);
             }
           }
@@ -368,14 +369,14 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
           for (int it = 0; it < 4; ++it) {
             const int rr = it * 8 + (lane >> 2);
             uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (lane & 3) * 16);
-            if (OP == kDgrad2Mask) {                          // ReLU'(u) = [u > 0]: bits saved by the forward GEMM
+            if (OP == kDgrad2Mask && !p.plain) {              // ReLU'(u) = [u > 0]: bits saved by the forward GEMM
               const uint32_t bits = __shfl_sync(0xffffffffu, q_mw[0], rr) >> ((lane & 3) * 8);
               uint32_t* w = reinterpret_cast<uint32_t*>(&val);
 #pragma unroll
               for (int q = 0; q < 4; ++q)
                 w[q] &= ((bits >> (2 * q)) & 1u ? 0x0000FFFFu : 0u) | ((bits >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u);
             }
-            if (OP == kGemm1Relu) {                           // save [H > 0] as one bit per element for the backward pass
+            if (OP == kGemm1Relu && !p.plain) {               // save [H > 0] as one bit per element for the backward pass
               const uint32_t* w = reinterpret_cast<const uint32_t*>(&val);
               uint32_t m8 = 0;
 #pragma unroll
@@ -496,6 +497,8 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   const void* h = ws_ptr<char>(ws, p.h);
   const void* dyd = ws_ptr<char>(ws, p.dyd);
   const void* dh = ws_ptr<char>(ws, p.dh);
+  const int fin = s.fin;                                      // columns of W_in: f, or 2 f for GEGLU experts
+  const void* du = s.geglu ? ws_ptr<char>(ws, p.dab) : dh;    // gradient of the pre-activation(s)
 
   PairParams q{};
   q.op = (int)op;
@@ -512,9 +515,10 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   int K = 0;
   switch (op) {
     case kGemm1Relu:       // A = W_in [E][d (k)][f (m)]: m contiguous -> MN-major; B = X_d [E][C][d] K-major
-      q.token_op = 1; q.a_mn_major = 1; q.Mw = s.f; K = s.d;
-      rc = make_map(&tmA, a.W_in, s.E, s.d, s.f, 64); rc2 = make_map(&tmB, xd, s.E, s.C, s.d, 128);
-      q.out = ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = s.f; break;
+      q.token_op = 1; q.a_mn_major = 1; q.Mw = fin; K = s.d;   // GEGLU: [a | b], 2 f output columns, no ReLU
+      rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 64); rc2 = make_map(&tmB, xd, s.E, s.C, s.d, 128);
+      q.out = s.geglu ? ws_ptr<__nv_bfloat16>(ws, p.ab) : ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = fin;
+      q.plain = s.geglu; break;
     case kGemm2Combine:    // A = W_out [E][f (k)][d (m)] MN-major; B = H [E][C][f] K-major
       q.token_op = 1; q.a_mn_major = 1; q.Mw = s.d; K = s.f;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 64); rc2 = make_map(&tmB, h, s.E, s.C, s.f, 128);
@@ -524,10 +528,10 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
     case kDgrad2Mask:      // A = W_out [E][f (m)][d (k)] K-major; B = dY_d [E][C][d] K-major
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.f; K = s.d;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 128); rc2 = make_map(&tmB, dyd, s.E, s.C, s.d, 128);
-      q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.ld_out = s.f; break;
-    case kDgrad1Scatter:   // A = W_in [E][d (m)][f (k)] K-major; B = dH [E][C][f] K-major
-      q.token_op = 1; q.a_mn_major = 0; q.Mw = s.d; K = s.f;
-      rc = make_map(&tmA, a.W_in, s.E, s.d, s.f, 128); rc2 = make_map(&tmB, dh, s.E, s.C, s.f, 128);
+      q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.ld_out = s.f; q.plain = s.geglu; break;
+    case kDgrad1Scatter:   // A = W_in [E][d (m)][f (k)] K-major; B = dH [E][C][f] K-major  (GEGLU: d[a | b], K = 2 f)
+      q.token_op = 1; q.a_mn_major = 0; q.Mw = s.d; K = fin;
+      rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 128); rc2 = make_map(&tmB, du, s.E, s.C, fin, 128);
       q.out = static_cast<__nv_bfloat16*>(a.dx); q.ld_out = s.d;
       if (s.residual) q.res = static_cast<const __nv_bfloat16*>(a.dy);
       break;
@@ -535,10 +539,10 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
       q.token_op = 0; q.a_mn_major = 1; q.Mw = s.f; q.Nfix = s.d;
       rc = make_map(&tmA, h, s.E, s.C, s.f, 64); rc2 = make_map(&tmB, dyd, s.E, s.C, s.d, 64);
       q.out = static_cast<__nv_bfloat16*>(a.dW_out); q.ld_out = s.d; break;
-    case kWgrad1:          // dW_in [d][f] = X_d^T dH
-      q.token_op = 0; q.a_mn_major = 1; q.Mw = s.d; q.Nfix = s.f;
-      rc = make_map(&tmA, xd, s.E, s.C, s.d, 64); rc2 = make_map(&tmB, dh, s.E, s.C, s.f, 64);
-      q.out = static_cast<__nv_bfloat16*>(a.dW_in); q.ld_out = s.f; break;
+    case kWgrad1:          // dW_in [d][f] = X_d^T dH  (GEGLU: X_d^T d[a | b], 2 f columns)
+      q.token_op = 0; q.a_mn_major = 1; q.Mw = s.d; q.Nfix = fin;
+      rc = make_map(&tmA, xd, s.E, s.C, s.d, 64); rc2 = make_map(&tmB, du, s.E, s.C, fin, 64);
+      q.out = static_cast<__nv_bfloat16*>(a.dW_in); q.ld_out = fin; break;
     default: return SWITCH_MOE_INVALID_ARGUMENT;
   }
   if (rc != SWITCH_MOE_OK || rc2 != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;

@@ -18,6 +18,7 @@ struct SimtProblem {
   void* out; const void* mask_src; int ld_out;
   const void* res;   // combine / scatter with the skip path inside the layer: row added to the output (x or dy)
   void* out2;        // combine with the skip path: second copy of the output without it
+  int plain;         // GEMM1 / dgrad2 without ReLU and mask (GEGLU experts gate elsewhere)
 };
 
 __device__ __forceinline__ float ldf(const float* p) { return *p; }
@@ -93,8 +94,8 @@ __global__ void __launch_bounds__(256) simt_grouped_gemm_kernel(SimtProblem pr) 
       const int n = n0 + tx * 4 + j;
       if (n >= pr.N) continue;
       float v = acc[i][j] * scale;
-      if (OP == kGemm1Relu) v = fmaxf(v, 0.f);
-      if (OP == kDgrad2Mask) v = ldf(static_cast<const ET*>(pr.mask_src) + row + n) > 0.f ? v : 0.f;
+      if (OP == kGemm1Relu && !pr.plain) v = fmaxf(v, 0.f);
+      if (OP == kDgrad2Mask && !pr.plain) v = ldf(static_cast<const ET*>(pr.mask_src) + row + n) > 0.f ? v : 0.f;
       if (OP == kGemm2Combine && pr.out2 != nullptr) stf(static_cast<ET*>(pr.out2) + row + n, v);
       if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && pr.res != nullptr)   // the expert term is rounded first
         v = rnd(static_cast<const ET*>(nullptr), v) + ldf(static_cast<const ET*>(pr.res) + row + n);
@@ -113,31 +114,36 @@ int launch_t(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* 
   pr.gate = ws_ptr<float>(ws, p.gate);
   void* xd = ws_ptr<char>(ws, p.xd); void* h = ws_ptr<char>(ws, p.h);
   void* dyd = ws_ptr<char>(ws, p.dyd); void* dh = ws_ptr<char>(ws, p.dh);
+  const long long fin = s.fin;                               // columns of W_in: f, or 2 f for GEGLU experts
+  void* ab = ws_ptr<char>(ws, p.ab);
+  void* du = s.geglu ? ws_ptr<char>(ws, p.dab) : dh;         // gradient of the pre-activation(s)
   int max_m;
   switch (op) {
-    case kGemm1Relu:      // H[e] (C x f) = ReLU(X_d[e] (C x d) . W_in[e] (d x f))
-      pr = SimtProblem{xd, C * d, d, 1, a.W_in, d * f, f, 1, -1, s.d, s.f, s.C, pr.kept, pr.token_of_slot, pr.gate,
-                       h, nullptr, s.f};
+    case kGemm1Relu:      // H[e] (C x f) = ReLU(X_d[e] (C x d) . W_in[e] (d x f));  GEGLU: [a | b] (C x 2f), no ReLU
+      pr = SimtProblem{xd, C * d, d, 1, a.W_in, d * fin, fin, 1, -1, s.d, s.fin, s.C, pr.kept, pr.token_of_slot,
+                       pr.gate, s.geglu ? ab : h, nullptr, s.fin};
+      pr.plain = s.geglu;
       max_m = s.C; break;
     case kGemm2Combine:   // y[token] = g . (H[e] (C x f) . W_out[e] (f x d))
       pr = SimtProblem{h, C * f, f, 1, a.W_out, f * d, d, 1, -1, s.f, s.d, s.C, pr.kept, pr.token_of_slot, pr.gate,
                        a.y, nullptr, s.d};
       max_m = s.C; break;
-    case kDgrad2Mask:     // dH[e] = (dY_d[e] (C x d) . W_out[e]^T (d x f)) * [H > 0]
+    case kDgrad2Mask:     // dH[e] = (dY_d[e] (C x d) . W_out[e]^T (d x f)) * [H > 0];  GEGLU: no mask
       pr = SimtProblem{dyd, C * d, d, 1, a.W_out, f * d, 1, d, -1, s.d, s.f, s.C, pr.kept, pr.token_of_slot, pr.gate,
                        dh, h, s.f};
+      pr.plain = s.geglu;
       max_m = s.C; break;
-    case kDgrad1Scatter:  // dx[token] = dH[e] (C x f) . W_in[e]^T (f x d)
-      pr = SimtProblem{dh, C * f, f, 1, a.W_in, d * f, 1, f, -1, s.f, s.d, s.C, pr.kept, pr.token_of_slot, pr.gate,
-                       a.dx, nullptr, s.d};
+    case kDgrad1Scatter:  // dx[token] = dH[e] (C x f) . W_in[e]^T (f x d);  GEGLU: d[a | b] (C x 2f)
+      pr = SimtProblem{du, C * fin, fin, 1, a.W_in, d * fin, 1, fin, -1, s.fin, s.d, s.C, pr.kept, pr.token_of_slot,
+                       pr.gate, a.dx, nullptr, s.d};
       max_m = s.C; break;
     case kWgrad2:         // dW_out[e] (f x d) = H[e]^T (f x kept) . dY_d[e] (kept x d)
       pr = SimtProblem{h, C * f, 1, f, dyd, C * d, d, 1, s.f, -1, s.d, s.C, pr.kept, pr.token_of_slot, pr.gate,
                        a.dW_out, nullptr, s.d};
       max_m = s.f; break;
-    case kWgrad1:         // dW_in[e] (d x f) = X_d[e]^T (d x kept) . dH[e] (kept x f)
-      pr = SimtProblem{xd, C * d, 1, d, dh, C * f, f, 1, s.d, -1, s.f, s.C, pr.kept, pr.token_of_slot, pr.gate,
-                       a.dW_in, nullptr, s.f};
+    case kWgrad1:         // dW_in[e] (d x f) = X_d[e]^T (d x kept) . dH[e] (kept x f);  GEGLU: d[a | b], 2f columns
+      pr = SimtProblem{xd, C * d, 1, d, du, C * fin, fin, 1, s.d, -1, s.fin, s.C, pr.kept, pr.token_of_slot, pr.gate,
+                       a.dW_in, nullptr, s.fin};
       max_m = s.d; break;
     default: return SWITCH_MOE_INVALID_ARGUMENT;
   }

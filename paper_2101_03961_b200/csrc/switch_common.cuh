@@ -32,6 +32,8 @@ struct Shape {
   int router_blocks, plan_blocks, max_mtiles, dwr_chunks;
   int residual;     // 1: y = x + layer(x), dx = dy + d layer / dx (SWITCH_MOE_FLAG_RESIDUAL)
   int reroute;      // 1: overflowed tokens are offered to their second-choice expert (SWITCH_MOE_FLAG_REROUTE)
+  int geglu;        // 1: GEGLU experts: W_in is [E, d, 2 f] (SWITCH_MOE_FLAG_GEGLU)
+  int fin;          // columns of W_in per expert: f, or 2 f for GEGLU
   int jitter;       // 1: the router's input is x . u (SWITCH_MOE_FLAG_INPUT_JITTER)
   const void* jitter_u;   // device [T, d] factors u (activation dtype); may be null when only sizes are asked for
 };
@@ -39,7 +41,7 @@ struct Shape {
 // Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
 struct Plan {
   size_t status, expert_index, gate, slot, token_of_slot, count, kept, count_g, group_base, psum, psum_partial, hist, hist_base,
-      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, layer_y, alt, expert_proc, xr, total;
+      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, layer_y, alt, expert_proc, xr, ab, dab, total;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -60,7 +62,8 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (cfg->T % G != 0) return SWITCH_MOE_INVALID_ARGUMENT;
   if (G > 1 && ((cfg->T / G) % kPlanBlockTokens != 0 || cfg->T > 65536 || G > kMaxGroups))
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
-  if ((cfg->flags & ~(SWITCH_MOE_FLAG_RESIDUAL | SWITCH_MOE_FLAG_REROUTE | SWITCH_MOE_FLAG_INPUT_JITTER)) != 0)
+  if ((cfg->flags & ~(SWITCH_MOE_FLAG_RESIDUAL | SWITCH_MOE_FLAG_REROUTE | SWITCH_MOE_FLAG_INPUT_JITTER |
+                      SWITCH_MOE_FLAG_GEGLU)) != 0)
     return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->E > kMaxExperts) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if (cfg->d_model % 8 != 0 || cfg->d_ff % 8 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
@@ -83,6 +86,9 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (s->gemm_path != 1 && (cfg->d_model % 64 != 0 || cfg->d_ff % 64 != 0)) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   s->residual = (cfg->flags & SWITCH_MOE_FLAG_RESIDUAL) ? 1 : 0;
   if (s->residual && s->gemm_path == SWITCH_MOE_GEMM_TC_1CTA) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->geglu = (cfg->flags & SWITCH_MOE_FLAG_GEGLU) ? 1 : 0;
+  s->fin = s->geglu ? 2 * cfg->d_ff : cfg->d_ff;
+  if (s->geglu && s->gemm_path == SWITCH_MOE_GEMM_TC_1CTA) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   s->jitter = (cfg->flags & SWITCH_MOE_FLAG_INPUT_JITTER) ? 1 : 0;
   s->jitter_u = s->jitter ? cfg->router_jitter : nullptr;
   s->reroute = (cfg->flags & SWITCH_MOE_FLAG_REROUTE) ? 1 : 0;
@@ -148,6 +154,8 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->alt = s.reroute ? take(T * 4) : 0;                     // second choice of overflowed tokens, -1 for the others
   p->expert_proc = s.reroute ? take(T * 4) : p->expert_index;   // the expert that processes each token
   p->xr = s.jitter ? take(T * d * s.elt) : 0;               // the router's input x . u, rounded to the activation dtype
+  p->ab = s.geglu ? take(E * C * 2 * f * s.elt) : 0;        // GEGLU: [a | b] = X_d [W_0 | W_1] per slot
+  p->dab = s.geglu ? take(E * C * 2 * f * s.elt) : 0;       // GEGLU: gradient of [a | b] per slot
   p->total = off;
 }
 
@@ -227,5 +235,8 @@ struct GemmArgs {
 int launch_simt_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
 int launch_tc_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
 int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
+// GEGLU gating over the kept rows: H = GELU(a) . b, and its derivative d[a | b] from dH (element-wise).
+int launch_geglu_fwd(const Shape& s, const Plan& p, void* ws, cudaStream_t st);
+int launch_geglu_bwd(const Shape& s, const Plan& p, void* ws, cudaStream_t st);
 
 }  // namespace swmoe

@@ -41,6 +41,11 @@ class SwitchConfig:
     dtype: int = DTYPE_BF16          # DTYPE_BF16: x, W_in, W_out, dy in bf16, router in fp32; DTYPE_F32: all fp32
     bias_std: float = 0.0            # std of the fixed per-expert router-logit bias (0 = no bias)
     init_scale: float = 0.1          # the paper's s in sigma = sqrt(s / fan_in)
+    geglu: bool = False              # GEGLU experts: W_in holds [W_0 | W_1], 2 d_ff columns per expert
+
+    @property
+    def w_in_cols(self) -> int:
+        return 2 * self.d_ff if self.geglu else self.d_ff
 
     def with_(self, **kw) -> "SwitchConfig":
         return replace(self, **kw)
@@ -59,6 +64,8 @@ CONFIGS = {
     # a quarter of switch_base (same tokens per expert, same d_model / d_ff): small enough for profiler captures,
     # still larger than L2 (2 x 151 MB of weights)
     "switch_base_quarter": SwitchConfig("switch_base_quarter", 8192, 768, 3072, 32, 1.25),
+    # the paper's own Switch-Base layer shape with GEGLU experts (its hyper-parameter table: d_model 768, d_ff 2048)
+    "geglu_base": SwitchConfig("geglu_base", 32768, 768, 2048, 128, 1.25, geglu=True),
 }
 
 
@@ -151,9 +158,9 @@ def storage_round(cfg: SwitchConfig):
 
 
 def gen_W_in_expert(cfg: SwitchConfig, e: int, seed: int = 0) -> np.ndarray:
-    """Expert e's expansion matrix [d_model, d_ff] (fan-in d_model)."""
+    """Expert e's expansion matrix [d_model, d_ff] (fan-in d_model); [d_model, 2 d_ff] = [W_0 | W_1] for GEGLU experts."""
     sigma = math.sqrt(cfg.init_scale / cfg.d_model)
-    return _finish(cfg, _truncated_normal(_rng(seed, _TENSOR_WIN, e), (cfg.d_model, cfg.d_ff), sigma))
+    return _finish(cfg, _truncated_normal(_rng(seed, _TENSOR_WIN, e), (cfg.d_model, cfg.w_in_cols), sigma))
 
 
 def gen_W_out_expert(cfg: SwitchConfig, e: int, seed: int = 0) -> np.ndarray:
@@ -180,7 +187,7 @@ def _stack_experts(fn, cfg: SwitchConfig, seed: int, shape, as_bits: bool, threa
 
 def gen_W_in(cfg: SwitchConfig, seed: int = 0, as_bits: bool = False, threads: int = 8) -> np.ndarray:
     """All experts' W_in [E, d_model, d_ff]; float32 values, or uint16 bf16 patterns if as_bits."""
-    return _stack_experts(gen_W_in_expert, cfg, seed, (cfg.d_model, cfg.d_ff), as_bits, threads)
+    return _stack_experts(gen_W_in_expert, cfg, seed, (cfg.d_model, cfg.w_in_cols), as_bits, threads)
 
 
 def gen_W_out(cfg: SwitchConfig, seed: int = 0, as_bits: bool = False, threads: int = 8) -> np.ndarray:

@@ -42,13 +42,15 @@ class GpuLayer:
     """Device buffers of one layer call plus the library calls on them."""
 
     def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0,
-                 residual=False, groups=1, reroute=False):
+                 residual=False, groups=1, reroute=False, geglu=False):
         sbuild.build()
+        geglu = geglu or cfg.geglu
         jit = data.get("router_jitter")
         self.scfg = cfg
         self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
                                   dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path,
-                                  residual=residual, groups=groups, reroute=reroute, input_jitter=jit is not None)
+                                  residual=residual, groups=groups, reroute=reroute, input_jitter=jit is not None,
+                                  geglu=geglu)
         dt = cfg.dtype
         self.x = to_dev(data["x"], dt)
         self.dy = to_dev(data["dy"], dt)
@@ -120,13 +122,13 @@ def check_second_choice(gpu_alt: np.ndarray, p: np.ndarray, e: np.ndarray, overf
 
 
 def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capacity=None, experts=None,
-                     residual=False, groups=1, gpu_alt=None):
+                     residual=False, groups=1, gpu_alt=None, geglu=False):
     """Oracle forward with the device's expert choice (identical unless a near-tie flipped), after checking flips."""
-    jit_kw = {}
+    jit_kw = {"geglu": True} if (geglu or cfg.geglu) else {}
     if data.get("router_jitter") is not None:                  # the router sees x . u rounded to the activation type
-        jit_kw = {"router_jitter": data["router_jitter"], "storage_round": si.storage_round(cfg)}
+        jit_kw.update({"router_jitter": data["router_jitter"], "storage_round": si.storage_round(cfg)})
     if groups > 1:
-        assert capacity is None
+        assert capacity is None and not jit_kw
         first = so.switch_forward_groups(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
                                          cfg.alpha, groups, router_bias=data.get("router_bias"), experts=[])
         flips = check_flips(gpu_e, first)
@@ -169,3 +171,12 @@ def expert_preactivation(fwd: dict, i: int):
         return fwd["u"].get(i)
     rows = [q["u"][i] for q in fwd["parts"] if i in q["u"]]
     return np.concatenate(rows, axis=0) if rows else None
+
+
+def expert_hidden(fwd: dict, i: int):
+    """The hidden activations of expert i's rows in slot order: ReLU(u), or GELU(a) . b for GEGLU experts."""
+    u = expert_preactivation(fwd, i)
+    if fwd.get("geglu", False):
+        fh = u.shape[1] // 2
+        return so.gelu(u[:, :fh]) * u[:, fh:]
+    return np.maximum(u, 0.0)

@@ -12,7 +12,7 @@ from oracle import switch_oracle as so
 from paper_2101_03961_b200 import build as sbuild
 from paper_2101_03961_b200 import inputs as si
 from paper_2101_03961_b200 import switch_moe as sm
-from tests.gpu_helpers import (TOL_BF16, TOL_ROUTER, check_flips, check_second_choice, expert_preactivation, rel_err,
+from tests.gpu_helpers import (TOL_BF16, TOL_ROUTER, check_flips, check_second_choice, expert_hidden, rel_err,
                                skip_path_ok, to_np)
 
 pytestmark = pytest.mark.gpu
@@ -34,7 +34,7 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False, groups=1, reroute=Fal
     W_r = torch.from_numpy(W_r_np).cuda()
     bias = None if b_np is None else torch.from_numpy(b_np).cuda()
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, residual=residual,
-                          groups=groups, reroute=reroute)
+                          groups=groups, reroute=reroute, geglu=cfg.geglu)
     ws = sm.allocate_workspace(mcfg)
     ws.fill_(0xFF)
     y, dx = torch.full_like(x, float("nan")), torch.full_like(x, float("nan"))
@@ -88,7 +88,8 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False, groups=1, reroute=Fal
     W_out_s = {i: si.gen_W_out_expert(cfg, i, seed) for i in sample}
     if groups == 1:
         fwd = so.switch_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, router_bias=b_np,
-                                expert_index=gpu_e, experts=sample, residual=residual, reroute=reroute, alt_index=alt)
+                                expert_index=gpu_e, experts=sample, residual=residual, reroute=reroute, alt_index=alt,
+                                geglu=cfg.geglu)
         bwd = so.switch_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
     else:
         fwd = so.switch_forward_groups(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, groups,
@@ -101,7 +102,7 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False, groups=1, reroute=Fal
         k = int(plan["kept"][i])
         tok = plan["token_of_slot"][i * C:i * C + k]           # the expert's tokens in slot order
         tt = torch.from_numpy(tok).cuda()
-        errs[f"H[{i}]"] = rel_err(to_np(hid[i, :k]), np.maximum(expert_preactivation(fwd, i), 0.0))
+        errs[f"H[{i}]"] = rel_err(to_np(hid[i, :k]), expert_hidden(fwd, i))
         if residual:
             layer_y = view(sm.WS_LAYER_Y).view(T, cfg.d_model)
             errs[f"layer_y[{i}]"] = rel_err(to_np(layer_y[tt]), fwd["layer_y"][tok])
@@ -175,3 +176,7 @@ def test_overflow_stress_with_rerouting_full_size():
     out = _run_fullsize("stress_calibrated", reroute=True)
     # capacity factor 1: the experts' slots add up to exactly T, so only part of the 31% overflow finds a second home
     assert out["dropped"] < 0.25 * 32768
+
+
+def test_geglu_experts_at_the_papers_switch_base_shape_full_size():
+    _run_fullsize("geglu_base")

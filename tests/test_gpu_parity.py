@@ -12,8 +12,8 @@ import torch
 from oracle import switch_oracle as so
 from paper_2101_03961_b200 import inputs as si
 from paper_2101_03961_b200 import switch_moe as sm
-from tests.gpu_helpers import (TOL_BF16, TOL_F32, TOL_ROUTER, GpuLayer, check_flips, expert_preactivation,
-                               oracle_following, rel_err, skip_path_ok, to_np)
+from tests.gpu_helpers import (TOL_BF16, TOL_F32, TOL_ROUTER, GpuLayer, check_flips, expert_hidden, oracle_following,
+                               rel_err, skip_path_ok, to_np)
 
 pytestmark = pytest.mark.gpu
 
@@ -120,19 +120,22 @@ def test_dispatch_plan_is_deterministic():
 
 # ---------------------------------------------------------------------------------------------- whole layer
 def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False, groups=1,
-                 reroute=False, noise_eps=0.0, jitter_eps=0.0):
+                 reroute=False, noise_eps=0.0, jitter_eps=0.0, geglu=False):
+    if geglu:                                                  # W_in = [W_0 | W_1]: twice the columns
+        cfg = cfg.with_(geglu=True)
     data = si.gen_layer(cfg, seed=seed)
     if jitter_eps:
         data["router_jitter"] = si.gen_router_jitter(cfg, jitter_eps, seed)
     if noise_eps:
         data["router_noise"] = si.gen_router_noise(cfg, noise_eps, seed)
     g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual,
-                 groups=groups, reroute=reroute)
+                 groups=groups, reroute=reroute, geglu=geglu)
     g.fwd()
     gpu_e = g.expert_index()
     cap = capacity_override if capacity_override else None
     gpu_alt = g.view(sm.WS_SECOND_CHOICE).cpu().numpy().astype(np.int64) if reroute else None
-    fwd = oracle_following(cfg, data, gpu_e, capacity=cap, residual=residual, groups=groups, gpu_alt=gpu_alt)
+    fwd = oracle_following(cfg, data, gpu_e, capacity=cap, residual=residual, groups=groups, gpu_alt=gpu_alt,
+                           geglu=geglu)
     if reroute:
         np.testing.assert_array_equal(g.view(sm.WS_EXPERT_PROC).cpu().numpy(), fwd["e_proc"])
         np.testing.assert_allclose(to_np(g.view(sm.WS_GATE))[fwd["keep"]], fwd["g"][fwd["keep"]], rtol=2e-5)
@@ -158,7 +161,7 @@ def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, re
             continue
         tok = fwd["token_of_slot"][i * C:i * C + k]
         np.testing.assert_array_equal(xd[i, :k], x64[tok])
-        errs[f"H[{i}]"] = rel_err(hid[i, :k], np.maximum(expert_preactivation(fwd, i), 0.0))
+        errs[f"H[{i}]"] = rel_err(hid[i, :k], expert_hidden(fwd, i))
     y = to_np(g.y)
     assert np.isfinite(y).all()
     if residual:
@@ -295,6 +298,15 @@ def test_jitter_flag_without_the_factors_is_refused():
     W_r = torch.zeros(MID.d_model, MID.E, device="cuda")
     with pytest.raises(sm.SwitchMoeError):
         sm.switch_moe_router_fwd(cfg, x, W_r, None, ws)
+
+
+@pytest.mark.parametrize("cfg,path,tol,residual", [
+    (TINY, sm.GEMM_DEFAULT, TOL_F32, False), (MID, sm.GEMM_SIMT, TOL_BF16, False), (MID, sm.GEMM_DEFAULT, TOL_BF16, False),
+    (RAGGED, sm.GEMM_DEFAULT, TOL_BF16, False), (MANY, sm.GEMM_DEFAULT, TOL_BF16, True)],
+    ids=["tiny_f32", "mid_fma", "mid_tc", "ragged_tc", "many_tc_skip"])
+def test_geglu_experts_match_oracle(cfg, path, tol, residual):
+    """hidden = GELU(x W_0) . (x W_1) (Table 9): one grouped GEMM with 2 d_ff columns, gating and its derivative after."""
+    _check_layer(cfg, path, tol, geglu=True, residual=residual, d_aux=0.7)
 
 
 def test_rerouting_is_refused_with_several_routing_groups():
