@@ -343,12 +343,43 @@ def run_ours(args, cfg):
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         host_step()                                           # synchronises the stream before returning
+    blocking_s = (time.perf_counter() - t0) / e2e_steps
+
+    # the same step kept two deep with the non-blocking call: step i + 1 uploads while step i computes and step i - 1
+    # downloads; every step still copies its own inputs in and its own results out
+    slots = []
+    for _ in range(2):
+        slots.append({"x": torch.empty_like(x), "dy": torch.empty_like(dy), "y": torch.empty_like(y),
+                      "dx": torch.empty_like(dx), "aux": torch.zeros(1, device="cuda"),
+                      "yh": torch.empty_like(xh).pin_memory(), "dxh": torch.empty_like(xh).pin_memory(),
+                      "auxh": torch.zeros(1).pin_memory(), "done": None})
+
+    def pipelined(n):
+        for i in range(n):
+            sl = slots[i % 2]
+            done = torch.cuda.Event()
+            sm.switch_moe_step_host_enqueue(mcfg, xh, dyh, 1.0, W_r, bias, W_in, W_out, sl["x"], sl["dy"], sl["y"],
+                                            sl["dx"], sl["aux"], dW_r, dW_in, dW_out, sl["yh"], sl["dxh"], sl["auxh"],
+                                            ws, stream, up_stream, down_stream, sl["done"], done)
+            sl["done"] = done
+        for sl in slots:
+            if sl["done"] is not None:
+                sl["done"].synchronize()
+
+    pipelined(2)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    pipelined(e2e_steps)
     e2e_s = (time.perf_counter() - t0) / e2e_steps
+    sm.switch_moe_check_device_status(mcfg, ws, stream)
+    assert torch.equal(slots[0]["yh"], yh) and torch.equal(slots[1]["dxh"], dxh)   # same results as the blocking call
     act_bytes = cfg.T * row_bytes
     e2e = {"value": world * cfg.T / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 2 * act_bytes,
            "d2h_bytes_per_step": 2 * act_bytes + 4, "ms_per_step": e2e_s * 1e3,
-           "note": "x, dy copied from pinned host memory; y, dx, aux copied back (dy upload overlaps forward, y "
-                   "download overlaps backward); weights and weight gradients resident"}
+           "blocking_call_value": world * cfg.T / blocking_s, "blocking_call_ms_per_step": blocking_s * 1e3,
+           "note": "switch_moe_step_host_enqueue, two steps in flight: every step copies x, dy from pinned host memory "
+                   "and y, dx, aux back; weights and weight gradients resident.  blocking_call_*: switch_moe_step_host, "
+                   "one step at a time (dy upload overlaps forward, y download overlaps backward)"}
 
     # ---- CPU baseline: the oracle on a bounded sample, this machine's host cores
     cpu = None

@@ -224,6 +224,21 @@ int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const
                          void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host, void* workspace,
                          size_t workspace_bytes, void* stream, void* h2d_stream, void* d2h_stream);
 
+/* The same step without the final synchronisation, for callers that keep several steps in flight: everything is
+ * enqueued and the call returns.  h2d_stream and d2h_stream are required.  slot_free_event (cudaEvent_t, may be NULL):
+ * the uploads into x_dev / dy_dev wait for it instead of for the work already enqueued on `stream` -- pass the
+ * step_done_event of the step that last used these staging buffers.  step_done_event (cudaEvent_t, required) is
+ * recorded on d2h_stream after the last download: y_host, dx_host and aux_host are valid, and the host inputs and all
+ * staging buffers reusable, once it has completed.  The kernels of all steps share `stream`, so one workspace and one
+ * set of weight-gradient buffers serve every step in flight; only the five staging buffers (and the host result
+ * buffers) need one copy per step in flight. */
+int switch_moe_step_host_enqueue(const switch_moe_config* cfg, const void* x_host, const void* dy_host, float d_aux,
+                                 const float* W_r, const float* router_bias, const void* W_in, const void* W_out,
+                                 void* x_dev, void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r,
+                                 void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host,
+                                 void* workspace, size_t workspace_bytes, void* stream, void* h2d_stream,
+                                 void* d2h_stream, void* slot_free_event, void* step_done_event);
+
 /* Synchronises `stream`, reads the workspace's status word and returns SWITCH_MOE_DEVICE_TIMEOUT if a kernel
  * gave up on a bounded wait (its results are then invalid), SWITCH_MOE_CUDA_ERROR if the stream reports an
  * error, else SWITCH_MOE_OK.  info_out (HOST int32[16], may be NULL) receives the raw status words. */

@@ -192,28 +192,32 @@ int switch_moe_router_bwd(const switch_moe_config* cfg, const void* x, const flo
                            static_cast<cudaStream_t>(stream));
 }
 
-int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const void* dy_host, float d_aux,
-                         const float* W_r, const float* router_bias, const void* W_in, const void* W_out,
-                         void* x_dev, void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r,
-                         void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host, void* workspace,
-                         size_t workspace_bytes, void* stream, void* h2d_stream, void* d2h_stream) {
+namespace {
+// Shared body of the two host-activation entry points.  `slot_free` (may be null): event the uploads wait for instead
+// of the work already enqueued on `stream`; `step_done` (may be null): recorded on the download stream after the last
+// copy.  Returns with everything enqueued; nothing is synchronised here.
+int step_host_enqueue(const switch_moe_config* cfg, const void* x_host, const void* dy_host, float d_aux,
+                      const float* W_r, const float* router_bias, const void* W_in, const void* W_out, void* x_dev,
+                      void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r, void* dW_in, void* dW_out,
+                      void* y_host, void* dx_host, float* aux_host, void* workspace, size_t workspace_bytes,
+                      cudaStream_t st, cudaStream_t up, cudaStream_t down, cudaEvent_t slot_free,
+                      cudaEvent_t step_done) {
   Ctx c;
   SWMOE_TRY(prepare(cfg, workspace, workspace_bytes, true, &c));
   if (!x_host || !dy_host || !x_dev || !dy_dev || !y_dev || !dx_dev || !aux_dev || !y_host || !dx_host || !aux_host)
     return SWITCH_MOE_INVALID_ARGUMENT;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // Optional copy streams let dy travel to the device during the forward pass and y travel back during the
-  // backward pass.  Without them (NULL) every copy is ordered on `stream`.
-  cudaStream_t up = h2d_stream ? static_cast<cudaStream_t>(h2d_stream) : st;
-  cudaStream_t down = d2h_stream ? static_cast<cudaStream_t>(d2h_stream) : st;
   const size_t act = (size_t)c.s.T * c.s.d * c.s.elt;
   cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // start, x up, dy up, fwd done, bwd done
   int rc = SWITCH_MOE_OK;
   auto ck = [&](cudaError_t e) { if (e != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR; };
   for (int i = 0; i < 5; ++i) ck(cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming));
   if (rc == SWITCH_MOE_OK) {
-    ck(cudaEventRecord(ev[0], st));                            // copies start after earlier work on `stream`
-    if (up != st) ck(cudaStreamWaitEvent(up, ev[0], 0));
+    if (slot_free != nullptr) {
+      ck(cudaStreamWaitEvent(up, slot_free, 0));               // the staging buffers' previous user has finished
+    } else {
+      ck(cudaEventRecord(ev[0], st));                          // copies start after earlier work on `stream`
+      if (up != st) ck(cudaStreamWaitEvent(up, ev[0], 0));
+    }
     ck(cudaMemcpyAsync(x_dev, x_host, act, cudaMemcpyHostToDevice, up));
     ck(cudaEventRecord(ev[1], up));
     ck(cudaMemcpyAsync(dy_dev, dy_host, act, cudaMemcpyHostToDevice, up));
@@ -221,7 +225,7 @@ int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const
     if (up != st) ck(cudaStreamWaitEvent(st, ev[1], 0));
   }
   if (rc == SWITCH_MOE_OK)
-    rc = switch_moe_fwd(cfg, x_dev, W_r, router_bias, W_in, W_out, y_dev, aux_dev, workspace, workspace_bytes, stream);
+    rc = switch_moe_fwd(cfg, x_dev, W_r, router_bias, W_in, W_out, y_dev, aux_dev, workspace, workspace_bytes, st);
   if (rc == SWITCH_MOE_OK) {
     ck(cudaEventRecord(ev[3], st));
     if (down != st) ck(cudaStreamWaitEvent(down, ev[3], 0));
@@ -231,19 +235,52 @@ int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const
   }
   if (rc == SWITCH_MOE_OK)
     rc = switch_moe_bwd(cfg, dy_dev, d_aux, x_dev, W_r, W_in, W_out, y_dev, workspace, workspace_bytes, dx_dev, dW_r,
-                        dW_in, dW_out, stream);
+                        dW_in, dW_out, st);
   if (rc == SWITCH_MOE_OK) {
     ck(cudaEventRecord(ev[4], st));
     if (down != st) ck(cudaStreamWaitEvent(down, ev[4], 0));
     ck(cudaMemcpyAsync(dx_host, dx_dev, act, cudaMemcpyDeviceToHost, down));
+    if (step_done != nullptr) ck(cudaEventRecord(step_done, down));
   }
-  // always drain what was enqueued, also after an error, before the events go away
-  if (cudaStreamSynchronize(up) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
-  if (cudaStreamSynchronize(st) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
-  if (cudaStreamSynchronize(down) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
+  // an event that has been recorded but not reached yet is released when it completes
   for (int i = 0; i < 5; ++i)
     if (ev[i] != nullptr) cudaEventDestroy(ev[i]);
   return rc;
+}
+}  // namespace
+
+int switch_moe_step_host(const switch_moe_config* cfg, const void* x_host, const void* dy_host, float d_aux,
+                         const float* W_r, const float* router_bias, const void* W_in, const void* W_out,
+                         void* x_dev, void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r,
+                         void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host, void* workspace,
+                         size_t workspace_bytes, void* stream, void* h2d_stream, void* d2h_stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // Optional copy streams let dy travel to the device during the forward pass and y travel back during the
+  // backward pass.  Without them (NULL) every copy is ordered on `stream`.
+  cudaStream_t up = h2d_stream ? static_cast<cudaStream_t>(h2d_stream) : st;
+  cudaStream_t down = d2h_stream ? static_cast<cudaStream_t>(d2h_stream) : st;
+  int rc = step_host_enqueue(cfg, x_host, dy_host, d_aux, W_r, router_bias, W_in, W_out, x_dev, dy_dev, y_dev, dx_dev,
+                             aux_dev, dW_r, dW_in, dW_out, y_host, dx_host, aux_host, workspace, workspace_bytes, st,
+                             up, down, nullptr, nullptr);
+  // always drain what was enqueued, also after an error
+  if (cudaStreamSynchronize(up) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
+  if (cudaStreamSynchronize(st) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
+  if (cudaStreamSynchronize(down) != cudaSuccess && rc == SWITCH_MOE_OK) rc = SWITCH_MOE_CUDA_ERROR;
+  return rc;
+}
+
+int switch_moe_step_host_enqueue(const switch_moe_config* cfg, const void* x_host, const void* dy_host, float d_aux,
+                                 const float* W_r, const float* router_bias, const void* W_in, const void* W_out,
+                                 void* x_dev, void* dy_dev, void* y_dev, void* dx_dev, float* aux_dev, float* dW_r,
+                                 void* dW_in, void* dW_out, void* y_host, void* dx_host, float* aux_host,
+                                 void* workspace, size_t workspace_bytes, void* stream, void* h2d_stream,
+                                 void* d2h_stream, void* slot_free_event, void* step_done_event) {
+  if (h2d_stream == nullptr || d2h_stream == nullptr || step_done_event == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
+  return step_host_enqueue(cfg, x_host, dy_host, d_aux, W_r, router_bias, W_in, W_out, x_dev, dy_dev, y_dev, dx_dev,
+                           aux_dev, dW_r, dW_in, dW_out, y_host, dx_host, aux_host, workspace, workspace_bytes,
+                           static_cast<cudaStream_t>(stream), static_cast<cudaStream_t>(h2d_stream),
+                           static_cast<cudaStream_t>(d2h_stream), static_cast<cudaEvent_t>(slot_free_event),
+                           static_cast<cudaEvent_t>(step_done_event));
 }
 
 int switch_moe_check_device_status(const switch_moe_config* cfg, void* workspace, int32_t* info_out, void* stream) {

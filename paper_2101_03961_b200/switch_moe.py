@@ -29,8 +29,8 @@ FLAG_RESIDUAL, FLAG_REROUTE, FLAG_INPUT_JITTER, FLAG_GEGLU = 1, 2, 4, 8
 EXPORTED_SYMBOLS = [
     "switch_moe_capacity", "switch_moe_workspace_bytes", "switch_moe_workspace_view", "switch_moe_fwd",
     "switch_moe_bwd", "switch_moe_router_fwd", "switch_moe_dispatch_plan", "switch_moe_router_bwd",
-    "switch_moe_dispatch_plan_static", "switch_moe_step_host", "switch_moe_check_device_status", "switch_moe_launches_per_step",
-    "switch_moe_status_string",
+    "switch_moe_dispatch_plan_static", "switch_moe_step_host", "switch_moe_step_host_enqueue",
+    "switch_moe_check_device_status", "switch_moe_launches_per_step", "switch_moe_status_string",
 ]
 
 
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.switch_moe_dispatch_plan_static.argtypes = [cp, vp, vp, vp, vp, vp, vp]
     lib.switch_moe_router_bwd.argtypes = [cp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp, vp, vp]
     lib.switch_moe_step_host.argtypes = [cp, vp, vp, ctypes.c_float] + [vp] * 15 + [vp, ctypes.c_size_t, vp, vp, vp]
+    lib.switch_moe_step_host_enqueue.argtypes = lib.switch_moe_step_host.argtypes + [vp, vp]
     lib.switch_moe_check_device_status.argtypes = [cp, vp, i32p, vp]
     lib.switch_moe_launches_per_step.argtypes = [cp, i32p]
     lib.switch_moe_status_string.argtypes = [ctypes.c_int]
@@ -225,6 +226,23 @@ def switch_moe_step_host(cfg, x_host, dy_host, d_aux, W_r, router_bias, W_in, W_
         _ptr(dW_out), _ptr(y_host), _ptr(dx_host), _ptr(aux_host), _ptr(workspace), workspace.numel(),
         _stream(stream), None if h2d_stream is None else _stream(h2d_stream),
         None if d2h_stream is None else _stream(d2h_stream)), "switch_moe_step_host")
+
+
+def switch_moe_step_host_enqueue(cfg, x_host, dy_host, d_aux, W_r, router_bias, W_in, W_out, x_dev, dy_dev, y_dev, dx_dev,
+                                 aux_dev, dW_r, dW_in, dW_out, y_host, dx_host, aux_host, workspace, stream, h2d_stream,
+                                 d2h_stream, slot_free_event, step_done_event) -> None:
+    """Non-blocking step: `slot_free_event` / `step_done_event` are torch.cuda.Event objects (the first may be None).
+    torch creates the CUDA event behind an Event object on its first record(), so `step_done_event` is recorded once
+    on `d2h_stream` here before its handle is passed down (the library records it again after the last download)."""
+    if not step_done_event.cuda_event:
+        step_done_event.record(d2h_stream)
+    _check(load_library().switch_moe_step_host_enqueue(
+        ctypes.byref(cfg), _ptr(x_host), _ptr(dy_host), float(d_aux), _ptr(W_r), _ptr(router_bias), _ptr(W_in),
+        _ptr(W_out), _ptr(x_dev), _ptr(dy_dev), _ptr(y_dev), _ptr(dx_dev), _ptr(aux_dev), _ptr(dW_r), _ptr(dW_in),
+        _ptr(dW_out), _ptr(y_host), _ptr(dx_host), _ptr(aux_host), _ptr(workspace), workspace.numel(),
+        _stream(stream), _stream(h2d_stream), _stream(d2h_stream),
+        None if slot_free_event is None else ctypes.c_void_p(slot_free_event.cuda_event),
+        ctypes.c_void_p(step_done_event.cuda_event)), "switch_moe_step_host_enqueue")
 
 
 def switch_moe_check_device_status(cfg, workspace, stream=None) -> list:

@@ -5,6 +5,8 @@ the tolerances in gpu_helpers (router 1e-5; bf16 tensors 2e-2 relative Frobenius
 Argmax flips are counted and allowed only inside a top-2 probability gap of 1e-4; the oracle then follows the
 device's expert choice, because a single flip moves every later slot of two experts.
 """
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -416,3 +418,51 @@ def test_step_with_host_activations_equals_device_calls(extra_streams):
     assert torch.equal(yh.cuda(), y_ref) and torch.equal(dxh.cuda(), dx_ref)
     assert float(auxh.item()) == aux_ref
     assert torch.equal(g.dW_in, dW_in_ref)
+
+
+def test_steps_kept_in_flight_give_the_results_of_the_blocking_call():
+    """switch_moe_step_host_enqueue with two staging slots and different inputs per step: every step's host results
+    equal those of a blocking call on the same inputs."""
+    cfg = MID
+    layers = [GpuLayer(cfg, si.gen_layer(cfg, seed=s)) for s in (7, 8, 9)]
+    g = layers[0]                                            # its weights, workspace and gradient buffers serve all steps
+    hosts = []
+    for other in layers:
+        xh, dyh = other.x.cpu().pin_memory(), other.dy.cpu().pin_memory()
+        yh, dxh = torch.empty_like(xh).pin_memory(), torch.empty_like(xh).pin_memory()
+        auxh = torch.zeros(1).pin_memory()
+        x_dev, dy_dev = torch.zeros_like(g.x), torch.zeros_like(g.x)
+        sm.switch_moe_step_host(g.cfg, xh, dyh, 1.0, g.W_r, g.bias, g.W_in, g.W_out, x_dev, dy_dev, g.y, g.dx, g.aux,
+                                g.dW_r, g.dW_in, g.dW_out, yh, dxh, auxh, g.ws)
+        hosts.append({"xh": xh, "dyh": dyh, "y": yh.clone(), "dx": dxh.clone(), "aux": float(auxh.item()),
+                      "dW_in": g.dW_in.clone()})
+    slots = [{"x": torch.zeros_like(g.x), "dy": torch.zeros_like(g.x), "y": torch.zeros_like(g.x),
+              "dx": torch.zeros_like(g.x), "aux": torch.zeros(1, device="cuda"), "done": None} for _ in range(2)]
+    main, up, down = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = []
+    for i, h in enumerate(hosts):
+        sl = slots[i % 2]
+        yh, dxh = torch.empty_like(h["xh"]).pin_memory(), torch.empty_like(h["xh"]).pin_memory()
+        auxh = torch.zeros(1).pin_memory()
+        done = torch.cuda.Event()
+        sm.switch_moe_step_host_enqueue(g.cfg, h["xh"], h["dyh"], 1.0, g.W_r, g.bias, g.W_in, g.W_out, sl["x"],
+                                        sl["dy"], sl["y"], sl["dx"], sl["aux"], g.dW_r, g.dW_in, g.dW_out, yh, dxh,
+                                        auxh, g.ws, main, up, down, sl["done"], done)
+        sl["done"] = done
+        outs.append((yh, dxh, auxh, done))
+    for (yh, dxh, auxh, done), h in zip(outs, hosts):
+        done.synchronize()
+        assert torch.equal(yh, h["y"]) and torch.equal(dxh, h["dx"]) and float(auxh.item()) == h["aux"]
+    torch.cuda.synchronize()
+    assert torch.equal(g.dW_in, hosts[-1]["dW_in"])           # the gradient buffers hold the last step's gradients
+    sm.switch_moe_check_device_status(g.cfg, g.ws)
+    # the copy streams and the completion event are required
+    h = hosts[0]
+    rc = sm.load_library().switch_moe_step_host_enqueue(
+        ctypes.byref(g.cfg), h["xh"].data_ptr(), h["dyh"].data_ptr(), 1.0, g.W_r.data_ptr(), None, g.W_in.data_ptr(),
+        g.W_out.data_ptr(), slots[0]["x"].data_ptr(), slots[0]["dy"].data_ptr(), slots[0]["y"].data_ptr(),
+        slots[0]["dx"].data_ptr(), slots[0]["aux"].data_ptr(), g.dW_r.data_ptr(), g.dW_in.data_ptr(),
+        g.dW_out.data_ptr(), outs[0][0].data_ptr(), outs[0][1].data_ptr(), outs[0][2].data_ptr(), g.ws.data_ptr(),
+        g.ws.numel(), main.cuda_stream, None, None, None, None)
+    assert rc == sm.INVALID_ARGUMENT
