@@ -466,3 +466,34 @@ def test_steps_kept_in_flight_give_the_results_of_the_blocking_call():
         g.dW_out.data_ptr(), outs[0][0].data_ptr(), outs[0][1].data_ptr(), outs[0][2].data_ptr(), g.ws.data_ptr(),
         g.ws.numel(), main.cuda_stream, None, None, None, None)
     assert rc == sm.INVALID_ARGUMENT
+
+
+def test_forward_and_backward_can_be_captured_in_a_cuda_graph():
+    """Both calls only enqueue work on the caller's stream (no allocation, no synchronisation), so a step can be
+    captured once and replayed; the replay on new inputs gives what direct calls give."""
+    cfg = MID
+    g = GpuLayer(cfg, si.gen_layer(cfg, seed=11))
+    g.fwd()
+    g.bwd()                                                  # first calls outside the capture (one-time set-up)
+    other = si.gen_layer(cfg, seed=12)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            sm.switch_moe_fwd(g.cfg, g.x, g.W_r, g.bias, g.W_in, g.W_out, g.y, g.aux, g.ws, side)
+            sm.switch_moe_bwd(g.cfg, g.dy, 1.0, g.x, g.W_r, g.W_in, g.W_out, g.y, g.ws, g.dx, g.dW_r, g.dW_in, g.dW_out,
+                              side)
+    torch.cuda.synchronize()
+    from tests.gpu_helpers import to_dev
+    g.x.copy_(to_dev(other["x"], cfg.dtype))
+    g.dy.copy_(to_dev(other["dy"], cfg.dtype))
+    for t in (g.y, g.dx, g.dW_in, g.dW_out):
+        t.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    got = [t.clone() for t in (g.y, g.dx, g.dW_r, g.dW_in, g.dW_out, g.aux)]
+    g.fwd()
+    g.bwd()
+    for a, b in zip(got, (g.y, g.dx, g.dW_r, g.dW_in, g.dW_out, g.aux)):
+        assert torch.equal(a, b)
