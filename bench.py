@@ -122,15 +122,32 @@ def run_reference(args, cfg):
 
 # ----------------------------------------------------------------------------------------------- clocks sampler
 class ClockSampler:
+    """SM clock, power and throttle reasons of one GPU while the timed region runs: NVML polled every 2 ms from a
+    thread (read-only queries); nvidia-smi's own loop as the fall-back where NVML cannot be loaded."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    REASON_BITS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, pci_bus_id: str | None = None):
         self.rows, self.proc, self.thread = [], None, None
-        self.gpu_index = gpu_index
+        self.gpu_index, self.pci_bus_id = gpu_index, pci_bus_id
+        self.nvml, self.handle, self.stop_flag, self.source = None, None, threading.Event(), "nvidia-smi"
+        self.sm, self.power, self.reason_mask, self.sm_max = [], [], 0, None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.handle = (pynvml.nvmlDeviceGetHandleByPciBusId(self.pci_bus_id.encode()) if self.pci_bus_id
+                           else pynvml.nvmlDeviceGetHandleByIndex(self.gpu_index))
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.nvml, self.source = pynvml, "nvml"
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
@@ -141,11 +158,29 @@ class ClockSampler:
         self.thread = threading.Thread(target=self._read, daemon=True)
         self.thread.start()
 
+    def _poll(self):
+        n = self.nvml
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)))
+                self.power.append(n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0)
+                self.reason_mask |= int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
 
     def stop(self):
+        if self.nvml is not None:
+            self.stop_flag.set()
+            self.thread.join(timeout=2)
+            reasons = sorted(k for k, bit in self.REASON_BITS.items() if self.reason_mask & bit)
+            return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_min_mhz": min(self.sm) if self.sm else None,
+                    "sm_max_mhz": self.sm_max, "power_w_max": max(self.power) if self.power else None,
+                    "samples": len(self.sm), "reasons": reasons, "source": "nvml, polled every 2 ms"}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
@@ -167,7 +202,8 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons),
+                "source": "nvidia-smi -lms 100"}
 
 
 # ----------------------------------------------------------------------------------------------- GPU arm
@@ -243,7 +279,10 @@ def run_ours(args, cfg):
         for ev in evs:
             ev.record(stream)                                 # creates the underlying cudaEvent_t handles
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank)
+    props = torch.cuda.get_device_properties(local_rank)
+    bus_id = (f"{props.pci_domain_id:08x}:{props.pci_bus_id:02x}:{props.pci_device_id:02x}.0"
+              if hasattr(props, "pci_bus_id") else None)           # NVML's index need not be CUDA's
+    sampler = ClockSampler(local_rank, bus_id)
     barrier()
     sampler.start()
     t_start.record(stream)
