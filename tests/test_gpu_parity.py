@@ -497,3 +497,15 @@ def test_forward_and_backward_can_be_captured_in_a_cuda_graph():
     g.bwd()
     for a, b in zip(got, (g.y, g.dx, g.dW_r, g.dW_in, g.dW_out, g.aux)):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("cfg", [
+    si.SwitchConfig("five_tokens", 5, 64, 64, 2, 1.0),                       # fewer tokens than any tile
+    si.SwitchConfig("one_token", 1, 64, 64, 1, 1.0),                         # the smallest call there is
+    si.SwitchConfig("max_experts", 2048, 64, 128, 256, 2.0, bias_std=0.2),   # E = 256, the library's limit
+    si.SwitchConfig("more_experts_than_tokens", 128, 64, 64, 256, 4.0),      # most experts stay empty, capacity 2
+    si.SwitchConfig("capacity_is_everything", 300, 64, 128, 3, 3.0),         # cf = E: capacity = T, nothing can drop
+], ids=lambda c: c.name)
+def test_extreme_shapes_match_oracle(cfg):
+    errs = _check_layer(cfg, sm.GEMM_DEFAULT, TOL_BF16, d_aux=0.5)
+    assert errs
