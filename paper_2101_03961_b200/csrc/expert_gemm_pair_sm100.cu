@@ -325,6 +325,64 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       tc_fence_after();
       const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * 256u;
       bool released = false;
+      if (!kTok) {
+        // Weight gradients (row = weight row): 64 output columns at a time, so that a row is a whole 128-byte line.
+        // The warp's 2 KB of shared memory hold 16 rows x 128 bytes: rows 0-15 and 16-31 of the warp take turns, and
+        // every store instruction then writes 4 complete lines (the store path's cost grows with the number of lines
+        // an instruction touches).
+#pragma unroll 1
+        for (int c = half; c < 4; c += 2) {
+          uint32_t v[64];
+          if (have_acc) {
+            tc_ld32(t_addr + c * 64, v);
+            tc_ld32(t_addr + c * 64 + 32, v + 32);
+            tc_wait_ld();
+          } else {
+#pragma unroll
+            for (int i = 0; i < 64; ++i) v[i] = 0u;
+          }
+          if (c + 2 >= 4) {                                   // last chunk of this warp: accumulator read out
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
+          }
+          uint4 ch[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + 2 * h]),
+                                                        __uint_as_float(v[q * 8 + 2 * h + 1]));
+              w[h] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            ch[q] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+          const int chunk = lane & 7;
+          const int col = t.n0 + c * 64 + chunk * 8;
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            if ((lane >> 4) == hf) {
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                *reinterpret_cast<uint4*>(tr + (lane & 15) * 128 + ((q ^ (lane & 7)) << 4)) = ch[q];
+            }
+            __syncwarp();
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+              const int rr = it * 4 + (lane >> 3);
+              const uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 128 + ((chunk ^ (rr & 7)) << 4));
+              const int orow = m_warp + hf * 16 + rr;
+              if (orow < p.Mw && col < p.Nfix)
+                *reinterpret_cast<uint4*>(p.out + ((long long)t.e * p.Mw + orow) * p.ld_out + col) = val;
+            }
+            __syncwarp();
+          }
+        }
+        acc ^= 1u;
+        if (acc == 0) acc_phase ^= 1u;
+        continue;
+      }
 
 #pragma unroll 1
       for (int c = half; c < n_chunks; c += 2) {
