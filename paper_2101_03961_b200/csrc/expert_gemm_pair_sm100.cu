@@ -51,8 +51,9 @@ struct PairParams {
   const int* token_of_slot;
   const float* gate;
   __nv_bfloat16* out;
-  uint32_t* hmask;          // [E*C][d_ff/32] bit i of word w: H[row][32w + i] > 0 (written by GEMM1, read by dgrad2)
-  int hmask_ld;
+  uint32_t* hmask;          // [d_ff/32][E*C]: bit i of word [w][row]: H[row][32w + i] > 0 (written by GEMM1, read by
+                            // dgrad2); rows are contiguous so that 32 token rows are one 128-byte store / load
+  long long hmask_rows;     // E*C
   long long ld_out;
   int* status;
   const __nv_bfloat16* res;   // combine / scatter with the skip path inside the layer: rows added to the output (x or dy)
@@ -316,7 +317,8 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             if (q_off[k] >= 0)
-              q_mw[k] = p.hmask[((long long)t.e * p.C + t.row0 + (half + 2 * k) * 32 + lane) * p.hmask_ld + (m_warp >> 5)];
+              q_mw[k] = p.hmask[(long long)(m_warp >> 5) * p.hmask_rows + (long long)t.e * p.C + t.row0 +
+                                (half + 2 * k) * 32 + lane];
         }
       }
       ok = mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag, p.status, 24);
@@ -423,6 +425,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             }
           }
           __syncwarp();
+          uint32_t mword[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
           for (int it = 0; it < 4; ++it) {
             const int rr = it * 8 + (lane >> 2);
@@ -443,8 +446,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
               uint32_t word = m8 << ((lane & 3) * 8);
               word |= __shfl_xor_sync(0xffffffffu, word, 1);
               word |= __shfl_xor_sync(0xffffffffu, word, 2);
-              if ((lane & 3) == 0 && offs[it] >= 0 && m_warp < p.Mw)
-                p.hmask[((long long)t.e * p.C + t.row0 + c * 32 + rr) * p.hmask_ld + (m_warp >> 5)] = word;
+              mword[it] = word;                               // the word of token row rr, in all four lanes of its group
             }
             if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[it] >= 0 && mcol < p.Mw) {
               // skip path inside the layer: y = x + g E(x), dx = dy + dH W_in^T (the expert term is already bf16)
@@ -459,6 +461,16 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
               }
             }
             if (offs[it] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[it] + mcol) = val;
+          }
+          if (OP == kGemm1Relu && !p.plain) {                 // lane i stores the mask word of token row i: one 128-byte line
+            uint32_t mine = 0;
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+              const uint32_t w = __shfl_sync(0xffffffffu, mword[it], 4 * (lane & 7));
+              if ((lane >> 3) == it) mine = w;
+            }
+            if (q_off[0] >= 0 && m_warp < p.Mw)
+              p.hmask[(long long)(m_warp >> 5) * p.hmask_rows + (long long)t.e * p.C + t.row0 + c * 32 + lane] = mine;
           }
 #pragma unroll
           for (int k = 0; k < 3; ++k) {                       // advance the queue
@@ -567,7 +579,7 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   q.gate = ws_ptr<float>(ws, p.gate);
   q.status = ws_ptr<int>(ws, p.status);
   q.hmask = ws_ptr<uint32_t>(ws, p.hmask);
-  q.hmask_ld = s.f / 32;
+  q.hmask_rows = (long long)s.E * s.C;
   CUtensorMap tmA, tmB;
   int rc = SWITCH_MOE_OK, rc2 = SWITCH_MOE_OK;
   int K = 0;
