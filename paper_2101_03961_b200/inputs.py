@@ -66,6 +66,8 @@ CONFIGS = {
     "switch_base_quarter": SwitchConfig("switch_base_quarter", 8192, 768, 3072, 32, 1.25),
     # the paper's own Switch-Base layer shape with GEGLU experts (its hyper-parameter table: d_model 768, d_ff 2048)
     "geglu_base": SwitchConfig("geglu_base", 32768, 768, 2048, 128, 1.25, geglu=True),
+    # many tokens, narrow layer: exercises the token-count limits of the router's partial sums and of the plan's scan
+    "long_batch": SwitchConfig("long_batch", 131072, 256, 512, 128, 1.25),
 }
 
 

@@ -180,3 +180,8 @@ def test_overflow_stress_with_rerouting_full_size():
 
 def test_geglu_experts_at_the_papers_switch_base_shape_full_size():
     _run_fullsize("geglu_base")
+
+
+def test_batch_of_131072_tokens_full_size():
+    out = _run_fullsize("long_batch")
+    assert out["dropped"] < 0.05 * 131072
