@@ -375,3 +375,89 @@ def switch_backward_groups(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, exp
             res["dW_in"][i] = sum(q["dW_in"][i] for q in outs)
             res["dW_out"][i] = sum(q["dW_out"][i] for q in outs)
     return res
+
+
+# ------------------------------------------------------------------------------------------------------------
+# Top-2 routing: the Mixture-of-Experts layer the paper compares with (Eq. 1-2 with the two highest-probability
+# experts; "MoE Transformers using top-2 routing" in its comparison tables).  Readings, where the paper gives none:
+# the combine weights are the softmax probabilities of Eq. 1 themselves (Eq. 2, no renormalisation over the two);
+# every token's first choice is placed before any second choice (token order inside each round), all against the
+# same expert capacity; f in the auxiliary loss counts the first choice (the argmax of Eq. 5).
+def top2_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None, first_index=None,
+                 second_index=None, experts=None):
+    """Forward of the top-2 layer.  Assignments are numbered v = t for the first choice of token t and v = T + t for
+    its second choice; "slot" [2T], "token_of_slot" [E*C] (holding v) and "keep" [2T] describe the plan in that
+    numbering, "e" [2T] the expert and "g" [2T] the combine weight of every assignment."""
+    x64 = np.asarray(x, dtype=F64)
+    T, d = x64.shape
+    E = np.asarray(W_r).shape[1]
+    h = router_logits(x64, W_r, router_bias)
+    p = router_probs(h)
+    a = top1(p)[0] if first_index is None else np.asarray(first_index, dtype=np.int64)
+    b = second_choice(p, a) if second_index is None else np.asarray(second_index, dtype=np.int64)
+    aux, f, P = load_balance_loss(p, a, alpha)                  # f: first choices only
+    C = expert_capacity(T, E, capacity_factor)
+    e = np.concatenate([a, b])
+    plan = dispatch_plan(e, E, C)                                # first choices of all tokens, then second choices
+    keep = plan["keep"]
+    tok_of = np.concatenate([np.arange(T), np.arange(T)])       # the token behind an assignment
+    g = p[tok_of, e]
+    y = np.zeros((T, d), dtype=F64)
+    o = np.zeros((2 * T, d), dtype=F64)                          # un-weighted expert output per assignment
+    u = {}
+    todo = range(E) if experts is None else experts
+    for i in todo:
+        v = plan["token_of_slot"][i * C:i * C + int(plan["kept"][i])]   # the expert's assignments in slot order
+        if v.size == 0:
+            continue
+        u_i = x64[tok_of[v]] @ np.asarray(W_in[i], dtype=F64)
+        o_i = np.maximum(u_i, 0.0) @ np.asarray(W_out[i], dtype=F64)
+        u[i] = u_i
+        o[v] = o_i
+        np.add.at(y, tok_of[v], g[v, None] * o_i)                # Eq. 2: sum over the selected experts
+    out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "y": y, "o": o, "u": u, "T": T, "E": E,
+           "alpha": alpha, "tok_of": tok_of, "first": a, "second": b}
+    out.update(plan)
+    out["count_first"] = np.bincount(a, minlength=E)
+    return out
+
+
+def top2_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=None, want_weight_grads=True):
+    """Backward of top2_forward: both kept assignments of a token send gradient to x, to their expert's weights and,
+    through their combine weight p[t, e], to the router; f has no gradient."""
+    x64 = np.asarray(x, dtype=F64)
+    dy64 = np.asarray(dy, dtype=F64)
+    W_r64 = np.asarray(W_r, dtype=F64)
+    T, d = x64.shape
+    E, C = fwd["E"], fwd["C"]
+    p, e, g, keep, tok_of, alpha = fwd["p"], fwd["e"], fwd["g"], fwd["keep"], fwd["tok_of"], fwd["alpha"]
+    dx = np.zeros((T, d), dtype=F64)
+    dgate = np.zeros(2 * T, dtype=F64)
+    dW_in, dW_out = {}, {}
+    todo = range(E) if experts is None else experts
+    for i in todo:
+        v = fwd["token_of_slot"][i * C:i * C + int(fwd["kept"][i])]
+        W_in_i = np.asarray(W_in[i], dtype=F64)
+        W_out_i = np.asarray(W_out[i], dtype=F64)
+        if v.size == 0:
+            if want_weight_grads:
+                dW_in[i] = np.zeros_like(W_in_i)
+                dW_out[i] = np.zeros_like(W_out_i)
+            continue
+        t = tok_of[v]
+        u_i = fwd["u"][i]
+        a_i = np.maximum(u_i, 0.0)
+        do_i = g[v, None] * dy64[t]
+        dgate[v] = np.sum(dy64[t] * fwd["o"][v], axis=1)
+        du_i = (do_i @ W_out_i.T) * (u_i > 0.0)
+        np.add.at(dx, t, du_i @ W_in_i.T)
+        if want_weight_grads:
+            dW_out[i] = a_i.T @ do_i
+            dW_in[i] = x64[t].T @ du_i
+    G = np.broadcast_to((d_aux * alpha * E / T) * fwd["f"][None, :], (T, E)).copy()
+    kept_v = np.flatnonzero(keep)
+    np.add.at(G, (tok_of[kept_v], e[kept_v]), dgate[kept_v])
+    dh = p * (G - np.sum(p * G, axis=1, keepdims=True))
+    dx_router = dh @ W_r64.T
+    return {"dx": dx + dx_router, "dW_r": x64.T @ dh, "db": dh.sum(axis=0), "dW_in": dW_in, "dW_out": dW_out,
+            "dgate": dgate, "dh": dh, "dx_router": dx_router}

@@ -728,3 +728,77 @@ def test_geglu_single_expert_is_the_dense_geglu_ffn_and_gradients_match_finite_d
             num.append((lp - lm) / (2 * eps))
         ana = np.array([grad[i] for i in idxs])
         assert np.linalg.norm(np.array(num) - ana) / np.linalg.norm(ana) < 1e-7, name
+
+
+# ------------------------------------------------------------------ top-2 routing (the Mixture-of-Experts comparator, Eq. 1-2)
+def _literal_top2_layer(x, W_r, W_in, W_out, C):
+    """Eq. 1-2 with the two highest-probability experts, one token at a time: first choices of all tokens are
+    placed before any second choice; an assignment beyond the expert's capacity contributes nothing."""
+    T, d = x.shape
+    E = W_r.shape[1]
+    logits = x @ W_r
+    probs = np.exp(logits - logits.max(1, keepdims=True))
+    probs /= probs.sum(1, keepdims=True)
+    order = np.argsort(-probs, axis=1, kind="stable")
+    load = np.zeros(E, dtype=int)
+    y = np.zeros((T, d))
+    placed = []
+    for rnd in (0, 1):
+        for t in range(T):
+            i = order[t, rnd]
+            if load[i] < C:
+                load[i] += 1
+                placed.append((rnd, t, i))
+                y[t] += probs[t, i] * (np.maximum(x[t] @ W_in[i], 0.0) @ W_out[i])
+    return y, placed, load
+
+
+@pytest.mark.parametrize("T,d,f,E,cf,seed", [(40, 6, 9, 4, 2.0, 0), (48, 5, 8, 6, 1.0, 1), (30, 4, 6, 3, 0.5, 2)])
+def test_top2_layer_equals_token_by_token_definition(T, d, f, E, cf, seed):
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=seed, scale=2.0)
+    out = so.top2_forward(x, W_r, W_in, W_out, cf, 0.01)
+    y, placed, load = _literal_top2_layer(x, W_r, W_in, W_out, out["C"])
+    np.testing.assert_allclose(out["y"], y, rtol=1e-12, atol=1e-14)
+    assert out["kept"].tolist() == load.tolist()
+    assert sorted((v // T, v % T, int(out["e"][v])) for v in np.flatnonzero(out["keep"])) == sorted(placed)
+    plain = so.switch_forward(x, W_r, W_in, W_out, cf, 0.01)
+    assert out["aux"] == plain["aux"]                                        # f counts the first choice only
+    assert np.array_equal(out["first"], plain["e"]) and np.all(out["second"] != out["first"])
+    assert np.array_equal(out["slot"][:T][plain["keep"]], plain["slot"][plain["keep"]])   # round one is Switch routing
+    if cf >= 2.0:
+        assert out["keep"][:T].all()
+
+
+def test_top2_backward_matches_finite_differences():
+    T, d, f, E, cf, alpha, d_aux = 14, 5, 7, 4, 1.0, 0.04, 0.9
+    rng = np.random.default_rng(81)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=81, scale=2.0)
+    R = rng.standard_normal((T, d))
+    fwd = so.top2_forward(x, W_r, W_in, W_out, cf, alpha)
+    srt = np.sort(fwd["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-3 and (srt[:, -2] - srt[:, -3]).min() > 1e-3 and (~fwd["keep"]).any()
+    bwd = so.top2_backward(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    a, b, eps = fwd["first"], fwd["second"], 1e-6
+
+    def loss():
+        o = so.top2_forward(x, W_r, W_in, W_out, cf, alpha, first_index=a, second_index=b)
+        return float(np.sum(o["y"] * R) + d_aux * o["aux"])
+
+    dW_in = np.stack([bwd["dW_in"][i] for i in range(E)])
+    dW_out = np.stack([bwd["dW_out"][i] for i in range(E)])
+    for name, arr, grad in [("dx", x, bwd["dx"]), ("dW_r", W_r, bwd["dW_r"]), ("dW_in", W_in, dW_in),
+                            ("dW_out", W_out, dW_out)]:
+        idxs = list(np.ndindex(arr.shape))
+        if len(idxs) > 150:
+            idxs = [idxs[i] for i in rng.choice(len(idxs), 150, replace=False)]
+        num = []
+        for idx in idxs:
+            old = arr[idx]
+            arr[idx] = old + eps
+            lp = loss()
+            arr[idx] = old - eps
+            lm = loss()
+            arr[idx] = old
+            num.append((lp - lm) / (2 * eps))
+        ana = np.array([grad[i] for i in idxs])
+        assert np.linalg.norm(np.array(num) - ana) / np.linalg.norm(ana) < 1e-7, name
