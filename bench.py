@@ -245,7 +245,7 @@ def run_ours(args, cfg):
 
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype,
                           residual=args.residual, groups=args.groups, reroute=args.reroute,
-                          input_jitter=args.input_jitter > 0.0, geglu=cfg.geglu)
+                          input_jitter=args.input_jitter > 0.0, geglu=cfg.geglu, top2=args.top2)
     noise = None
     if args.router_noise > 0.0:                              # exploration noise on the logits: an input of the layer
         noise = torch.from_numpy(si.gen_router_noise(cfg, args.router_noise, seed)).cuda()
@@ -437,7 +437,7 @@ def run_ours(args, cfg):
                    "geglu_experts": cfg.geglu,
                    "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha, "capacity": sm.switch_moe_capacity(mcfg),
                    "kept_tokens": kept, "parallelism": "replicas" if world > 1 else "single",
-                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "router_noise_eps": args.router_noise, "input_jitter_eps": args.input_jitter,
+                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "top2_routing": bool(args.top2), "router_noise_eps": args.router_noise, "input_jitter_eps": args.input_jitter,
                    "l2": "inputs larger than L2 (weights 2 x %.0f MB per pass), no flush" %
                          (cfg.E * cfg.d_model * cfg.d_ff * elt / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": sm.switch_moe_launches_per_step(mcfg) * args.steps,
@@ -469,6 +469,9 @@ def main():
     ap.add_argument("--input-jitter", type=float, default=0.0,
                     help="multiply the router's input by uniform(1 - eps, 1 + eps) factors (a seeded input tensor); "
                          "the headline configuration has none")
+    ap.add_argument("--top2", action="store_true",
+                    help="top-2 routing (the Mixture-of-Experts comparator): two assignments per token, so about twice "
+                         "the expert work of the headline configuration at a capacity factor that keeps them")
     ap.add_argument("--reroute", action="store_true",
                     help="offer tokens that overflow their expert to their second choice (stage 2 of "
                          "No-Token-Left-Behind routing); not the headline configuration")

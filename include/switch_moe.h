@@ -62,9 +62,17 @@ enum switch_moe_gemm_path {
    weights which are non-linearly combined"): W_in is [E, d_model, 2 d_ff] = [W_0 | W_1] per expert (and dW_in
    likewise), hidden = GELU(x W_0) . (x W_1) with the exact GELU z Phi(z), y = hidden W_out.  The two products are
    one grouped GEMM with 2 d_ff output columns; the gating and its derivative are element-wise kernels over the
-   kept rows.  Not available on SWITCH_MOE_GEMM_TC_1CTA. */
+   kept rows.  Not available on SWITCH_MOE_GEMM_TC_1CTA.
+   SWITCH_MOE_FLAG_TOP2: top-2 routing, the Mixture-of-Experts layer the paper compares with (Eq. 1-2 with the two
+   highest-probability experts): y_t = p_a E_a(x_t) + p_b E_b(x_t) with the softmax probabilities of Eq. 1 as they
+   are.  Every token's first choice is placed before any second choice (token order within each round), all against
+   the capacity of Eq. 3; f in the auxiliary loss counts the first choice.  The library numbers the 2T assignments
+   v = t (first choice of token t) and v = T + t (second choice): the workspace regions EXPERT_INDEX, GATE, SLOT and
+   DGATE then have 2T entries and TOKEN_OF_SLOT holds v.  Needs T to be a multiple of 256; not together with
+   RESIDUAL, REROUTE or several routing groups. */
 enum switch_moe_flags {
-  SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2, SWITCH_MOE_FLAG_INPUT_JITTER = 4, SWITCH_MOE_FLAG_GEGLU = 8
+  SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2, SWITCH_MOE_FLAG_INPUT_JITTER = 4, SWITCH_MOE_FLAG_GEGLU = 8,
+  SWITCH_MOE_FLAG_TOP2 = 16
 };
 
 typedef enum switch_moe_status {

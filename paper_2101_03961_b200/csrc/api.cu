@@ -75,9 +75,9 @@ int switch_moe_workspace_view(const switch_moe_config* cfg, void* workspace, int
   size_t off, bytes;
   switch (region) {
     case SWITCH_MOE_WS_STATUS: off = p.status; bytes = 16 * 4; break;
-    case SWITCH_MOE_WS_EXPERT_INDEX: off = p.expert_index; bytes = T * 4; break;
-    case SWITCH_MOE_WS_GATE: off = p.gate; bytes = T * 4; break;
-    case SWITCH_MOE_WS_SLOT: off = p.slot; bytes = T * 4; break;
+    case SWITCH_MOE_WS_EXPERT_INDEX: off = p.expert_index; bytes = (size_t)s.Tv * 4; break;
+    case SWITCH_MOE_WS_GATE: off = p.gate; bytes = (size_t)s.Tv * 4; break;
+    case SWITCH_MOE_WS_SLOT: off = p.slot; bytes = (size_t)s.Tv * 4; break;
     case SWITCH_MOE_WS_TOKEN_OF_SLOT: off = p.token_of_slot; bytes = E * C * 4; break;
     case SWITCH_MOE_WS_COUNT: off = p.count; bytes = E * 4; break;
     case SWITCH_MOE_WS_KEPT: off = p.kept; bytes = E * 4; break;
@@ -87,7 +87,7 @@ int switch_moe_workspace_view(const switch_moe_config* cfg, void* workspace, int
     case SWITCH_MOE_WS_H: off = p.h; bytes = E * C * s.f * s.elt; break;
     case SWITCH_MOE_WS_DYD: off = p.dyd; bytes = E * C * s.d * s.elt; break;
     case SWITCH_MOE_WS_DH: off = p.dh; bytes = E * C * s.f * s.elt; break;
-    case SWITCH_MOE_WS_DGATE: off = p.dgate; bytes = T * 4; break;
+    case SWITCH_MOE_WS_DGATE: off = p.dgate; bytes = (size_t)s.Tv * 4; break;
     case SWITCH_MOE_WS_DLOGITS: off = p.dlogits; bytes = T * E * 4; break;
     case SWITCH_MOE_WS_EXPERT_PROC:
       if (!s.reroute) return SWITCH_MOE_INVALID_ARGUMENT;
@@ -134,17 +134,21 @@ int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r
   if (cudaMemsetAsync(ws_ptr<char>(workspace, c.p.status), 0, 16 * 4, st) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
   SWMOE_TRY(mark(cfg, 0, st));
   SWMOE_TRY(launch_router_fwd(c.s, c.p, x, W_r, router_bias, cfg->router_noise, workspace, st));
+  if (c.s.top2) SWMOE_TRY(launch_top2_choice(c.s, c.p, workspace, st));     // assignments T .. 2T - 1
   SWMOE_TRY(mark(cfg, 1, st));
   SWMOE_TRY(launch_dispatch_plan(c.s, c.p, nullptr, aux_loss, workspace, st));
   SWMOE_TRY(mark(cfg, 2, st));
-  SWMOE_TRY(launch_gather_x(c.s, c.p, x, y, workspace, st));
+  // top-2 routing: the experts write one weighted output row per assignment; the two rows of a token are summed last
+  void* y_rows = c.s.top2 ? ws_ptr<void>(workspace, c.p.yv) : y;
+  SWMOE_TRY(launch_gather_x(c.s, c.p, x, y_rows, workspace, st));
   GemmArgs a{};
-  a.W_in = W_in; a.W_out = W_out; a.y = y; a.x = x;
+  a.W_in = W_in; a.W_out = W_out; a.y = y_rows; a.x = x;
   SWMOE_TRY(mark(cfg, 3, st));
   SWMOE_TRY(run_gemm(kGemm1Relu, c, a, workspace, st));
   if (c.s.geglu) SWMOE_TRY(launch_geglu_fwd(c.s, c.p, workspace, st));     // hidden = GELU(a) . b
   SWMOE_TRY(mark(cfg, 4, st));
   SWMOE_TRY(run_gemm(kGemm2Combine, c, a, workspace, st));
+  if (c.s.top2) SWMOE_TRY(launch_top2_sum(c.s, c.p, y_rows, y, workspace, st));   // Eq. 2: sum over the two experts
   SWMOE_TRY(mark(cfg, 5, st));
   return SWITCH_MOE_OK;
 }
@@ -161,9 +165,12 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   GemmArgs a{};
-  a.W_in = W_in; a.W_out = W_out; a.dx = dx; a.dW_in = dW_in; a.dW_out = dW_out; a.dy = dy;
+  // top-2 routing: gradients are formed per assignment (the gate's from the per-assignment outputs the forward pass
+  // left in the workspace) and the two input-gradient rows of a token are summed before the router adds its part
+  void* dx_rows = c.s.top2 ? ws_ptr<void>(workspace, c.p.dxv) : dx;
+  a.W_in = W_in; a.W_out = W_out; a.dx = dx_rows; a.dW_in = dW_in; a.dW_out = dW_out; a.dy = dy;
   SWMOE_TRY(mark(cfg, 6, st));
-  SWMOE_TRY(launch_gather_dy(c.s, c.p, dy, y, dx, workspace, st));
+  SWMOE_TRY(launch_gather_dy(c.s, c.p, dy, c.s.top2 ? ws_ptr<void>(workspace, c.p.yv) : y, dx, workspace, st));
   SWMOE_TRY(mark(cfg, 7, st));
   SWMOE_TRY(run_gemm(kDgrad2Mask, c, a, workspace, st));
   if (c.s.geglu) SWMOE_TRY(launch_geglu_bwd(c.s, c.p, workspace, st));     // d[a | b] from dH
@@ -173,6 +180,7 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
   SWMOE_TRY(run_gemm(kDgrad1Scatter, c, a, workspace, st));
   SWMOE_TRY(mark(cfg, 10, st));
   SWMOE_TRY(run_gemm(kWgrad1, c, a, workspace, st));
+  if (c.s.top2) SWMOE_TRY(launch_top2_sum(c.s, c.p, dx_rows, dx, workspace, st));
   SWMOE_TRY(mark(cfg, 11, st));
   SWMOE_TRY(launch_router_bwd(c.s, c.p, x, W_r, ws_ptr<float>(workspace, c.p.dgate), d_aux, workspace, dx, true, dW_r,
                               st));
@@ -304,8 +312,8 @@ int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches
   // Tensor-core router: forward = operand split, router, column sums; backward = logit gradients, two products, reduce.
   // Rerouting of overflowed tokens adds four plan kernels to the forward pass.
   // Input jitter adds the element-wise product kernel.
-  // GEGLU experts add the gating kernel to each pass.
-  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0) + (s.geglu ? 2 : 0);
+  // GEGLU experts add the gating kernel to each pass.  Top-2 routing adds the second-choice kernel and two row sums.
+  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0) + (s.geglu ? 2 : 0) + (s.top2 ? 3 : 0);
   return SWITCH_MOE_OK;
 }
 

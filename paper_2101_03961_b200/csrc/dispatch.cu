@@ -71,7 +71,7 @@ __device__ __forceinline__ void write_tile_lists(const float* term, const int* k
 constexpr int kScanThreads = 1024;
 constexpr int kScanRows = 16;
 __global__ void __launch_bounds__(kScanThreads)
-plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __restrict__ psum_partial,
+plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, int loss_blocks, const float* __restrict__ psum_partial,
                  int router_blocks, int T, int E, int Ew, int C, float alpha, int* __restrict__ hist_base,
                  int* __restrict__ count, int* __restrict__ kept, float* __restrict__ psum,
                  float* __restrict__ aux_loss, int* __restrict__ tile_expert, int* __restrict__ tile_row0,
@@ -79,6 +79,7 @@ plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __r
   pdl_launch_dependents();
   pdl_wait();
   __shared__ int qsum[kScanThreads];                         // [g][e], Ew columns per row
+  __shared__ int qfirst[kScanThreads];                       // the same over rows < loss_blocks (top-2: first choices)
   __shared__ float qps[kScanThreads];
   __shared__ float term[kMaxExperts];
   __shared__ int kept_s[kMaxExperts];
@@ -93,15 +94,20 @@ plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __r
     float pv[kScanRows];
 #pragma unroll
     for (int j = 0; j < kScanRows; ++j) pv[j] = r0 + j < r1 ? psum_partial[(size_t)(r0 + j) * E + e] : 0.f;
-    int sum = 0;
+    int sum = 0, first = 0;
 #pragma unroll
-    for (int j = 0; j < kScanRows; ++j) sum += hv[j];
-    for (int b = h0 + kScanRows; b < h1; ++b) sum += hist[(size_t)b * E + e];
+    for (int j = 0; j < kScanRows; ++j) { sum += hv[j]; if (h0 + j < loss_blocks) first += hv[j]; }
+    for (int b = h0 + kScanRows; b < h1; ++b) {
+      const int v = hist[(size_t)b * E + e];
+      sum += v;
+      if (b < loss_blocks) first += v;
+    }
     float ps = 0.f;
 #pragma unroll
     for (int j = 0; j < kScanRows; ++j) ps += pv[j];                                   // fixed order
     for (int b = r0 + kScanRows; b < r1; ++b) ps += psum_partial[(size_t)b * E + e];
     qsum[g * Ew + e] = sum;
+    qfirst[g * Ew + e] = first;
     qps[g * Ew + e] = ps;
   }
   __syncthreads();
@@ -113,17 +119,17 @@ plan_scan_kernel(const int* __restrict__ hist, int plan_blocks, const float* __r
       if (h0 + j < h1) { hist_base[(size_t)(h0 + j) * E + e] = run; run += hv[j]; }
     for (int b = h0 + kScanRows; b < h1; ++b) { hist_base[(size_t)b * E + e] = run; run += hist[(size_t)b * E + e]; }
     if (g == 0) {
-      int total = 0;
+      int total = 0, first = 0;
       float ps = 0.f;
-      for (int q = 0; q < G; ++q) { total += qsum[q * Ew + e]; ps += qps[q * Ew + e]; }
-      count[e] = total;
-      count_g[e] = total;                                                              // one routing group
+      for (int q = 0; q < G; ++q) { total += qsum[q * Ew + e]; first += qfirst[q * Ew + e]; ps += qps[q * Ew + e]; }
+      count[e] = first;                                                                // f counts the argmax (Eq. 5)
+      count_g[e] = first;                                                              // one routing group
       group_base[e] = 0;
       const int k = min(total, C);
       kept[e] = k;
       kept_s[e] = k;
       psum[e] = ps;
-      term[e] = ((float)total / (float)T) * (ps / (float)T);                           // f_i . P_i  (Eq. 5, 6)
+      term[e] = ((float)first / (float)T) * (ps / (float)T);                           // f_i . P_i  (Eq. 5, 6)
     }
   }
   write_tile_lists(term, kept_s, E, alpha * (float)E, aux_loss, tile_expert, tile_row0, ntile);
@@ -201,12 +207,13 @@ plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__
   for (int i = tid; i < kWarps * kMaxExperts; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
   __syncthreads();
   const int t = blockIdx.x * kPlanBlockTokens + tid;
-  const int e = t < T ? expert_index[t] : -1 - lane;          // distinct dummies for out-of-range lanes
-  const unsigned same = __match_any_sync(0xffffffffu, e);
+  const int e = t < T ? expert_index[t] : -1;                 // negative: no expert (takes no slot)
+  const unsigned same = __match_any_sync(0xffffffffu, e >= 0 ? e : -1 - lane);   // distinct dummies for those lanes
   const int rank = __popc(same & ((1u << lane) - 1u));
-  if (t < T && rank == 0) warp_cnt[warp][e] = __popc(same);
+  if (e >= 0 && rank == 0) warp_cnt[warp][e] = __popc(same);
   __syncthreads();
-  if (t < T) {
+  if (t < T && e < 0) slot[t] = -1;
+  if (e >= 0) {
     int pos = hist_base[(size_t)blockIdx.x * E + e] + rank;                  // position inside the token's own group
     for (int w = 0; w < warp; ++w) pos += warp_cnt[w][e];
     const int grp = blockIdx.x / blocks_per_group;
@@ -320,6 +327,75 @@ reroute_assign_kernel(const int* __restrict__ alt, const int* __restrict__ exper
   }
 }
 
+// ---- top-2 routing ------------------------------------------------------------------------------------------
+// Second choice of every token: the expert with the second-highest probability (lowest index on ties) and its
+// probability, stored as assignment T + t.  One warp per token.
+__global__ void __launch_bounds__(256)
+top2_choice_kernel(const float* __restrict__ probs, int T, int E, int* __restrict__ expert_index,
+                   float* __restrict__ gate) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= T) return;
+  const int e1 = expert_index[t];
+  float best = -1.f;
+  int arg = 0x7fffffff;
+  for (int e = lane; e < E; e += 32) {
+    const float v = probs[(size_t)t * E + e];
+    if (e != e1 && v > best) { best = v; arg = e; }          // ascending e: the first maximum wins
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+    const int oa = __shfl_xor_sync(0xffffffffu, arg, off);
+    if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+  }
+  if (lane == 0) {
+    expert_index[T + t] = arg < E ? arg : -1;                 // E == 1: no second choice (a negative index takes no slot)
+    gate[T + t] = arg < E ? best : 0.f;
+  }
+}
+
+// out[t] = rows[t] + rows[T + t], a dropped assignment (slot < 0) counting as zero: y from the weighted expert outputs
+// of the two choices, dx from their input gradients.  One warp per token, float32 sum.
+template <bool kBf16>
+__global__ void __launch_bounds__(256)
+top2_sum_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot, int T, int row_vec,
+                uint4* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= T) return;
+  const bool k1 = slot[t] >= 0, k2 = slot[T + t] >= 0;
+  const uint4* r1 = rows + (size_t)t * row_vec;
+  const uint4* r2 = rows + (size_t)(T + t) * row_vec;
+  uint4* dst = out + (size_t)t * row_vec;
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  for (int v = lane; v < row_vec; v += 32) {
+    const uint4 a = k1 ? r1[v] : zero, b = k2 ? r2[v] : zero;
+    uint4 o;
+    if (kBf16) {
+      const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+      __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 fa = __bfloat1622float2(pa[i]), fb = __bfloat1622float2(pb[i]);
+        po[i] = __floats2bfloat162_rn(fa.x + fb.x, fa.y + fb.y);
+      }
+    } else {
+      const float* fa = reinterpret_cast<const float*>(&a);
+      const float* fb = reinterpret_cast<const float*>(&b);
+      float* fo = reinterpret_cast<float*>(&o);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) fo[i] = fa[i] + fb[i];
+    }
+    dst[v] = o;
+  }
+}
+
 // Forward gather.  Part 1 (blockIdx.x < slot_blocks): one warp per slot row; kept slots copy the token's row
 // with 128-bit loads and stores, slots in [kept_i, roundup(kept_i, kTileM)) are zero-filled so that tensor-core
 // tiles never read stale rows.  Part 2: one warp per token; dropped tokens get a zero output row (their
@@ -329,6 +405,7 @@ __global__ void __launch_bounds__(256)
 gather_x_kernel(const uint4* __restrict__ x, const int* __restrict__ token_of_slot, const int* __restrict__ kept,
                 const int* __restrict__ slot, int T, int E, int C, int row_vec, int slot_blocks, int residual,
                 uint4* __restrict__ xd, uint4* __restrict__ y) {
+  // top-2 routing: slot s may hold assignment T + t (the second choice of token t): its source row is still x[t]
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -338,7 +415,9 @@ gather_x_kernel(const uint4* __restrict__ x, const int* __restrict__ token_of_sl
     const int ex = s / C, pos = s - ex * C, k = kept[ex];
     uint4* dst = xd + (size_t)s * row_vec;
     if (pos < k) {
-      const uint4* src = x + (size_t)token_of_slot[s] * row_vec;
+      int tok = token_of_slot[s];
+      if (tok >= T) tok -= T;
+      const uint4* src = x + (size_t)tok * row_vec;
       for (int v = lane; v < row_vec; v += 32) dst[v] = src[v];
     } else if (pos < (k + kTileM - 1) / kTileM * kTileM) {
       for (int v = lane; v < row_vec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
@@ -402,9 +481,9 @@ gather_dy_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ y, cons
   const int ex = s / C, pos = s - ex * C, k = kept[ex];
   uint4* dst = dyd + (size_t)s * row_vec;
   if (pos < k) {
-    const int t = token_of_slot[s];
+    const int t = token_of_slot[s];                           // top-2 routing: assignment t or T + t of token t mod T
     const float g = gate[t];
-    const uint4* src = dy + (size_t)t * row_vec;
+    const uint4* src = dy + (size_t)(t >= T ? t - T : t) * row_vec;
     const uint4* ysrc = y + (size_t)t * row_vec;
     float dot = 0.f;
     for (int v = lane; v < row_vec; v += 32) {
@@ -426,10 +505,10 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
                          cudaStream_t st) {
   int* ei = ws_ptr<int>(ws, p.expert_index);
   if (expert_index != nullptr && expert_index != ei) {
-    if (cudaMemcpyAsync(ei, expert_index, (size_t)s.T * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    if (cudaMemcpyAsync(ei, expert_index, (size_t)s.Tv * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return SWITCH_MOE_CUDA_ERROR;
   }
-  launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, s.T, s.E, ws_ptr<int>(ws, p.hist));
+  launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, s.Tv, s.E, ws_ptr<int>(ws, p.hist));
   int Ew = 32;
   while (Ew < s.E) Ew *= 2;
   const int blocks_per_group = s.plan_blocks / s.G;
@@ -437,7 +516,8 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
   int* group_base = ws_ptr<int>(ws, p.group_base);
   if (s.G == 1) {
     launch_k(plan_scan_kernel, dim3(1), dim3(kScanThreads), 0, st, ws_ptr<int>(ws, p.hist), s.plan_blocks,
-             ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, Ew, s.Cg, s.alpha,
+             s.top2 ? s.plan_blocks / 2 : s.plan_blocks, ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, Ew,
+             s.Cg, s.alpha,
              ws_ptr<int>(ws, p.hist_base), ws_ptr<int>(ws, p.count), ws_ptr<int>(ws, p.kept),
              ws_ptr<float>(ws, p.psum), aux_loss, ws_ptr<int>(ws, p.tile_expert), ws_ptr<int>(ws, p.tile_row0),
              ws_ptr<int4>(ws, p.ntile), count_g, group_base);
@@ -450,7 +530,7 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
              ws_ptr<int4>(ws, p.ntile), count_g, group_base);
   }
   launch_k(plan_assign_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, ws_ptr<int>(ws, p.hist_base),
-           ws_ptr<int>(ws, p.kept), group_base, blocks_per_group, s.T, s.E, s.C, s.Cg, ws_ptr<int>(ws, p.slot),
+           ws_ptr<int>(ws, p.kept), group_base, blocks_per_group, s.Tv, s.E, s.C, s.Cg, ws_ptr<int>(ws, p.slot),
            ws_ptr<int>(ws, p.token_of_slot));
   if (s.reroute) {
     int* alt = ws_ptr<int>(ws, p.alt);
@@ -470,7 +550,8 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
 
 int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void* ws, cudaStream_t st) {
   const int row_vec = (int)((size_t)s.d * s.elt / 16);
-  const int slot_blocks = (s.E * s.C + 7) / 8, tok_blocks = (s.T + 7) / 8;
+  // top-2 routing: the output rows of dropped assignments are skipped by the kernel that sums the two choices
+  const int slot_blocks = (s.E * s.C + 7) / 8, tok_blocks = s.top2 ? 0 : (s.T + 7) / 8;
   launch_k(gather_x_kernel, dim3(slot_blocks + tok_blocks), dim3(256), 0, st, 
       static_cast<const uint4*>(x), ws_ptr<int>(ws, p.token_of_slot), ws_ptr<int>(ws, p.kept),
       ws_ptr<int>(ws, p.slot), s.T, s.E, s.C, row_vec, slot_blocks, s.residual, ws_ptr<uint4>(ws, p.xd),
@@ -494,6 +575,23 @@ int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* 
              static_cast<const uint4*>(ysrc), ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
              ws_ptr<int>(ws, p.kept), ws_ptr<int>(ws, p.slot), s.T, s.E, s.C, row_vec, slot_blocks,
              ws_ptr<uint4>(ws, p.dyd), ws_ptr<float>(ws, p.dgate), static_cast<uint4*>(dx));
+  return launch_status();
+}
+
+int launch_top2_choice(const Shape& s, const Plan& p, void* ws, cudaStream_t st) {
+  launch_k(top2_choice_kernel, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs), s.T, s.E,
+           ws_ptr<int>(ws, p.expert_index), ws_ptr<float>(ws, p.gate));
+  return launch_status();
+}
+
+int launch_top2_sum(const Shape& s, const Plan& p, const void* per_assignment, void* out, void* ws, cudaStream_t st) {
+  const int row_vec = (int)((size_t)s.d * s.elt / 16);
+  if (s.dtype == SWITCH_MOE_BF16)
+    launch_k(top2_sum_kernel<true>, dim3((s.T + 7) / 8), dim3(256), 0, st, static_cast<const uint4*>(per_assignment),
+             ws_ptr<int>(ws, p.slot), s.T, row_vec, static_cast<uint4*>(out));
+  else
+    launch_k(top2_sum_kernel<false>, dim3((s.T + 7) / 8), dim3(256), 0, st, static_cast<const uint4*>(per_assignment),
+             ws_ptr<int>(ws, p.slot), s.T, row_vec, static_cast<uint4*>(out));
   return launch_status();
 }
 

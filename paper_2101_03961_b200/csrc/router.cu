@@ -204,12 +204,13 @@ router_jitter_kernel(const uint4* __restrict__ x, const uint4* __restrict__ u, s
 }
 
 // dh[t,i] = p[t,i] (G[t,i] - sum_j p[t,j] G[t,j]),  G[t,i] = cG.count_gi + [i = e_t and t kept].dgate_t,
-// count_gi counted inside the token's own routing group g = t / Tg
+// count_gi counted inside the token's own routing group g = t / Tg.  Top-2 routing (second > 0): the token's second
+// assignment T + t adds its own gate gradient at its own expert.
 template <int NE>
 __global__ void __launch_bounds__(256)
 router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ expert_index,
                       const int* __restrict__ slot, const int* __restrict__ count, const float* __restrict__ dgate,
-                      float cG, int T, int Tg, int E, float* __restrict__ dlogits,
+                      float cG, int T, int Tg, int E, int second, float* __restrict__ dlogits,
                       __nv_bfloat16* __restrict__ dhsplit, int Epad64) {
   pdl_launch_dependents();
   pdl_wait();
@@ -218,13 +219,15 @@ router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ e
   if (t >= T) return;
   const int et = expert_index[t];
   const float dg = slot[t] >= 0 ? dgate[t] : 0.f;
+  const int et2 = second ? expert_index[T + t] : -1;
+  const float dg2 = (second && slot[T + t] >= 0) ? dgate[T + t] : 0.f;
   count += (size_t)(t / Tg) * E;
   float p[NE], G[NE], s = 0.f;
 #pragma unroll
   for (int n = 0; n < NE; ++n) {
     const int e = lane * NE + n;
     p[n] = e < E ? probs[(size_t)t * E + e] : 0.f;
-    G[n] = e < E ? cG * (float)count[e] + (e == et ? dg : 0.f) : 0.f;
+    G[n] = e < E ? cG * (float)count[e] + (e == et ? dg : 0.f) + (e == et2 ? dg2 : 0.f) : 0.f;
     s = fmaf(p[n], G[n], s);
   }
 #pragma unroll
@@ -424,7 +427,7 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
   float* dlogits = ws_ptr<float>(ws, p.dlogits);
   launch_k(router_dlogits_kernel<NE>, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs),
                                                             ws_ptr<int>(ws, p.expert_proc), ws_ptr<int>(ws, p.slot),
-                                                            ws_ptr<int>(ws, p.count_g), dgate, cG, s.T, s.Tg, s.E, dlogits,
+                                                            ws_ptr<int>(ws, p.count_g), dgate, cG, s.T, s.Tg, s.E, s.top2, dlogits,
                                                             (s.router_tc && sizeof(XT) == 2)
                                                                 ? ws_ptr<__nv_bfloat16>(ws, p.dhsplit) : nullptr,
                                                             s.Epad64);
@@ -452,7 +455,7 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
       cudaSuccess)
     return SWITCH_MOE_CUDA_ERROR;
   launch_k(router_dx_kernel<XT, NE>, dim3((s.T + 63) / 64), dim3(256), smem, st, dlogits, W_r, ws_ptr<int>(ws, p.slot), s.T, s.d, s.E,
-                                                              accumulate_dx ? (s.residual ? 2 : 1) : 0,
+                                                              accumulate_dx ? ((s.residual || s.top2) ? 2 : 1) : 0,
                                                               static_cast<const XT*>(s.jitter_u), static_cast<XT*>(dx));
   return launch_status();
 }

@@ -762,7 +762,7 @@ int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const flo
   q.mma_n = kBN;
   q.n_mtiles = (s.T + kTileM - 1) / kTileM; q.n_ntiles = (s.d + kBN - 1) / kBN;
   q.wrap = s.Epad64 / kBK;
-  q.dx = static_cast<__nv_bfloat16*>(dx); q.slot = ws_ptr<int>(ws, p.slot); q.accumulate = accumulate_dx ? (s.residual ? 2 : 1) : 0;   // 2: every row (skip path inside the layer)
+  q.dx = static_cast<__nv_bfloat16*>(dx); q.slot = ws_ptr<int>(ws, p.slot); q.accumulate = accumulate_dx ? ((s.residual || s.top2) ? 2 : 1) : 0;   // 2: every row already holds a value
   q.jitter_u = static_cast<const __nv_bfloat16*>(s.jitter_u);
   return launch_op<kRDx>(tmA, tmB, q, st);
 }

@@ -34,6 +34,8 @@ struct Shape {
   int reroute;      // 1: overflowed tokens are offered to their second-choice expert (SWITCH_MOE_FLAG_REROUTE)
   int geglu;        // 1: GEGLU experts: W_in is [E, d, 2 f] (SWITCH_MOE_FLAG_GEGLU)
   int fin;          // columns of W_in per expert: f, or 2 f for GEGLU
+  int top2;         // 1: top-2 routing (SWITCH_MOE_FLAG_TOP2)
+  int Tv;           // assignments the dispatch plan places: T, or 2 T for top-2 routing (first choices, then second)
   int jitter;       // 1: the router's input is x . u (SWITCH_MOE_FLAG_INPUT_JITTER)
   const void* jitter_u;   // device [T, d] factors u (activation dtype); may be null when only sizes are asked for
 };
@@ -41,7 +43,7 @@ struct Shape {
 // Workspace layout: byte offsets from the (1024-byte aligned) workspace base.
 struct Plan {
   size_t status, expert_index, gate, slot, token_of_slot, count, kept, count_g, group_base, psum, psum_partial, hist, hist_base,
-      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, layer_y, alt, expert_proc, xr, ab, dab, total;
+      tile_expert, tile_row0, ntile, probs, dlogits, xd, h, dyd, dh, dgate, dwr_partial, wsplit, dhsplit, hmask, layer_y, alt, expert_proc, xr, ab, dab, yv, dxv, total;
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -63,7 +65,7 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (G > 1 && ((cfg->T / G) % kPlanBlockTokens != 0 || cfg->T > 65536 || G > kMaxGroups))
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if ((cfg->flags & ~(SWITCH_MOE_FLAG_RESIDUAL | SWITCH_MOE_FLAG_REROUTE | SWITCH_MOE_FLAG_INPUT_JITTER |
-                      SWITCH_MOE_FLAG_GEGLU)) != 0)
+                      SWITCH_MOE_FLAG_GEGLU | SWITCH_MOE_FLAG_TOP2)) != 0)
     return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->E > kMaxExperts) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if (cfg->d_model % 8 != 0 || cfg->d_ff % 8 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
@@ -89,6 +91,10 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   s->geglu = (cfg->flags & SWITCH_MOE_FLAG_GEGLU) ? 1 : 0;
   s->fin = s->geglu ? 2 * cfg->d_ff : cfg->d_ff;
   if (s->geglu && s->gemm_path == SWITCH_MOE_GEMM_TC_1CTA) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->top2 = (cfg->flags & SWITCH_MOE_FLAG_TOP2) ? 1 : 0;
+  if (s->top2 && (s->residual || (cfg->flags & SWITCH_MOE_FLAG_REROUTE) || G > 1 || cfg->T % kPlanBlockTokens != 0))
+    return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->Tv = s->top2 ? 2 * cfg->T : cfg->T;
   s->jitter = (cfg->flags & SWITCH_MOE_FLAG_INPUT_JITTER) ? 1 : 0;
   s->jitter_u = s->jitter ? cfg->router_jitter : nullptr;
   s->reroute = (cfg->flags & SWITCH_MOE_FLAG_REROUTE) ? 1 : 0;
@@ -99,7 +105,7 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   s->Epad = 32 * ne_pow2;
   s->Epad64 = (cfg->E + 63) / 64 * 64;
   s->router_tc = s->gemm_path != 1 ? 1 : 0;
-  s->plan_blocks = (cfg->T + kPlanBlockTokens - 1) / kPlanBlockTokens;
+  s->plan_blocks = (s->Tv + kPlanBlockTokens - 1) / kPlanBlockTokens;
   s->max_mtiles = cfg->E * ((s->C + kTileM - 1) / kTileM);
   if (s->router_tc) {
     // dW_r split so that tiles x splits fills the GPU
@@ -122,11 +128,11 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
 inline void make_plan(const Shape& s, Plan* p) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
-  const size_t T = s.T, E = s.E, C = s.C, d = s.d, f = s.f;
+  const size_t T = s.T, E = s.E, C = s.C, d = s.d, f = s.f, Tv = s.Tv;
   p->status = take(16 * sizeof(int32_t));
-  p->expert_index = take(T * 4);
-  p->gate = take(T * 4);
-  p->slot = take(T * 4);
+  p->expert_index = take(Tv * 4);
+  p->gate = take(Tv * 4);
+  p->slot = take(Tv * 4);
   p->token_of_slot = take(E * C * 4);
   p->count = take(E * 4);
   p->kept = take(E * 4);
@@ -145,7 +151,7 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->h = take(E * C * f * s.elt);
   p->dyd = take(E * C * d * s.elt);
   p->dh = take(E * C * f * s.elt);
-  p->dgate = take(T * 4);
+  p->dgate = take(Tv * 4);
   p->dwr_partial = take((size_t)s.dwr_chunks * d * E * 4);
   p->wsplit = take(3 * d * (size_t)s.Epad64 * 2);
   p->dhsplit = take(3 * T * (size_t)s.Epad64 * 2);
@@ -156,6 +162,8 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->xr = s.jitter ? take(T * d * s.elt) : 0;               // the router's input x . u, rounded to the activation dtype
   p->ab = s.geglu ? take(E * C * 2 * f * s.elt) : 0;        // GEGLU: [a | b] = X_d [W_0 | W_1] per slot
   p->dab = s.geglu ? take(E * C * 2 * f * s.elt) : 0;       // GEGLU: gradient of [a | b] per slot
+  p->yv = s.top2 ? take(Tv * d * s.elt) : 0;                // top-2: weighted expert output per assignment
+  p->dxv = s.top2 ? take(Tv * d * s.elt) : 0;               // top-2: input gradient per assignment
   p->total = off;
 }
 
@@ -208,6 +216,9 @@ int launch_router_fwd(const Shape& s, const Plan& p, const void* x, const float*
 int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_index, float* aux_loss, void* ws,
                          cudaStream_t st);
 int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void* ws, cudaStream_t st);
+// Top-2 routing: second choices (expert and weight) of every token; sums of the two assignments' rows.
+int launch_top2_choice(const Shape& s, const Plan& p, void* ws, cudaStream_t st);
+int launch_top2_sum(const Shape& s, const Plan& p, const void* per_assignment, void* out, void* ws, cudaStream_t st);
 int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* dx, void* ws, cudaStream_t st);
 int launch_router_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* dgate, float d_aux,
                       void* ws, void* dx, bool accumulate_dx, float* dW_r, cudaStream_t st);

@@ -42,7 +42,7 @@ class GpuLayer:
     """Device buffers of one layer call plus the library calls on them."""
 
     def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0,
-                 residual=False, groups=1, reroute=False, geglu=False):
+                 residual=False, groups=1, reroute=False, geglu=False, top2=False):
         sbuild.build()
         geglu = geglu or cfg.geglu
         jit = data.get("router_jitter")
@@ -50,7 +50,7 @@ class GpuLayer:
         self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
                                   dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path,
                                   residual=residual, groups=groups, reroute=reroute, input_jitter=jit is not None,
-                                  geglu=geglu)
+                                  geglu=geglu, top2=top2)
         dt = cfg.dtype
         self.x = to_dev(data["x"], dt)
         self.dy = to_dev(data["dy"], dt)

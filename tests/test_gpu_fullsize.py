@@ -185,3 +185,70 @@ def test_geglu_experts_at_the_papers_switch_base_shape_full_size():
 def test_batch_of_131072_tokens_full_size():
     out = _run_fullsize("long_batch")
     assert out["dropped"] < 0.05 * 131072
+
+
+def test_top2_routing_at_the_switch_base_shape_full_size():
+    """Top-2 routing at T=32768, E=128 with the capacity factor 2.0 of the paper's Mixture-of-Experts baselines: the
+    plan for all 65536 assignments bit for bit, sampled experts' rows and gradients within tolerance."""
+    sbuild.build()
+    cfg = si.CONFIGS["switch_base"].with_(capacity_factor=2.0)
+    seed = 0
+    x_np, dy_np, W_r_np = si.gen_x(cfg, seed), si.gen_dy(cfg, seed), si.gen_W_r(cfg, seed)
+    x, dy = _bits_to_dev(si.to_bf16_bits(x_np)), _bits_to_dev(si.to_bf16_bits(dy_np))
+    W_in = _bits_to_dev(si.gen_W_in(cfg, seed, as_bits=True, threads=16))
+    W_out = _bits_to_dev(si.gen_W_out(cfg, seed, as_bits=True, threads=16))
+    W_r = torch.from_numpy(W_r_np).cuda()
+    mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, top2=True)
+    ws = sm.allocate_workspace(mcfg)
+    ws.fill_(0xFF)
+    y, dx = torch.full_like(x, float("nan")), torch.full_like(x, float("nan"))
+    dW_in, dW_out = torch.full_like(W_in, float("nan")), torch.full_like(W_out, float("nan"))
+    dW_r = torch.full_like(W_r, float("nan"))
+    aux = torch.zeros(1, device="cuda")
+    sm.switch_moe_fwd(mcfg, x, W_r, None, W_in, W_out, y, aux, ws)
+    sm.switch_moe_bwd(mcfg, dy, 1.0, x, W_r, W_in, W_out, y, ws, dx, dW_r, dW_in, dW_out)
+    sm.switch_moe_check_device_status(mcfg, ws)
+    view = lambda r: sm.switch_moe_workspace_view(mcfg, ws, r)
+    T, E, C = cfg.T, cfg.E, sm.switch_moe_capacity(mcfg)
+    gpu_e = view(sm.WS_EXPERT_INDEX).cpu().numpy().astype(np.int64)
+    p = so.router_probs(so.router_logits(x_np, W_r_np))
+    first = gpu_e[:T]
+    assert check_flips(first, {"e": so.top1(p)[0], "p": p}) <= 8
+    second = check_second_choice(gpu_e[T:], p, first, np.ones(T, dtype=bool))
+    plan = so.top2_forward(x_np, W_r_np, {}, {}, cfg.capacity_factor, cfg.alpha, first_index=first, second_index=second,
+                           experts=[])
+    assert C == plan["C"] == 512
+    np.testing.assert_array_equal(view(sm.WS_SLOT).cpu().numpy(), plan["slot"])
+    np.testing.assert_array_equal(view(sm.WS_TOKEN_OF_SLOT).cpu().numpy(), plan["token_of_slot"])
+    np.testing.assert_array_equal(view(sm.WS_COUNT).cpu().numpy(), plan["count_first"])
+    np.testing.assert_array_equal(view(sm.WS_KEPT).cpu().numpy(), plan["kept"])
+    assert abs(float(aux.item()) - plan["aux"]) <= TOL_ROUTER * plan["aux"]
+    assert plan["keep"].mean() > 0.9                           # twice the capacity holds most of the assignments
+    kept = plan["kept"]
+    sample = sorted({int(np.argmax(kept)), int(np.argmin(kept)), 7, 100})
+    W_in_s = {i: si.gen_W_in_expert(cfg, i, seed) for i in sample}
+    W_out_s = {i: si.gen_W_out_expert(cfg, i, seed) for i in sample}
+    fwd = so.top2_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, first_index=first,
+                          second_index=second, experts=sample)
+    bwd = so.top2_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
+    yv = None
+    errs = {}
+    hid = view(sm.WS_H).view(E, C, cfg.d_ff)
+    for i in sample:
+        k = int(kept[i])
+        v = plan["token_of_slot"][i * C:i * C + k]
+        errs[f"H[{i}]"] = rel_err(to_np(hid[i, :k]), np.maximum(fwd["u"][i], 0.0))
+        errs[f"dW_in[{i}]"] = rel_err(to_np(dW_in[i]), bwd["dW_in"][i])
+        errs[f"dW_out[{i}]"] = rel_err(to_np(dW_out[i]), bwd["dW_out"][i])
+        vv = torch.from_numpy(v).cuda()
+        errs[f"dgate[{i}]"] = rel_err(to_np(view(sm.WS_DGATE)[vv]), bwd["dgate"][v])
+    # tokens both of whose assignments went to sampled experts: their whole output row is known to the oracle
+    in_sample = np.isin(plan["e"], sample) & plan["keep"]
+    whole = np.flatnonzero((in_sample[:T] | ~plan["keep"][:T]) & (in_sample[T:] | ~plan["keep"][T:])
+                           & (plan["keep"][:T] | plan["keep"][T:]))
+    assert whole.size > 10
+    wt = torch.from_numpy(whole).cuda()
+    errs["y"] = rel_err(to_np(y[wt]), fwd["y"][whole])
+    bad = {k: v for k, v in errs.items() if not v <= TOL_BF16}
+    assert not bad, (bad, errs)
+    assert bool(torch.isfinite(y).all()) and bool(torch.isfinite(dx).all()) and bool(torch.isfinite(dW_in).all())

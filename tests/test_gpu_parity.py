@@ -509,3 +509,79 @@ def test_forward_and_backward_can_be_captured_in_a_cuda_graph():
 def test_extreme_shapes_match_oracle(cfg):
     errs = _check_layer(cfg, sm.GEMM_DEFAULT, TOL_BF16, d_aux=0.5)
     assert errs
+
+
+# ---------------------------------------------------------------------------------------------- top-2 routing
+def _check_top2(cfg, gemm_path, tol, seed=0, d_aux=0.7):
+    from tests.gpu_helpers import check_second_choice
+    data = si.gen_layer(cfg, seed=seed)
+    g = GpuLayer(cfg, data, gemm_path=gemm_path, top2=True)
+    g.fwd()
+    T, E, C = cfg.T, cfg.E, g.C
+    gpu_e = g.expert_index()
+    assert gpu_e.shape == (2 * T,)
+    first, second = gpu_e[:T], gpu_e[T:]
+    probe = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
+                              router_bias=data.get("router_bias"), experts=[])
+    check_flips(first, probe)
+    second = check_second_choice(second, probe["p"], first, np.ones(T, dtype=bool))
+    fwd = so.top2_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
+                          router_bias=data.get("router_bias"), first_index=first, second_index=second)
+    assert C == fwd["C"]
+    keep = fwd["keep"]
+    assert keep[T:].any() and (~keep).any()                   # second choices do get slots, and some assignments overflow
+    np.testing.assert_array_equal(g.view(sm.WS_SLOT).cpu().numpy(), fwd["slot"])
+    np.testing.assert_array_equal(g.view(sm.WS_TOKEN_OF_SLOT).cpu().numpy(), fwd["token_of_slot"])
+    np.testing.assert_array_equal(g.view(sm.WS_COUNT).cpu().numpy(), fwd["count_first"])   # f counts first choices
+    np.testing.assert_array_equal(g.view(sm.WS_KEPT).cpu().numpy(), fwd["kept"])
+    assert rel_err(to_np(g.view(sm.WS_PROBS)).reshape(T, E), fwd["p"]) <= TOL_ROUTER
+    assert abs(float(g.aux.item()) - fwd["aux"]) <= TOL_ROUTER * abs(fwd["aux"])
+    np.testing.assert_allclose(to_np(g.view(sm.WS_GATE))[keep], fwd["g"][keep], rtol=2e-5)
+    xd = to_np(g.view(sm.WS_XD)).reshape(E, C, cfg.d_model)
+    hid = to_np(g.view(sm.WS_H)).reshape(E, C, cfg.d_ff)
+    x64 = np.asarray(data["x"], dtype=np.float64)
+    errs = {}
+    for i in range(E):
+        k = int(fwd["kept"][i])
+        if k == 0:
+            continue
+        v = fwd["token_of_slot"][i * C:i * C + k]
+        np.testing.assert_array_equal(xd[i, :k], x64[fwd["tok_of"][v]])
+        errs[f"H[{i}]"] = rel_err(hid[i, :k], np.maximum(fwd["u"][i], 0.0))
+    y = to_np(g.y)
+    assert np.isfinite(y).all()
+    both_dropped = ~keep[:T] & ~keep[T:]
+    assert np.all(y[both_dropped] == 0.0)
+    errs["y"] = rel_err(y, fwd["y"])
+    g.bwd(d_aux=d_aux)
+    bwd = so.top2_backward(fwd, data["x"], data["W_r"], data["W_in"], data["W_out"], data["dy"], d_aux=d_aux)
+    kept_v = np.flatnonzero(keep)
+    errs["dgate"] = rel_err(to_np(g.view(sm.WS_DGATE))[kept_v], bwd["dgate"][kept_v])
+    errs["dx"] = rel_err(to_np(g.dx), bwd["dx"])
+    errs["dW_r"] = rel_err(to_np(g.dW_r), bwd["dW_r"])
+    errs["dW_in"] = rel_err(to_np(g.dW_in), _stack(bwd["dW_in"]))
+    errs["dW_out"] = rel_err(to_np(g.dW_out), _stack(bwd["dW_out"]))
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, (bad, errs)
+
+
+TOP2 = si.SwitchConfig("top2", 2048, 128, 256, 8, 1.5, bias_std=0.3)
+TOP2_F32 = si.SwitchConfig("top2_f32", 512, 64, 128, 4, 1.5, dtype=si.DTYPE_F32, bias_std=0.3)
+
+
+@pytest.mark.parametrize("cfg,path,tol", [(TOP2_F32, sm.GEMM_DEFAULT, TOL_F32), (TOP2, sm.GEMM_SIMT, TOL_BF16),
+                                          (TOP2, sm.GEMM_DEFAULT, TOL_BF16), (TOP2, sm.GEMM_TC_1CTA, TOL_BF16),
+                                          (si.SwitchConfig("top2_many", 4096, 64, 128, 96, 2.0, bias_std=0.2),
+                                           sm.GEMM_DEFAULT, TOL_BF16)],
+                         ids=["f32", "fma", "tc", "tc1", "many_tc"])
+def test_top2_routing_matches_oracle(cfg, path, tol):
+    """y = p_a E_a(x) + p_b E_b(x): first choices placed before second choices, one capacity, f from the first choice."""
+    _check_top2(cfg, path, tol)
+
+
+def test_top2_is_refused_with_the_options_it_does_not_combine_with():
+    for kw in (dict(residual=True), dict(reroute=True), dict(groups=2), dict(T=2000)):
+        base = dict(T=2048, d_model=128, d_ff=256, E=8, capacity_factor=1.5, top2=True)
+        base.update(kw)
+        with pytest.raises(sm.SwitchMoeError):
+            sm.switch_moe_workspace_bytes(sm.make_config(**base))
