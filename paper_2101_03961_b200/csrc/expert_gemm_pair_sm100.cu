@@ -327,7 +327,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       tc_fence_after();
       const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * 256u;
       bool released = false;
-      if (!kTok) {
+      if constexpr (!kTok) {
         // Weight gradients (row = weight row): 64 output columns at a time, so that a row is a whole 128-byte line.
         // The warp's 2 KB of shared memory hold 16 rows x 128 bytes: rows 0-15 and 16-31 of the warp take turns, and
         // every store instruction then writes 4 complete lines (the store path's cost grows with the number of lines
@@ -384,8 +384,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         acc ^= 1u;
         if (acc == 0) acc_phase ^= 1u;
         continue;
-      }
-
+      } else {
 #pragma unroll 1
       for (int c = half; c < n_chunks; c += 2) {
         uint32_t v[32];
@@ -402,7 +401,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
           if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
           released = true;
         }
-        if (kTok) {
+        {
           long long offs[4];
 #pragma unroll
           for (int it = 0; it < 4; ++it) offs[it] = __shfl_sync(0xffffffffu, q_off[0], it * 8 + (lane >> 2));
@@ -479,31 +478,6 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             q_mw[k] = q_mw[k + 1];
           }
           __syncwarp();
-        } else {
-          // weight gradient: row = weight row, 32 output columns per chunk
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint32_t w[4];
-#pragma unroll
-            for (int h = 0; h < 4; ++h) {
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + 2 * h]),
-                                                        __uint_as_float(v[q * 8 + 2 * h + 1]));
-              w[h] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-            *reinterpret_cast<uint4*>(tr + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
-                make_uint4(w[0], w[1], w[2], w[3]);
-          }
-          __syncwarp();
-          const int col = t.n0 + c * 32 + (lane & 3) * 8;
-#pragma unroll
-          for (int it = 0; it < 4; ++it) {
-            const int rr = it * 8 + (lane >> 2);
-            const uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (((lane & 3) ^ ((rr >> 1) & 3)) << 4));
-            const int orow = m_warp + rr;
-            if (orow < p.Mw && col < p.Nfix)
-              *reinterpret_cast<uint4*>(p.out + ((long long)t.e * p.Mw + orow) * p.ld_out + col) = val;
-          }
-          __syncwarp();
         }
       }
       if (!released) {                                        // this warp had no chunk in this tile
@@ -513,6 +487,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       }
       acc ^= 1u;
       if (acc == 0) acc_phase ^= 1u;
+      }
     }
   }
 
