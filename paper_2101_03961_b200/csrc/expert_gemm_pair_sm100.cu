@@ -386,107 +386,107 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         continue;
       } else {
 #pragma unroll 1
-      for (int c = half; c < n_chunks; c += 2) {
-        uint32_t v[32];
-        if (have_acc) {
-          tc_ld32(t_addr + c * 32, v);
-          tc_wait_ld();
-        } else {
+        for (int c = half; c < n_chunks; c += 2) {
+          uint32_t v[32];
+          if (have_acc) {
+            tc_ld32(t_addr + c * 32, v);
+            tc_wait_ld();
+          } else {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = 0u;
+            for (int i = 0; i < 32; ++i) v[i] = 0u;
+          }
+          if (c + 2 >= n_chunks) {                              // last chunk of this warp: accumulator read out
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
+            released = true;
+          }
+          {
+            long long offs[4];
+#pragma unroll
+            for (int it = 0; it < 4; ++it) offs[it] = __shfl_sync(0xffffffffu, q_off[0], it * 8 + (lane >> 2));
+            if (OP == kGemm2Combine) gate_s[lane] = q_gate[0];
+            __syncwarp();
+            // transpose: this lane holds weight row m_warp + lane for 32 tokens -> tr[token][lane]
+#pragma unroll
+            for (int i4 = 0; i4 < 32; i4 += 4) {
+              float g[4] = {1.f, 1.f, 1.f, 1.f};
+              if (OP == kGemm2Combine) {
+                const float4 g4 = *reinterpret_cast<const float4*>(gate_s + i4);
+                g[0] = g4.x; g[1] = g4.y; g[2] = g4.z; g[3] = g4.w;
+              }
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                float a = __uint_as_float(v[i4 + u]);
+                if (OP == kGemm2Combine) a *= g[u];
+                if (OP == kGemm1Relu && !p.plain) a = fmaxf(a, 0.f);
+                *reinterpret_cast<__nv_bfloat16*>(tr + (i4 + u) * 64 + lane * 2) = __float2bfloat16(a);
+              }
+            }
+            __syncwarp();
+            uint32_t mword[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+              const int rr = it * 8 + (lane >> 2);
+              uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (lane & 3) * 16);
+              if (OP == kDgrad2Mask && !p.plain) {              // ReLU'(u) = [u > 0]: bits saved by the forward GEMM
+                const uint32_t bits = __shfl_sync(0xffffffffu, q_mw[0], rr) >> ((lane & 3) * 8);
+                uint32_t* w = reinterpret_cast<uint32_t*>(&val);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  w[q] &= ((bits >> (2 * q)) & 1u ? 0x0000FFFFu : 0u) | ((bits >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u);
+              }
+              if (OP == kGemm1Relu && !p.plain) {               // save [H > 0] as one bit per element for the backward pass
+                const uint32_t* w = reinterpret_cast<const uint32_t*>(&val);
+                uint32_t m8 = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  m8 |= ((w[q] & 0x00007FFFu) ? 1u << (2 * q) : 0u) | ((w[q] & 0x7FFF0000u) ? 1u << (2 * q + 1) : 0u);
+                uint32_t word = m8 << ((lane & 3) * 8);
+                word |= __shfl_xor_sync(0xffffffffu, word, 1);
+                word |= __shfl_xor_sync(0xffffffffu, word, 2);
+                mword[it] = word;                               // the word of token row rr, in all four lanes of its group
+              }
+              if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[it] >= 0 && mcol < p.Mw) {
+                // skip path inside the layer: y = x + g E(x), dx = dy + dH W_in^T (the expert term is already bf16)
+                if (OP == kGemm2Combine) *reinterpret_cast<uint4*>(p.out2 + offs[it] + mcol) = val;
+                const uint4 r = *reinterpret_cast<const uint4*>(p.res + offs[it] + mcol);
+                const __nv_bfloat162* rv = reinterpret_cast<const __nv_bfloat162*>(&r);
+                __nv_bfloat162* vv = reinterpret_cast<__nv_bfloat162*>(&val);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const float2 a2 = __bfloat1622float2(vv[q]), b2 = __bfloat1622float2(rv[q]);
+                  vv[q] = __floats2bfloat162_rn(a2.x + b2.x, a2.y + b2.y);
+                }
+              }
+              if (offs[it] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[it] + mcol) = val;
+            }
+            if (OP == kGemm1Relu && !p.plain) {                 // lane i stores the mask word of token row i: one 128-byte line
+              uint32_t mine = 0;
+#pragma unroll
+              for (int it = 0; it < 4; ++it) {
+                const uint32_t w = __shfl_sync(0xffffffffu, mword[it], 4 * (lane & 7));
+                if ((lane >> 3) == it) mine = w;
+              }
+              if (q_off[0] >= 0 && m_warp < p.Mw)
+                p.hmask[(long long)(m_warp >> 5) * p.hmask_rows + (long long)t.e * p.C + t.row0 + c * 32 + lane] = mine;
+            }
+#pragma unroll
+            for (int k = 0; k < 3; ++k) {                       // advance the queue
+              q_off[k] = q_off[k + 1];
+              q_gate[k] = q_gate[k + 1];
+              q_mw[k] = q_mw[k + 1];
+            }
+            __syncwarp();
+          }
         }
-        if (c + 2 >= n_chunks) {                              // last chunk of this warp: accumulator read out
+        if (!released) {                                        // this warp had no chunk in this tile
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
-          released = true;
         }
-        {
-          long long offs[4];
-#pragma unroll
-          for (int it = 0; it < 4; ++it) offs[it] = __shfl_sync(0xffffffffu, q_off[0], it * 8 + (lane >> 2));
-          if (OP == kGemm2Combine) gate_s[lane] = q_gate[0];
-          __syncwarp();
-          // transpose: this lane holds weight row m_warp + lane for 32 tokens -> tr[token][lane]
-#pragma unroll
-          for (int i4 = 0; i4 < 32; i4 += 4) {
-            float g[4] = {1.f, 1.f, 1.f, 1.f};
-            if (OP == kGemm2Combine) {
-              const float4 g4 = *reinterpret_cast<const float4*>(gate_s + i4);
-              g[0] = g4.x; g[1] = g4.y; g[2] = g4.z; g[3] = g4.w;
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              float a = __uint_as_float(v[i4 + u]);
-              if (OP == kGemm2Combine) a *= g[u];
-              if (OP == kGemm1Relu && !p.plain) a = fmaxf(a, 0.f);
-              *reinterpret_cast<__nv_bfloat16*>(tr + (i4 + u) * 64 + lane * 2) = __float2bfloat16(a);
-            }
-          }
-          __syncwarp();
-          uint32_t mword[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-          for (int it = 0; it < 4; ++it) {
-            const int rr = it * 8 + (lane >> 2);
-            uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (lane & 3) * 16);
-            if (OP == kDgrad2Mask && !p.plain) {              // ReLU'(u) = [u > 0]: bits saved by the forward GEMM
-              const uint32_t bits = __shfl_sync(0xffffffffu, q_mw[0], rr) >> ((lane & 3) * 8);
-              uint32_t* w = reinterpret_cast<uint32_t*>(&val);
-#pragma unroll
-              for (int q = 0; q < 4; ++q)
-                w[q] &= ((bits >> (2 * q)) & 1u ? 0x0000FFFFu : 0u) | ((bits >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u);
-            }
-            if (OP == kGemm1Relu && !p.plain) {               // save [H > 0] as one bit per element for the backward pass
-              const uint32_t* w = reinterpret_cast<const uint32_t*>(&val);
-              uint32_t m8 = 0;
-#pragma unroll
-              for (int q = 0; q < 4; ++q)
-                m8 |= ((w[q] & 0x00007FFFu) ? 1u << (2 * q) : 0u) | ((w[q] & 0x7FFF0000u) ? 1u << (2 * q + 1) : 0u);
-              uint32_t word = m8 << ((lane & 3) * 8);
-              word |= __shfl_xor_sync(0xffffffffu, word, 1);
-              word |= __shfl_xor_sync(0xffffffffu, word, 2);
-              mword[it] = word;                               // the word of token row rr, in all four lanes of its group
-            }
-            if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[it] >= 0 && mcol < p.Mw) {
-              // skip path inside the layer: y = x + g E(x), dx = dy + dH W_in^T (the expert term is already bf16)
-              if (OP == kGemm2Combine) *reinterpret_cast<uint4*>(p.out2 + offs[it] + mcol) = val;
-              const uint4 r = *reinterpret_cast<const uint4*>(p.res + offs[it] + mcol);
-              const __nv_bfloat162* rv = reinterpret_cast<const __nv_bfloat162*>(&r);
-              __nv_bfloat162* vv = reinterpret_cast<__nv_bfloat162*>(&val);
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const float2 a2 = __bfloat1622float2(vv[q]), b2 = __bfloat1622float2(rv[q]);
-                vv[q] = __floats2bfloat162_rn(a2.x + b2.x, a2.y + b2.y);
-              }
-            }
-            if (offs[it] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[it] + mcol) = val;
-          }
-          if (OP == kGemm1Relu && !p.plain) {                 // lane i stores the mask word of token row i: one 128-byte line
-            uint32_t mine = 0;
-#pragma unroll
-            for (int it = 0; it < 4; ++it) {
-              const uint32_t w = __shfl_sync(0xffffffffu, mword[it], 4 * (lane & 7));
-              if ((lane >> 3) == it) mine = w;
-            }
-            if (q_off[0] >= 0 && m_warp < p.Mw)
-              p.hmask[(long long)(m_warp >> 5) * p.hmask_rows + (long long)t.e * p.C + t.row0 + c * 32 + lane] = mine;
-          }
-#pragma unroll
-          for (int k = 0; k < 3; ++k) {                       // advance the queue
-            q_off[k] = q_off[k + 1];
-            q_gate[k] = q_gate[k + 1];
-            q_mw[k] = q_mw[k + 1];
-          }
-          __syncwarp();
-        }
-      }
-      if (!released) {                                        // this warp had no chunk in this tile
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
-      }
-      acc ^= 1u;
-      if (acc == 0) acc_phase ^= 1u;
+        acc ^= 1u;
+        if (acc == 0) acc_phase ^= 1u;
       }
     }
   }
