@@ -585,3 +585,28 @@ def test_top2_is_refused_with_the_options_it_does_not_combine_with():
         base.update(kw)
         with pytest.raises(sm.SwitchMoeError):
             sm.switch_moe_workspace_bytes(sm.make_config(**base))
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(residual=True), dict(reroute=True), dict(top2=True), dict(geglu=True)],
+                         ids=["plain", "skip", "reroute", "top2", "geglu"])
+def test_results_are_bitwise_reproducible(kw):
+    """No floating-point atomics and fixed reduction orders everywhere: two runs on the same inputs give the same bits,
+    whatever ran in between."""
+    cfg = si.SwitchConfig("repro", 2048, 128, 256, 8, 1.0, bias_std=0.5)
+    if kw.get("geglu"):
+        cfg = cfg.with_(geglu=True)
+    data = si.gen_layer(cfg, seed=3)
+    g = GpuLayer(cfg, data, **{k: v for k, v in kw.items() if k != "geglu"})
+    outs = []
+    for rep in range(3):
+        for t in (g.y, g.dx, g.dW_r, g.dW_in, g.dW_out):
+            t.fill_(float("nan"))
+        if rep == 1:
+            g.ws.fill_(0x5A)                                  # different stale workspace contents
+            g.view(sm.WS_STATUS).zero_()
+        g.fwd()
+        g.bwd(d_aux=0.3)
+        outs.append([t.clone() for t in (g.y, g.dx, g.dW_r, g.dW_in, g.dW_out, g.aux)])
+    for other in outs[1:]:
+        for a, b in zip(outs[0], other):
+            assert torch.equal(a, b)
