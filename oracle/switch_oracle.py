@@ -319,7 +319,8 @@ def router_backward_given_dgate(p, e, keep, count, dgate, x, W_r, alpha: float, 
 # the experts are shared, and the loss is the mean over cores and experts times num_experts^2, i.e. the mean of the
 # groups' losses.  Here a group is T / G consecutive rows of x.
 def switch_forward_groups(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, groups: int, router_bias=None,
-                          expert_index=None, experts=None, residual: bool = False):
+                          expert_index=None, experts=None, residual: bool = False, router_noise=None,
+                          router_jitter=None, storage_round=None, geglu: bool = False):
     """Forward for G routing groups: switch_forward on each group, results concatenated in token order.
 
     The merged plan numbers an expert's rows group by group (group 0's kept tokens in token order, then group 1's,
@@ -336,8 +337,11 @@ def switch_forward_groups(x, W_r, W_in, W_out, capacity_factor: float, alpha: fl
     for g in range(G):
         rows = slice(g * Tg, (g + 1) * Tg)
         ei = None if expert_index is None else np.asarray(expert_index)[rows]
+        noise = None if router_noise is None else np.asarray(router_noise)[rows]
+        jitter = None if router_jitter is None else np.asarray(router_jitter)[rows]
         parts.append(switch_forward(x64[rows], W_r, W_in, W_out, capacity_factor, alpha, router_bias=router_bias,
-                                    expert_index=ei, experts=experts, residual=residual))
+                                    expert_index=ei, experts=experts, residual=residual, router_noise=noise,
+                                    router_jitter=jitter, storage_round=storage_round, geglu=geglu))
     C = parts[0]["C"]
     cat = lambda k: np.concatenate([q[k] for q in parts], axis=0)
     kept_g = np.stack([q["kept"] for q in parts])                       # [G, E]
@@ -349,6 +353,7 @@ def switch_forward_groups(x, W_r, W_in, W_out, capacity_factor: float, alpha: fl
     token_of_slot = np.full(E * G * C, -1, dtype=np.int64)
     token_of_slot[slot[keep]] = np.flatnonzero(keep)
     out = {"parts": parts, "G": G, "Tg": Tg, "C": C, "E": E, "T": T, "alpha": alpha, "residual": bool(residual),
+           "geglu": bool(geglu),
            "aux": float(np.mean([q["aux"] for q in parts])),
            "y": cat("y"), "layer_y": cat("layer_y"), "o": cat("o"), "p": cat("p"), "h": cat("h"), "g": cat("g"),
            "e": e, "pos": pos, "keep": keep, "slot": slot, "token_of_slot": token_of_slot,

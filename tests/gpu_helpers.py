@@ -128,13 +128,15 @@ def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capaci
     if data.get("router_jitter") is not None:                  # the router sees x . u rounded to the activation type
         jit_kw.update({"router_jitter": data["router_jitter"], "storage_round": si.storage_round(cfg)})
     if groups > 1:
-        assert capacity is None and not jit_kw
+        assert capacity is None
         first = so.switch_forward_groups(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
-                                         cfg.alpha, groups, router_bias=data.get("router_bias"), experts=[])
+                                         cfg.alpha, groups, router_bias=data.get("router_bias"), experts=[],
+                                         router_noise=data.get("router_noise"), **jit_kw)
         flips = check_flips(gpu_e, first)
         fwd = so.switch_forward_groups(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
                                        cfg.alpha, groups, router_bias=data.get("router_bias"), expert_index=gpu_e,
-                                       experts=experts, residual=residual)
+                                       experts=experts, residual=residual, router_noise=data.get("router_noise"),
+                                       **jit_kw)
         fwd["flips"] = flips
         return fwd
     first = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,

@@ -610,3 +610,14 @@ def test_results_are_bitwise_reproducible(kw):
     for other in outs[1:]:
         for a, b in zip(outs[0], other):
             assert torch.equal(a, b)
+
+
+def test_options_combine():
+    """Rerouting + the skip path + GEGLU experts + logit noise + input jitter in one call; several groups + GEGLU."""
+    cfg = si.SwitchConfig("combo", 2048, 128, 256, 8, 1.0, bias_std=0.5)
+    _check_layer(cfg, sm.GEMM_DEFAULT, TOL_BF16, reroute=True, residual=True, geglu=True, noise_eps=0.3, jitter_eps=0.2,
+                 d_aux=0.4)
+    _check_layer(cfg, sm.GEMM_SIMT, TOL_BF16, reroute=True, residual=True, geglu=True, noise_eps=0.3, jitter_eps=0.2,
+                 d_aux=0.4)
+    _check_layer(si.SwitchConfig("combo_groups", 2048, 128, 256, 8, 1.0, bias_std=0.3), sm.GEMM_DEFAULT, TOL_BF16,
+                 groups=4, geglu=True, noise_eps=0.3, d_aux=0.4)
