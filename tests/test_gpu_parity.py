@@ -621,3 +621,19 @@ def test_options_combine():
                  d_aux=0.4)
     _check_layer(si.SwitchConfig("combo_groups", 2048, 128, 256, 8, 1.0, bias_std=0.3), sm.GEMM_DEFAULT, TOL_BF16,
                  groups=4, geglu=True, noise_eps=0.3, d_aux=0.4)
+
+
+def test_top2_with_a_single_expert_has_no_second_choice():
+    cfg = si.SwitchConfig("top2_one_expert", 256, 64, 64, 1, 1.0)
+    data = si.gen_layer(cfg, seed=0)
+    g = GpuLayer(cfg, data, top2=True)
+    g.fwd()
+    g.bwd()
+    e = g.expert_index()
+    assert np.all(e[:256] == 0) and np.all(e[256:] == -1)
+    assert np.all(g.view(sm.WS_SLOT).cpu().numpy()[256:] == -1)
+    plain = GpuLayer(cfg, data)
+    plain.fwd()
+    plain.bwd()
+    for a, b in ((g.y, plain.y), (g.dx, plain.dx), (g.dW_in, plain.dW_in), (g.dW_out, plain.dW_out), (g.dW_r, plain.dW_r)):
+        assert torch.equal(a, b)
