@@ -160,7 +160,7 @@ def reroute_overflow(plan, e, alt, E: int, C: int):
 def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None,
                    capacity: int | None = None, expert_index=None, experts=None, residual: bool = False,
                    reroute: bool = False, alt_index=None, router_noise=None, router_jitter=None, storage_round=None,
-                   geglu: bool = False):
+                   geglu: bool = False, expert_keep=None, expert_dropout: float = 0.0):
     """Forward of the Switch FFN layer for one routing group.
 
     x [T, d]; W_r [d, E]; W_in [E, d, f]; W_out [E, f, d].  `capacity` overrides Eq. 3 when given.
@@ -182,6 +182,10 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     `geglu` replaces the expert's ReLU FFN by the GEGLU FFN of the paper's Table 9 ("the expansion matrix is
     substituted with two sets of weights which are non-linearly combined"): W_in[i] is [d, 2 f] = [W_0 | W_1],
     a = x W_0, b = x W_1, hidden = GELU(a) . b, output = hidden W_out.  "u" then holds the rows [a | b].
+    `expert_keep` [E * C, f] (booleans, indexed by slot row) with `expert_dropout` = rate applies expert dropout
+    (Section 2.4 / fine-tuning regularisation table: a larger dropout rate "at the interim feed-forward computation at
+    each expert layer"): the hidden activations are multiplied by keep / (1 - rate), the usual inverted dropout; the
+    mask is an input (the caller draws it).
     Returns a dict with every intermediate the staged comparisons need.
     """
     x64 = np.asarray(x, dtype=F64)
@@ -225,6 +229,8 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
             a_i = gelu(u_i[:, :fh]) * u_i[:, fh:]                # GELU(x W_0) . (x W_1)
         else:
             a_i = np.maximum(u_i, 0.0)                           # ReLU(h)
+        if expert_keep is not None:                              # expert dropout on the hidden activations
+            a_i = a_i * (np.asarray(expert_keep)[i * C:i * C + tok.size] / (1.0 - expert_dropout))
         o_i = a_i @ np.asarray(W_out[i], dtype=F64)              # y = ReLU(h) W_out
         u[i] = u_i
         o[tok] = o_i
@@ -232,6 +238,7 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "layer_y": y,
            "y": x64 + y if residual else y, "o": o, "u": u, "T": T, "E": E, "alpha": alpha, "residual": bool(residual),
            "e_proc": e_proc, "x_router": x_router, "geglu": bool(geglu),
+           "expert_keep": None if expert_keep is None else np.asarray(expert_keep, dtype=F64) / (1.0 - expert_dropout),
            "router_jitter": None if router_jitter is None else np.asarray(router_jitter, dtype=F64)}
     out.update(plan)
     return out
@@ -269,6 +276,10 @@ def switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=No
         do_i = g[tok, None] * dy64[tok]                 # y = g . o        =>  do = g . dy
         dgate[tok] = np.sum(dy64[tok] * fwd["o"][tok], axis=1)   #          =>  dg = <dy, o>
         da_i = do_i @ W_out_i.T                         # o = a W_out
+        keep_i = None
+        if fwd.get("expert_keep") is not None:          # a = dropout(act(u)): the same factors on the way back
+            keep_i = fwd["expert_keep"][i * C:i * C + tok.size]
+            da_i = da_i * keep_i
         if fwd.get("geglu", False):
             fh = u_i.shape[1] // 2
             ua, ub = u_i[:, :fh], u_i[:, fh:]
@@ -277,6 +288,8 @@ def switch_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=No
         else:
             a_i = np.maximum(u_i, 0.0)
             du_i = da_i * (u_i > 0.0)                   # a = ReLU(u), ReLU'(0) = 0
+        if keep_i is not None:
+            a_i = a_i * keep_i                          # the hidden activations that entered W_out
         dx[tok] = du_i @ W_in_i.T                       # u = x W_in
         if want_weight_grads:
             dW_out[i] = a_i.T @ do_i

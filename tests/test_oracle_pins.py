@@ -802,3 +802,49 @@ def test_top2_backward_matches_finite_differences():
             num.append((lp - lm) / (2 * eps))
         ana = np.array([grad[i] for i in idxs])
         assert np.linalg.norm(np.array(num) - ana) / np.linalg.norm(ana) < 1e-7, name
+
+
+# ------------------------------------------------------------------ expert dropout (fine-tuning regularisation)
+def test_expert_dropout_scales_kept_hidden_units_and_gradients_match_finite_differences():
+    T, d, f, E, cf, alpha, rate = 16, 5, 8, 3, 0.75, 0.03, 0.4
+    rng = np.random.default_rng(91)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=91, scale=2.0)
+    plain = so.switch_forward(x, W_r, W_in, W_out, cf, alpha)
+    C = plain["C"]
+    keep = rng.random((E * C, f)) >= rate
+    fwd = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, expert_keep=keep, expert_dropout=rate)
+    assert np.array_equal(fwd["slot"], plain["slot"]) and fwd["aux"] == plain["aux"]      # routing is untouched
+    for t in np.flatnonzero(fwd["keep"])[:6]:
+        i, s = fwd["e"][t], fwd["slot"][t]
+        hidden = np.maximum(x[t] @ W_in[i], 0.0) * keep[s] / (1.0 - rate)
+        np.testing.assert_allclose(fwd["y"][t], fwd["g"][t] * (hidden @ W_out[i]), rtol=1e-12, atol=1e-14)
+    ones = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, expert_keep=np.ones((E * C, f), bool), expert_dropout=0.0)
+    assert np.array_equal(ones["y"], plain["y"])
+    R = rng.standard_normal((T, d))
+    srt = np.sort(fwd["p"], axis=1)
+    assert (srt[:, -1] - srt[:, -2]).min() > 1e-3
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, R, d_aux=0.6)
+    e_frozen, eps = fwd["e"], 1e-6
+
+    def loss():
+        o = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, expert_index=e_frozen, expert_keep=keep, expert_dropout=rate)
+        return float(np.sum(o["y"] * R) + 0.6 * o["aux"])
+
+    dW_in = np.stack([bwd["dW_in"][i] for i in range(E)])
+    dW_out = np.stack([bwd["dW_out"][i] for i in range(E)])
+    for name, arr, grad in [("dx", x, bwd["dx"]), ("dW_r", W_r, bwd["dW_r"]), ("dW_in", W_in, dW_in),
+                            ("dW_out", W_out, dW_out)]:
+        idxs = list(np.ndindex(arr.shape))
+        if len(idxs) > 150:
+            idxs = [idxs[i] for i in rng.choice(len(idxs), 150, replace=False)]
+        num = []
+        for idx in idxs:
+            old = arr[idx]
+            arr[idx] = old + eps
+            lp = loss()
+            arr[idx] = old - eps
+            lm = loss()
+            arr[idx] = old
+            num.append((lp - lm) / (2 * eps))
+        ana = np.array([grad[i] for i in idxs])
+        assert np.linalg.norm(np.array(num) - ana) / np.linalg.norm(ana) < 1e-7, name
