@@ -245,11 +245,18 @@ def run_ours(args, cfg):
 
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype,
                           residual=args.residual, groups=args.groups, reroute=args.reroute,
-                          input_jitter=args.input_jitter > 0.0, geglu=cfg.geglu, top2=args.top2)
+                          input_jitter=args.input_jitter > 0.0, geglu=cfg.geglu, top2=args.top2,
+                          expert_dropout=args.expert_dropout if args.expert_dropout > 0.0 else None)
     noise = None
     if args.router_noise > 0.0:                              # exploration noise on the logits: an input of the layer
         noise = torch.from_numpy(si.gen_router_noise(cfg, args.router_noise, seed)).cuda()
         mcfg.router_noise = noise.data_ptr()
+    keep_bits = None
+    if args.expert_dropout > 0.0:                            # expert dropout: the keep mask is a seeded input as well
+        rows = cfg.E * sm.switch_moe_capacity(mcfg) * max(args.groups, 1)
+        keep_bits = torch.from_numpy(si.pack_keep_bits(si.gen_expert_keep(cfg, rows, args.expert_dropout, seed))
+                                     .view(np.int32)).cuda()
+        mcfg.expert_keep = keep_bits.data_ptr()
     jitter = None
     if args.input_jitter > 0.0:                              # multiplicative jitter on the router's input: an input too
         jitter = dev(si.gen_router_jitter(cfg, args.input_jitter, seed))
@@ -437,7 +444,7 @@ def run_ours(args, cfg):
                    "geglu_experts": cfg.geglu,
                    "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha, "capacity": sm.switch_moe_capacity(mcfg),
                    "kept_tokens": kept, "parallelism": "replicas" if world > 1 else "single",
-                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "top2_routing": bool(args.top2), "router_noise_eps": args.router_noise, "input_jitter_eps": args.input_jitter,
+                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "top2_routing": bool(args.top2), "expert_dropout": args.expert_dropout, "router_noise_eps": args.router_noise, "input_jitter_eps": args.input_jitter,
                    "l2": "inputs larger than L2 (weights 2 x %.0f MB per pass), no flush" %
                          (cfg.E * cfg.d_model * cfg.d_ff * elt / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": sm.switch_moe_launches_per_step(mcfg) * args.steps,
@@ -472,6 +479,8 @@ def main():
     ap.add_argument("--top2", action="store_true",
                     help="top-2 routing (the Mixture-of-Experts comparator): two assignments per token, so about twice "
                          "the expert work of the headline configuration at a capacity factor that keeps them")
+    ap.add_argument("--expert-dropout", type=float, default=0.0,
+                    help="dropout rate on the experts' hidden activations (fine-tuning regularisation; seeded keep mask)")
     ap.add_argument("--reroute", action="store_true",
                     help="offer tokens that overflow their expert to their second choice (stage 2 of "
                          "No-Token-Left-Behind routing); not the headline configuration")

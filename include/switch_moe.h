@@ -69,10 +69,14 @@ enum switch_moe_gemm_path {
    the capacity of Eq. 3; f in the auxiliary loss counts the first choice.  The library numbers the 2T assignments
    v = t (first choice of token t) and v = T + t (second choice): the workspace regions EXPERT_INDEX, GATE, SLOT and
    DGATE then have 2T entries and TOKEN_OF_SLOT holds v.  Needs T to be a multiple of 256; not together with
-   RESIDUAL, REROUTE or several routing groups. */
+   RESIDUAL, REROUTE or several routing groups.
+   SWITCH_MOE_FLAG_EXPERT_DROPOUT: expert dropout (the fine-tuning regularisation of Section 2.4: a larger dropout
+   rate "at the interim feed-forward computation at each expert layer"): the experts' hidden activations are
+   multiplied by keep / (1 - expert_dropout), and so is their gradient on the way back.  The keep mask is an input
+   (expert_keep), one bit per hidden unit of every slot row; the caller draws it. */
 enum switch_moe_flags {
   SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2, SWITCH_MOE_FLAG_INPUT_JITTER = 4, SWITCH_MOE_FLAG_GEGLU = 8,
-  SWITCH_MOE_FLAG_TOP2 = 16
+  SWITCH_MOE_FLAG_TOP2 = 16, SWITCH_MOE_FLAG_EXPERT_DROPOUT = 32
 };
 
 typedef enum switch_moe_status {
@@ -117,6 +121,9 @@ typedef struct switch_moe_config {
                                 (e.g. uniform(1 - eps, 1 + eps), drawn by the caller); must be set, 16-byte aligned,
                                 when the flag is, and is ignored otherwise.  Needed by fwd, router_fwd, bwd and
                                 router_bwd alike. */
+  const uint32_t* expert_keep; /* DEVICE uint32[E * G * C][d_ff / 32]: bit i of word [row][w] = keep hidden unit 32 w + i
+                                  of slot row `row` (SWITCH_MOE_FLAG_EXPERT_DROPOUT; d_ff a multiple of 32) */
+  float expert_dropout;        /* the dropout rate of that flag, in [0, 1) */
 } switch_moe_config;
 
 #define SWITCH_MOE_STAGE_EVENTS 13

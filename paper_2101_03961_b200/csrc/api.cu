@@ -146,6 +146,7 @@ int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r
   SWMOE_TRY(mark(cfg, 3, st));
   SWMOE_TRY(run_gemm(kGemm1Relu, c, a, workspace, st));
   if (c.s.geglu) SWMOE_TRY(launch_geglu_fwd(c.s, c.p, workspace, st));     // hidden = GELU(a) . b
+  if (c.s.dropout) SWMOE_TRY(launch_expert_dropout(c.s, c.p, false, workspace, st));
   SWMOE_TRY(mark(cfg, 4, st));
   SWMOE_TRY(run_gemm(kGemm2Combine, c, a, workspace, st));
   if (c.s.top2) SWMOE_TRY(launch_top2_sum(c.s, c.p, y_rows, y, workspace, st));   // Eq. 2: sum over the two experts
@@ -173,6 +174,7 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
   SWMOE_TRY(launch_gather_dy(c.s, c.p, dy, c.s.top2 ? ws_ptr<void>(workspace, c.p.yv) : y, dx, workspace, st));
   SWMOE_TRY(mark(cfg, 7, st));
   SWMOE_TRY(run_gemm(kDgrad2Mask, c, a, workspace, st));
+  if (c.s.dropout) SWMOE_TRY(launch_expert_dropout(c.s, c.p, true, workspace, st));   // same factors on the way back
   if (c.s.geglu) SWMOE_TRY(launch_geglu_bwd(c.s, c.p, workspace, st));     // d[a | b] from dH
   SWMOE_TRY(mark(cfg, 8, st));
   SWMOE_TRY(run_gemm(kWgrad2, c, a, workspace, st));
@@ -313,7 +315,7 @@ int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches
   // Rerouting of overflowed tokens adds four plan kernels to the forward pass.
   // Input jitter adds the element-wise product kernel.
   // GEGLU experts add the gating kernel to each pass.  Top-2 routing adds the second-choice kernel and two row sums.
-  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0) + (s.geglu ? 2 : 0) + (s.top2 ? 3 : 0);
+  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0) + (s.geglu ? 2 : 0) + (s.top2 ? 3 : 0) + (s.dropout ? 2 : 0);
   return SWITCH_MOE_OK;
 }
 

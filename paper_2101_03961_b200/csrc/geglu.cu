@@ -82,6 +82,33 @@ geglu_kernel(const uint4* __restrict__ ab, const int* __restrict__ kept, int E, 
   }
 }
 
+// Expert dropout: one warp per slot row, consecutive lanes on consecutive 16-byte pieces of the row; a piece's keep
+// bits are one byte (bf16: 8 hidden units) or half a byte (fp32: 4) of the row's mask words.
+template <typename ET>
+__global__ void __launch_bounds__(256)
+expert_dropout_kernel(const uint32_t* __restrict__ keep_bits, const int* __restrict__ kept, int E, int C, int f,
+                      float scale, ET* __restrict__ rows) {
+  pdl_launch_dependents();
+  pdl_wait();
+  constexpr int N = Pack<ET>::n;                             // elements per 16 bytes
+  const int lane = threadIdx.x & 31;
+  const int s = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (s >= E * C) return;
+  const int ex = s / C, pos = s - ex * C;
+  if (pos >= min(C, (kept[ex] + 15) / 16 * 16)) return;
+  const uint32_t* words = keep_bits + (size_t)s * (f / 32);
+  uint4* row = reinterpret_cast<uint4*>(rows + (size_t)s * f);
+  for (int v = lane; v < f / N; v += 32) {
+    const int first = v * N;                                   // first hidden unit of this piece
+    const uint32_t bits = words[first >> 5] >> (first & 31);
+    float x[N];
+    Pack<ET>::load(row[v], x);
+#pragma unroll
+    for (int i = 0; i < N; ++i) x[i] = ((bits >> i) & 1u) ? x[i] * scale : 0.f;
+    row[v] = Pack<ET>::store(x);
+  }
+}
+
 template <bool kBackward>
 int launch(const Shape& s, const Plan& p, void* ws, cudaStream_t st) {
   const int f_vec = (int)((size_t)s.f * s.elt / 16);
@@ -102,5 +129,18 @@ int launch(const Shape& s, const Plan& p, void* ws, cudaStream_t st) {
 
 int launch_geglu_fwd(const Shape& s, const Plan& p, void* ws, cudaStream_t st) { return launch<false>(s, p, ws, st); }
 int launch_geglu_bwd(const Shape& s, const Plan& p, void* ws, cudaStream_t st) { return launch<true>(s, p, ws, st); }
+
+int launch_expert_dropout(const Shape& s, const Plan& p, bool backward, void* ws, cudaStream_t st) {
+  if (s.keep_bits == nullptr || (reinterpret_cast<uintptr_t>(s.keep_bits) & 3u) != 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  const int blocks = (s.E * s.C + 7) / 8;
+  void* rows = ws_ptr<char>(ws, backward ? p.dh : p.h);
+  if (s.dtype == SWITCH_MOE_BF16)
+    launch_k(expert_dropout_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, s.keep_bits, ws_ptr<int>(ws, p.kept), s.E,
+             s.C, s.f, s.keep_scale, static_cast<__nv_bfloat16*>(rows));
+  else
+    launch_k(expert_dropout_kernel<float>, dim3(blocks), dim3(256), 0, st, s.keep_bits, ws_ptr<int>(ws, p.kept), s.E, s.C,
+             s.f, s.keep_scale, static_cast<float*>(rows));
+  return launch_status();
+}
 
 }  // namespace swmoe

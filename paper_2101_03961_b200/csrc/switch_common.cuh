@@ -34,6 +34,9 @@ struct Shape {
   int reroute;      // 1: overflowed tokens are offered to their second-choice expert (SWITCH_MOE_FLAG_REROUTE)
   int geglu;        // 1: GEGLU experts: W_in is [E, d, 2 f] (SWITCH_MOE_FLAG_GEGLU)
   int fin;          // columns of W_in per expert: f, or 2 f for GEGLU
+  int dropout;      // 1: expert dropout on the hidden activations (SWITCH_MOE_FLAG_EXPERT_DROPOUT)
+  const uint32_t* keep_bits;   // device [E C][f / 32] keep mask; may be null when only sizes are asked for
+  float keep_scale;            // 1 / (1 - rate)
   int top2;         // 1: top-2 routing (SWITCH_MOE_FLAG_TOP2)
   int Tv;           // assignments the dispatch plan places: T, or 2 T for top-2 routing (first choices, then second)
   int jitter;       // 1: the router's input is x . u (SWITCH_MOE_FLAG_INPUT_JITTER)
@@ -65,7 +68,7 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (G > 1 && ((cfg->T / G) % kPlanBlockTokens != 0 || cfg->T > 65536 || G > kMaxGroups))
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if ((cfg->flags & ~(SWITCH_MOE_FLAG_RESIDUAL | SWITCH_MOE_FLAG_REROUTE | SWITCH_MOE_FLAG_INPUT_JITTER |
-                      SWITCH_MOE_FLAG_GEGLU | SWITCH_MOE_FLAG_TOP2)) != 0)
+                      SWITCH_MOE_FLAG_GEGLU | SWITCH_MOE_FLAG_TOP2 | SWITCH_MOE_FLAG_EXPERT_DROPOUT)) != 0)
     return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->E > kMaxExperts) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   if (cfg->d_model % 8 != 0 || cfg->d_ff % 8 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
@@ -91,6 +94,14 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   s->geglu = (cfg->flags & SWITCH_MOE_FLAG_GEGLU) ? 1 : 0;
   s->fin = s->geglu ? 2 * cfg->d_ff : cfg->d_ff;
   if (s->geglu && s->gemm_path == SWITCH_MOE_GEMM_TC_1CTA) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  s->dropout = (cfg->flags & SWITCH_MOE_FLAG_EXPERT_DROPOUT) ? 1 : 0;
+  s->keep_bits = s->dropout ? cfg->expert_keep : nullptr;
+  s->keep_scale = 1.f;
+  if (s->dropout) {
+    if (!(cfg->expert_dropout >= 0.f) || !(cfg->expert_dropout < 1.f)) return SWITCH_MOE_INVALID_ARGUMENT;
+    if (cfg->d_ff % 32 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+    s->keep_scale = 1.f / (1.f - cfg->expert_dropout);
+  }
   s->top2 = (cfg->flags & SWITCH_MOE_FLAG_TOP2) ? 1 : 0;
   if (s->top2 && (s->residual || (cfg->flags & SWITCH_MOE_FLAG_REROUTE) || G > 1 || cfg->T % kPlanBlockTokens != 0))
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
@@ -249,5 +260,8 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
 // GEGLU gating over the kept rows: H = GELU(a) . b, and its derivative d[a | b] from dH (element-wise).
 int launch_geglu_fwd(const Shape& s, const Plan& p, void* ws, cudaStream_t st);
 int launch_geglu_bwd(const Shape& s, const Plan& p, void* ws, cudaStream_t st);
+// Expert dropout: rows[slot][j] *= keep bit / (1 - rate) over the kept rows of the hidden activations (forward) or of
+// their gradient (backward).
+int launch_expert_dropout(const Shape& s, const Plan& p, bool backward, void* ws, cudaStream_t st);
 
 }  // namespace swmoe

@@ -24,7 +24,7 @@ import numpy as np
 DTYPE_BF16 = 0
 DTYPE_F32 = 1
 
-_TENSOR_X, _TENSOR_DY, _TENSOR_WR, _TENSOR_WIN, _TENSOR_WOUT, _TENSOR_BIAS, _TENSOR_NOISE, _TENSOR_JITTER = 1, 2, 3, 4, 5, 6, 7, 8
+_TENSOR_X, _TENSOR_DY, _TENSOR_WR, _TENSOR_WIN, _TENSOR_WOUT, _TENSOR_BIAS, _TENSOR_NOISE, _TENSOR_JITTER, _TENSOR_KEEP = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
 
 @dataclass(frozen=True)
@@ -150,6 +150,20 @@ def gen_router_jitter(cfg: SwitchConfig, eps: float, seed: int = 0) -> np.ndarra
     (bf16-representable where cfg.dtype is bf16); an input of the layer like x."""
     u = _rng(seed, _TENSOR_JITTER).random((cfg.T, cfg.d_model), dtype=np.float32)
     return _finish(cfg, (np.float32(1.0 - eps) + np.float32(2.0 * eps) * u).astype(np.float32))
+
+
+def gen_expert_keep(cfg: SwitchConfig, slot_rows: int, rate: float, seed: int = 0) -> np.ndarray:
+    """Keep mask of expert dropout, booleans [slot_rows, d_ff] (slot_rows = experts x rows per expert), each True with
+    probability 1 - rate; an input of the layer."""
+    return _rng(seed, _TENSOR_KEEP).random((slot_rows, cfg.d_ff), dtype=np.float32) >= np.float32(rate)
+
+
+def pack_keep_bits(keep: np.ndarray) -> np.ndarray:
+    """Booleans [rows, d_ff] -> uint32 [rows, d_ff / 32]: bit i of word w is hidden unit 32 w + i."""
+    rows, f = keep.shape
+    assert f % 32 == 0
+    packed = np.packbits(keep.reshape(rows, f // 32, 32), axis=-1, bitorder="little")
+    return np.ascontiguousarray(packed).view("<u4").reshape(rows, f // 32)
 
 
 def storage_round(cfg: SwitchConfig):

@@ -24,7 +24,7 @@ INVALID_ARGUMENT, UNSUPPORTED_SHAPE, WORKSPACE_TOO_SMALL, CUDA_ERROR, DEVICE_TIM
 
 WS_STATUS, WS_EXPERT_INDEX, WS_GATE, WS_SLOT, WS_TOKEN_OF_SLOT, WS_COUNT, WS_KEPT, WS_PSUM, WS_PROBS, WS_XD, WS_H, \
     WS_DYD, WS_DH, WS_DGATE, WS_DLOGITS, WS_LAYER_Y, WS_EXPERT_PROC, WS_SECOND_CHOICE = range(18)
-FLAG_RESIDUAL, FLAG_REROUTE, FLAG_INPUT_JITTER, FLAG_GEGLU, FLAG_TOP2 = 1, 2, 4, 8, 16
+FLAG_RESIDUAL, FLAG_REROUTE, FLAG_INPUT_JITTER, FLAG_GEGLU, FLAG_TOP2, FLAG_EXPERT_DROPOUT = 1, 2, 4, 8, 16, 32
 
 EXPORTED_SYMBOLS = [
     "switch_moe_capacity", "switch_moe_workspace_bytes", "switch_moe_workspace_view", "switch_moe_fwd",
@@ -45,6 +45,8 @@ class SwitchMoeConfig(ctypes.Structure):
         ("stage_events", ctypes.POINTER(ctypes.c_void_p)),
         ("router_noise", ctypes.c_void_p),
         ("router_jitter", ctypes.c_void_p),
+        ("expert_keep", ctypes.c_void_p),
+        ("expert_dropout", ctypes.c_float),
     ]
 
 
@@ -92,14 +94,15 @@ def load_library() -> ctypes.CDLL:
 
 
 def make_config(T, d_model, d_ff, E, capacity_factor, alpha=0.01, dtype=BF16, capacity_override=0,
-                gemm_path=GEMM_DEFAULT, residual=False, groups=1, reroute=False, input_jitter=False, geglu=False, top2=False) -> SwitchMoeConfig:
+                gemm_path=GEMM_DEFAULT, residual=False, groups=1, reroute=False, input_jitter=False, geglu=False, top2=False, expert_dropout=None) -> SwitchMoeConfig:
     cfg = SwitchMoeConfig()
     cfg.T, cfg.d_model, cfg.d_ff, cfg.E = int(T), int(d_model), int(d_ff), int(E)
     cfg.capacity_factor, cfg.alpha = float(capacity_factor), float(alpha)
     cfg.capacity_override, cfg.dtype, cfg.gemm_path = int(capacity_override), int(dtype), int(gemm_path)
     cfg.flags = ((FLAG_RESIDUAL if residual else 0) | (FLAG_REROUTE if reroute else 0)
                  | (FLAG_INPUT_JITTER if input_jitter else 0) | (FLAG_GEGLU if geglu else 0)
-                 | (FLAG_TOP2 if top2 else 0))     # set cfg.router_jitter to the device pointer of u
+                 | (FLAG_TOP2 if top2 else 0) | (FLAG_EXPERT_DROPOUT if expert_dropout is not None else 0))
+    cfg.expert_dropout = float(expert_dropout or 0.0)              # set cfg.expert_keep to the device pointer of the mask     # set cfg.router_jitter to the device pointer of u
     cfg.groups = int(groups)
     return cfg
 

@@ -44,13 +44,15 @@ class GpuLayer:
     def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0,
                  residual=False, groups=1, reroute=False, geglu=False, top2=False):
         sbuild.build()
+        keep = data.get("expert_keep")
         geglu = geglu or cfg.geglu
         jit = data.get("router_jitter")
         self.scfg = cfg
         self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
                                   dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path,
                                   residual=residual, groups=groups, reroute=reroute, input_jitter=jit is not None,
-                                  geglu=geglu, top2=top2)
+                                  geglu=geglu, top2=top2,
+                                  expert_dropout=data.get("expert_dropout") if keep is not None else None)
         dt = cfg.dtype
         self.x = to_dev(data["x"], dt)
         self.dy = to_dev(data["dy"], dt)
@@ -64,6 +66,10 @@ class GpuLayer:
         self.jitter = None if jit is None else to_dev(jit, dt)
         if self.jitter is not None:
             self.cfg.router_jitter = self.jitter.data_ptr()
+        self.keep = None
+        if keep is not None:
+            self.keep = torch.from_numpy(si.pack_keep_bits(keep).view(np.int32)).cuda()
+            self.cfg.expert_keep = self.keep.data_ptr()
         self.W_in = to_dev(data["W_in"], dt)
         self.W_out = to_dev(data["W_out"], dt)
         tdt = torch.bfloat16 if dt == sm.BF16 else torch.float32
@@ -125,6 +131,8 @@ def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capaci
                      residual=False, groups=1, gpu_alt=None, geglu=False):
     """Oracle forward with the device's expert choice (identical unless a near-tie flipped), after checking flips."""
     jit_kw = {"geglu": True} if (geglu or cfg.geglu) else {}
+    if data.get("expert_keep") is not None:
+        jit_kw.update({"expert_keep": data["expert_keep"], "expert_dropout": data["expert_dropout"]})
     if data.get("router_jitter") is not None:                  # the router sees x . u rounded to the activation type
         jit_kw.update({"router_jitter": data["router_jitter"], "storage_round": si.storage_round(cfg)})
     if groups > 1:
@@ -180,5 +188,9 @@ def expert_hidden(fwd: dict, i: int):
     u = expert_preactivation(fwd, i)
     if fwd.get("geglu", False):
         fh = u.shape[1] // 2
-        return so.gelu(u[:, :fh]) * u[:, fh:]
-    return np.maximum(u, 0.0)
+        hidden = so.gelu(u[:, :fh]) * u[:, fh:]
+    else:
+        hidden = np.maximum(u, 0.0)
+    if fwd.get("expert_keep") is not None:                       # factors keep / (1 - rate), by slot row
+        hidden = hidden * fwd["expert_keep"][i * fwd["C"]:i * fwd["C"] + hidden.shape[0]]
+    return hidden

@@ -122,12 +122,15 @@ def test_dispatch_plan_is_deterministic():
 
 # ---------------------------------------------------------------------------------------------- whole layer
 def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False, groups=1,
-                 reroute=False, noise_eps=0.0, jitter_eps=0.0, geglu=False):
+                 reroute=False, noise_eps=0.0, jitter_eps=0.0, geglu=False, dropout=0.0):
     if geglu:                                                  # W_in = [W_0 | W_1]: twice the columns
         cfg = cfg.with_(geglu=True)
     data = si.gen_layer(cfg, seed=seed)
     if jitter_eps:
         data["router_jitter"] = si.gen_router_jitter(cfg, jitter_eps, seed)
+    if dropout:
+        rows = cfg.E * so.expert_capacity(cfg.T, cfg.E, cfg.capacity_factor)
+        data["expert_keep"], data["expert_dropout"] = si.gen_expert_keep(cfg, rows, dropout, seed), dropout
     if noise_eps:
         data["router_noise"] = si.gen_router_noise(cfg, noise_eps, seed)
     g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual,
@@ -637,3 +640,12 @@ def test_top2_with_a_single_expert_has_no_second_choice():
     plain.bwd()
     for a, b in ((g.y, plain.y), (g.dx, plain.dx), (g.dW_in, plain.dW_in), (g.dW_out, plain.dW_out), (g.dW_r, plain.dW_r)):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("cfg,path,tol,kw", [
+    (TINY, sm.GEMM_DEFAULT, TOL_F32, {}), (MID, sm.GEMM_SIMT, TOL_BF16, {}), (MID, sm.GEMM_DEFAULT, TOL_BF16, {}),
+    (RAGGED, sm.GEMM_DEFAULT, TOL_BF16, dict(reroute=True)), (MANY, sm.GEMM_DEFAULT, TOL_BF16, dict(geglu=True, residual=True))],
+    ids=["tiny_f32", "mid_fma", "mid_tc", "ragged_tc_reroute", "many_tc_geglu_skip"])
+def test_expert_dropout_matches_oracle(cfg, path, tol, kw):
+    """Hidden activations and their gradient are multiplied by keep / (1 - rate); the mask is a seeded input."""
+    _check_layer(cfg, path, tol, dropout=0.4, d_aux=0.7, **kw)
