@@ -111,7 +111,9 @@ typedef struct switch_moe_config {
                                 When set, fwd records event i on the stream before its stage i (0 router, 1 dispatch
                                 plan, 2 gather, 3 GEMM1+ReLU, 4 GEMM2+combine) and event 5 after the last one; bwd
                                 records events 6..11 before (6 gather dy, 7 dgrad2, 8 wgrad2, 9 dgrad1, 10 wgrad1,
-                                11 router backward) and event 12 after.  For per-kernel timing only. */
+                                11 router backward) and event 12 after.  With gemm_path 0 dgrad1 and wgrad1 are one
+                                launch: event 10 follows it, so stage 9 spans both products and stage 10 is empty.
+                                For per-kernel timing only. */
   const float* router_noise; /* DEVICE float[T, E] added to the router logits before the softmax, or NULL (default).
                                 The router pseudo-code of the appendix adds uniform(1 - eps, 1 + eps) noise to the
                                 logits in training (the text instead speaks of multiplicative jitter on the router's

@@ -179,9 +179,15 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
   SWMOE_TRY(mark(cfg, 8, st));
   SWMOE_TRY(run_gemm(kWgrad2, c, a, workspace, st));
   SWMOE_TRY(mark(cfg, 9, st));
-  SWMOE_TRY(run_gemm(kDgrad1Scatter, c, a, workspace, st));
-  SWMOE_TRY(mark(cfg, 10, st));
-  SWMOE_TRY(run_gemm(kWgrad1, c, a, workspace, st));
+  if (c.s.gemm_path == 0) {
+    // both products of dH in one launch (they share its rows through L2); the stage event between them falls after both
+    SWMOE_TRY(launch_pair_dgrad1_wgrad1(c.s, c.p, a, workspace, st));
+    SWMOE_TRY(mark(cfg, 10, st));
+  } else {
+    SWMOE_TRY(run_gemm(kDgrad1Scatter, c, a, workspace, st));
+    SWMOE_TRY(mark(cfg, 10, st));
+    SWMOE_TRY(run_gemm(kWgrad1, c, a, workspace, st));
+  }
   if (c.s.top2) SWMOE_TRY(launch_top2_sum(c.s, c.p, dx_rows, dx, workspace, st));
   SWMOE_TRY(mark(cfg, 11, st));
   SWMOE_TRY(launch_router_bwd(c.s, c.p, x, W_r, ws_ptr<float>(workspace, c.p.dgate), d_aux, workspace, dx, true, dW_r,
@@ -315,7 +321,8 @@ int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches
   // Rerouting of overflowed tokens adds four plan kernels to the forward pass.
   // Input jitter adds the element-wise product kernel.
   // GEGLU experts add the gating kernel to each pass.  Top-2 routing adds the second-choice kernel and two row sums.
-  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0) + (s.geglu ? 2 : 0) + (s.top2 ? 3 : 0) + (s.dropout ? 2 : 0);
+  // The paired-CTA path runs the two products of dH (dgrad1, wgrad1) as one launch.
+  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) - (s.gemm_path == 0 ? 1 : 0) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0) + (s.geglu ? 2 : 0) + (s.top2 ? 3 : 0) + (s.dropout ? 2 : 0);
   return SWITCH_MOE_OK;
 }
 

@@ -135,10 +135,12 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
 
 // One instantiation per product (OP is a GemmOp): each kernel carries only its own epilogue, and the operand
 // orientations are compile-time constants, which keeps the code footprint of every role small.
+//
+// `pair` of `n_pairs` is this CTA pair's place among the pairs that work on this product: the whole grid for a
+// launch of one product, a share of it when two products run side by side in one launch (below).
 template <int OP>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
-expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                        const PairParams p) {
+__device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairParams& p,
+                                          const int pair, const int n_pairs) {
   constexpr bool kTok = OP <= kDgrad1Scatter;                 // tokens on N, transposed epilogue
   constexpr bool kAMn = (OP == kGemm1Relu || OP == kGemm2Combine || OP == kWgrad2 || OP == kWgrad1);
   constexpr bool kBMn = !kTok;
@@ -160,7 +162,6 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();                   // 0 = leader (issues the MMAs)
-  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kPStages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
@@ -502,14 +503,33 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 }
 
 template <int OP>
-int launch_pair_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairParams& q, int dev, int sm_count,
-                   cudaStream_t st) {
-  if (cudaFuncSetAttribute(expert_gemm_pair_kernel<OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmemBytes) !=
-      cudaSuccess)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                        const PairParams p) {
+  pair_body<OP>(tmA, tmB, p, (int)(blockIdx.x >> 1), (int)(gridDim.x >> 1));
+}
+
+// Two products that read the same activations, side by side in one launch: the first `split` CTA pairs work on
+// product A, the others on product B, each walking the experts in the same order.  dgrad1 (dx = dH W_in^T) and wgrad1
+// (dW_in = X_d^T dH) both read dH and nothing of each other; run one after the other each reads its 0.2 GB from HBM,
+// run together the expert's rows that one of them fetched are still in L2 when the other asks for them (whichever
+// runs ahead pays the HBM latency and so falls back: the two stay within a few experts of each other).
+template <int OPA, int OPB>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+expert_gemm_pair_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                             const PairParams p0, const __grid_constant__ CUtensorMap tmA1,
+                             const __grid_constant__ CUtensorMap tmB1, const PairParams p1, const int split) {
+  const int cl = (int)(blockIdx.x >> 1), n = (int)(gridDim.x >> 1);
+  if (cl < split) pair_body<OPA>(tmA0, tmB0, p0, cl, split);
+  else pair_body<OPB>(tmA1, tmB1, p1, cl - split, n - split);
+}
+
+// persistent grid: as many CTA pairs as can be resident at once (at most one CTA per SM).  The occupancy query
+// costs tens of microseconds of host time, so its answer is kept per device and kernel.
+template <typename Kernel>
+int pair_grid(Kernel kernel, int* cached_grid, int dev, int sm_count, cudaStream_t st, int* grid_out) {
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmemBytes) != cudaSuccess)
     return SWITCH_MOE_CUDA_ERROR;
-  // persistent grid: as many CTA pairs as can be resident at once (at most one CTA per SM).  The occupancy query
-  // costs tens of microseconds of host time, so its answer is kept per device.
-  static int cached_grid[64] = {0};
   int grid = (dev >= 0 && dev < 64) ? cached_grid[dev] : 0;
   if (grid == 0) {
     cudaLaunchConfig_t lc = {};
@@ -518,8 +538,7 @@ int launch_pair_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairPar
     lc.dynamicSmemBytes = kPSmemBytes;
     lc.stream = st;
     int max_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&max_clusters, expert_gemm_pair_kernel<OP>, &lc) != cudaSuccess ||
-        max_clusters < 1) {
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &lc) != cudaSuccess || max_clusters < 1) {
       (void)cudaGetLastError();
       max_clusters = sm_count / 2;
     }
@@ -527,17 +546,24 @@ int launch_pair_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairPar
     if (grid < 2) return SWITCH_MOE_CUDA_ERROR;
     if (dev >= 0 && dev < 64) cached_grid[dev] = grid;
   }
+  *grid_out = grid;
+  return SWITCH_MOE_OK;
+}
+
+template <int OP>
+int launch_pair_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairParams& q, int dev, int sm_count,
+                   cudaStream_t st) {
+  static int cached_grid[64] = {0};
+  int grid = 0;
+  const int rc = pair_grid(expert_gemm_pair_kernel<OP>, cached_grid, dev, sm_count, st, &grid);
+  if (rc != SWITCH_MOE_OK) return rc;
   launch_k(expert_gemm_pair_kernel<OP>, dim3(grid), dim3(kPThreads), kPSmemBytes, st, tmA, tmB, q);
   return launch_status();
 }
 
-}  // namespace
-
-int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st) {
-  int dev = 0, sm_count = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
-  if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return SWITCH_MOE_CUDA_ERROR;
+// Operands, output and tile counts of one product.
+int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, PairParams* out,
+                 CUtensorMap* tmA_out, CUtensorMap* tmB_out) {
   const void* xd = ws_ptr<char>(ws, p.xd);
   const void* h = ws_ptr<char>(ws, p.h);
   const void* dyd = ws_ptr<char>(ws, p.dyd);
@@ -555,7 +581,8 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   q.status = ws_ptr<int>(ws, p.status);
   q.hmask = ws_ptr<uint32_t>(ws, p.hmask);
   q.hmask_rows = (long long)s.E * s.C;
-  CUtensorMap tmA, tmB;
+  CUtensorMap& tmA = *tmA_out;
+  CUtensorMap& tmB = *tmB_out;
   int rc = SWITCH_MOE_OK, rc2 = SWITCH_MOE_OK;
   int K = 0;
   switch (op) {
@@ -594,6 +621,26 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   q.n_mpairs = (q.Mw + 255) / 256;
   q.n_ntiles_fixed = q.token_op ? 0 : (q.Nfix + 255) / 256;
   q.k_blocks_fixed = q.token_op ? K / kBK : 0;
+  *out = q;
+  return SWITCH_MOE_OK;
+}
+
+int device_and_sms(int* dev, int* sm_count) {
+  if (cudaGetDevice(dev) != cudaSuccess) return SWITCH_MOE_CUDA_ERROR;
+  if (cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, *dev) != cudaSuccess)
+    return SWITCH_MOE_CUDA_ERROR;
+  return SWITCH_MOE_OK;
+}
+
+}  // namespace
+
+int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st) {
+  int dev = 0, sm_count = 0;
+  if (device_and_sms(&dev, &sm_count) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  PairParams q;
+  CUtensorMap tmA, tmB;
+  const int rc = pair_problem(op, s, p, a, ws, &q, &tmA, &tmB);
+  if (rc != SWITCH_MOE_OK) return rc;
   switch (op) {
     case kGemm1Relu: return launch_pair_op<kGemm1Relu>(tmA, tmB, q, dev, sm_count, st);
     case kGemm2Combine: return launch_pair_op<kGemm2Combine>(tmA, tmB, q, dev, sm_count, st);
@@ -602,6 +649,35 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
     case kWgrad2: return launch_pair_op<kWgrad2>(tmA, tmB, q, dev, sm_count, st);
     default: return launch_pair_op<kWgrad1>(tmA, tmB, q, dev, sm_count, st);
   }
+}
+
+// dgrad1 and wgrad1 in one launch (see expert_gemm_pair_dual_kernel).  The two products have the same flops; the
+// weight gradient's tiles are the slower ones, so it gets the larger share of the CTA pairs (39 of 74 measured best
+// on B200 at the bench shape: 1.3% of the step against two launches).
+int launch_pair_dgrad1_wgrad1(const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st) {
+  int dev = 0, sm_count = 0;
+  if (device_and_sms(&dev, &sm_count) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  PairParams q0, q1;
+  CUtensorMap tmA0, tmB0, tmA1, tmB1;
+  int rc = pair_problem(kDgrad1Scatter, s, p, a, ws, &q0, &tmA0, &tmB0);
+  if (rc != SWITCH_MOE_OK) return rc;
+  rc = pair_problem(kWgrad1, s, p, a, ws, &q1, &tmA1, &tmB1);
+  if (rc != SWITCH_MOE_OK) return rc;
+  static int cached_grid[64] = {0};
+  int grid = 0;
+  auto kernel = expert_gemm_pair_dual_kernel<kDgrad1Scatter, kWgrad1>;
+  rc = pair_grid(kernel, cached_grid, dev, sm_count, st, &grid);
+  if (rc != SWITCH_MOE_OK) return rc;
+  const int n_pairs = grid / 2;
+  if (n_pairs < 2) {                                          // nothing to share a launch with: one after the other
+    rc = launch_pair_op<kDgrad1Scatter>(tmA0, tmB0, q0, dev, sm_count, st);
+    return rc != SWITCH_MOE_OK ? rc : launch_pair_op<kWgrad1>(tmA1, tmB1, q1, dev, sm_count, st);
+  }
+  int split = (n_pairs * 35 + 37) / 74;
+  if (split < 1) split = 1;
+  if (split > n_pairs - 1) split = n_pairs - 1;
+  launch_k(kernel, dim3(grid), dim3(kPThreads), kPSmemBytes, st, tmA0, tmB0, q0, tmA1, tmB1, q1, split);
+  return launch_status();
 }
 
 }  // namespace swmoe

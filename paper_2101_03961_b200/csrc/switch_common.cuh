@@ -257,6 +257,7 @@ struct GemmArgs {
 int launch_simt_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
 int launch_tc_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
 int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
+int launch_pair_dgrad1_wgrad1(const Shape& s, const Plan& p, const GemmArgs& a, void* ws, cudaStream_t st);
 // GEGLU gating over the kept rows: H = GELU(a) . b, and its derivative d[a | b] from dH (element-wise).
 int launch_geglu_fwd(const Shape& s, const Plan& p, void* ws, cudaStream_t st);
 int launch_geglu_bwd(const Shape& s, const Plan& p, void* ws, cudaStream_t st);

@@ -87,7 +87,8 @@ def test_status_strings(lib):
 
 def test_launch_count_is_reported(lib):
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, dtype=sm.F32)) == 16
-    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 18
+    # bf16 default path: 18 kernels, of which the two products of dH share one launch
+    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 17
     # options add launches: four plan kernels for rerouting, one product kernel for input jitter, two GEGLU gating kernels
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, reroute=True, input_jitter=True,
-                                                          geglu=True, expert_dropout=0.4)) == 18 + 4 + 1 + 2 + 2
+                                                          geglu=True, expert_dropout=0.4)) == 17 + 4 + 1 + 2 + 2
