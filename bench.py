@@ -341,9 +341,9 @@ def run_ours(args, cfg):
     achieved_tf = flops_per_launch / (gemm_ms_avg * 1e-3) / 1e12
     if cfg.dtype == si.DTYPE_BF16:
         peak_tf = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
-        # DRAM bytes per launch from the ncu capture of the quarter-size workload (195.4 MB per launch at E=32,
+        # DRAM bytes per product from the ncu capture of the quarter-size workload (191.3 MB per product at E=32,
         # proportional to E); see profiles/expert_gemm_pair_kernel__switch_base_quarter.md
-        traffic = 195.4e6 * cfg.E / 32 if (cfg.d_model, cfg.d_ff) == (768, 3072) and cfg.T == 256 * cfg.E else None
+        traffic = 191.3e6 * cfg.E / 32 if (cfg.d_model, cfg.d_ff) == (768, 3072) and cfg.T == 256 * cfg.E else None
         hbm_peak = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
         roofline = {"bound": "tensor", "kernel": "expert_gemm_pair_kernel (6 products per step in 5 launches, mean per product)",
                     "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
