@@ -430,6 +430,7 @@ def run_ours(args, cfg):
     act_bytes = cfg.T * row_bytes
     e2e = {"value": world * cfg.T / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 2 * act_bytes,
            "d2h_bytes_per_step": 2 * act_bytes + 4, "ms_per_step": e2e_s * 1e3,
+           "pcie_gbs_each_way": 2 * act_bytes / e2e_s / 1e9,   # both directions carry this at once
            "blocking_call_value": world * cfg.T / blocking_s, "blocking_call_ms_per_step": blocking_s * 1e3,
            "note": "switch_moe_step_host_enqueue, two steps in flight: every step copies x, dy from pinned host memory "
                    "and y, dx, aux back; weights and weight gradients resident.  blocking_call_*: switch_moe_step_host, "
