@@ -544,8 +544,9 @@ def run_ours(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    # defaults: long enough for the GPU to settle at its power-capped clock before the timed steps (about 0.4 s of
-    # warm-up), so that the default line is a sustained figure; the whole run still takes seconds
+    # defaults (300 warm-up, 500 timed steps): long enough for the GPU to settle at its power-capped clock before the
+    # timed steps (about 0.4 s of warm-up) and to average over the cap's swings (0.7 s per timed region), so that the
+    # default line is a sustained figure; the whole run still takes seconds
     # (the reference arm's steps take seconds each on the host: its defaults are 3 timed steps after 1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
@@ -580,7 +581,7 @@ def main():
     args = ap.parse_args()
     cfg = si.CONFIGS[args.workload]
     if args.steps is None:
-        args.steps = 3 if args.impl == "reference" else 200
+        args.steps = 3 if args.impl == "reference" else 500
     if args.warmup is None:
         args.warmup = 1 if args.impl == "reference" else 300
     if args.oracle_experts is None:
