@@ -384,7 +384,7 @@ def run_ours(args, cfg):
     gemm_names = ["gemm1_relu", "gemm2_combine", "dgrad2_mask", "wgrad2", "dgrad1_scatter", "wgrad1"]
     gemm_ms_avg = statistics.mean(stage_ms[n] for n in gemm_names)
     # useful flops of one expert GEMM (kept rows only); with GEGLU experts the three GEMMs that touch W_in have twice
-    # the columns, and the figure is the mean over the six launches
+    # the columns, and the figure is the mean over the six products
     gemm_weight = {n: 1.0 for n in gemm_names}
     if cfg.geglu:
         gemm_weight.update({"gemm1_relu": 2.0, "dgrad1_scatter": 2.0, "wgrad1": 2.0})
