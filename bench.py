@@ -416,7 +416,10 @@ def run_ours(args, cfg):
                     "frac_of_burst_peak": achieved_tf / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
                     "hbm_gbs_at_measured_traffic": None if traffic is None else traffic / (gemm_ms_avg * 1e-3) / 1e9,
                     "hbm_frac_at_measured_traffic": None if traffic is None
-                    else traffic / (gemm_ms_avg * 1e-3) / 1e9 / hbm_peak}
+                    else traffic / (gemm_ms_avg * 1e-3) / 1e9 / hbm_peak,
+                    # nominal figures for context: 2250 TFLOP/s dense bf16, 8000 GB/s HBM3e
+                    "frac_of_nominal_peak": achieved_tf / 2250.0,
+                    "hbm_frac_of_nominal": None if traffic is None else traffic / (gemm_ms_avg * 1e-3) / 1e9 / 8000.0}
     else:
         peak_tf = 148 * 128 * 2 * 1.965e9 / 1e12
         roofline = {"bound": "alu", "kernel": "simt_grouped_gemm_kernel", "achieved": achieved_tf, "peak": peak_tf,
