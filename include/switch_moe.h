@@ -54,13 +54,12 @@ enum switch_moe_gemm_path {
    second-highest probability and takes that expert's next free slot if one is left; its gate is that expert's
    probability.  Tokens kept by the first stage keep their slots, and f in the auxiliary loss still counts the
    argmax.  One routing group only.
-   SWITCH_MOE_FLAG_INPUT_JITTER: the router's input is x . u, element by element, with u = router_jitter (the text's
-   "multiplicative jitter noise on the incoming representation", Appendix C); the experts still see x.  The product
+   SWITCH_MOE_FLAG_INPUT_JITTER: the router's input is x . u, element by element, with u = router_jitter (input
+   jitter as the text describes it, Appendix C); the experts still see x.  The product
    is rounded to the activation dtype (the router's input is a tensor of that type) and kept in the workspace for
    the backward pass, where dW_r uses it and the router's part of dx is multiplied by u.
-   SWITCH_MOE_FLAG_GEGLU: the experts are GEGLU FFNs (Table 9: "the expansion matrix is substituted with two sets of
-   weights which are non-linearly combined"): W_in is [E, d_model, 2 d_ff] = [W_0 | W_1] per expert (and dW_in
-   likewise), hidden = GELU(x W_0) . (x W_1) with the exact GELU z Phi(z), y = hidden W_out.  The two products are
+   SWITCH_MOE_FLAG_GEGLU: the experts are GEGLU FFNs (Table 9: two expansion matrices whose outputs are combined
+   non-linearly): W_in is [E, d_model, 2 d_ff] = [W_0 | W_1] per expert (and dW_in likewise), hidden = GELU(x W_0) . (x W_1) with the exact GELU z Phi(z), y = hidden W_out.  The two products are
    one grouped GEMM with 2 d_ff output columns; the gating and its derivative are element-wise kernels over the
    kept rows.  Not available on SWITCH_MOE_GEMM_TC_1CTA.
    SWITCH_MOE_FLAG_TOP2: top-2 routing, the Mixture-of-Experts layer the paper compares with (Eq. 1-2 with the two
@@ -71,7 +70,7 @@ enum switch_moe_gemm_path {
    DGATE then have 2T entries and TOKEN_OF_SLOT holds v.  Needs T to be a multiple of 256; not together with
    RESIDUAL, REROUTE or several routing groups.
    SWITCH_MOE_FLAG_EXPERT_DROPOUT: expert dropout (the fine-tuning regularisation of Section 2.4: a larger dropout
-   rate "at the interim feed-forward computation at each expert layer"): the experts' hidden activations are
+   rate on the hidden activations inside every expert): the experts' hidden activations are
    multiplied by keep / (1 - expert_dropout), and so is their gradient on the way back.  The keep mask is an input
    (expert_keep), one bit per hidden unit of every slot row; the caller draws it. */
 enum switch_moe_flags {
@@ -132,7 +131,8 @@ typedef struct switch_moe_config {
 
 /* Regions of the workspace that switch_moe_workspace_view can expose (all written by the library). */
 enum switch_moe_ws_region {
-  SWITCH_MOE_WS_STATUS = 0,         /* int32[16]; [0] != 0 after a device-side timeout */
+  SWITCH_MOE_WS_STATUS = 0,         /* int32[16]; [0] != 0 after a device-side timeout ([0] = code of the wait that gave
+                                       up, [1] = its block, [2] = the barrier phase) */
   SWITCH_MOE_WS_EXPERT_INDEX = 1,   /* int32[T]   e_t */
   SWITCH_MOE_WS_GATE = 2,           /* float[T]   g_t (the un-masked top-1 probability, also for dropped tokens) */
   SWITCH_MOE_WS_SLOT = 3,           /* int32[T]   row of the token in the slot buffers: e_t * (G C) + (kept tokens of
@@ -202,7 +202,11 @@ int switch_moe_dispatch_plan(const switch_moe_config* cfg, const int32_t* expert
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /* Staged: the router's backward alone for a caller-supplied gate gradient (device float[T]; entries of dropped
- * tokens are ignored): G = d_aux.alpha.E.f_i/T + [i = e_t, kept].dgate_t, dh = p (G - <p,G>), dW_r = x^T dh,
+ * tokens are ignored).  The paper states no backward pass; this is the derivative of its forward definitions: the
+ * gate value p_i(x) of Eq. 2 carries the gradient into the router (Section 2.1: the gate keeps the router
+ * differentiable), the softmax of Eq. 1 is differentiated as usual, and the auxiliary loss of Eq. 4 contributes
+ * through P_i only, because f_i (Eq. 5) is not differentiable (Section 2.2):
+ * G = d_aux.alpha.E.f_i/T + [i = e_t, kept].dgate_t, dh = p (G - <p,G>), dW_r = x^T dh,
  * dx_router = dh W_r^T.  Uses PROBS, EXPERT_INDEX, SLOT, COUNT of the workspace.  dx_router [T,d_model] is written
  * in the config's dtype (not accumulated). */
 int switch_moe_router_bwd(const switch_moe_config* cfg, const void* x, const float* W_r, const float* dgate,
@@ -216,10 +220,13 @@ int switch_moe_router_bwd(const switch_moe_config* cfg, const void* x, const flo
  * scratch the plan needs -- per-block expert histograms and their scan -- is a 512 KiB array compiled into the
  * library, resident on every GPU that loads it until the process exits; the call itself allocates and frees
  * nothing (no cudaMalloc / cudaFree, no allocating library routine).
- *   expert_index device int32[T] (in).  Outputs, all caller-owned device buffers: count int32[E], kept int32[E],
- *   slot int32[T] (e*C + position, or -1 if dropped), token_of_slot int32[E*C] (-1 for empty slots) -- the same
- *   values switch_moe_dispatch_plan leaves in its workspace regions of those names.
- * Limits: T <= SWITCH_MOE_STATIC_PLAN_MAX_TOKENS (else SWITCH_MOE_UNSUPPORTED_SHAPE), E <= 256.
+ *   expert_index device int32[T] (in; an entry that is negative or >= E means "no expert" and takes no slot).
+ *   Outputs, all caller-owned device buffers: count int32[E], kept int32[E], slot int32[T] (e*C + position, or -1
+ *   if dropped), token_of_slot int32[E*C] (-1 for empty slots) -- the same values switch_moe_dispatch_plan leaves
+ *   in its workspace regions of those names.
+ * Limits: T <= SWITCH_MOE_STATIC_PLAN_MAX_TOKENS, E <= 256, one routing group, and the top-1 plan of Section 2.2
+ * only: a config with SWITCH_MOE_FLAG_TOP2 or SWITCH_MOE_FLAG_REROUTE is refused like an oversized one
+ * (SWITCH_MOE_UNSUPPORTED_SHAPE), since those plans place more assignments than the array is sized for.
  * The first call on each device looks up the array's device address (with that device current); make that first
  * call before starting any stream capture.  All calls on a device share the one array: nothing in it needs
  * clearing between calls (every word read is written earlier in the same call), but two calls whose kernels
@@ -263,6 +270,11 @@ int switch_moe_check_device_status(const switch_moe_config* cfg, void* workspace
 
 /* HOST call.  Number of this library's kernels that one switch_moe_fwd plus one switch_moe_bwd launch. */
 int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches_out);
+
+/* HOST call.  The same count per stage: launches_out (HOST int32[SWITCH_MOE_STAGE_EVENTS - 1]) entry i is the number
+ * of kernels launched between stage event i and stage event i + 1 (see switch_moe_config::stage_events; entry 5, the
+ * gap between the forward and the backward pass, is 0). */
+int switch_moe_stage_launches(const switch_moe_config* cfg, int32_t* launches_out);
 
 /* HOST call.  Static description of a status code. */
 const char* switch_moe_status_string(int status);

@@ -175,16 +175,16 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     expert where it has room, and their gate is that expert's probability (Eq. 2 with the expert that processes the
     token); f in the auxiliary loss still counts the argmax (Eq. 5).  `alt_index`, when given, replaces the second
     choice (to follow a legitimate near-tie flip of the device).
-    `router_jitter` [T, d], when given, multiplies the router's input element by element (the text's "multiplicative
-    jitter noise on the incoming representation", Appendix C): the router sees x . u, the experts see x.  It is an
+    `router_jitter` [T, d], when given, multiplies the router's input element by element (input jitter as the text
+    describes it, Appendix C): the router sees x . u, the experts see x.  It is an
     input (the caller draws it).  `storage_round`, when given, is applied to x . u: the router's input is a tensor
     of the layer's activation type, so the product is rounded to that type before the router's float32 arithmetic.
-    `geglu` replaces the expert's ReLU FFN by the GEGLU FFN of the paper's Table 9 ("the expansion matrix is
-    substituted with two sets of weights which are non-linearly combined"): W_in[i] is [d, 2 f] = [W_0 | W_1],
+    `geglu` replaces the expert's ReLU FFN by the GEGLU FFN of the paper's Table 9 (two expansion matrices whose
+    outputs are combined non-linearly): W_in[i] is [d, 2 f] = [W_0 | W_1],
     a = x W_0, b = x W_1, hidden = GELU(a) . b, output = hidden W_out.  "u" then holds the rows [a | b].
     `expert_keep` [E * C, f] (booleans, indexed by slot row) with `expert_dropout` = rate applies expert dropout
-    (Section 2.4 / fine-tuning regularisation table: a larger dropout rate "at the interim feed-forward computation at
-    each expert layer"): the hidden activations are multiplied by keep / (1 - rate), the usual inverted dropout; the
+    (Section 2.4 / fine-tuning regularisation table: a larger dropout rate on the hidden activations inside every
+    expert): the hidden activations are multiplied by keep / (1 - rate), the usual inverted dropout; the
     mask is an input (the caller draws it).
     Returns a dict with every intermediate the staged comparisons need.
     """

@@ -312,17 +312,36 @@ int switch_moe_check_device_status(const switch_moe_config* cfg, void* workspace
   return host[0] != 0 ? SWITCH_MOE_DEVICE_TIMEOUT : SWITCH_MOE_OK;
 }
 
-int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches_out) {
+int switch_moe_stage_launches(const switch_moe_config* cfg, int32_t* launches_out) {
   if (launches_out == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
   Shape s;
   SWMOE_TRY(resolve_shape(cfg, &s));
-  // fwd: router, 3 plan kernels, gather, 2 GEMMs; bwd: gather, 4 GEMMs, 4 router-backward kernels.
-  // Tensor-core router: forward = operand split, router, column sums; backward = logit gradients, two products, reduce.
-  // Rerouting of overflowed tokens adds four plan kernels to the forward pass.
-  // Input jitter adds the element-wise product kernel.
-  // GEGLU experts add the gating kernel to each pass.  Top-2 routing adds the second-choice kernel and two row sums.
-  // The paired-CTA path runs the two products of dH (dgrad1, wgrad1) as one launch.
-  *launches_out = (s.router_tc ? (9 + 9) : (7 + 9)) - (s.gemm_path == 0 ? 1 : 0) + (s.reroute ? 4 : 0) + (s.jitter ? 1 : 0) + (s.geglu ? 2 : 0) + (s.top2 ? 3 : 0) + (s.dropout ? 2 : 0);
+  int32_t* n = launches_out;
+  for (int i = 0; i < SWITCH_MOE_STAGE_EVENTS - 1; ++i) n[i] = 0;
+  // forward.  Router: the kernel itself; on the tensor cores also the bf16 split of W_r and the column sums of the
+  // probabilities; input jitter adds the element-wise product, top-2 routing the second-choice kernel.
+  n[0] = (s.router_tc ? 3 : 1) + (s.jitter ? 1 : 0) + (s.top2 ? 1 : 0);
+  n[1] = 3 + (s.reroute ? 4 : 0);                     // histogram, scan, assign; stage 2 of rerouting adds four
+  n[2] = 1;                                           // gather
+  n[3] = 1 + (s.geglu ? 1 : 0) + (s.dropout ? 1 : 0); // GEMM1 (+ GEGLU gating, + expert dropout)
+  n[4] = 1 + (s.top2 ? 1 : 0);                        // GEMM2 + combine (+ sum of the two assignments' rows)
+  // backward.  With the paired-CTA path the two products of dH are one launch (stage 9).
+  n[6] = 1;
+  n[7] = 1 + (s.dropout ? 1 : 0) + (s.geglu ? 1 : 0);
+  n[8] = 1;
+  n[9] = 1;
+  n[10] = (s.gemm_path == 0 ? 0 : 1) + (s.top2 ? 1 : 0);
+  n[11] = 4;                                          // logit gradients, x^T dh partials, their reduction, dx += dh W_r^T
+  return SWITCH_MOE_OK;
+}
+
+int switch_moe_launches_per_step(const switch_moe_config* cfg, int32_t* launches_out) {
+  if (launches_out == nullptr) return SWITCH_MOE_INVALID_ARGUMENT;
+  int32_t n[SWITCH_MOE_STAGE_EVENTS];
+  SWMOE_TRY(switch_moe_stage_launches(cfg, n));
+  int total = 0;
+  for (int i = 0; i < SWITCH_MOE_STAGE_EVENTS - 1; ++i) total += n[i];
+  *launches_out = total;
   return SWITCH_MOE_OK;
 }
 

@@ -21,14 +21,14 @@ plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int* __rest
   __syncthreads();
   const int t = blockIdx.x * kPlanBlockTokens + threadIdx.x;
   const int e = t < T ? expert_index[t] : -1;
-  if (e >= 0) atomicAdd(&h[e], 1);                           // integer counts: order-independent; negative = no vote
+  if ((unsigned)e < (unsigned)E) atomicAdd(&h[e], 1);        // integer counts: order-independent; negative or >= E: no vote
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) hist[(size_t)blockIdx.x * E + e] = h[e];
 }
 
 // Tile lists, shared by both scan kernels: 128-row token tiles (single-CTA GEMM) and, for the paired-CTA GEMM, each
-// expert's kept rows cut into the fewest pieces of at most 256 rows, equal up to rounding each piece to a multiple of
-// 16 (the MMA's N granularity).  Thread 0 adds the loss terms and scans the per-expert tile counts; the first E
+// expert's kept rows cut into the fewest pieces of at most kPairTileTokens rows, equal up to rounding each piece to a
+// multiple of 16 (the MMA's N granularity).  Thread 0 adds the loss terms and scans the per-expert tile counts; the first E
 // threads write their expert's entries.  `term` and `kept_s` are shared-memory arrays filled before the call.
 __device__ __forceinline__ void write_tile_lists(const float* term, const int* kept_s, int E, float loss_scale,
                                                  float* __restrict__ aux_loss, int* __restrict__ tile_expert,
@@ -43,7 +43,7 @@ __device__ __forceinline__ void write_tile_lists(const float* term, const int* k
     for (int i = 0; i < E; ++i) {
       start128[i] = n; startn[i] = m;
       n += (kept_s[i] + kTileM - 1) / kTileM;
-      m += (kept_s[i] + 255) / 256;
+      m += (kept_s[i] + kPairTileTokens - 1) / kPairTileTokens;
     }
     tile_expert[0] = n;
     tile_row0[0] = n;
@@ -56,7 +56,7 @@ __device__ __forceinline__ void write_tile_lists(const float* term, const int* k
     int n = start128[e];
     for (int r = 0; r < k; r += kTileM, ++n) { tile_expert[1 + n] = e; tile_row0[1 + n] = r; }
     if (k > 0) {
-      const int pieces = (k + 255) / 256;
+      const int pieces = (k + kPairTileTokens - 1) / kPairTileTokens;
       const int rows = ((k + pieces - 1) / pieces + 15) / 16 * 16;
       int m = startn[e];
       for (int r = 0; r < k; r += rows, ++m) ntile[1 + m] = make_int4(e, r, min(rows, (k - r + 15) / 16 * 16), 0);
@@ -207,7 +207,8 @@ plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__
   for (int i = tid; i < kWarps * kMaxExperts; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
   __syncthreads();
   const int t = blockIdx.x * kPlanBlockTokens + tid;
-  const int e = t < T ? expert_index[t] : -1;                 // negative: no expert (takes no slot)
+  int e = t < T ? expert_index[t] : -1;                       // negative: no expert (takes no slot)
+  if (e >= E) e = -1;                                         // an index no expert has is treated the same way
   const unsigned same = __match_any_sync(0xffffffffu, e >= 0 ? e : -1 - lane);   // distinct dummies for those lanes
   const int rank = __popc(same & ((1u << lane) - 1u));
   if (e >= 0 && rank == 0) warp_cnt[warp][e] = __popc(same);
@@ -304,7 +305,8 @@ reroute_assign_kernel(const int* __restrict__ alt, const int* __restrict__ exper
   for (int i = tid; i < kWarps * kMaxExperts; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
   __syncthreads();
   const int t = blockIdx.x * kPlanBlockTokens + tid;
-  const int a = t < T ? alt[t] : -1;
+  int a = t < T ? alt[t] : -1;
+  if (a >= E) a = -1;
   const int key = a >= 0 ? a : -1 - lane;                     // distinct dummies for tokens that do not move
   const unsigned same = __match_any_sync(0xffffffffu, key);
   const int rank = __popc(same & ((1u << lane) - 1u));

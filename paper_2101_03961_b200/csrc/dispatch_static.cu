@@ -34,7 +34,8 @@ static_plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int*
   for (int e = threadIdx.x; e < E; e += blockDim.x) h[e] = 0;
   __syncthreads();
   const int t = blockIdx.x * kPlanBlockTokens + threadIdx.x;
-  if (t < T) atomicAdd(&h[expert_index[t]], 1);
+  const int e = t < T ? expert_index[t] : -1;
+  if ((unsigned)e < (unsigned)E) atomicAdd(&h[e], 1);        // negative or out-of-range index: no vote
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) hist[(size_t)blockIdx.x * E + e] = h[e];
 }
@@ -63,12 +64,14 @@ static_plan_assign_kernel(const int* __restrict__ expert_index, const int* __res
   for (int i = tid; i < kWarps * kMaxExperts; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
   __syncthreads();
   const int t = blockIdx.x * kPlanBlockTokens + tid;
-  const int e = t < T ? expert_index[t] : -1 - lane;
-  const unsigned same = __match_any_sync(0xffffffffu, e);
+  int e = t < T ? expert_index[t] : -1;
+  if ((unsigned)e >= (unsigned)E) e = -1;                     // "no expert" (-1, as the library's own marker) takes no slot
+  const unsigned same = __match_any_sync(0xffffffffu, e >= 0 ? e : -1 - lane);   // distinct dummies for those lanes
   const int rank = __popc(same & ((1u << lane) - 1u));
-  if (t < T && rank == 0) warp_cnt[warp][e] = __popc(same);
+  if (e >= 0 && rank == 0) warp_cnt[warp][e] = __popc(same);
   __syncthreads();
-  if (t < T) {
+  if (t < T && e < 0) slot[t] = -1;
+  if (e >= 0) {
     int pos = hist_base[(size_t)blockIdx.x * E + e] + rank;
     for (int w = 0; w < warp; ++w) pos += warp_cnt[w][e];
     const int s = pos < C ? e * C + pos : -1;
@@ -109,16 +112,22 @@ extern "C" int switch_moe_dispatch_plan_static(const switch_moe_config* cfg, con
   int rc = resolve_shape(cfg, &s);
   if (rc != SWITCH_MOE_OK) return rc;
   if (!expert_index || !count || !kept || !slot || !token_of_slot) return SWITCH_MOE_INVALID_ARGUMENT;
-  if (s.T > kStaticMaxTokens || s.G != 1) return SWITCH_MOE_UNSUPPORTED_SHAPE;      // the static scratch holds 256 x 256 counters twice
+  // This entry point is the top-1 plan of one routing group only: the variants that place more than T assignments
+  // or run a second stage need the workspace-based call.
+  if (s.G != 1 || (cfg->flags & (SWITCH_MOE_FLAG_TOP2 | SWITCH_MOE_FLAG_REROUTE)) != 0)
+    return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  const int blocks = (s.T + kPlanBlockTokens - 1) / kPlanBlockTokens;
+  if (s.T > kStaticMaxTokens || blocks > kStaticMaxBlocks)   // the static scratch holds 256 x 256 counters twice
+    return SWITCH_MOE_UNSUPPORTED_SHAPE;
   int32_t* scratch = nullptr;
   rc = scratch_for_current_device(&scratch);
   if (rc != SWITCH_MOE_OK) return rc;
   int32_t* hist = scratch;
   int32_t* hist_base = scratch + (size_t)kStaticMaxBlocks * kMaxExperts;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  static_plan_hist_kernel<<<s.plan_blocks, kPlanBlockTokens, 0, st>>>(expert_index, s.T, s.E, hist);
-  static_plan_scan_kernel<<<1, kMaxExperts, 0, st>>>(hist, s.plan_blocks, s.E, s.C, hist_base, count, kept);
-  static_plan_assign_kernel<<<s.plan_blocks, kPlanBlockTokens, 0, st>>>(expert_index, hist_base, kept, s.T, s.E, s.C,
+  static_plan_hist_kernel<<<blocks, kPlanBlockTokens, 0, st>>>(expert_index, s.T, s.E, hist);
+  static_plan_scan_kernel<<<1, kMaxExperts, 0, st>>>(hist, blocks, s.E, s.C, hist_base, count, kept);
+  static_plan_assign_kernel<<<blocks, kPlanBlockTokens, 0, st>>>(expert_index, hist_base, kept, s.T, s.E, s.C,
                                                                         slot, token_of_slot);
   return launch_status();
 }

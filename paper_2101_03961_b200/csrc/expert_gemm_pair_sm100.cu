@@ -11,11 +11,19 @@
 // transposes 32x32 blocks through shared memory to write token-major rows.  The weight gradients keep the natural
 // orientation (dW_out = H^T dY_d, dW_in = X_d^T dH: M = weight rows, N = weight columns, contraction over tokens).
 //
-// A CTA pair shares the B operand: each CTA stages its own 128 A rows and half of B (32 KB per 64-deep k-block, six
-// stages), the leader CTA's single MMA thread issues M=256 instructions that read both CTAs' shared memory, and
-// tcgen05.commit with a cluster mask releases stages and publishes accumulators in both CTAs.  TMA loads carry no
-// multicast.  Each CTA drains its own 128 TMEM lanes with 8 epilogue warps while the next tile's MMAs run into the
-// second accumulator.
+// A CTA pair shares the B operand: each CTA stages its own 128 A rows and half of B per 64-deep k-block, the leader
+// CTA's single MMA thread issues M=256 instructions that read both CTAs' shared memory, and tcgen05.commit with a
+// cluster mask releases stages and publishes accumulators in both CTAs.  TMA loads carry no multicast.  Each CTA
+// drains its own 128 TMEM lanes with 8 epilogue warps while the next tile's MMAs run.
+//
+// One pass per expert.  A token tile holds up to 320 tokens (the capacity of the paper's layers at capacity factor
+// 1.25), so an expert's weights cross shared memory once; a tile wider than the MMA's N limit of 256 is two column
+// segments, i.e. two MMAs per k-step that read the same A block.  The token operand's TMA box is exactly the rows
+// the tile has (one tensor map per box height), so no byte enters shared memory that no MMA reads.
+// Two accumulators of up to 320 columns do not fit 512 TMEM columns side by side, so they overlap in the middle:
+// even tiles of a CTA pair use columns [0, n), odd tiles [512 - n, 512).  The epilogue drains a tile starting from
+// the middle columns and tells the MMA thread (barrier `tmid`) once the columns the next tile also uses have been
+// read; the next tile's MMAs then start while the rest of the tile is still being drained.
 //
 // Every mbarrier wait is bounded in time (status word + abort flag); both CTAs always reach the final cluster
 // barrier, so tensor memory is freed and no CTA exits while its peer can still address its shared memory.
@@ -25,15 +33,17 @@ namespace swmoe {
 using namespace tc;
 namespace {
 
-constexpr int kPStages = 6;
+constexpr int kPStages = 6;                            // weight gradients: six stages of A (16 KB) + half of B (16 KB)
+constexpr int kPMaxStages = 8;                         // token products: as many stages as fit, at most this
 constexpr int kPHalfBytes = 16384;                     // A tile (128 x 64) and B half tile (<= 128 x 64)
 constexpr int kPStageBytes = 2 * kPHalfBytes;
+constexpr int kPRingBytes = kPStages * kPStageBytes;   // 192 KB of operand stages
 constexpr int kPTransBytes = 8 * 2048;                 // 8 epilogue warps x (32 x 64 B)
 constexpr int kPAuxBytes = 8 * 128;                    // 8 epilogue warps x 32 gates
 constexpr int kPKeptCache = kMaxExperts;                 // kept[e] for every expert
 constexpr int kPTileCache = 448;                        // first token tiles of the list ({expert, row, rows})
 constexpr int kPCacheBytes = kPKeptCache * 4 + kPTileCache * 16;
-constexpr int kPSmemBytes = 1024 + kPStages * kPStageBytes + kPTransBytes + kPAuxBytes + 256 + kPCacheBytes;
+constexpr int kPSmemBytes = 1024 + kPRingBytes + kPTransBytes + kPAuxBytes + 256 + kPCacheBytes;
 constexpr int kPThreads = 320;
 constexpr uint32_t kPeerMask = 0xFEFFFFFFu;            // clears the CTA-rank bit of a shared::cluster address
 
@@ -59,10 +69,18 @@ struct PairParams {
   const __nv_bfloat16* res;   // combine / scatter with the skip path inside the layer: rows added to the output (x or dy)
   __nv_bfloat16* out2;        // combine with the skip path: second copy of the output without it
   int plain;                  // GEMM1 / dgrad2 without ReLU and without the ReLU mask (GEGLU experts gate elsewhere)
+  int stages, stage_bytes;    // operand ring: token products size a stage for the widest tile the capacity allows
+};
+
+// Token products: the token operand's TMA box is exactly this CTA's share of the tile (n / 2 rows, a multiple of 8):
+// one tensor map per height 8, 16, .., 128.  Weight gradients use entry 0 (a 64-row box of the token contraction).
+constexpr int kBMaps = 16;
+struct BMapSet {
+  CUtensorMap m[kBMaps];
 };
 
 struct PTile {
-  int e, m0, n0, row0, n, k_blocks, last_mmas;
+  int e, m0, n0, row0, n, n1, k_blocks, last_mmas;   // n1: columns of the first segment (n if n <= 256)
 };
 
 // Tile decode reads the plan through shared-memory copies made at kernel start: a dependent global load per tile
@@ -73,6 +91,7 @@ __device__ __forceinline__ PTile p_decode(const PairParams& p, int id, const int
     const int nt = id / p.n_mpairs;
     const int4 q = nt < kPTileCache ? tile_s[nt] : p.ntile[1 + nt];
     t.e = q.x; t.row0 = q.y; t.n = q.z; t.n0 = 0;
+    t.n1 = t.n <= 256 ? t.n : ((t.n >> 1) + 15) & ~15;         // two segments: both multiples of 16, both <= 256
     t.m0 = (id - nt * p.n_mpairs) * 256;
     t.k_blocks = p.k_blocks_fixed;
     t.last_mmas = kBK / kUmmaK;
@@ -83,7 +102,7 @@ __device__ __forceinline__ PTile p_decode(const PairParams& p, int id, const int
     const int mp = rem / p.n_ntiles_fixed;
     t.m0 = mp * 256;
     t.n0 = (rem - mp * p.n_ntiles_fixed) * 256;
-    t.row0 = 0; t.n = 256;
+    t.row0 = 0; t.n = 256; t.n1 = 256;
     const int k = kept_s[t.e];
     t.k_blocks = (k + kBK - 1) / kBK;
     const int rem_rows = k - (t.k_blocks - 1) * kBK;          // rows of the last k-block that hold tokens
@@ -139,7 +158,7 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
 // `pair` of `n_pairs` is this CTA pair's place among the pairs that work on this product: the whole grid for a
 // launch of one product, a share of it when two products run side by side in one launch (below).
 template <int OP>
-__device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairParams& p,
+__device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet& bm, const PairParams& p,
                                           const int pair, const int n_pairs) {
   constexpr bool kTok = OP <= kDgrad1Scatter;                 // tokens on N, transposed epilogue
   constexpr bool kAMn = (OP == kGemm1Relu || OP == kGemm2Combine || OP == kWgrad2 || OP == kWgrad1);
@@ -148,24 +167,28 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  uint8_t* trans_gen = smem_gen + kPStages * kPStageBytes;
+  uint8_t* trans_gen = smem_gen + kPRingBytes;
   uint8_t* aux_gen = trans_gen + kPTransBytes;
   uint8_t* bar_gen = aux_gen + kPAuxBytes;
-  const uint32_t bar_base = smem_base + kPStages * kPStageBytes + kPTransBytes + kPAuxBytes;
-  // barrier block: full[S] | empty[S] | tmem_full[2] | tmem_empty[2] | tmem_ptr | abort
-  const uint32_t full0 = bar_base, empty0 = bar_base + 8u * kPStages;
-  const uint32_t tfull0 = bar_base + 16u * kPStages, tempty0 = tfull0 + 16u;
-  volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kPStages + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kPStages + 4) + 4);
+  const uint32_t bar_base = smem_base + kPRingBytes + kPTransBytes + kPAuxBytes;
+  // barrier block: full[S] | empty[S] | tmem_full[2] | tmem_empty[2] | tmem_mid[2] | tmem_ptr | abort   (S = kPMaxStages)
+  const uint32_t full0 = bar_base, empty0 = bar_base + 8u * kPMaxStages;
+  const uint32_t tfull0 = bar_base + 16u * kPMaxStages, tempty0 = tfull0 + 16u, tmid0 = tfull0 + 32u;
+  volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kPMaxStages + 6));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kPMaxStages + 6) + 4);
   int* kept_s = reinterpret_cast<int*>(bar_gen + 256);
   int4* tile_s = reinterpret_cast<int4*>(bar_gen + 256 + kPKeptCache * 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();                   // 0 = leader (issues the MMAs)
+  const uint32_t n_stages = kTok ? (uint32_t)p.stages : (uint32_t)kPStages;
+  const uint32_t stage_bytes = kTok ? (uint32_t)p.stage_bytes : (uint32_t)kPStageBytes;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kPStages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 16); }
+    for (int s = 0; s < kPMaxStages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 16); mbar_init(tmid0 + 8u * a, 16);
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -185,6 +208,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
   const uint32_t tmem_base = *tmem_ptr_s;
   const int n_tiles = kTok ? n_ntiles_listed * p.n_mpairs : p.E * p.n_mpairs * p.n_ntiles_fixed;
 
+  // Accumulator columns of this pair's `it`-th tile: even tiles [0, n), odd tiles [512 - n, 512).  Consecutive tiles
+  // share the middle columns when n + n_next > 512.
   if (warp == 0) {
     // ------------------------------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
@@ -194,31 +219,40 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
         const PTile t = p_decode(p, id, kept_s, tile_s);
         // coordinates of this CTA's boxes; only the contraction coordinate moves inside the tile
         const int a_m = t.m0 + 128 * (int)rank;
-        const int b_r = kTok ? t.row0 + (int)rank * (t.n >> 1) : t.n0 + 128 * (int)rank;
         const int e = t.e, kbs = t.k_blocks;
+        // token products: this CTA's half of each column segment's token rows, in boxes of exactly that height;
+        // weight gradients: this CTA's 128 of the 256 output columns
+        const int h1 = t.n1 >> 1, h2 = (t.n - t.n1) >> 1;
+        const int b_r = kTok ? t.row0 + (int)rank * h1 : t.n0 + 128 * (int)rank;
+        const int b_r2 = t.row0 + t.n1 + (int)rank * h2;
+        const CUtensorMap* tmB = kTok ? &bm.m[(h1 >> 3) - 1] : &bm.m[0];
+        const CUtensorMap* tmB2 = (kTok && h2 > 0) ? &bm.m[(h2 >> 3) - 1] : tmB;
+        // both CTAs' bytes land on the leader's barrier
+        const uint32_t tx_bytes = kTok ? 2u * (uint32_t)(kPHalfBytes + (t.n >> 1) * 128) : 2u * (uint32_t)kPStageBytes;
 #pragma unroll 1
         for (int kb = 0; kb < kbs; ++kb) {
           const uint32_t eb = empty0 + 8u * stage;
           ok = mbar_wait(eb, phase ^ 1u, abort_flag, p.status, 21);
           if (!ok) break;
-          const uint32_t a_dst = smem_base + stage * kPStageBytes, b_dst = a_dst + kPHalfBytes;
+          const uint32_t a_dst = smem_base + stage * stage_bytes, b_dst = a_dst + kPHalfBytes;
           const uint32_t fb = full0 + 8u * stage;
           const uint32_t lead_full = fb & kPeerMask;
           const int k0 = kb * kBK;
-          if (rank == 0) mbar_arrive_expect_tx(fb, 2 * kPStageBytes);     // both CTAs' bytes land on the leader
+          if (rank == 0) mbar_arrive_expect_tx(fb, tx_bytes);
           if (kAMn) {
             tma_load_3d_pair(a_dst, &tmA, lead_full, a_m, k0, e);
             tma_load_3d_pair(a_dst + kAtomBytes, &tmA, lead_full, a_m + 64, k0, e);
           } else {
             tma_load_3d_pair(a_dst, &tmA, lead_full, k0, a_m, e);
           }
-          if (kBMn) {                                         // this CTA's 128 of the 256 output columns
-            tma_load_3d_pair(b_dst, &tmB, lead_full, b_r, k0, e);
-            tma_load_3d_pair(b_dst + kAtomBytes, &tmB, lead_full, b_r + 64, k0, e);
-          } else {                                            // this CTA's half of the expert's token rows
-            tma_load_3d_pair(b_dst, &tmB, lead_full, k0, b_r, e);
+          if (kBMn) {
+            tma_load_3d_pair(b_dst, tmB, lead_full, b_r, k0, e);
+            tma_load_3d_pair(b_dst + kAtomBytes, tmB, lead_full, b_r + 64, k0, e);
+          } else {
+            tma_load_3d_pair(b_dst, tmB, lead_full, k0, b_r, e);
+            if (h2 > 0) tma_load_3d_pair(b_dst + (uint32_t)h1 * 128u, tmB2, lead_full, k0, b_r2, e);
           }
-          if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
         }
       }
       if (*abort_flag != 0) {
@@ -236,40 +270,57 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
       constexpr uint32_t b_kstep = (kBMn ? kUmmaK * 128u : kUmmaK * 2u) >> 4;
       const uint64_t a_desc0 = make_smem_desc(smem_base, kAMn ? kAtomBytes : 16u, 1024u);
       const uint64_t b_desc0 = make_smem_desc(smem_base + kPHalfBytes, kBMn ? kAtomBytes : 16u, 1024u);
-      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+      uint32_t stage = 0, phase = 0, it = 0;
+      int n_prev = 0;
       bool ok = true;
-      for (int id = pair; id < n_tiles && ok; id += n_pairs) {
+      for (int id = pair; id < n_tiles && ok; id += n_pairs, ++it) {
         const PTile t = p_decode(p, id, kept_s, tile_s);
-        const uint32_t idesc = idesc_base | ((uint32_t)(t.n >> 3) << 17);
+        const uint32_t side = it & 1u, use = it >> 1;          // this side's `use`-th tile
+        const uint32_t idesc1 = idesc_base | ((uint32_t)(t.n1 >> 3) << 17);
+        const int n2 = t.n - t.n1;
+        const uint32_t idesc2 = idesc_base | ((uint32_t)(n2 >> 3) << 17);
+        const uint32_t b2_off = ((uint32_t)(t.n1 >> 1) * 128u) >> 4;    // second segment's rows in this CTA's half of B
         const int kbs = t.k_blocks, last_mmas = t.last_mmas;
-        ok = mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag, p.status, 22);
+        // the side's previous tile has been read out completely ...
+        ok = mbar_wait(tempty0 + 8u * side, (use & 1u) ^ 1u, abort_flag, p.status, 22);
         if (!ok) break;
+        // ... and so have the middle columns of the other side's tile, if this tile reaches into them
+        if (kTok && it > 0 && n_prev + t.n > kTmemCols) {
+          ok = mbar_wait(tmid0 + 8u * (side ^ 1u), ((it - 1u) >> 1) & 1u, abort_flag, p.status, 25);
+          if (!ok) break;
+        }
+        n_prev = t.n;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * 256u;
+        const uint32_t d_tmem = tmem_base + (side ? (uint32_t)(kTmemCols - t.n) : 0u);
+        const uint32_t d_tmem2 = d_tmem + (uint32_t)t.n1;
 #pragma unroll 1
         for (int kb = 0; kb < kbs; ++kb) {
           ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 23);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t ad = a_desc0 + (uint64_t)(stage * (kPStageBytes >> 4));
-          const uint64_t bd = b_desc0 + (uint64_t)(stage * (kPStageBytes >> 4));
+          const uint64_t ad = a_desc0 + (uint64_t)(stage * (stage_bytes >> 4));
+          const uint64_t bd = b_desc0 + (uint64_t)(stage * (stage_bytes >> 4));
           const int n_mma = (!kTok && kb == kbs - 1) ? last_mmas : kBK / kUmmaK;
-          tc_mma_bf16_pair(d_tmem, ad, bd, idesc, kb > 0 ? 1u : 0u);
-          if (n_mma > 1) tc_mma_bf16_pair(d_tmem, ad + a_kstep, bd + b_kstep, idesc, 1u);
-          if (n_mma > 2) tc_mma_bf16_pair(d_tmem, ad + 2 * a_kstep, bd + 2 * b_kstep, idesc, 1u);
-          if (n_mma > 3) tc_mma_bf16_pair(d_tmem, ad + 3 * a_kstep, bd + 3 * b_kstep, idesc, 1u);
+          const uint32_t acc0 = kb > 0 ? 1u : 0u;
+          tc_mma_bf16_pair(d_tmem, ad, bd, idesc1, acc0);
+          if (kTok && n2 > 0) tc_mma_bf16_pair(d_tmem2, ad, bd + b2_off, idesc2, acc0);
+#pragma unroll
+          for (int ks = 1; ks < kBK / kUmmaK; ++ks) {
+            if (ks < n_mma) {
+              tc_mma_bf16_pair(d_tmem, ad + ks * a_kstep, bd + ks * b_kstep, idesc1, 1u);
+              if (kTok && n2 > 0) tc_mma_bf16_pair(d_tmem2, ad + ks * a_kstep, bd + b2_off + ks * b_kstep, idesc2, 1u);
+            }
+          }
           tc_commit_pair(empty0 + 8u * stage);                // frees this stage in both CTAs
-          if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+          if (++stage == n_stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         if (kbs > 0) {
-          tc_commit_pair(tfull0 + 8u * acc);                  // accumulator complete, in both CTAs
+          tc_commit_pair(tfull0 + 8u * side);                 // accumulator complete, in both CTAs
         } else {                                              // nothing to contract: epilogues write zeros
-          mbar_arrive(tfull0 + 8u * acc);
-          mbar_arrive_remote(tfull0 + 8u * acc, 1);
+          mbar_arrive(tfull0 + 8u * side);
+          mbar_arrive_remote(tfull0 + 8u * side, 1);
         }
-        acc ^= 1u;
-        if (acc == 0) acc_phase ^= 1u;
       }
     }
   } else {
@@ -278,27 +329,34 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
     const int half = (warp - 2) >> 2;
     uint8_t* tr = trans_gen + (warp - 2) * 2048;              // this warp's 32 x 64 B transpose tile
     float* gate_s = reinterpret_cast<float*>(aux_gen + (warp - 2) * 128);
-    uint32_t acc = 0, acc_phase = 0;
+    uint32_t it = 0;
     bool ok = true;
-    for (int id = pair; id < n_tiles && ok; id += n_pairs) {
+    for (int id = pair; id < n_tiles && ok; id += n_pairs, ++it) {
       const PTile t = p_decode(p, id, kept_s, tile_s);
+      const uint32_t side = it & 1u, use = it >> 1;
       const int m_warp = t.m0 + 128 * (int)rank + 32 * lg;    // first M row (weight row) this warp holds
       const int n_chunks = kTok ? (t.n + 31) >> 5 : 8;
       const bool have_acc = t.k_blocks > 0;
-      // Token products: lane i describes token column c*32 + i of the chunk being processed: the element offset of
-      // its output row (or -1) and its gate.  The first chunk's description (and ReLU mask) is fetched before the
-      // accumulator is awaited, each later one while the previous chunk is being written.
+      const int c0 = side ? kTmemCols - t.n : 0;              // first accumulator column of the tile
+      // Token products.  Chunks of 32 accumulator columns are numbered so that chunk j of an even tile holds the
+      // tile's tokens [32 j, 32 j + 32) and chunk j of an odd tile its tokens [n - 32 (j + 1), n - 32 j): a chunk is
+      // then always inside the 512 columns, and counting j down from the last chunk starts in the middle columns, the
+      // ones the next tile may also use.  Lane i describes token column (chunk's first token) + i: the element offset
+      // of its output row (or -1) and its gate.  This warp's chunks are j = n_chunks - 1 - half, then every second
+      // one down to 0; their descriptions (and ReLU masks) are fetched before the accumulator is awaited.
       constexpr bool kSlotRows = (OP == kGemm1Relu || OP == kDgrad2Mask);
+      constexpr int kQueue = 5;                                // (320 / 32) chunks over two warps
       int row_limit = 0;
-      long long q_off[4] = {-1, -1, -1, -1};                   // this warp's (up to) four chunks, head = next to process
-      float q_gate[4] = {1.f, 1.f, 1.f, 1.f};
-      uint32_t q_mw[4] = {0u, 0u, 0u, 0u};                      // dgrad2: ReLU mask bits of weight rows m_warp..+31 per token
+      long long q_off[kQueue] = {-1, -1, -1, -1, -1};           // head = next chunk to process
+      float q_gate[kQueue] = {1.f, 1.f, 1.f, 1.f, 1.f};
+      uint32_t q_mw[kQueue] = {0u, 0u, 0u, 0u, 0u};             // dgrad2: ReLU mask bits of weight rows m_warp..+31 per token
       const int mcol = m_warp + (lane & 3) * 8;               // store `it` writes weight rows mcol .. mcol + 7
-      auto describe = [&](int c, long long* off, float* g) {
-        const int col = c * 32 + lane, slot_row = t.row0 + col;
+      auto chunk_tok0 = [&](int j) { return side ? t.n - 32 * (j + 1) : 32 * j; };
+      auto describe = [&](int j, long long* off, float* g) {
+        const int col = chunk_tok0(j) + lane, slot_row = t.row0 + col;
         *off = -1;
         *g = 1.f;
-        if (c < n_chunks && col < t.n && slot_row < row_limit) {
+        if (j >= 0 && col >= 0 && col < t.n && slot_row < row_limit) {
           if (kSlotRows) {
             *off = ((long long)t.e * p.C + slot_row) * p.ld_out;
           } else {
@@ -308,26 +366,29 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
           }
         }
       };
+      int j_mid = 0;                                            // chunks j >= j_mid hold columns the next tile uses too
       if (kTok) {
         const int kept_e = kept_s[t.e];
         row_limit = kSlotRows ? min(p.C, (kept_e + 15) / 16 * 16) : kept_e;
+        const int id_next = id + n_pairs;
+        const int n_next = id_next < n_tiles ? p_decode(p, id_next, kept_s, tile_s).n : 0;
+        j_mid = (t.n - max(0, t.n + n_next - kTmemCols)) >> 5;
         // everything the epilogue needs from global memory is requested here, before the accumulator is awaited
 #pragma unroll
-        for (int k = 0; k < 4; ++k) describe(half + 2 * k, &q_off[k], &q_gate[k]);
+        for (int k = 0; k < kQueue; ++k) describe(n_chunks - 1 - half - 2 * k, &q_off[k], &q_gate[k]);
         if (OP == kDgrad2Mask && !p.plain && m_warp < p.Mw) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
+          for (int k = 0; k < kQueue; ++k)
             if (q_off[k] >= 0)
               q_mw[k] = p.hmask[(long long)(m_warp >> 5) * p.hmask_rows + (long long)t.e * p.C + t.row0 +
-                                (half + 2 * k) * 32 + lane];
+                                chunk_tok0(n_chunks - 1 - half - 2 * k) + lane];
         }
       }
-      ok = mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag, p.status, 24);
+      ok = mbar_wait(tfull0 + 8u * side, use & 1u, abort_flag, p.status, 24);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * 256u;
-      bool released = false;
+      const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)c0;
       if constexpr (!kTok) {
         // Weight gradients (row = weight row): 64 output columns at a time, so that a row is a whole 128-byte line.
         // The warp's 2 KB of shared memory hold 16 rows x 128 bytes: rows 0-15 and 16-31 of the warp take turns, and
@@ -347,7 +408,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
           if (c + 2 >= 4) {                                   // last chunk of this warp: accumulator read out
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
+            if (lane == 0) mbar_arrive_remote(tempty0 + 8u * side, 0);
           }
           uint4 ch[8];
 #pragma unroll
@@ -372,8 +433,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
             }
             __syncwarp();
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-              const int rr = it * 4 + (lane >> 3);
+            for (int st = 0; st < 4; ++st) {
+              const int rr = st * 4 + (lane >> 3);
               const uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 128 + ((chunk ^ (rr & 7)) << 4));
               const int orow = m_warp + hf * 16 + rr;
               if (orow < p.Mw && col < p.Nfix)
@@ -382,30 +443,36 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
             __syncwarp();
           }
         }
-        acc ^= 1u;
-        if (acc == 0) acc_phase ^= 1u;
         continue;
       } else {
+        bool released = false, mid_sent = false;
 #pragma unroll 1
-        for (int c = half; c < n_chunks; c += 2) {
+        for (int j = n_chunks - 1 - half; j >= 0; j -= 2) {
+          const int tok0 = chunk_tok0(j);                       // token column of lane 0 (-16 in an odd tile's last chunk)
           uint32_t v[32];
           if (have_acc) {
-            tc_ld32(t_addr + c * 32, v);
+            tc_ld32(t_addr + (uint32_t)(tok0 + 0), v);
             tc_wait_ld();
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0u;
           }
-          if (c + 2 >= n_chunks) {                              // last chunk of this warp: accumulator read out
+          if (!mid_sent && j - 2 < j_mid) {                     // this warp's share of the middle columns is read out
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
+            if (lane == 0) mbar_arrive_remote(tmid0 + 8u * side, 0);
+            mid_sent = true;
+          }
+          if (j - 2 < 0) {                                      // last chunk of this warp: accumulator read out
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(tempty0 + 8u * side, 0);
             released = true;
           }
           {
             long long offs[4];
 #pragma unroll
-            for (int it = 0; it < 4; ++it) offs[it] = __shfl_sync(0xffffffffu, q_off[0], it * 8 + (lane >> 2));
+            for (int st = 0; st < 4; ++st) offs[st] = __shfl_sync(0xffffffffu, q_off[0], st * 8 + (lane >> 2));
             if (OP == kGemm2Combine) gate_s[lane] = q_gate[0];
             __syncwarp();
             // transpose: this lane holds weight row m_warp + lane for 32 tokens -> tr[token][lane]
@@ -427,8 +494,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
             __syncwarp();
             uint32_t mword[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-              const int rr = it * 8 + (lane >> 2);
+            for (int st = 0; st < 4; ++st) {
+              const int rr = st * 8 + (lane >> 2);
               uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (lane & 3) * 16);
               if (OP == kDgrad2Mask && !p.plain) {              // ReLU'(u) = [u > 0]: bits saved by the forward GEMM
                 const uint32_t bits = __shfl_sync(0xffffffffu, q_mw[0], rr) >> ((lane & 3) * 8);
@@ -446,12 +513,12 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
                 uint32_t word = m8 << ((lane & 3) * 8);
                 word |= __shfl_xor_sync(0xffffffffu, word, 1);
                 word |= __shfl_xor_sync(0xffffffffu, word, 2);
-                mword[it] = word;                               // the word of token row rr, in all four lanes of its group
+                mword[st] = word;                               // the word of token row rr, in all four lanes of its group
               }
-              if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[it] >= 0 && mcol < p.Mw) {
+              if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[st] >= 0 && mcol < p.Mw) {
                 // skip path inside the layer: y = x + g E(x), dx = dy + dH W_in^T (the expert term is already bf16)
-                if (OP == kGemm2Combine) *reinterpret_cast<uint4*>(p.out2 + offs[it] + mcol) = val;
-                const uint4 r = *reinterpret_cast<const uint4*>(p.res + offs[it] + mcol);
+                if (OP == kGemm2Combine) *reinterpret_cast<uint4*>(p.out2 + offs[st] + mcol) = val;
+                const uint4 r = *reinterpret_cast<const uint4*>(p.res + offs[st] + mcol);
                 const __nv_bfloat162* rv = reinterpret_cast<const __nv_bfloat162*>(&r);
                 __nv_bfloat162* vv = reinterpret_cast<__nv_bfloat162*>(&val);
 #pragma unroll
@@ -460,20 +527,20 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
                   vv[q] = __floats2bfloat162_rn(a2.x + b2.x, a2.y + b2.y);
                 }
               }
-              if (offs[it] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[it] + mcol) = val;
+              if (offs[st] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[st] + mcol) = val;
             }
             if (OP == kGemm1Relu && !p.plain) {                 // lane i stores the mask word of token row i: one 128-byte line
               uint32_t mine = 0;
 #pragma unroll
-              for (int it = 0; it < 4; ++it) {
-                const uint32_t w = __shfl_sync(0xffffffffu, mword[it], 4 * (lane & 7));
-                if ((lane >> 3) == it) mine = w;
+              for (int st = 0; st < 4; ++st) {
+                const uint32_t w = __shfl_sync(0xffffffffu, mword[st], 4 * (lane & 7));
+                if ((lane >> 3) == st) mine = w;
               }
               if (q_off[0] >= 0 && m_warp < p.Mw)
-                p.hmask[(long long)(m_warp >> 5) * p.hmask_rows + (long long)t.e * p.C + t.row0 + c * 32 + lane] = mine;
+                p.hmask[(long long)(m_warp >> 5) * p.hmask_rows + (long long)t.e * p.C + t.row0 + tok0 + lane] = mine;
             }
 #pragma unroll
-            for (int k = 0; k < 3; ++k) {                       // advance the queue
+            for (int k = 0; k < kQueue - 1; ++k) {              // advance the queue
               q_off[k] = q_off[k + 1];
               q_gate[k] = q_gate[k + 1];
               q_mw[k] = q_mw[k + 1];
@@ -481,13 +548,16 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
             __syncwarp();
           }
         }
-        if (!released) {                                        // this warp had no chunk in this tile
+        if (!mid_sent) {                                        // this warp had no chunk in this tile
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive_remote(tempty0 + 8u * acc, 0);
+          if (lane == 0) mbar_arrive_remote(tmid0 + 8u * side, 0);
         }
-        acc ^= 1u;
-        if (acc == 0) acc_phase ^= 1u;
+        if (!released) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(tempty0 + 8u * side, 0);
+        }
       }
     }
   }
@@ -504,9 +574,9 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const CUtensor
 
 template <int OP>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
-expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ BMapSet bm,
                         const PairParams p) {
-  pair_body<OP>(tmA, tmB, p, (int)(blockIdx.x >> 1), (int)(gridDim.x >> 1));
+  pair_body<OP>(tmA, bm, p, (int)(blockIdx.x >> 1), (int)(gridDim.x >> 1));
 }
 
 // Two products that read the same activations, side by side in one launch: the first `split` CTA pairs work on
@@ -516,9 +586,9 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 // runs ahead pays the HBM latency and so falls back: the two stay within a few experts of each other).
 template <int OPA, int OPB>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
-expert_gemm_pair_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+expert_gemm_pair_dual_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ BMapSet tmB0,
                              const PairParams p0, const __grid_constant__ CUtensorMap tmA1,
-                             const __grid_constant__ CUtensorMap tmB1, const PairParams p1, const int split) {
+                             const __grid_constant__ BMapSet tmB1, const PairParams p1, const int split) {
   const int cl = (int)(blockIdx.x >> 1), n = (int)(gridDim.x >> 1);
   if (cl < split) pair_body<OPA>(tmA0, tmB0, p0, cl, split);
   else pair_body<OPB>(tmA1, tmB1, p1, cl - split, n - split);
@@ -551,7 +621,7 @@ int pair_grid(Kernel kernel, int* cached_grid, int dev, int sm_count, cudaStream
 }
 
 template <int OP>
-int launch_pair_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairParams& q, int dev, int sm_count,
+int launch_pair_op(const CUtensorMap& tmA, const BMapSet& tmB, const PairParams& q, int dev, int sm_count,
                    cudaStream_t st) {
   static int cached_grid[64] = {0};
   int grid = 0;
@@ -562,8 +632,15 @@ int launch_pair_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const PairPar
 }
 
 // Operands, output and tile counts of one product.
+// The token operand's maps: one per box height (8 j rows, j = 1..16).
+int make_token_maps(BMapSet* bm, const void* base, long long E, long long rows, long long cols) {
+  for (int j = 1; j <= kBMaps; ++j)
+    if (make_map(&bm->m[j - 1], base, E, rows, cols, 8 * j) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
+  return SWITCH_MOE_OK;
+}
+
 int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* ws, PairParams* out,
-                 CUtensorMap* tmA_out, CUtensorMap* tmB_out) {
+                 CUtensorMap* tmA_out, BMapSet* tmB_out) {
   const void* xd = ws_ptr<char>(ws, p.xd);
   const void* h = ws_ptr<char>(ws, p.h);
   const void* dyd = ws_ptr<char>(ws, p.dyd);
@@ -582,28 +659,29 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
   q.hmask = ws_ptr<uint32_t>(ws, p.hmask);
   q.hmask_rows = (long long)s.E * s.C;
   CUtensorMap& tmA = *tmA_out;
-  CUtensorMap& tmB = *tmB_out;
+  BMapSet& bm = *tmB_out;
+  CUtensorMap& tmB = bm.m[0];
   int rc = SWITCH_MOE_OK, rc2 = SWITCH_MOE_OK;
   int K = 0;
   switch (op) {
     case kGemm1Relu:       // A = W_in [E][d (k)][f (m)]: m contiguous -> MN-major; B = X_d [E][C][d] K-major
       q.token_op = 1; q.a_mn_major = 1; q.Mw = fin; K = s.d;   // GEGLU: [a | b], 2 f output columns, no ReLU
-      rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 64); rc2 = make_map(&tmB, xd, s.E, s.C, s.d, 128);
+      rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 64); rc2 = make_token_maps(&bm, xd, s.E, s.C, s.d);
       q.out = s.geglu ? ws_ptr<__nv_bfloat16>(ws, p.ab) : ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = fin;
       q.plain = s.geglu; break;
     case kGemm2Combine:    // A = W_out [E][f (k)][d (m)] MN-major; B = H [E][C][f] K-major
       q.token_op = 1; q.a_mn_major = 1; q.Mw = s.d; K = s.f;
-      rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 64); rc2 = make_map(&tmB, h, s.E, s.C, s.f, 128);
+      rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 64); rc2 = make_token_maps(&bm, h, s.E, s.C, s.f);
       q.out = static_cast<__nv_bfloat16*>(a.y); q.ld_out = s.d;
       if (s.residual) { q.res = static_cast<const __nv_bfloat16*>(a.x); q.out2 = ws_ptr<__nv_bfloat16>(ws, p.layer_y); }
       break;
     case kDgrad2Mask:      // A = W_out [E][f (m)][d (k)] K-major; B = dY_d [E][C][d] K-major
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.f; K = s.d;
-      rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 128); rc2 = make_map(&tmB, dyd, s.E, s.C, s.d, 128);
+      rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 128); rc2 = make_token_maps(&bm, dyd, s.E, s.C, s.d);
       q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.ld_out = s.f; q.plain = s.geglu; break;
     case kDgrad1Scatter:   // A = W_in [E][d (m)][f (k)] K-major; B = dH [E][C][f] K-major  (GEGLU: d[a | b], K = 2 f)
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.d; K = fin;
-      rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 128); rc2 = make_map(&tmB, du, s.E, s.C, fin, 128);
+      rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 128); rc2 = make_token_maps(&bm, du, s.E, s.C, fin);
       q.out = static_cast<__nv_bfloat16*>(a.dx); q.ld_out = s.d;
       if (s.residual) q.res = static_cast<const __nv_bfloat16*>(a.dy);
       break;
@@ -619,6 +697,11 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
   }
   if (rc != SWITCH_MOE_OK || rc2 != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
   q.n_mpairs = (q.Mw + 255) / 256;
+  // operand ring of the token products: a stage holds A (16 KB) and this CTA's half of the widest token tile the
+  // capacity allows (at most kPairTileTokens / 2 rows of 128 bytes, rounded up to whole 1 KB swizzle atoms)
+  const int widest = s.C < kPairTileTokens ? (s.C + 15) / 16 * 16 : kPairTileTokens;
+  q.stage_bytes = kPHalfBytes + ((widest / 2) * 128 + 1023) / 1024 * 1024;
+  q.stages = kPRingBytes / q.stage_bytes < kPMaxStages ? kPRingBytes / q.stage_bytes : kPMaxStages;
   q.n_ntiles_fixed = q.token_op ? 0 : (q.Nfix + 255) / 256;
   q.k_blocks_fixed = q.token_op ? K / kBK : 0;
   *out = q;
@@ -638,7 +721,8 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   int dev = 0, sm_count = 0;
   if (device_and_sms(&dev, &sm_count) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
   PairParams q;
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA;
+  BMapSet tmB;
   const int rc = pair_problem(op, s, p, a, ws, &q, &tmA, &tmB);
   if (rc != SWITCH_MOE_OK) return rc;
   switch (op) {
@@ -658,7 +742,8 @@ int launch_pair_dgrad1_wgrad1(const Shape& s, const Plan& p, const GemmArgs& a, 
   int dev = 0, sm_count = 0;
   if (device_and_sms(&dev, &sm_count) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
   PairParams q0, q1;
-  CUtensorMap tmA0, tmB0, tmA1, tmB1;
+  CUtensorMap tmA0, tmA1;
+  BMapSet tmB0, tmB1;
   int rc = pair_problem(kDgrad1Scatter, s, p, a, ws, &q0, &tmA0, &tmB0);
   if (rc != SWITCH_MOE_OK) return rc;
   rc = pair_problem(kWgrad1, s, p, a, ws, &q1, &tmA1, &tmB1);

@@ -15,6 +15,9 @@ constexpr int kMaxExperts = 256;        // router kernels keep ceil(E/32) <= 8 e
 constexpr int kRouterBlockTokens = 64;  // tokens per router-forward block (one partial P-sum row each)
 constexpr int kPlanBlockTokens = 256;   // tokens per dispatch-plan block (one histogram row each)
 constexpr int kTileM = 128;             // token rows per tensor-core tile; tails are zero-filled to this
+constexpr int kPairTileTokens = 320;    // widest token tile of the paired-CTA GEMM (tokens on the MMA's N side, two
+                                        // column segments above 256): an expert within the capacity of the paper's
+                                        // layers (capacity factor 1.25 at 256 tokens per expert) is one tile
 constexpr int kDwrChunkTokens = 512;    // tokens per split of the dW_r reduction
 constexpr int kMaxGroups = 64;          // routing groups per call
 

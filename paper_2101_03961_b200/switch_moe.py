@@ -30,7 +30,8 @@ EXPORTED_SYMBOLS = [
     "switch_moe_capacity", "switch_moe_workspace_bytes", "switch_moe_workspace_view", "switch_moe_fwd",
     "switch_moe_bwd", "switch_moe_router_fwd", "switch_moe_dispatch_plan", "switch_moe_router_bwd",
     "switch_moe_dispatch_plan_static", "switch_moe_step_host", "switch_moe_step_host_enqueue",
-    "switch_moe_check_device_status", "switch_moe_launches_per_step", "switch_moe_status_string",
+    "switch_moe_check_device_status", "switch_moe_launches_per_step", "switch_moe_stage_launches",
+    "switch_moe_status_string",
 ]
 
 
@@ -84,6 +85,7 @@ def load_library() -> ctypes.CDLL:
     lib.switch_moe_step_host_enqueue.argtypes = lib.switch_moe_step_host.argtypes + [vp, vp]
     lib.switch_moe_check_device_status.argtypes = [cp, vp, i32p, vp]
     lib.switch_moe_launches_per_step.argtypes = [cp, i32p]
+    lib.switch_moe_stage_launches.argtypes = [cp, i32p]
     lib.switch_moe_status_string.argtypes = [ctypes.c_int]
     lib.switch_moe_status_string.restype = ctypes.c_char_p
     for name in EXPORTED_SYMBOLS:
@@ -263,3 +265,10 @@ def switch_moe_launches_per_step(cfg) -> int:
     _check(load_library().switch_moe_launches_per_step(ctypes.byref(cfg), ctypes.byref(out)),
            "switch_moe_launches_per_step")
     return out.value
+
+
+def switch_moe_stage_launches(cfg) -> dict:
+    """Kernel launches per stage, keyed by STAGE_NAMES."""
+    out = (ctypes.c_int32 * (STAGE_EVENTS - 1))()
+    _check(load_library().switch_moe_stage_launches(ctypes.byref(cfg), out), "switch_moe_stage_launches")
+    return {name: int(out[i]) for i, name in enumerate(STAGE_NAMES) if name is not None}

@@ -1,8 +1,10 @@
 """Full-size parity in the launch configuration the benchmark times: the whole layer runs on the device at the
-workload's real shape; the oracle checks everything it can afford exactly -- the router and the dispatch plan for
-all tokens (bit-exact integers), the auxiliary loss, and, for a sample of experts (the fullest, the emptiest
-non-empty one and two others), every output row and gradient those experts produce.  Properties that hold at any
-size cover the rest: dropped tokens give zero rows, experts without tokens give zero gradients, nothing is NaN.
+workload's real shape and the oracle checks all of it -- the router and the dispatch plan for all tokens (bit-exact
+integers), the auxiliary loss, and every expert's hidden activations, output rows and gradients (the whole of y, dx,
+dW_r, dW_in, dW_out), each tensor by its relative Frobenius error and element by element.  Only the wide-expert
+workload (8 TFLOP of float64 work for the oracle) samples experts: the fullest, the emptiest non-empty one and one
+other.  Properties that hold at any size are asserted as well: dropped tokens give zero rows, experts without
+tokens give zero gradients, nothing is NaN.
 """
 import numpy as np
 import pytest
@@ -12,8 +14,8 @@ from oracle import switch_oracle as so
 from paper_2101_03961_b200 import build as sbuild
 from paper_2101_03961_b200 import inputs as si
 from paper_2101_03961_b200 import switch_moe as sm
-from tests.gpu_helpers import (TOL_BF16, TOL_ROUTER, check_flips, check_second_choice, expert_hidden, rel_err,
-                               skip_path_ok, to_np)
+from tests.gpu_helpers import (TOL_BF16, TOL_ROUTER, check_flips, check_second_choice, expert_hidden,
+                               follow_relu_flips, rel_err, skip_path_ok, to_np)
 
 pytestmark = pytest.mark.gpu
 
@@ -22,15 +24,27 @@ def _bits_to_dev(bits: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def _run_fullsize(name, seed=0, n_extra=2, residual=False, groups=1, reroute=False):
+class _ExpertWeights:
+    """Expert i's weights as float32, decoded on demand from the bfloat16 bits the device was given (the oracle only
+    ever indexes by expert, so host memory stays flat)."""
+
+    def __init__(self, bits: np.ndarray):
+        self.bits = bits
+
+    def __getitem__(self, i):
+        return si.from_bf16_bits(self.bits[i])
+
+
+def _run_fullsize(name, seed=0, n_extra=None, residual=False, groups=1, reroute=False):
     sbuild.build()
     cfg = si.CONFIGS[name]
     assert cfg.dtype == si.DTYPE_BF16
     x_np, dy_np = si.gen_x(cfg, seed), si.gen_dy(cfg, seed)
     W_r_np, b_np = si.gen_W_r(cfg, seed), si.gen_router_bias(cfg, seed)
     x, dy = _bits_to_dev(si.to_bf16_bits(x_np)), _bits_to_dev(si.to_bf16_bits(dy_np))
-    W_in = _bits_to_dev(si.gen_W_in(cfg, seed, as_bits=True, threads=16))
-    W_out = _bits_to_dev(si.gen_W_out(cfg, seed, as_bits=True, threads=16))
+    W_in_bits = si.gen_W_in(cfg, seed, as_bits=True, threads=16)
+    W_out_bits = si.gen_W_out(cfg, seed, as_bits=True, threads=16)
+    W_in, W_out = _bits_to_dev(W_in_bits), _bits_to_dev(W_out_bits)
     W_r = torch.from_numpy(W_r_np).cuda()
     bias = None if b_np is None else torch.from_numpy(b_np).cuda()
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, residual=residual,
@@ -77,29 +91,38 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False, groups=1, reroute=Fal
     np.testing.assert_array_equal(view(sm.WS_KEPT).cpu().numpy(), plan["kept"])
     assert abs(float(aux.item()) - aux_ref) <= TOL_ROUTER * aux_ref
 
-    # sampled experts: fullest, emptiest non-empty, and a few fixed ones
+    # every expert; or (n_extra given) a sample: the fullest, the emptiest non-empty one and n_extra others
     count = plan["count"]
     nonempty = np.flatnonzero(count > 0)
-    sample = {int(np.argmax(count)), int(nonempty[np.argmin(count[nonempty])])}
-    rng = np.random.default_rng(seed)
-    sample.update(int(v) for v in rng.choice(nonempty, size=min(n_extra, nonempty.size), replace=False))
-    sample = sorted(sample)
-    W_in_s = {i: si.gen_W_in_expert(cfg, i, seed) for i in sample}
-    W_out_s = {i: si.gen_W_out_expert(cfg, i, seed) for i in sample}
+    if n_extra is None:
+        sample = list(range(E))
+    else:
+        sample = {int(np.argmax(count)), int(nonempty[np.argmin(count[nonempty])])}
+        rng = np.random.default_rng(seed)
+        sample.update(int(v) for v in rng.choice(nonempty, size=min(n_extra, nonempty.size), replace=False))
+        sample = sorted(sample)
+    W_in_s, W_out_s = _ExpertWeights(W_in_bits), _ExpertWeights(W_out_bits)
+    for i in sample[:2]:                                       # the decoded bits are the seeded generator's values
+        np.testing.assert_array_equal(W_in_s[i], si.gen_W_in_expert(cfg, i, seed))
     if groups == 1:
         fwd = so.switch_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, router_bias=b_np,
                                 expert_index=gpu_e, experts=sample, residual=residual, reroute=reroute, alt_index=alt,
                                 geglu=cfg.geglu)
-        bwd = so.switch_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
     else:
         fwd = so.switch_forward_groups(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, groups,
                                        router_bias=b_np, expert_index=gpu_e, experts=sample, residual=residual)
+    hid = view(sm.WS_H).view(E, C, cfg.d_ff)
+    relu_flips = follow_relu_flips(fwd, lambda i, k: to_np(hid[i, :k]), experts=sample)
+    if groups == 1:
+        bwd = so.switch_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
+    else:
         bwd = so.switch_backward_groups(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
     keep = plan["keep"]
-    hid = view(sm.WS_H).view(E, C, cfg.d_ff)
     errs = {}
     for i in sample:
         k = int(plan["kept"][i])
+        if k == 0:
+            continue                                           # zero gradients are asserted below
         tok = plan["token_of_slot"][i * C:i * C + k]           # the expert's tokens in slot order
         tt = torch.from_numpy(tok).cuda()
         errs[f"H[{i}]"] = rel_err(to_np(hid[i, :k]), expert_hidden(fwd, i))
@@ -108,15 +131,20 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False, groups=1, reroute=Fal
             errs[f"layer_y[{i}]"] = rel_err(to_np(layer_y[tt]), fwd["layer_y"][tok])
             assert skip_path_ok(to_np(y[tt]), fwd["y"][tok], fwd["layer_y"][tok], TOL_BF16, sm.BF16)
             assert skip_path_ok(to_np(dx[tt]), bwd["dx"][tok], bwd["dx"][tok] - dy_np[tok].astype(np.float64),
-                                TOL_BF16, sm.BF16)
+                                TOL_BF16, sm.BF16, roundings=3)
         else:
             errs[f"y[{i}]"] = rel_err(to_np(y[tt]), fwd["y"][tok])
             errs[f"dx[{i}]"] = rel_err(to_np(dx[tt]), bwd["dx"][tok])
         errs[f"dW_in[{i}]"] = rel_err(to_np(dW_in[i]), bwd["dW_in"][i])
         errs[f"dW_out[{i}]"] = rel_err(to_np(dW_out[i]), bwd["dW_out"][i])
         errs[f"dgate[{i}]"] = rel_err(to_np(view(sm.WS_DGATE)[tt]), bwd["dgate"][tok])
+    if n_extra is None and not residual:
+        # all experts were run: the whole output, the whole input gradient and the router's weight gradient
+        errs["y"] = rel_err(to_np(y), fwd["y"])
+        errs["dx"] = rel_err(to_np(dx), bwd["dx"])
+        errs["dW_r"] = rel_err(to_np(dW_r), bwd["dW_r"])
     bad = {k: v for k, v in errs.items() if not v <= TOL_BF16}
-    assert not bad, (bad, errs)
+    assert not bad, bad
 
     # properties that hold at any size
     dropped = torch.from_numpy(np.flatnonzero(~keep)).cuda()
@@ -136,7 +164,7 @@ def _run_fullsize(name, seed=0, n_extra=2, residual=False, groups=1, reroute=Fal
     for i in np.flatnonzero(count == 0):
         assert bool((dW_in[int(i)] == 0).all()) and bool((dW_out[int(i)] == 0).all())
     # dropped tokens receive only the router's gradient: finite and small, never the expert path
-    return {"flips": flips, "dropped": int((~keep).sum()), "errs": errs}
+    return {"flips": flips, "relu_flips": relu_flips, "dropped": int((~keep).sum()), "errs": errs}
 
 
 def test_switch_base_full_size():
@@ -159,7 +187,7 @@ def test_switch_large_full_size():
 
 
 def test_wide_expert_full_size():
-    _run_fullsize("wide", n_extra=1)
+    _run_fullsize("wide", n_extra=1)                          # sampled experts: the oracle pass would take minutes
 
 
 def test_overflow_stress_with_the_skip_path_inside_full_size():
@@ -195,8 +223,9 @@ def test_top2_routing_at_the_switch_base_shape_full_size():
     seed = 0
     x_np, dy_np, W_r_np = si.gen_x(cfg, seed), si.gen_dy(cfg, seed), si.gen_W_r(cfg, seed)
     x, dy = _bits_to_dev(si.to_bf16_bits(x_np)), _bits_to_dev(si.to_bf16_bits(dy_np))
-    W_in = _bits_to_dev(si.gen_W_in(cfg, seed, as_bits=True, threads=16))
-    W_out = _bits_to_dev(si.gen_W_out(cfg, seed, as_bits=True, threads=16))
+    W_in_bits = si.gen_W_in(cfg, seed, as_bits=True, threads=16)
+    W_out_bits = si.gen_W_out(cfg, seed, as_bits=True, threads=16)
+    W_in, W_out = _bits_to_dev(W_in_bits), _bits_to_dev(W_out_bits)
     W_r = torch.from_numpy(W_r_np).cuda()
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, top2=True)
     ws = sm.allocate_workspace(mcfg)
@@ -225,15 +254,14 @@ def test_top2_routing_at_the_switch_base_shape_full_size():
     assert abs(float(aux.item()) - plan["aux"]) <= TOL_ROUTER * plan["aux"]
     assert plan["keep"].mean() > 0.9                           # twice the capacity holds most of the assignments
     kept = plan["kept"]
-    sample = sorted({int(np.argmax(kept)), int(np.argmin(kept)), 7, 100})
-    W_in_s = {i: si.gen_W_in_expert(cfg, i, seed) for i in sample}
-    W_out_s = {i: si.gen_W_out_expert(cfg, i, seed) for i in sample}
+    sample = list(range(E))                                    # every expert
+    W_in_s, W_out_s = _ExpertWeights(W_in_bits), _ExpertWeights(W_out_bits)
     fwd = so.top2_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, first_index=first,
                           second_index=second, experts=sample)
-    bwd = so.top2_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
-    yv = None
-    errs = {}
     hid = view(sm.WS_H).view(E, C, cfg.d_ff)
+    follow_relu_flips(fwd, lambda i, k: to_np(hid[i, :k]), experts=sample)
+    bwd = so.top2_backward(fwd, x_np, W_r_np, W_in_s, W_out_s, dy_np, experts=sample)
+    errs = {}
     for i in sample:
         k = int(kept[i])
         v = plan["token_of_slot"][i * C:i * C + k]
@@ -242,13 +270,9 @@ def test_top2_routing_at_the_switch_base_shape_full_size():
         errs[f"dW_out[{i}]"] = rel_err(to_np(dW_out[i]), bwd["dW_out"][i])
         vv = torch.from_numpy(v).cuda()
         errs[f"dgate[{i}]"] = rel_err(to_np(view(sm.WS_DGATE)[vv]), bwd["dgate"][v])
-    # tokens both of whose assignments went to sampled experts: their whole output row is known to the oracle
-    in_sample = np.isin(plan["e"], sample) & plan["keep"]
-    whole = np.flatnonzero((in_sample[:T] | ~plan["keep"][:T]) & (in_sample[T:] | ~plan["keep"][T:])
-                           & (plan["keep"][:T] | plan["keep"][T:]))
-    assert whole.size > 10
-    wt = torch.from_numpy(whole).cuda()
-    errs["y"] = rel_err(to_np(y[wt]), fwd["y"][whole])
+    errs["y"] = rel_err(to_np(y), fwd["y"])
+    errs["dx"] = rel_err(to_np(dx), bwd["dx"])
+    errs["dW_r"] = rel_err(to_np(dW_r), bwd["dW_r"])
     bad = {k: v for k, v in errs.items() if not v <= TOL_BF16}
-    assert not bad, (bad, errs)
+    assert not bad, bad
     assert bool(torch.isfinite(y).all()) and bool(torch.isfinite(dx).all()) and bool(torch.isfinite(dW_in).all())
