@@ -147,7 +147,9 @@ enum switch_moe_ws_region {
   SWITCH_MOE_WS_DYD = 11,           /* [E,C,d_model] g . dy per slot (backward) */
   SWITCH_MOE_WS_DH = 12,            /* [E,C,d_ff]    gradient of the pre-activation per slot (backward) */
   SWITCH_MOE_WS_DGATE = 13,         /* float[T]   <dy_t, o_t> for kept tokens (backward) */
-  SWITCH_MOE_WS_DLOGITS = 14,       /* float[T,E] gradient of the router logits (backward) */
+  SWITCH_MOE_WS_DLOGITS = 14,       /* float[T,E] gradient of the router logits: written by switch_moe_router_bwd, and
+                                       by switch_moe_bwd only where the router runs on the FP32 FMA path (the
+                                       tensor-core path keeps just the bfloat16 parts it multiplies) */
   SWITCH_MOE_WS_LAYER_Y = 15,       /* [T,d_model] g_t E(x_t) without the skip path (only with SWITCH_MOE_FLAG_RESIDUAL;
                                        rows of dropped tokens are not written) */
   SWITCH_MOE_WS_EXPERT_PROC = 16,   /* int32[T] the expert that processes the token: e_t unless stage 2 rerouted it

@@ -510,7 +510,10 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
     if (cudaMemcpyAsync(ei, expert_index, (size_t)s.Tv * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
       return SWITCH_MOE_CUDA_ERROR;
   }
-  launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, s.Tv, s.E, ws_ptr<int>(ws, p.hist));
+  // the tensor-core router's forward kernel leaves the histograms of its own expert choices in the workspace
+  const bool have_hist = expert_index == nullptr && s.router_hist;
+  if (!have_hist)
+    launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, s.Tv, s.E, ws_ptr<int>(ws, p.hist));
   int Ew = 32;
   while (Ew < s.E) Ew *= 2;
   const int blocks_per_group = s.plan_blocks / s.G;

@@ -236,10 +236,10 @@ router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ e
   for (int n = 0; n < NE; ++n) {
     const int e = lane * NE + n;
     const float dh = p[n] * (G[n] - s);
-    if (e < E) dlogits[(size_t)t * E + e] = dh;
+    if (dlogits != nullptr && e < E) dlogits[(size_t)t * E + e] = dh;
     G[n] = e < E ? dh : 0.f;
   }
-  if (dhsplit != nullptr && lane * NE < Epad64) {             // bf16 hi/mid/lo parts for the tensor-core products
+  if (dhsplit != nullptr && lane * NE < Epad64) {             // bf16 hi / mid parts for the tensor-core products
     __align__(16) __nv_bfloat16 hi[NE], mid[NE], lo[NE];
 #pragma unroll
     for (int n = 0; n < NE; ++n) split3(G[n], &hi[n], &mid[n], &lo[n]);
@@ -247,14 +247,13 @@ router_dlogits_kernel(const float* __restrict__ probs, const int* __restrict__ e
     using Vec = typename BfVec<NE>::type;
     *reinterpret_cast<Vec*>(dhsplit + at) = *reinterpret_cast<const Vec*>(hi);
     *reinterpret_cast<Vec*>(dhsplit + plane + at) = *reinterpret_cast<const Vec*>(mid);
-    *reinterpret_cast<Vec*>(dhsplit + 2 * plane + at) = *reinterpret_cast<const Vec*>(lo);
   }
   if (dhsplit != nullptr) {                                   // padding columns beyond the lanes' experts
     const __nv_bfloat16 z = __float2bfloat16(0.f);
     const size_t plane = (size_t)T * Epad64;
     for (int e = 32 * NE + lane; e < Epad64; e += 32) {
       const size_t at = (size_t)t * Epad64 + e;
-      dhsplit[at] = z; dhsplit[plane + at] = z; dhsplit[2 * plane + at] = z;
+      dhsplit[at] = z; dhsplit[plane + at] = z;
     }
   }
 }
@@ -425,9 +424,13 @@ int router_bwd_t(const Shape& s, const Plan& p, const void* x, const float* W_r,
   // the loss is the mean over the routing groups, and T = G . Tg)
   const float cG = (float)((double)d_aux * (double)s.alpha * (double)s.E / ((double)s.T * (double)s.Tg));
   float* dlogits = ws_ptr<float>(ws, p.dlogits);
+  // The float32 logit gradients are an output of the staged call (and the operand of the FP32-FMA products); the
+  // whole-layer backward pass on the tensor cores only needs their bfloat16 parts.
+  const bool tc_products = s.router_tc && sizeof(XT) == 2;
   launch_k(router_dlogits_kernel<NE>, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs),
                                                             ws_ptr<int>(ws, p.expert_proc), ws_ptr<int>(ws, p.slot),
-                                                            ws_ptr<int>(ws, p.count_g), dgate, cG, s.T, s.Tg, s.E, s.top2, dlogits,
+                                                            ws_ptr<int>(ws, p.count_g), dgate, cG, s.T, s.Tg, s.E, s.top2,
+                                                            (tc_products && accumulate_dx) ? nullptr : dlogits,
                                                             (s.router_tc && sizeof(XT) == 2)
                                                                 ? ws_ptr<__nv_bfloat16>(ws, p.dhsplit) : nullptr,
                                                             s.Epad64);

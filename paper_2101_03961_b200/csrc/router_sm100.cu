@@ -1,13 +1,14 @@
 // Router of the Switch FFN layer on the B200 tensor cores with float32-grade accuracy (Section 2.4: the router is the
 // part of the layer that must not run in bfloat16).
 //
-// x is bfloat16, hence exact in float32.  A float32 operand w is written as the sum of three bfloat16 numbers
-// (w = hi + mid + lo exactly up to 2^-24 relative), every bf16 x bf16 product is exact in float32, and tcgen05
-// accumulates in float32.  So
-//   logits   h = x W_r            = x (W_hi + W_mid + W_lo)                       (Section 2.1; Eq. 1 follows in the epilogue)
-//   dW_r       = x^T dh           = x^T (dh_hi + dh_mid + dh_lo)                  (contraction over tokens, split over CTAs)
+// x is bfloat16, hence exact in float32.  A float32 operand w is written as the sum of two bfloat16 numbers
+// (w = hi + mid up to 2^-18 relative: each part carries 8 significant bits and a third part would add what the 1e-5
+// tolerance of the router never sees), every bf16 x bf16 product is exact in float32, and tcgen05 accumulates in
+// float32.  So
+//   logits   h = x W_r            = x (W_hi + W_mid)                              (Section 2.1; Eq. 1 follows in the epilogue)
+//   dW_r       = x^T dh           = x^T (dh_hi + dh_mid)                          (contraction over tokens, split over CTAs)
 //   dx_router  = dh W_r^T         ~ dh_hi W_hi^T + dh_hi W_mid^T + dh_mid W_hi^T  (the output is bfloat16: 2^-16 suffices)
-// are bfloat16 tensor-core products whose results agree with the float32 definition to about 1e-7 relative, and the
+// are bfloat16 tensor-core products whose results agree with the float32 definition to a few 1e-6 relative, and the
 // router stops being bound by the FP32 FMA pipes (E flop per byte of x) and becomes a streaming kernel.
 //
 // The forward epilogue keeps one token per thread (a TMEM lane holds all E logits of a token): softmax, top-1 with
@@ -18,12 +19,9 @@ namespace swmoe {
 using namespace tc;
 namespace {
 
-constexpr int kRThreads = 192;                       // forward kernel: TMA warp, MMA warp, 4 epilogue warps
 constexpr int kRTcThreads = 320;                     // generic kernel: TMA warp, MMA warp, 8 epilogue warps
 constexpr int kRTcOutStageBytes = 8 * 32 * 128;
 constexpr int kRTcSmemBytes = 1024 + kStages * kStageBytes + kRTcOutStageBytes + 128;
-constexpr int kROutStageBytes = 4 * 32 * 128;
-constexpr int kRSmemBytes = 1024 + kStages * kStageBytes + kROutStageBytes + 128;
 
 enum RouterOp { kRFwd = 0, kRDwr = 1, kRDx = 2 };
 
@@ -33,6 +31,7 @@ struct RouterTcParams {
   int n_mtiles, n_ntiles;
   int splits, chunk_kblocks, total_kblocks;   // dwr: split of the token contraction
   int wrap;                  // k-blocks per part: d/64 (fwd), Epad64/64 (dx); dwr derives it per tile
+  int both_parts;            // dwr: 1 = a stage holds the x block and both parts of dh (2 x mma_n columns <= 256)
   const float* bias; const float* noise; float* probs; int* expert_index; float* gate;   // fwd
   float* partial;                                                                         // dwr
   __nv_bfloat16* dx; const int* slot; int accumulate; const __nv_bfloat16* jitter_u;      // dx
@@ -68,7 +67,9 @@ __device__ __forceinline__ RTile r_decode(const RouterTcParams& p, int id) {
     t.n0 = (id - mt * p.n_ntiles) * kBN;
     t.wrap = p.wrap;
   }
-  t.k_blocks = 3 * t.wrap;
+  // forward: W_r = hi + mid, one part after the other; dW_r: dh = hi + mid, both parts staged with the x block they
+  // multiply when they fit (up to 128 experts), else one after the other; dx: three cross terms
+  t.k_blocks = (OP == kRDx ? 3 : (OP == kRDwr && p.both_parts) ? 1 : 2) * t.wrap;
   return t;
 }
 
@@ -111,7 +112,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   pdl_wait();                                                 // the previous kernel's results are needed from here on
   const int n_tiles = r_total_tiles<OP>(p);
   const int b_atoms = (p.mma_n + 63) / 64;
-  const uint32_t stage_tx = kABytes + (kBMn ? (uint32_t)b_atoms * kAtomBytes : (uint32_t)kBBytes);
+  const bool both = OP == kRDwr && p.both_parts;
+  const uint32_t stage_tx = kABytes + (kBMn ? (uint32_t)(both ? 2 : 1) * b_atoms * kAtomBytes : (uint32_t)kBBytes);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -135,6 +137,9 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tma_load_3d(a_dst + kAtomBytes, &tmA, full_bar(stage), t.m0 + 64, kblk * kBK, 0);
             for (int j = 0; j < b_atoms; ++j)                                                // dh part [64 tok][64 e]
               tma_load_3d(b_dst + j * kAtomBytes, &tmB, full_bar(stage), 64 * j, kblk * kBK, part);
+            if (both)                                                                        // the other part, behind it
+              for (int j = 0; j < b_atoms; ++j)
+                tma_load_3d(b_dst + (b_atoms + j) * kAtomBytes, &tmB, full_bar(stage), 64 * j, kblk * kBK, 1);
           } else {
             const int a_part = part == 2 ? 1 : 0, b_part = part == 1 ? 1 : 0;               // (hi,hi) (hi,mid) (mid,hi)
             tma_load_3d(a_dst, &tmA, full_bar(stage), kblk * kBK, t.m0, a_part);            // dh part [128 tok][64 e]
@@ -174,6 +179,14 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint64_t ad = make_smem_desc(a_src + ks * a_kstep, a_lbo, 1024u);
             const uint64_t bd = make_smem_desc(b_src + ks * b_kstep, b_lbo, 1024u);
             tc_mma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+          }
+          if (both) {
+#pragma unroll
+            for (int ks = 0; ks < kBK / kUmmaK; ++ks) {
+              const uint64_t ad = make_smem_desc(a_src + ks * a_kstep, a_lbo, 1024u);
+              const uint64_t bd = make_smem_desc(b_src + (uint32_t)b_atoms * kAtomBytes + ks * b_kstep, b_lbo, 1024u);
+              tc_mma_bf16(d_tmem, ad, bd, idesc, 1u);
+            }
           }
           tc_commit(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -415,35 +428,46 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------------------------------------
-// Forward router for E <= 128: the x tile of a k-block is staged once and multiplied with all three parts of W_r;
-// the epilogue keeps a token's logits in registers (one TMEM pass, one expf per logit) and writes the probabilities
-// through a 32x32 shared-memory transpose so that global stores are 128-byte rows.
+// Forward router for E <= 128.  A CTA works on 256 consecutive tokens at a time -- two 128-token tiles that share every
+// staged k-block of W_r, so the weight parts cross shared memory once per 256 tokens -- and those 256 tokens are
+// exactly one block of the dispatch plan.  The epilogue (one token per thread: a TMEM lane holds all E logits of a
+// token) therefore also produces what the plan needs from the router: the block's histogram of expert choices
+// (Section 2.2: the counts behind Eq. 3's capacity cut and Eq. 5's f) and, per 128-token tile, the column sums of the
+// probabilities (Eq. 6's P), both in a fixed order.
 struct RouterFwdParams {
-  int T, d, E, Epad64, n_mtiles, k_blocks, b_atoms, stages, stage_bytes;
+  int T, d, E, Epad64, n_ptiles, k_blocks, b_atoms, stages, stage_bytes;
   const float* bias; const float* noise; float* probs; int* expert_index; float* gate;
+  float* psum_partial;       // [2 n_ptiles][E]: column sums of p over each 128-token tile
+  int* hist;                 // [n_ptiles][E]: tokens of each 256-token block per expert
   int* status;
 };
+constexpr int kRFParts = 2;                                    // W_r = hi + mid (bfloat16 each): exact to 2^-18 relative
+constexpr int kRFThreads = 320;                                // TMA warp, MMA warp, 8 epilogue warps (4 per token tile)
 constexpr int kRFRingBytes = kStages * kStageBytes;            // 192 KB of operand stages
+constexpr int kRFOutBytes = 8 * 128 * 4;                       // the eight epilogue warps' column sums (E <= 128 floats each)
+constexpr int kRFTailBytes = 2048;                             // barriers, TMEM pointer, abort flag, the block's histogram
+constexpr int kRFSmemBytes = 1024 + kRFRingBytes + kRFOutBytes + kRFTailBytes;
 
 template <int NCH>                                             // 32-logit chunks per token: 2 (E <= 64) or 4 (E <= 128)
-__global__ void __launch_bounds__(kRThreads, 1)
+__global__ void __launch_bounds__(kRFThreads, 1)
 router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const RouterFwdParams p) {
   pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + kRFRingBytes + kROutStageBytes;
-  uint8_t* bar_gen = smem_gen + kRFRingBytes + kROutStageBytes;
+  const uint32_t bar_base = smem_base + kRFRingBytes + kRFOutBytes;
+  uint8_t* bar_gen = smem_gen + kRFRingBytes + kRFOutBytes;
   const uint32_t full0 = bar_base, empty0 = bar_base + 8u * kStages;
   const uint32_t tfull0 = bar_base + 16u * kStages, tempty0 = tfull0 + 16u;
   volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kStages + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kStages + 4) + 4);
+  int* hist_s = reinterpret_cast<int*>(bar_gen + 1024);        // kMaxExperts counters
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -453,12 +477,13 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                      smem_u32(const_cast<uint32_t*>(tmem_ptr_s))), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  for (int i = threadIdx.x; i < kMaxExperts; i += kRFThreads) hist_s[i] = 0;
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_s;
   pdl_wait();                                                 // the previous kernel's results are needed from here on
-  const int n_tiles = p.n_mtiles, kbs = p.k_blocks, b_atoms = p.b_atoms;
+  const int n_tiles = p.n_ptiles, kbs = p.k_blocks, b_atoms = p.b_atoms;
   const uint32_t n_stages = (uint32_t)p.stages, stage_bytes = (uint32_t)p.stage_bytes;
 
   if (warp == 0) {
@@ -466,7 +491,7 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
-        const int m0 = id * kTileM;
+        const int m0 = id * 2 * kTileM;
 #pragma unroll 1
         for (int kb = 0; kb < kbs; ++kb) {
           ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag, p.status, 31);
@@ -477,9 +502,10 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           // the same L2 lines of W_r at the same moment
           int kr = kb + (int)(blockIdx.x % (unsigned)kbs);
           if (kr >= kbs) kr -= kbs;
-          tma_load_3d(a_dst, &tmA, fb, kr * kBK, m0, 0);                              // x tile [128 tok][64 k]
-          uint32_t b_dst = a_dst + kABytes;
-          for (int part = 0; part < 3; ++part)
+          tma_load_3d(a_dst, &tmA, fb, kr * kBK, m0, 0);                              // x tiles [128 tok][64 k]
+          tma_load_3d(a_dst + kABytes, &tmA, fb, kr * kBK, m0 + kTileM, 0);
+          uint32_t b_dst = a_dst + 2 * kABytes;
+          for (int part = 0; part < kRFParts; ++part)
             for (int j = 0; j < b_atoms; ++j, b_dst += kAtomBytes)                     // W part [64 k][64 e]
               tma_load_3d(b_dst, &tmB, fb, 64 * j, kr * kBK, part);
           if (++stage == n_stages) { stage = 0; phase ^= 1u; }
@@ -495,7 +521,7 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(p.Epad64 >> 3) << 17) |
                              ((uint32_t)(kTileM >> 4) << 24);
       const uint64_t a_desc0 = make_smem_desc(smem_base, 16u, 1024u);
-      const uint64_t b_desc0 = make_smem_desc(smem_base + kABytes, kAtomBytes, 1024u);
+      const uint64_t b_desc0 = make_smem_desc(smem_base + 2 * kABytes, kAtomBytes, 1024u);
       const uint32_t part_step = (uint32_t)(b_atoms * kAtomBytes) >> 4;
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
@@ -503,20 +529,24 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ok = mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag, p.status, 32);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * (uint32_t)kBN;
+        const uint32_t d_tmem = tmem_base + acc * (uint32_t)kBN;      // tile 0: 128 columns here, tile 1: the next 128
 #pragma unroll 1
         for (int kb = 0; kb < kbs; ++kb) {
           ok = mbar_wait(full0 + 8u * stage, phase, abort_flag, p.status, 33);
           if (!ok) break;
           tc_fence_after();
           const uint64_t ad = a_desc0 + (uint64_t)(stage * (stage_bytes >> 4));
-          uint64_t bd = b_desc0 + (uint64_t)(stage * (stage_bytes >> 4));
+          const uint64_t bd0 = b_desc0 + (uint64_t)(stage * (stage_bytes >> 4));
 #pragma unroll
-          for (int part = 0; part < 3; ++part, bd += part_step) {
+          for (int tile = 0; tile < 2; ++tile) {
+            uint64_t bd = bd0;
 #pragma unroll
-            for (int ks = 0; ks < kBK / kUmmaK; ++ks)
-              tc_mma_bf16(d_tmem, ad + (uint64_t)(ks * ((kUmmaK * 2) >> 4)), bd + (uint64_t)(ks * ((kUmmaK * 128) >> 4)),
-                          idesc, (kb > 0 || part > 0 || ks > 0) ? 1u : 0u);
+            for (int part = 0; part < kRFParts; ++part, bd += part_step) {
+#pragma unroll
+              for (int ks = 0; ks < kBK / kUmmaK; ++ks)
+                tc_mma_bf16(d_tmem + tile * 128u, ad + (uint64_t)(tile * (kABytes >> 4) + ks * ((kUmmaK * 2) >> 4)),
+                            bd + (uint64_t)(ks * ((kUmmaK * 128) >> 4)), idesc, (kb > 0 || part > 0 || ks > 0) ? 1u : 0u);
+            }
           }
           tc_commit(empty0 + 8u * stage);
           if (++stage == n_stages) { stage = 0; phase ^= 1u; }
@@ -528,33 +558,34 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
     }
   } else {
-    const int lg = warp & 3;
-    float* tile = reinterpret_cast<float*>(smem_gen + kRFRingBytes + (warp - 2) * 4096);   // 32 x 32 floats
+    const int lg = warp & 3, ti = (warp - 2) >> 2;            // TMEM lane group; which of the two token tiles
+    const int et = threadIdx.x - 64;                          // 0..255 over the epilogue warps
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
     for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
-      const int tok = id * kTileM + lg * 32 + lane;           // the token whose logits this lane holds
+      const int tok0 = id * 2 * kTileM + ti * kTileM + lg * 32;
+      const int tok = tok0 + lane;                            // the token whose logits this lane holds
       ok = mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag, p.status, 34);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * (uint32_t)kBN;
+      const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * (uint32_t)kBN + (uint32_t)ti * 128u;
       float h[NCH * 32];
+      {
+        uint32_t v[NCH * 32];
 #pragma unroll
-      for (int c = 0; c < NCH; ++c) {
-        uint32_t v[32];
-        tc_ld32(t_addr + c * 32, v);
+        for (int c = 0; c < NCH; ++c) tc_ld32(t_addr + c * 32, v + c * 32);       // all loads in flight together
         tc_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) h[c * 32 + i] = __uint_as_float(v[i]);
+        for (int i = 0; i < NCH * 32; ++i) h[i] = __uint_as_float(v[i]);
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty0 + 8u * acc);         // logits are in registers: the accumulator is free
-      // Eq. 1 and top-1 (first maximum wins), all within this lane.  Only four warps run here, so every dependent
-      // chain is paid in full: the maximum and the sum are kept as four interleaved chains, and the exponential is
-      // the hardware exp2 of a pre-scaled argument (relative error below 1e-6 for |h - m| < 10, inside the 1e-5
-      // the router is held to).
+      // Eq. 1 and top-1 (first maximum wins), all within this lane.  Few warps run here, so every dependent chain is
+      // paid in full: the maximum and the sum are kept as four interleaved chains, and the exponential is the
+      // hardware exp2 of a pre-scaled argument (relative error below 1e-6 for |h - m| < 10, inside the 1e-5 the
+      // router is held to).
       if (p.bias != nullptr) {
 #pragma unroll
         for (int e = 0; e < NCH * 32; ++e)
@@ -597,22 +628,68 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
       const float sum = (sq[0] + sq[1]) + (sq[2] + sq[3]);
       const float inv = 1.f / sum;
-      if (tok < p.T) { p.expert_index[tok] = am; p.gate[tok] = inv; }
-      // probabilities: 32 tokens x 32 experts at a time through shared memory, stored as 128-byte rows
+      const bool live = tok < p.T;
+      if (live) {
+        p.expert_index[tok] = am;
+        p.gate[tok] = inv;
+        atomicAdd(&hist_s[am], 1);                            // integer counts: the order does not matter
+      }
+      // Probabilities: every thread writes its own token's row, 16 bytes at a time (no transposition: the few warps
+      // of this kernel are bound by the number of memory instructions they issue, not by how the bytes coalesce).
+      // Column sums over the warp's 32 tokens (Eq. 6's sum over tokens) by a halving exchange: in each of five steps
+      // a lane hands half of its values to the lane whose index differs in one bit and adds what it receives, so that
+      // lane l ends with column 32 c + l summed over all lanes in a fixed (tree) order.
+      float* prow = p.probs + (size_t)(live ? tok : 0) * p.E;
+      float colsum[NCH];
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
+        float w[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) tile[lane * 32 + (i ^ lane)] = h[c * 32 + i] * inv;
-        __syncwarp();
-        const int e = c * 32 + lane;
-#pragma unroll 8
-        for (int rr = 0; rr < 32; ++rr) {
-          const int t2 = id * kTileM + lg * 32 + rr;
-          const float pv = tile[rr * 32 + (lane ^ rr)];
-          if (t2 < p.T && e < p.E) p.probs[(size_t)t2 * p.E + e] = pv;
+        for (int i = 0; i < 32; ++i) w[i] = h[c * 32 + i] * inv;
+        if (live) {
+          if ((p.E & 3) == 0) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              if (c * 32 + i < p.E) *reinterpret_cast<float4*>(prow + c * 32 + i) = make_float4(w[i], w[i + 1], w[i + 2], w[i + 3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i < p.E) prow[c * 32 + i] = w[i];
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) w[i] = 0.f;             // rows past the last token add nothing to the sums
         }
-        __syncwarp();
+#pragma unroll
+        for (int half = 16; half >= 1; half >>= 1) {
+          const bool upper = (lane & half) != 0;
+#pragma unroll
+          for (int j = 0; j < half; ++j) {
+            const float send = upper ? w[j] : w[j + half];
+            const float keep = upper ? w[j + half] : w[j];
+            w[j] = keep + __shfl_xor_sync(0xffffffffu, send, half);
+          }
+        }
+        colsum[c] = w[0];
       }
+      float* sums = reinterpret_cast<float*>(smem_gen + kRFRingBytes) + (warp - 2) * (NCH * 32);
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) sums[c * 32 + lane] = colsum[c];
+      asm volatile("bar.sync 1, 256;" ::: "memory");          // the eight epilogue warps: histogram and column sums complete
+      if (lg == 0) {                                          // the tile's four warps' sums, added in warp order
+        const float* t0 = reinterpret_cast<const float*>(smem_gen + kRFRingBytes) + (ti * 4) * (NCH * 32);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const int e = c * 32 + lane;
+          const float v = ((t0[e] + t0[NCH * 32 + e]) + t0[2 * NCH * 32 + e]) + t0[3 * NCH * 32 + e];
+          if (e < p.E) p.psum_partial[(size_t)(2 * id + ti) * p.E + e] = v;
+        }
+      }
+      if (et < p.E) {
+        p.hist[(size_t)id * p.E + et] = hist_s[et];
+        hist_s[et] = 0;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");          // before the next round reuses the tiles and the counters
       acc ^= 1u;
       if (acc == 0) acc_phase ^= 1u;
     }
@@ -651,7 +728,8 @@ probs_colsum_kernel(const float* __restrict__ probs, int T, int E, int rows_per_
   if (g == 0 && e < E) partial[(size_t)blockIdx.x * E + e] = ((part[0][e] + part[1][e]) + part[2][e]) + part[3][e];
 }
 
-// wsplit[part][k][e] for e < Epad64 (zero beyond E)
+// wsplit[part][k][e] for e < Epad64 (zero beyond E): W_r = hi + mid + (a remainder below 2^-18 relative that no
+// product uses: the forward logits and the backward dx both stop at hi + mid)
 __global__ void split_w_kernel(const float* __restrict__ W_r, int d, int E, int Epad64,
                                __nv_bfloat16* __restrict__ wsplit) {
   pdl_launch_dependents();
@@ -662,7 +740,7 @@ __global__ void split_w_kernel(const float* __restrict__ W_r, int d, int E, int 
   const int k = (int)(i / Epad64), e = (int)(i - (size_t)k * Epad64);
   __nv_bfloat16 h, m, l;
   split3(e < E ? W_r[(size_t)k * E + e] : 0.f, &h, &m, &l);
-  wsplit[i] = h; wsplit[n + i] = m; wsplit[2 * n + i] = l;
+  wsplit[i] = h; wsplit[n + i] = m;
 }
 
 int sm_count_or_default() {
@@ -692,42 +770,42 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
   CUtensorMap tmA, tmB;
   if (make_map(&tmA, x, 1, s.T, s.d, kTileM) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
   if (make_map(&tmB, wsplit, 3, s.d, s.Epad64, 64) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
-  const int n_mtiles = (s.T + kTileM - 1) / kTileM;
-  const int grid = n_mtiles < sm_count_or_default() ? n_mtiles : sm_count_or_default();
-  int rc;
   if (s.Epad64 <= 128) {
+    // 256 tokens per CTA and round; the epilogue also leaves the plan's histogram and the P-sum partials
     RouterFwdParams q{};
-    q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.n_mtiles = n_mtiles; q.k_blocks = s.d / kBK;
+    q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.n_ptiles = (s.T + 2 * kTileM - 1) / (2 * kTileM);
+    q.k_blocks = s.d / kBK;
     q.b_atoms = s.Epad64 / 64;
-    q.stage_bytes = kABytes + 3 * q.b_atoms * kAtomBytes;
+    q.stage_bytes = 2 * kABytes + kRFParts * q.b_atoms * kAtomBytes;
     q.stages = kRFRingBytes / q.stage_bytes < kStages ? kRFRingBytes / q.stage_bytes : kStages;
     q.bias = bias; q.noise = noise; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
     q.gate = ws_ptr<float>(ws, p.gate); q.status = ws_ptr<int>(ws, p.status);
+    q.psum_partial = ws_ptr<float>(ws, p.psum_partial); q.hist = ws_ptr<int>(ws, p.hist);
+    const int grid = q.n_ptiles < sm_count_or_default() ? q.n_ptiles : sm_count_or_default();
     if (s.Epad64 == 64) {
-      if (cudaFuncSetAttribute(router_fwd_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
+      if (cudaFuncSetAttribute(router_fwd_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRFSmemBytes) !=
           cudaSuccess)
         return SWITCH_MOE_CUDA_ERROR;
-      launch_k(router_fwd_tc_kernel<2>, dim3(grid), dim3(kRThreads), kRSmemBytes, st, tmA, tmB, q);
+      launch_k(router_fwd_tc_kernel<2>, dim3(grid), dim3(kRFThreads), kRFSmemBytes, st, tmA, tmB, q);
     } else {
-      if (cudaFuncSetAttribute(router_fwd_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes) !=
+      if (cudaFuncSetAttribute(router_fwd_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRFSmemBytes) !=
           cudaSuccess)
         return SWITCH_MOE_CUDA_ERROR;
-      launch_k(router_fwd_tc_kernel<4>, dim3(grid), dim3(kRThreads), kRSmemBytes, st, tmA, tmB, q);
+      launch_k(router_fwd_tc_kernel<4>, dim3(grid), dim3(kRFThreads), kRFSmemBytes, st, tmA, tmB, q);
     }
-    rc = launch_status();
-  } else {
-    RouterTcParams q{};
-    q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.mma_n = s.Epad64;
-    q.n_mtiles = n_mtiles; q.n_ntiles = 1; q.wrap = s.d / kBK;
-    q.bias = bias; q.noise = noise; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
-    q.gate = ws_ptr<float>(ws, p.gate); q.status = ws_ptr<int>(ws, p.status);
-    rc = launch_op<kRFwd>(tmA, tmB, q, st);
+    return launch_status();
   }
+  const int n_mtiles = (s.T + kTileM - 1) / kTileM;
+  RouterTcParams q{};
+  q.T = s.T; q.d = s.d; q.E = s.E; q.Epad64 = s.Epad64; q.mma_n = s.Epad64;
+  q.n_mtiles = n_mtiles; q.n_ntiles = 1; q.wrap = s.d / kBK;
+  q.bias = bias; q.noise = noise; q.probs = ws_ptr<float>(ws, p.probs); q.expert_index = ws_ptr<int>(ws, p.expert_index);
+  q.gate = ws_ptr<float>(ws, p.gate); q.status = ws_ptr<int>(ws, p.status);
+  const int rc = launch_op<kRFwd>(tmA, tmB, q, st);
   if (rc != SWITCH_MOE_OK) return rc;
-  // Eq. 6 partial sums: one row per block of tokens, reduced in a fixed order by the dispatch plan
-  const int rows = (s.T + s.router_blocks - 1) / s.router_blocks;
-  launch_k(probs_colsum_kernel, dim3(s.router_blocks), dim3(1024), 0, st, ws_ptr<float>(ws, p.probs), s.T, s.E, rows,
-                                                        ws_ptr<float>(ws, p.psum_partial));
+  // Eq. 6 partial sums: one row per 128 tokens, reduced in a fixed order by the dispatch plan
+  launch_k(probs_colsum_kernel, dim3(s.router_blocks), dim3(1024), 0, st, ws_ptr<float>(ws, p.probs), s.T, s.E, kTileM,
+           ws_ptr<float>(ws, p.psum_partial));
   return launch_status();
 }
 
@@ -749,6 +827,7 @@ int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const flo
   if (make_map(&tmA, x, 1, s.T, s.d, 64) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
   if (make_map(&tmB, dhsplit, 3, s.T, s.Epad64, 64) != SWITCH_MOE_OK) return SWITCH_MOE_CUDA_ERROR;
   q.mma_n = s.Epad64;
+  q.both_parts = s.Epad64 <= 128 ? 1 : 0;
   q.n_mtiles = (s.d + kTileM - 1) / kTileM; q.n_ntiles = 1;
   q.splits = s.dwr_chunks;
   q.total_kblocks = (s.T + kBK - 1) / kBK;

@@ -31,7 +31,8 @@ struct Shape {
   size_t elt;       // bytes per activation / expert-weight element
   int Epad;         // E rounded up to 32 * {1,2,4,8}
   int Epad64;       // E rounded up to a multiple of 64 (tensor-core router operands)
-  int router_tc;    // 1: router on the tensor cores (bf16 x, 3-way bf16 split of fp32 operands); 0: FP32 FMA
+  int router_tc;    // 1: router on the tensor cores (bf16 x, bf16 split of fp32 operands); 0: FP32 FMA
+  int router_hist;  // 1: the router's forward kernel also writes the dispatch plan's block histograms
   int router_blocks, plan_blocks, max_mtiles, dwr_chunks;
   int residual;     // 1: y = x + layer(x), dx = dy + d layer / dx (SWITCH_MOE_FLAG_RESIDUAL)
   int reroute;      // 1: overflowed tokens are offered to their second-choice expert (SWITCH_MOE_FLAG_REROUTE)
@@ -119,12 +120,12 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   s->Epad = 32 * ne_pow2;
   s->Epad64 = (cfg->E + 63) / 64 * 64;
   s->router_tc = s->gemm_path != 1 ? 1 : 0;
+  s->router_hist = (s->router_tc && s->Epad64 <= 128 && !s->top2) ? 1 : 0;
   s->plan_blocks = (s->Tv + kPlanBlockTokens - 1) / kPlanBlockTokens;
   s->max_mtiles = cfg->E * ((s->C + kTileM - 1) / kTileM);
   if (s->router_tc) {
     // dW_r split so that tiles x splits fills the GPU
-    s->router_blocks = (cfg->T + 255) / 256;                 // one partial P-sum row per 256 tokens, at most 256 rows
-    if (s->router_blocks > 256) s->router_blocks = 256;
+    s->router_blocks = 2 * ((cfg->T + 255) / 256);           // one partial P-sum row per 128-token tile (pairs of tiles)
     const int m_tiles = (cfg->d_model + kTileM - 1) / kTileM;
     const int k_blocks = (cfg->T + 63) / 64;
     int splits = 144 / m_tiles;
