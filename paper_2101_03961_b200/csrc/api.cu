@@ -322,7 +322,9 @@ int switch_moe_stage_launches(const switch_moe_config* cfg, int32_t* launches_ou
   // experts, the column sums of the probabilities (up to 128 experts the router kernel's epilogue leaves them, and
   // the plan's block histograms too); input jitter adds the element-wise product, top-2 routing the second-choice kernel.
   n[0] = (s.router_tc ? (s.Epad64 <= 128 ? 2 : 3) : 1) + (s.jitter ? 1 : 0) + (s.top2 ? 1 : 0);
-  n[1] = (s.router_hist ? 2 : 3) + (s.reroute ? 4 : 0);   // (histogram,) scan, assign; stage 2 of rerouting adds four
+  // plan: one fused kernel when the router left the histograms and there is one routing group; else (histogram,)
+  // scan, assign; stage 2 of rerouting adds four
+  n[1] = (s.router_hist ? (s.G == 1 ? 1 : 2) : 3) + (s.reroute ? 4 : 0);
   n[2] = 1;                                           // gather
   n[3] = 1 + (s.geglu ? 1 : 0) + (s.dropout ? 1 : 0); // GEMM1 (+ GEGLU gating, + expert dropout)
   n[4] = 1 + (s.top2 ? 1 : 0);                        // GEMM2 + combine (+ sum of the two assignments' rows)

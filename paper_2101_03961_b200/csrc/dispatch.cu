@@ -33,32 +33,49 @@ plan_hist_kernel(const int* __restrict__ expert_index, int T, int E, int* __rest
 __device__ __forceinline__ void write_tile_lists(const float* term, const int* kept_s, int E, float loss_scale,
                                                  float* __restrict__ aux_loss, int* __restrict__ tile_expert,
                                                  int* __restrict__ tile_row0, int4* __restrict__ ntile) {
-  __shared__ int start128[kMaxExperts + 1], startn[kMaxExperts + 1];
+  // Everything here is a sum or a running sum over the experts, done by the first kMaxExperts threads in log2 steps
+  // (a fixed tree, so the loss is the same number on every run): the loss terms, and the number of tiles before
+  // each expert in the two lists.
+  __shared__ int start128[kMaxExperts], startn[kMaxExperts];
+  __shared__ float lsum[kMaxExperts];
+  const int e = threadIdx.x;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    float s = 0.f;
-    for (int i = 0; i < E; ++i) s += term[i];
-    if (aux_loss != nullptr) *aux_loss = loss_scale * s;                              // Eq. 4
-    int n = 0, m = 0;
-    for (int i = 0; i < E; ++i) {
-      start128[i] = n; startn[i] = m;
-      n += (kept_s[i] + kTileM - 1) / kTileM;
-      m += (kept_s[i] + kPairTileTokens - 1) / kPairTileTokens;
-    }
+  int n128 = 0, npair = 0;
+  if (e < kMaxExperts) {
+    const int k = e < E ? kept_s[e] : 0;
+    n128 = (k + kTileM - 1) / kTileM;
+    npair = (k + kPairTileTokens - 1) / kPairTileTokens;
+    start128[e] = n128; startn[e] = npair;
+    lsum[e] = e < E ? term[e] : 0.f;
+  }
+  __syncthreads();
+  for (int off = 1; off < kMaxExperts; off <<= 1) {            // inclusive scans (counts), pairwise tree (loss)
+    int a = 0, b = 0;
+    float c = 0.f;
+    const bool scan = e < kMaxExperts && e >= off;
+    const bool tree = e < kMaxExperts && (e & (2 * off - 1)) == 0 && e + off < kMaxExperts;
+    if (scan) { a = start128[e - off]; b = startn[e - off]; }
+    if (tree) c = lsum[e + off];
+    __syncthreads();
+    if (scan) { start128[e] += a; startn[e] += b; }
+    if (tree) lsum[e] += c;
+    __syncthreads();
+  }
+  if (e == 0) {
+    if (aux_loss != nullptr) *aux_loss = loss_scale * lsum[0];                        // Eq. 4
+    const int n = start128[kMaxExperts - 1], m = startn[kMaxExperts - 1];
     tile_expert[0] = n;
     tile_row0[0] = n;
     ntile[0] = make_int4(m, 0, 0, 0);
   }
-  __syncthreads();
-  const int e = threadIdx.x;
   if (e < E) {
     const int k = kept_s[e];
-    int n = start128[e];
+    int n = start128[e] - n128;                                // tiles of earlier experts
     for (int r = 0; r < k; r += kTileM, ++n) { tile_expert[1 + n] = e; tile_row0[1 + n] = r; }
     if (k > 0) {
-      const int pieces = (k + kPairTileTokens - 1) / kPairTileTokens;
+      const int pieces = npair;
       const int rows = ((k + pieces - 1) / pieces + 15) / 16 * 16;
-      int m = startn[e];
+      int m = startn[e] - npair;
       for (int r = 0; r < k; r += rows, ++m) ntile[1 + m] = make_int4(e, r, min(rows, (k - r + 15) / 16 * 16), 0);
     }
   }
@@ -227,6 +244,111 @@ plan_assign_kernel(const int* __restrict__ expert_index, const int* __restrict__
   for (int s = blockIdx.x * blockDim.x + tid; s < total; s += gridDim.x * blockDim.x) {
     const int ex = s / C, pos = s - ex * C;
     if (pos >= kept[ex]) token_of_slot[s] = -1;
+  }
+}
+
+// The whole plan in one launch, for one routing group whose block histograms already exist (the tensor-core router's
+// forward kernel leaves hist[r][e] = tokens of the r-th block of 256 tokens routed to expert e).  Every block of 1024
+// tokens adds up the histogram columns itself -- all rows for the totals (kept_i = min(count_i, C), Eq. 3), the rows
+// before its own tokens for its position base -- instead of waiting for a scan kernel: the table is small (64 KB at
+// 128 x 128) and stays in L2.  Then, as in plan_assign_kernel, pos_t = base + (tokens of earlier warps with the same
+// expert) + (earlier lanes with it), in token order, with no atomics deciding a position.  One extra block writes the
+// counts, the P-sums, the auxiliary loss (Eq. 4-6) and the tile lists.
+constexpr int kFusedTokens = 1024;
+__global__ void __launch_bounds__(kFusedTokens)
+plan_fused_kernel(const int* __restrict__ expert_index, const int* __restrict__ hist, int hist_rows,
+                  const float* __restrict__ psum_partial, int router_blocks, int T, int E, int Ew, int C, float alpha,
+                  int* __restrict__ slot, int* __restrict__ token_of_slot, int* __restrict__ count,
+                  int* __restrict__ kept, float* __restrict__ psum, float* __restrict__ aux_loss,
+                  int* __restrict__ tile_expert, int* __restrict__ tile_row0, int4* __restrict__ ntile,
+                  int* __restrict__ count_g, int* __restrict__ group_base) {
+  pdl_launch_dependents();
+  pdl_wait();
+  __shared__ int part_pre[kFusedTokens], part_tot[kFusedTokens];    // [slice][column]; the extra block keeps floats here
+  __shared__ int base_s[kMaxExperts], kept_s[kMaxExperts];
+  __shared__ float term[kMaxExperts];
+  constexpr int kWarps = kFusedTokens / 32;
+  __shared__ int warp_cnt[kMaxExperts][kWarps];                // [expert][warp of the block]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_token_blocks = (int)gridDim.x - 1;
+  const bool summary = (int)blockIdx.x == n_token_blocks;
+  const int Q = kFusedTokens / Ew, q = tid / Ew, e = tid % Ew;
+  const int row_end = summary ? hist_rows : min(hist_rows, (int)blockIdx.x * (kFusedTokens / kPlanBlockTokens));
+  int pre = 0, tot = 0;
+  if (e < E) {
+    for (int r0 = q; r0 < hist_rows; r0 += 8 * Q) {
+      int v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = r0 + j * Q < hist_rows ? hist[(size_t)(r0 + j * Q) * E + e] : 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { tot += v[j]; if (r0 + j * Q < row_end) pre += v[j]; }
+    }
+  }
+  part_pre[tid] = pre;
+  part_tot[tid] = tot;
+  for (int i = tid; i < kWarps * kMaxExperts; i += kFusedTokens) (&warp_cnt[0][0])[i] = 0;
+  __syncthreads();
+  int total = 0;
+  if (tid < E) {
+    int b = 0;
+    for (int k = 0; k < Q; ++k) { b += part_pre[k * Ew + tid]; total += part_tot[k * Ew + tid]; }
+    base_s[tid] = b;
+    kept_s[tid] = min(total, C);
+  }
+  __syncthreads();
+  if (summary) {
+    // P-sums in a fixed order (slice by slice, rows ascending inside a slice), then the loss and the tile lists
+    float* part_ps = reinterpret_cast<float*>(part_pre);
+    float ps = 0.f;
+    if (e < E)
+      for (int r = q; r < router_blocks; r += Q) ps += psum_partial[(size_t)r * E + e];
+    __syncthreads();
+    part_ps[tid] = ps;
+    __syncthreads();
+    if (tid < E) {
+      float sum = 0.f;
+      for (int k = 0; k < Q; ++k) sum += part_ps[k * Ew + tid];
+      count[tid] = total;                                                              // f counts the argmax (Eq. 5)
+      count_g[tid] = total;
+      group_base[tid] = 0;
+      kept[tid] = kept_s[tid];
+      psum[tid] = sum;
+      term[tid] = ((float)total / (float)T) * (sum / (float)T);                        // f_i . P_i  (Eq. 5, 6)
+    }
+    write_tile_lists(term, kept_s, E, alpha * (float)E, aux_loss, tile_expert, tile_row0, ntile);
+    return;
+  }
+  const int t = (int)blockIdx.x * kFusedTokens + tid;
+  int et = t < T ? expert_index[t] : -1;                      // negative: no expert (takes no slot)
+  if (et >= E) et = -1;
+  const unsigned same = __match_any_sync(0xffffffffu, et >= 0 ? et : -1 - lane);   // distinct dummies for those lanes
+  const int rank = __popc(same & ((1u << lane) - 1u));
+  if (et >= 0 && rank == 0) warp_cnt[et][warp] = __popc(same);
+  __syncthreads();
+  for (int ex = warp; ex < E; ex += kWarps) {                  // exclusive scan over the block's warps, per expert
+    const int c = warp_cnt[ex][lane];
+    int incl = c;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += up;
+    }
+    warp_cnt[ex][lane] = incl - c;
+  }
+  __syncthreads();
+  if (t < T) {
+    int sl = -1;
+    if (et >= 0) {
+      const int pos = base_s[et] + warp_cnt[et][warp] + rank;
+      if (pos < C) { sl = et * C + pos; token_of_slot[sl] = t; }
+    }
+    slot[t] = sl;
+  }
+  // empty slots of every expert: -1 (disjoint from the kept slots written above)
+  const int total_slots = E * C;
+  for (int sidx = (int)blockIdx.x * kFusedTokens + tid; sidx < total_slots; sidx += n_token_blocks * kFusedTokens) {
+    const int ex = sidx / C, pos = sidx - ex * C;
+    if (pos >= kept_s[ex]) token_of_slot[sidx] = -1;
   }
 }
 
@@ -503,6 +625,8 @@ gather_dy_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ y, cons
 
 }  // namespace
 
+int launch_reroute(const Shape& s, const Plan& p, void* ws, cudaStream_t st);
+
 int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_index, float* aux_loss, void* ws,
                          cudaStream_t st) {
   int* ei = ws_ptr<int>(ws, p.expert_index);
@@ -512,6 +636,18 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
   }
   // the tensor-core router's forward kernel leaves the histograms of its own expert choices in the workspace
   const bool have_hist = expert_index == nullptr && s.router_hist;
+  if (have_hist && s.G == 1) {
+    int Ewf = 32;
+    while (Ewf < s.E) Ewf *= 2;
+    const int token_blocks = (s.T + kFusedTokens - 1) / kFusedTokens;
+    launch_k(plan_fused_kernel, dim3(token_blocks + 1), dim3(kFusedTokens), 0, st, ei, ws_ptr<int>(ws, p.hist),
+             s.plan_blocks, ws_ptr<float>(ws, p.psum_partial), s.router_blocks, s.T, s.E, Ewf, s.Cg, s.alpha,
+             ws_ptr<int>(ws, p.slot), ws_ptr<int>(ws, p.token_of_slot), ws_ptr<int>(ws, p.count),
+             ws_ptr<int>(ws, p.kept), ws_ptr<float>(ws, p.psum), aux_loss, ws_ptr<int>(ws, p.tile_expert),
+             ws_ptr<int>(ws, p.tile_row0), ws_ptr<int4>(ws, p.ntile), ws_ptr<int>(ws, p.count_g),
+             ws_ptr<int>(ws, p.group_base));
+    return launch_reroute(s, p, ws, st);
+  }
   if (!have_hist)
     launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, s.Tv, s.E, ws_ptr<int>(ws, p.hist));
   int Ew = 32;
@@ -537,6 +673,12 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
   launch_k(plan_assign_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, ei, ws_ptr<int>(ws, p.hist_base),
            ws_ptr<int>(ws, p.kept), group_base, blocks_per_group, s.Tv, s.E, s.C, s.Cg, ws_ptr<int>(ws, p.slot),
            ws_ptr<int>(ws, p.token_of_slot));
+  return launch_reroute(s, p, ws, st);
+}
+
+// Stage 2 of No-Token-Left-Behind routing, after either form of the first-stage plan.
+int launch_reroute(const Shape& s, const Plan& p, void* ws, cudaStream_t st) {
+  int* ei = ws_ptr<int>(ws, p.expert_index);
   if (s.reroute) {
     int* alt = ws_ptr<int>(ws, p.alt);
     launch_k(reroute_choice_kernel, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs), ei,

@@ -89,7 +89,7 @@ def test_launch_count_is_reported(lib):
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, dtype=sm.F32)) == 16
     # bf16 default path: the router's epilogue leaves the probabilities' column sums and the plan's histograms, and the
     # two products of dH share one launch
-    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 15
+    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 14
     # options add launches: four plan kernels for rerouting, one product kernel for input jitter, two GEGLU gating kernels
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, reroute=True, input_jitter=True,
-                                                          geglu=True, expert_dropout=0.4)) == 15 + 4 + 1 + 2 + 2
+                                                          geglu=True, expert_dropout=0.4)) == 14 + 4 + 1 + 2 + 2
