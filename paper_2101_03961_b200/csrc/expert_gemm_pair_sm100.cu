@@ -70,7 +70,14 @@ struct PairParams {
   __nv_bfloat16* out2;        // combine with the skip path: second copy of the output without it
   int plain;                  // GEMM1 / dgrad2 without ReLU and without the ReLU mask (GEGLU experts gate elsewhere)
   int stages, stage_bytes;    // operand ring: token products size a stage for the widest tile the capacity allows
+  // ceil(2^32 / divisor) for the three divisions of the tile decode (n_mpairs; n_mpairs * n_ntiles_fixed;
+  // n_ntiles_fixed): id / d = umulhi(id, magic) as long as id * d < 2^32
+  uint32_t magic_mpairs, magic_per_e, magic_nt;
 };
+
+__device__ __forceinline__ int fast_div(int id, uint32_t magic, int divisor) {
+  return divisor == 1 ? id : (int)__umulhi((uint32_t)id, magic);
+}
 
 // Token products: the token operand's TMA box is exactly this CTA's share of the tile (n / 2 rows, a multiple of 8):
 // one tensor map per height 8, 16, .., 128.  Weight gradients use entry 0 (a 64-row box of the token contraction).
@@ -88,7 +95,7 @@ struct PTile {
 __device__ __forceinline__ PTile p_decode(const PairParams& p, int id, const int* kept_s, const int4* tile_s) {
   PTile t;
   if (p.token_op) {
-    const int nt = id / p.n_mpairs;
+    const int nt = fast_div(id, p.magic_mpairs, p.n_mpairs);
     const int4 q = nt < kPTileCache ? tile_s[nt] : p.ntile[1 + nt];
     t.e = q.x; t.row0 = q.y; t.n = q.z; t.n0 = 0;
     t.n1 = t.n <= 256 ? t.n : ((t.n >> 1) + 15) & ~15;         // two segments: both multiples of 16, both <= 256
@@ -97,9 +104,9 @@ __device__ __forceinline__ PTile p_decode(const PairParams& p, int id, const int
     t.last_mmas = kBK / kUmmaK;
   } else {
     const int per_e = p.n_mpairs * p.n_ntiles_fixed;
-    t.e = id / per_e;
+    t.e = fast_div(id, p.magic_per_e, per_e);
     const int rem = id - t.e * per_e;
-    const int mp = rem / p.n_ntiles_fixed;
+    const int mp = fast_div(rem, p.magic_nt, p.n_ntiles_fixed);
     t.m0 = mp * 256;
     t.n0 = (rem - mp * p.n_ntiles_fixed) * 256;
     t.row0 = 0; t.n = 256; t.n1 = 256;
@@ -704,6 +711,17 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
   q.stages = kPRingBytes / q.stage_bytes < kPMaxStages ? kPRingBytes / q.stage_bytes : kPMaxStages;
   q.n_ntiles_fixed = q.token_op ? 0 : (q.Nfix + 255) / 256;
   q.k_blocks_fixed = q.token_op ? K / kBK : 0;
+  auto magic = [](int d) { return d > 1 ? (uint32_t)((0x100000000ull + (uint64_t)d - 1) / (uint64_t)d) : 0u; };
+  q.magic_mpairs = magic(q.n_mpairs);
+  q.magic_per_e = magic(q.n_mpairs * (q.n_ntiles_fixed > 0 ? q.n_ntiles_fixed : 1));
+  q.magic_nt = magic(q.n_ntiles_fixed > 0 ? q.n_ntiles_fixed : 1);
+  // the decode's divisions are exact only while id * divisor < 2^32: ids are below E * 16 * n_mpairs * n_ntiles
+  {
+    const uint64_t ids = q.token_op ? (uint64_t)s.max_mtiles * q.n_mpairs
+                                    : (uint64_t)s.E * q.n_mpairs * (q.n_ntiles_fixed > 0 ? q.n_ntiles_fixed : 1);
+    if (ids * (uint64_t)(q.n_mpairs * (q.n_ntiles_fixed > 0 ? q.n_ntiles_fixed : 1)) >= 0x100000000ull)
+      return SWITCH_MOE_UNSUPPORTED_SHAPE;
+  }
   *out = q;
   return SWITCH_MOE_OK;
 }
