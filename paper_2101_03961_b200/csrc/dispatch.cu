@@ -300,8 +300,15 @@ plan_fused_kernel(const int* __restrict__ expert_index, const int* __restrict__ 
     // P-sums in a fixed order (slice by slice, rows ascending inside a slice), then the loss and the tile lists
     float* part_ps = reinterpret_cast<float*>(part_pre);
     float ps = 0.f;
-    if (e < E)
-      for (int r = q; r < router_blocks; r += Q) ps += psum_partial[(size_t)r * E + e];
+    if (e < E) {
+      for (int r0 = q; r0 < router_blocks; r0 += 16 * Q) {      // 16 rows in flight, added in row order
+        float v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = r0 + j * Q < router_blocks ? psum_partial[(size_t)(r0 + j * Q) * E + e] : 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) ps += v[j];
+      }
+    }
     __syncthreads();
     part_ps[tid] = ps;
     __syncthreads();

@@ -432,12 +432,12 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // staged k-block of W_r, so the weight parts cross shared memory once per 256 tokens -- and those 256 tokens are
 // exactly one block of the dispatch plan.  The epilogue (one token per thread: a TMEM lane holds all E logits of a
 // token) therefore also produces what the plan needs from the router: the block's histogram of expert choices
-// (Section 2.2: the counts behind Eq. 3's capacity cut and Eq. 5's f) and, per 128-token tile, the column sums of the
+// (Section 2.2: the counts behind Eq. 3's capacity cut and Eq. 5's f) and the block's column sums of the
 // probabilities (Eq. 6's P), both in a fixed order.
 struct RouterFwdParams {
   int T, d, E, Epad64, n_ptiles, k_blocks, b_atoms, stages, stage_bytes;
   const float* bias; const float* noise; float* probs; int* expert_index; float* gate;
-  float* psum_partial;       // [2 n_ptiles][E]: column sums of p over each 128-token tile
+  float* psum_partial;       // [n_ptiles][E]: column sums of p over each block of 256 tokens
   int* hist;                 // [n_ptiles][E]: tokens of each 256-token block per expert
   int* status;
 };
@@ -676,13 +676,15 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
       for (int c = 0; c < NCH; ++c) sums[c * 32 + lane] = colsum[c];
       asm volatile("bar.sync 1, 256;" ::: "memory");          // the eight epilogue warps: histogram and column sums complete
-      if (lg == 0) {                                          // the tile's four warps' sums, added in warp order
-        const float* t0 = reinterpret_cast<const float*>(smem_gen + kRFRingBytes) + (ti * 4) * (NCH * 32);
+      if (warp == 2) {                                        // the eight warps' sums, added in warp order
+        const float* t0 = reinterpret_cast<const float*>(smem_gen + kRFRingBytes);
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const int e = c * 32 + lane;
-          const float v = ((t0[e] + t0[NCH * 32 + e]) + t0[2 * NCH * 32 + e]) + t0[3 * NCH * 32 + e];
-          if (e < p.E) p.psum_partial[(size_t)(2 * id + ti) * p.E + e] = v;
+          float v = t0[e];
+#pragma unroll
+          for (int w = 1; w < 8; ++w) v += t0[w * (NCH * 32) + e];
+          if (e < p.E) p.psum_partial[(size_t)id * p.E + e] = v;
         }
       }
       if (et < p.E) {
@@ -803,8 +805,8 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
   q.gate = ws_ptr<float>(ws, p.gate); q.status = ws_ptr<int>(ws, p.status);
   const int rc = launch_op<kRFwd>(tmA, tmB, q, st);
   if (rc != SWITCH_MOE_OK) return rc;
-  // Eq. 6 partial sums: one row per 128 tokens, reduced in a fixed order by the dispatch plan
-  launch_k(probs_colsum_kernel, dim3(s.router_blocks), dim3(1024), 0, st, ws_ptr<float>(ws, p.probs), s.T, s.E, kTileM,
+  // Eq. 6 partial sums: one row per 256 tokens, reduced in a fixed order by the dispatch plan
+  launch_k(probs_colsum_kernel, dim3(s.router_blocks), dim3(1024), 0, st, ws_ptr<float>(ws, p.probs), s.T, s.E, 2 * kTileM,
            ws_ptr<float>(ws, p.psum_partial));
   return launch_status();
 }

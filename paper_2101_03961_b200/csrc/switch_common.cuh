@@ -125,7 +125,7 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   s->max_mtiles = cfg->E * ((s->C + kTileM - 1) / kTileM);
   if (s->router_tc) {
     // dW_r split so that tiles x splits fills the GPU
-    s->router_blocks = 2 * ((cfg->T + 255) / 256);           // one partial P-sum row per 128-token tile (pairs of tiles)
+    s->router_blocks = (cfg->T + 255) / 256;                 // one partial P-sum row per block of 256 tokens
     const int m_tiles = (cfg->d_model + kTileM - 1) / kTileM;
     const int k_blocks = (cfg->T + 63) / 64;
     int splits = 144 / m_tiles;
