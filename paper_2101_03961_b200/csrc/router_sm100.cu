@@ -23,7 +23,10 @@ constexpr int kRTcThreads = 320;                     // generic kernel: TMA warp
 constexpr int kRTcOutStageBytes = 8 * 32 * 128;
 constexpr int kRTcSmemBytes = 1024 + kStages * kStageBytes + kRTcOutStageBytes + 128;
 
-enum RouterOp { kRFwd = 0, kRDwr = 1, kRDx = 2 };
+// kRDxRes: dx with the two parts of one 256-row block of W_r resident in shared memory for the CTA's whole life
+// (up to 128 experts): only the logit gradients stream, and every staged block of them meets the W_r parts it pairs
+// with in the three cross terms without a reload.
+enum RouterOp { kRFwd = 0, kRDwr = 1, kRDx = 2, kRDxRes = 3 };
 
 struct RouterTcParams {
   int T, d, E, Epad64;
@@ -46,6 +49,7 @@ template <int OP>
 __device__ __forceinline__ int r_total_tiles(const RouterTcParams& p) {
   if (OP == kRFwd) return p.n_mtiles;
   if (OP == kRDwr) return p.n_mtiles * p.splits;
+  if (OP == kRDxRes) return p.n_mtiles;
   return p.n_mtiles * p.n_ntiles;
 }
 
@@ -61,6 +65,10 @@ __device__ __forceinline__ RTile r_decode(const RouterTcParams& p, int id) {
     t.m0 = mt * kTileM;
     t.k_base = t.split * p.chunk_kblocks;
     t.wrap = max(0, min(p.chunk_kblocks, p.total_kblocks - t.k_base));
+  } else if (OP == kRDxRes) {                         // id = token tile; the CTA's block of W_r rows is fixed
+    t.m0 = id * kTileM;
+    t.n0 = (int)(blockIdx.x % (unsigned)p.n_ntiles) * kBN;
+    t.wrap = p.wrap;
   } else {
     const int mt = id / p.n_ntiles;
     t.m0 = mt * kTileM;
@@ -69,7 +77,7 @@ __device__ __forceinline__ RTile r_decode(const RouterTcParams& p, int id) {
   }
   // forward: W_r = hi + mid, one part after the other; dW_r: dh = hi + mid, both parts staged with the x block they
   // multiply when they fit (up to 128 experts), else one after the other; dx: three cross terms
-  t.k_blocks = (OP == kRDx ? 3 : (OP == kRDwr && p.both_parts) ? 1 : 2) * t.wrap;
+  t.k_blocks = (OP == kRDx ? 3 : (OP == kRDwr && p.both_parts) ? 1 : 2) * t.wrap;   // kRDxRes: hi and mid of dh
   return t;
 }
 
@@ -78,7 +86,8 @@ __global__ void __launch_bounds__(kRTcThreads, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const RouterTcParams p) {
   constexpr bool kAMn = (OP == kRDwr);                 // x^T: token rows are the contraction, d contiguous
-  constexpr bool kBMn = (OP != kRDx);                  // fwd: W [d][E]; dwr: dh [T][E]; dx: W as [d rows][E contiguous]
+  constexpr bool kDx = (OP == kRDx || OP == kRDxRes);
+  constexpr bool kBMn = !kDx;                          // fwd: W [d][E]; dwr: dh [T][E]; dx: W as [d rows][E contiguous]
   pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -91,11 +100,19 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
   volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kStages + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kStages + 4) + 4);
+  const uint32_t wfull_bar = bar_base + 8u * (2 * kStages + 5);     // kRDxRes: the resident W_r parts have landed
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // kRDxRes: the operand ring's first 64 KB are four 16 KB stages of logit-gradient blocks, the rest holds the
+  // resident W_r parts: [part][k-block] blocks of 256 rows x 64 experts (32 KB each)
+  const uint32_t w_res = smem_base + kStages * kABytes;
+  // tiles of this CTA: kRDxRes deals token tiles out among the CTAs that share a block of W_r rows
+  const int tile_first = OP == kRDxRes ? (int)(blockIdx.x / (unsigned)p.n_ntiles) : (int)blockIdx.x;
+  const int tile_step = OP == kRDxRes ? (int)(gridDim.x / (unsigned)p.n_ntiles) : (int)gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
+    mbar_init(wfull_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -120,12 +137,25 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+      if (OP == kRDxRes) {                                    // W_r parts hi, mid of this CTA's 256 rows, once
+        const int n0 = (int)(blockIdx.x % (unsigned)p.n_ntiles) * kBN;
+        mbar_arrive_expect_tx(wfull_bar, 2u * (uint32_t)p.wrap * kBBytes);
+        for (int part = 0; part < 2; ++part)
+          for (int kk = 0; kk < p.wrap; ++kk)
+            tma_load_3d(w_res + (uint32_t)(part * p.wrap + kk) * kBBytes, &tmB, wfull_bar, kk * kBK, n0, part);
+      }
+      for (int id = tile_first; id < n_tiles && ok; id += tile_step) {
         const RTile t = r_decode<OP>(p, id);
         for (int kb = 0; kb < t.k_blocks; ++kb) {
           const int part = kb / t.wrap, kblk = t.k_base + (kb - part * t.wrap);
           ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 11);
           if (!ok) break;
+          if (OP == kRDxRes) {                                // dh part [128 tok][64 e] only
+            mbar_arrive_expect_tx(full_bar(stage), kABytes);
+            tma_load_3d(smem_base + stage * kABytes, &tmA, full_bar(stage), kblk * kBK, t.m0, part);
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           const uint32_t a_dst = smem_base + stage * kStageBytes, b_dst = a_dst + kABytes;
           mbar_arrive_expect_tx(full_bar(stage), stage_tx);
           if (OP == kRFwd) {
@@ -163,7 +193,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+      if (OP == kRDxRes) ok = mbar_wait(wfull_bar, 0u, abort_flag, p.status, 15);
+      for (int id = tile_first; id < n_tiles && ok; id += tile_step) {
         const RTile t = r_decode<OP>(p, id);
         ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 12);
         if (!ok) break;
@@ -173,6 +204,24 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, 13);
           if (!ok) break;
           tc_fence_after();
+          if (OP == kRDxRes) {
+            // staged block: part `dpart` of dh, experts 64 kk .. 64 kk + 63.  dh_hi meets W_hi and W_mid, dh_mid meets W_hi.
+            const int dpart = kb / t.wrap, kk = kb - dpart * t.wrap;
+            const uint32_t a_src = smem_base + stage * kABytes;
+            const int n_w = dpart == 0 ? 2 : 1;
+            for (int wp = 0; wp < n_w; ++wp) {
+              const uint32_t b_src = w_res + (uint32_t)(wp * t.wrap + kk) * kBBytes;
+#pragma unroll
+              for (int ks = 0; ks < kBK / kUmmaK; ++ks) {
+                const uint64_t ad = make_smem_desc(a_src + ks * a_kstep, a_lbo, 1024u);
+                const uint64_t bd = make_smem_desc(b_src + ks * b_kstep, b_lbo, 1024u);
+                tc_mma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || wp > 0 || ks > 0) ? 1u : 0u);
+              }
+            }
+            tc_commit(empty_bar(stage));
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           const uint32_t a_src = smem_base + stage * kStageBytes, b_src = a_src + kABytes;
 #pragma unroll
           for (int ks = 0; ks < kBK / kUmmaK; ++ks) {
@@ -204,13 +253,13 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+    for (int id = tile_first; id < n_tiles && ok; id += tile_step) {
       const RTile t = r_decode<OP>(p, id);
       const int r = lg * 32 + lane;
       // dx: previous contents of the rows this thread will write (prefetched before the accumulator is ready)
       long long offs[8];
       unsigned add_mask = 0;
-      if (OP == kRDx) {
+      if (kDx) {
         const int tok = t.m0 + r;
         const long long row_off = tok < p.T ? (long long)tok * p.d : -1;
         const int add = (p.accumulate && tok < p.T && (p.accumulate == 2 || p.slot[tok] >= 0)) ? 1 : 0;
@@ -753,11 +802,12 @@ int sm_count_or_default() {
 }
 
 template <int OP>
-int launch_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const RouterTcParams& q, cudaStream_t st) {
+int launch_op(const CUtensorMap& tmA, const CUtensorMap& tmB, const RouterTcParams& q, cudaStream_t st, int grid = 0) {
   if (cudaFuncSetAttribute(router_tc_kernel<OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRTcSmemBytes) !=
       cudaSuccess)
     return SWITCH_MOE_CUDA_ERROR;
-  launch_k(router_tc_kernel<OP>, dim3(sm_count_or_default()), dim3(kRTcThreads), kRTcSmemBytes, st, tmA, tmB, q);
+  launch_k(router_tc_kernel<OP>, dim3(grid > 0 ? grid : sm_count_or_default()), dim3(kRTcThreads), kRTcSmemBytes, st,
+           tmA, tmB, q);
   return launch_status();
 }
 
@@ -845,6 +895,10 @@ int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const flo
   q.wrap = s.Epad64 / kBK;
   q.dx = static_cast<__nv_bfloat16*>(dx); q.slot = ws_ptr<int>(ws, p.slot); q.accumulate = accumulate_dx ? ((s.residual || s.top2) ? 2 : 1) : 0;   // 2: every row already holds a value
   q.jitter_u = static_cast<const __nv_bfloat16*>(s.jitter_u);
+  // up to 128 experts the two parts of a 256-row block of W_r (at most 128 KB) stay in shared memory: the CTAs are
+  // dealt out evenly over the row blocks and each walks its share of the token tiles
+  const int sms = sm_count_or_default();
+  if (s.Epad64 <= 128 && sms >= q.n_ntiles) return launch_op<kRDxRes>(tmA, tmB, q, st, sms / q.n_ntiles * q.n_ntiles);
   return launch_op<kRDx>(tmA, tmB, q, st);
 }
 
