@@ -437,7 +437,9 @@ def run_ours(args, cfg):
         reps.close()
         return
 
-    kept = int(sm.switch_moe_workspace_view(mcfg, ws, sm.WS_KEPT).sum().item())
+    kept_per_expert = sm.switch_moe_workspace_view(mcfg, ws, sm.WS_KEPT)
+    kept = int(kept_per_expert.sum().item())
+    busy = float((kept_per_expert > 0).sum().item()) / cfg.E   # experts without tokens: their weights are never read
     peaks, peak_kind = load_peaks()
     hbm = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
     elt = 2 if cfg.dtype == si.DTYPE_BF16 else 4
@@ -450,16 +452,18 @@ def run_ours(args, cfg):
         gemm_weight.update({"gemm1_relu": 2.0, "dgrad1_scatter": 2.0, "wgrad1": 2.0})
     flops_unit = 2.0 * kept * cfg.d_model * cfg.d_ff
     flops_per_launch = flops_unit * sum(gemm_weight.values()) / 6.0
-    # Algorithmic DRAM bytes of one product, mean over the six: its expert weights once (read, or written for a
-    # weight gradient) and its two activation operands once, over kept rows only (d-wide rows: X_d, dY_d, y, dx;
+    # Algorithmic DRAM bytes of one product, mean over the six: its expert weights once (read -- only of experts
+    # that kept a token -- or written for a weight gradient: every expert's, zeros included) and its two activation
+    # operands once, over kept rows only (d-wide rows: X_d, dY_d, y, dx;
     # f-wide rows: H, dH), plus the one-bit ReLU mask written by GEMM1 and read by dgrad2.
     fin = cfg.d_ff * (2 if cfg.geglu else 1)
     w_in_b, w_out_b = cfg.E * cfg.d_model * fin * elt, cfg.E * cfg.d_ff * cfg.d_model * elt
     rows_d, rows_f, rows_fin = kept * cfg.d_model * elt, kept * cfg.d_ff * elt, kept * fin * elt
     mask_b = 0 if cfg.geglu else kept * cfg.d_ff // 8
-    algo_bytes = {"gemm1_relu": w_in_b + rows_d + rows_fin + mask_b, "gemm2_combine": w_out_b + rows_f + rows_d,
-                  "dgrad2_mask": w_out_b + rows_d + rows_f + mask_b, "wgrad2": w_out_b + rows_f + rows_d,
-                  "dgrad1_scatter": w_in_b + rows_fin + rows_d, "wgrad1": w_in_b + rows_d + rows_fin}
+    algo_bytes = {"gemm1_relu": busy * w_in_b + rows_d + rows_fin + mask_b,
+                  "gemm2_combine": busy * w_out_b + rows_f + rows_d,
+                  "dgrad2_mask": busy * w_out_b + rows_d + rows_f + mask_b, "wgrad2": w_out_b + rows_f + rows_d,
+                  "dgrad1_scatter": busy * w_in_b + rows_fin + rows_d, "wgrad1": w_in_b + rows_d + rows_fin}
     traffic_algorithmic = sum(algo_bytes.values()) / 6.0
     captured = load_captured_traffic(cfg)
 
