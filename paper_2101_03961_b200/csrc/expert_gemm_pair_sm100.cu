@@ -38,7 +38,9 @@ constexpr int kPMaxStages = 8;                         // token products: as man
 constexpr int kPHalfBytes = 16384;                     // A tile (128 x 64) and B half tile (<= 128 x 64)
 constexpr int kPStageBytes = 2 * kPHalfBytes;
 constexpr int kPRingBytes = kPStages * kPStageBytes;   // 192 KB of operand stages
-constexpr int kPTransBytes = 8 * 2048;                 // 8 epilogue warps x (32 x 64 B)
+constexpr int kPTransWarp = 16 * 144;                  // per epilogue warp: 16 token pairs x (32 weight rows x 4 B, padded
+                                                       // to 144 B so that 16-byte reads of 8 rows do not collide)
+constexpr int kPTransBytes = 8 * kPTransWarp;
 constexpr int kPAuxBytes = 8 * 128;                    // 8 epilogue warps x 32 gates
 constexpr int kPKeptCache = kMaxExperts;                 // kept[e] for every expert
 constexpr int kPTileCache = 448;                        // first token tiles of the list ({expert, row, rows})
@@ -334,7 +336,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
     // ------------------------------------------------------------------------------------------ epilogue warps (both CTAs)
     const int lg = warp & 3;
     const int half = (warp - 2) >> 2;
-    uint8_t* tr = trans_gen + (warp - 2) * 2048;              // this warp's 32 x 64 B transpose tile
+    uint8_t* tr = trans_gen + (warp - 2) * kPTransWarp;       // this warp's transpose tile
     float* gate_s = reinterpret_cast<float*>(aux_gen + (warp - 2) * 128);
     uint32_t it = 0;
     bool ok = true;
@@ -477,12 +479,17 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
             released = true;
           }
           {
+            // Store `st` of this lane writes weight rows mcol .. mcol + 7 of token column tcol(st) of the chunk:
+            // eight lanes' token pairs x four row groups per instruction.
+            auto tcol = [&](int st) { return 16 * (st >> 1) + 2 * (lane >> 2) + (st & 1); };
             long long offs[4];
 #pragma unroll
-            for (int st = 0; st < 4; ++st) offs[st] = __shfl_sync(0xffffffffu, q_off[0], st * 8 + (lane >> 2));
+            for (int st = 0; st < 4; ++st) offs[st] = __shfl_sync(0xffffffffu, q_off[0], tcol(st));
             if (OP == kGemm2Combine) gate_s[lane] = q_gate[0];
             __syncwarp();
-            // transpose: this lane holds weight row m_warp + lane for 32 tokens -> tr[token][lane]
+            // transpose: this lane holds weight row m_warp + lane for 32 tokens.  Two tokens are packed into one
+            // 32-bit word, tr[token pair][lane]: half the shared-memory stores of a 16-bit layout, each a full
+            // 128-byte wavefront; a reader takes the words of eight rows (32 bytes) and separates the two tokens.
 #pragma unroll
             for (int i4 = 0; i4 < 32; i4 += 4) {
               float g[4] = {1.f, 1.f, 1.f, 1.f};
@@ -490,58 +497,69 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
                 const float4 g4 = *reinterpret_cast<const float4*>(gate_s + i4);
                 g[0] = g4.x; g[1] = g4.y; g[2] = g4.z; g[3] = g4.w;
               }
+              float a[4];
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
-                float a = __uint_as_float(v[i4 + u]);
-                if (OP == kGemm2Combine) a *= g[u];
-                if (OP == kGemm1Relu && !p.plain) a = fmaxf(a, 0.f);
-                *reinterpret_cast<__nv_bfloat16*>(tr + (i4 + u) * 64 + lane * 2) = __float2bfloat16(a);
+                a[u] = __uint_as_float(v[i4 + u]);
+                if (OP == kGemm2Combine) a[u] *= g[u];
+                if (OP == kGemm1Relu && !p.plain) a[u] = fmaxf(a[u], 0.f);
               }
+              *reinterpret_cast<__nv_bfloat162*>(tr + (i4 >> 1) * 144 + lane * 4) = __floats2bfloat162_rn(a[0], a[1]);
+              *reinterpret_cast<__nv_bfloat162*>(tr + ((i4 >> 1) + 1) * 144 + lane * 4) = __floats2bfloat162_rn(a[2], a[3]);
             }
             __syncwarp();
             uint32_t mword[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int st = 0; st < 4; ++st) {
-              const int rr = st * 8 + (lane >> 2);
-              uint4 val = *reinterpret_cast<const uint4*>(tr + rr * 64 + (lane & 3) * 16);
-              if (OP == kDgrad2Mask && !p.plain) {              // ReLU'(u) = [u > 0]: bits saved by the forward GEMM
-                const uint32_t bits = __shfl_sync(0xffffffffu, q_mw[0], rr) >> ((lane & 3) * 8);
-                uint32_t* w = reinterpret_cast<uint32_t*>(&val);
+            for (int pass = 0; pass < 2; ++pass) {
+              const uint8_t* src = tr + (8 * pass + (lane >> 2)) * 144 + (lane & 3) * 32;
+              const uint4 lo = *reinterpret_cast<const uint4*>(src);           // rows 8 g .. 8 g + 3, both tokens
+              const uint4 hi = *reinterpret_cast<const uint4*>(src + 16);      // rows 8 g + 4 .. 8 g + 7
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                  w[q] &= ((bits >> (2 * q)) & 1u ? 0x0000FFFFu : 0u) | ((bits >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u);
-              }
-              if (OP == kGemm1Relu && !p.plain) {               // save [H > 0] as one bit per element for the backward pass
-                const uint32_t* w = reinterpret_cast<const uint32_t*>(&val);
-                uint32_t m8 = 0;
+              for (int tb = 0; tb < 2; ++tb) {
+                const int st = 2 * pass + tb;
+                const uint32_t sel = tb ? 0x7632u : 0x5410u;                   // high halves: the pair's second token
+                uint4 val = make_uint4(__byte_perm(lo.x, lo.y, sel), __byte_perm(lo.z, lo.w, sel),
+                                       __byte_perm(hi.x, hi.y, sel), __byte_perm(hi.z, hi.w, sel));
+                if (OP == kDgrad2Mask && !p.plain) {            // ReLU'(u) = [u > 0]: bits saved by the forward GEMM
+                  const uint32_t bits = __shfl_sync(0xffffffffu, q_mw[0], tcol(st)) >> ((lane & 3) * 8);
+                  uint32_t* w = reinterpret_cast<uint32_t*>(&val);
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                  m8 |= ((w[q] & 0x00007FFFu) ? 1u << (2 * q) : 0u) | ((w[q] & 0x7FFF0000u) ? 1u << (2 * q + 1) : 0u);
-                uint32_t word = m8 << ((lane & 3) * 8);
-                word |= __shfl_xor_sync(0xffffffffu, word, 1);
-                word |= __shfl_xor_sync(0xffffffffu, word, 2);
-                mword[st] = word;                               // the word of token row rr, in all four lanes of its group
-              }
-              if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[st] >= 0 && mcol < p.Mw) {
-                // skip path inside the layer: y = x + g E(x), dx = dy + dH W_in^T (the expert term is already bf16)
-                if (OP == kGemm2Combine) *reinterpret_cast<uint4*>(p.out2 + offs[st] + mcol) = val;
-                const uint4 r = *reinterpret_cast<const uint4*>(p.res + offs[st] + mcol);
-                const __nv_bfloat162* rv = reinterpret_cast<const __nv_bfloat162*>(&r);
-                __nv_bfloat162* vv = reinterpret_cast<__nv_bfloat162*>(&val);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const float2 a2 = __bfloat1622float2(vv[q]), b2 = __bfloat1622float2(rv[q]);
-                  vv[q] = __floats2bfloat162_rn(a2.x + b2.x, a2.y + b2.y);
+                  for (int q = 0; q < 4; ++q)
+                    w[q] &= ((bits >> (2 * q)) & 1u ? 0x0000FFFFu : 0u) | ((bits >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u);
                 }
+                if (OP == kGemm1Relu && !p.plain) {             // save [H > 0] as one bit per element for the backward pass
+                  const uint32_t* w = reinterpret_cast<const uint32_t*>(&val);
+                  uint32_t m8 = 0;
+#pragma unroll
+                  for (int q = 0; q < 4; ++q)
+                    m8 |= ((w[q] & 0x00007FFFu) ? 1u << (2 * q) : 0u) | ((w[q] & 0x7FFF0000u) ? 1u << (2 * q + 1) : 0u);
+                  uint32_t word = m8 << ((lane & 3) * 8);
+                  word |= __shfl_xor_sync(0xffffffffu, word, 1);
+                  word |= __shfl_xor_sync(0xffffffffu, word, 2);
+                  mword[st] = word;                             // the word of token tcol(st), in all four lanes of its group
+                }
+                if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[st] >= 0 && mcol < p.Mw) {
+                  // skip path inside the layer: y = x + g E(x), dx = dy + dH W_in^T (the expert term is already bf16)
+                  if (OP == kGemm2Combine) *reinterpret_cast<uint4*>(p.out2 + offs[st] + mcol) = val;
+                  const uint4 r = *reinterpret_cast<const uint4*>(p.res + offs[st] + mcol);
+                  const __nv_bfloat162* rv = reinterpret_cast<const __nv_bfloat162*>(&r);
+                  __nv_bfloat162* vv = reinterpret_cast<__nv_bfloat162*>(&val);
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const float2 a2 = __bfloat1622float2(vv[q]), b2 = __bfloat1622float2(rv[q]);
+                    vv[q] = __floats2bfloat162_rn(a2.x + b2.x, a2.y + b2.y);
+                  }
+                }
+                if (offs[st] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[st] + mcol) = val;
               }
-              if (offs[st] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[st] + mcol) = val;
             }
             if (OP == kGemm1Relu && !p.plain) {                 // lane i stores the mask word of token row i: one 128-byte line
+              // token `lane` was handled as st = 2 (lane / 16) + (lane & 1) by the four lanes 4 ((lane / 2) & 7) ..
               uint32_t mine = 0;
 #pragma unroll
               for (int st = 0; st < 4; ++st) {
-                const uint32_t w = __shfl_sync(0xffffffffu, mword[st], 4 * (lane & 7));
-                if ((lane >> 3) == st) mine = w;
+                const uint32_t w = __shfl_sync(0xffffffffu, mword[st], 4 * ((lane >> 1) & 7));
+                if (2 * (lane >> 4) + (lane & 1) == st) mine = w;
               }
               if (q_off[0] >= 0 && m_warp < p.Mw)
                 p.hmask[(long long)(m_warp >> 5) * p.hmask_rows + (long long)t.e * p.C + t.row0 + tok0 + lane] = mine;
