@@ -402,10 +402,13 @@ def switch_backward_groups(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, exp
 # every token's first choice is placed before any second choice (token order inside each round), all against the
 # same expert capacity; f in the auxiliary loss counts the first choice (the argmax of Eq. 5).
 def top2_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None, first_index=None,
-                 second_index=None, experts=None):
+                 second_index=None, experts=None, residual: bool = False):
     """Forward of the top-2 layer.  Assignments are numbered v = t for the first choice of token t and v = T + t for
     its second choice; "slot" [2T], "token_of_slot" [E*C] (holding v) and "keep" [2T] describe the plan in that
-    numbering, "e" [2T] the expert and "g" [2T] the combine weight of every assignment."""
+    numbering, "e" [2T] the expert and "g" [2T] the combine weight of every assignment.
+    `residual` adds the layer's input to its output (the residual connection around the layer, Fig. 2; a token both of
+    whose assignments overflowed reaches the next layer through it unchanged, Section 2.2); "layer_y" holds the
+    output without it."""
     x64 = np.asarray(x, dtype=F64)
     T, d = x64.shape
     E = np.asarray(W_r).shape[1]
@@ -433,7 +436,8 @@ def top2_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, rout
         u[i] = u_i
         o[v] = o_i
         np.add.at(y, tok_of[v], g[v, None] * o_i)                # Eq. 2: sum over the selected experts
-    out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "y": y, "o": o, "u": u, "T": T, "E": E,
+    out = {"h": h, "p": p, "e": e, "g": g, "aux": aux, "f": f, "P": P, "C": C, "layer_y": y,
+           "y": x64 + y if residual else y, "residual": bool(residual), "o": o, "u": u, "T": T, "E": E,
            "alpha": alpha, "tok_of": tok_of, "first": a, "second": b}
     out.update(plan)
     out["count_first"] = np.bincount(a, minlength=E)
@@ -477,5 +481,8 @@ def top2_backward(fwd, x, W_r, W_in, W_out, dy, d_aux: float = 1.0, experts=None
     np.add.at(G, (tok_of[kept_v], e[kept_v]), dgate[kept_v])
     dh = p * (G - np.sum(p * G, axis=1, keepdims=True))
     dx_router = dh @ W_r64.T
-    return {"dx": dx + dx_router, "dW_r": x64.T @ dh, "db": dh.sum(axis=0), "dW_in": dW_in, "dW_out": dW_out,
+    dx = dx + dx_router
+    if fwd.get("residual", False):
+        dx = dx + dy64                                   # y = x + layer(x): the skip path carries dy to x unchanged
+    return {"dx": dx, "dW_r": x64.T @ dh, "db": dh.sum(axis=0), "dW_in": dW_in, "dW_out": dW_out,
             "dgate": dgate, "dh": dh, "dx_router": dx_router}

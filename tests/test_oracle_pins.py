@@ -769,19 +769,41 @@ def test_top2_layer_equals_token_by_token_definition(T, d, f, E, cf, seed):
         assert out["keep"][:T].all()
 
 
-def test_top2_backward_matches_finite_differences():
+def test_top2_with_the_skip_path_adds_the_input_and_passes_dy_through():
+    """Fig. 2: the layer sits inside a residual connection.  With it the output is the plain output plus x (a token
+    both of whose assignments overflowed comes out unchanged), and dx gains exactly dy."""
+    T, d, f, E, cf = 24, 5, 7, 4, 0.5
+    rng = np.random.default_rng(83)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=83, scale=2.0)
+    R = rng.standard_normal((T, d))
+    plain = so.top2_forward(x, W_r, W_in, W_out, cf, 0.02)
+    skip = so.top2_forward(x, W_r, W_in, W_out, cf, 0.02, residual=True)
+    np.testing.assert_array_equal(skip["layer_y"], plain["y"])
+    np.testing.assert_allclose(skip["y"] - x, plain["y"], rtol=0, atol=1e-14)
+    lost = ~plain["keep"][:T] & ~plain["keep"][T:]
+    assert lost.any()
+    np.testing.assert_array_equal(skip["y"][lost], x[lost])
+    b0 = so.top2_backward(plain, x, W_r, W_in, W_out, R)
+    b1 = so.top2_backward(skip, x, W_r, W_in, W_out, R)
+    np.testing.assert_allclose(b1["dx"], b0["dx"] + R, rtol=0, atol=1e-14)
+    for k in ("dW_r", "dgate"):
+        np.testing.assert_array_equal(b1[k], b0[k])
+
+
+@pytest.mark.parametrize("residual", [False, True], ids=["plain", "skip"])
+def test_top2_backward_matches_finite_differences(residual):
     T, d, f, E, cf, alpha, d_aux = 14, 5, 7, 4, 1.0, 0.04, 0.9
     rng = np.random.default_rng(81)
     x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=81, scale=2.0)
     R = rng.standard_normal((T, d))
-    fwd = so.top2_forward(x, W_r, W_in, W_out, cf, alpha)
+    fwd = so.top2_forward(x, W_r, W_in, W_out, cf, alpha, residual=residual)
     srt = np.sort(fwd["p"], axis=1)
     assert (srt[:, -1] - srt[:, -2]).min() > 1e-3 and (srt[:, -2] - srt[:, -3]).min() > 1e-3 and (~fwd["keep"]).any()
     bwd = so.top2_backward(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
     a, b, eps = fwd["first"], fwd["second"], 1e-6
 
     def loss():
-        o = so.top2_forward(x, W_r, W_in, W_out, cf, alpha, first_index=a, second_index=b)
+        o = so.top2_forward(x, W_r, W_in, W_out, cf, alpha, first_index=a, second_index=b, residual=residual)
         return float(np.sum(o["y"] * R) + d_aux * o["aux"])
 
     dW_in = np.stack([bwd["dW_in"][i] for i in range(E)])
