@@ -149,7 +149,8 @@ int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r
   if (c.s.dropout) SWMOE_TRY(launch_expert_dropout(c.s, c.p, false, workspace, st));
   SWMOE_TRY(mark(cfg, 4, st));
   SWMOE_TRY(run_gemm(kGemm2Combine, c, a, workspace, st));
-  if (c.s.top2) SWMOE_TRY(launch_top2_sum(c.s, c.p, y_rows, y, workspace, st));   // Eq. 2: sum over the two experts
+  if (c.s.top2)                                                                   // Eq. 2: sum over the two experts
+    SWMOE_TRY(launch_top2_sum(c.s, c.p, y_rows, c.s.residual ? x : nullptr, y, workspace, st));
   SWMOE_TRY(mark(cfg, 5, st));
   return SWITCH_MOE_OK;
 }
@@ -188,7 +189,7 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
     SWMOE_TRY(mark(cfg, 10, st));
     SWMOE_TRY(run_gemm(kWgrad1, c, a, workspace, st));
   }
-  if (c.s.top2) SWMOE_TRY(launch_top2_sum(c.s, c.p, dx_rows, dx, workspace, st));
+  if (c.s.top2) SWMOE_TRY(launch_top2_sum(c.s, c.p, dx_rows, c.s.residual ? dy : nullptr, dx, workspace, st));
   SWMOE_TRY(mark(cfg, 11, st));
   SWMOE_TRY(launch_router_bwd(c.s, c.p, x, W_r, ws_ptr<float>(workspace, c.p.dgate), d_aux, workspace, dx, true, dW_r,
                               st));

@@ -488,12 +488,13 @@ top2_choice_kernel(const float* __restrict__ probs, int T, int E, int* __restric
   }
 }
 
-// out[t] = rows[t] + rows[T + t], a dropped assignment (slot < 0) counting as zero: y from the weighted expert outputs
-// of the two choices, dx from their input gradients.  One warp per token, float32 sum.
+// out[t] = rows[t] + rows[T + t] (+ skip[t]), a dropped assignment (slot < 0) counting as zero: y from the weighted
+// expert outputs of the two choices, dx from their input gradients; `skip` is the layer's input (or dy) when the
+// layer carries its own residual connection.  One warp per token, float32 sum, one rounding.
 template <bool kBf16>
 __global__ void __launch_bounds__(256)
-top2_sum_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot, int T, int row_vec,
-                uint4* __restrict__ out) {
+top2_sum_kernel(const uint4* __restrict__ rows, const uint4* __restrict__ skip, const int* __restrict__ slot, int T,
+                int row_vec, uint4* __restrict__ out) {
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -502,26 +503,29 @@ top2_sum_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot, in
   const bool k1 = slot[t] >= 0, k2 = slot[T + t] >= 0;
   const uint4* r1 = rows + (size_t)t * row_vec;
   const uint4* r2 = rows + (size_t)(T + t) * row_vec;
+  const uint4* r3 = skip != nullptr ? skip + (size_t)t * row_vec : nullptr;
   uint4* dst = out + (size_t)t * row_vec;
   const uint4 zero = make_uint4(0, 0, 0, 0);
   for (int v = lane; v < row_vec; v += 32) {
-    const uint4 a = k1 ? r1[v] : zero, b = k2 ? r2[v] : zero;
+    const uint4 a = k1 ? r1[v] : zero, b = k2 ? r2[v] : zero, c = r3 != nullptr ? r3[v] : zero;
     uint4 o;
     if (kBf16) {
       const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
       const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+      const __nv_bfloat162* pc = reinterpret_cast<const __nv_bfloat162*>(&c);
       __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const float2 fa = __bfloat1622float2(pa[i]), fb = __bfloat1622float2(pb[i]);
-        po[i] = __floats2bfloat162_rn(fa.x + fb.x, fa.y + fb.y);
+        const float2 fa = __bfloat1622float2(pa[i]), fb = __bfloat1622float2(pb[i]), fc = __bfloat1622float2(pc[i]);
+        po[i] = __floats2bfloat162_rn((fa.x + fb.x) + fc.x, (fa.y + fb.y) + fc.y);
       }
     } else {
       const float* fa = reinterpret_cast<const float*>(&a);
       const float* fb = reinterpret_cast<const float*>(&b);
+      const float* fc = reinterpret_cast<const float*>(&c);
       float* fo = reinterpret_cast<float*>(&o);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) fo[i] = fa[i] + fb[i];
+      for (int i = 0; i < 4; ++i) fo[i] = (fa[i] + fb[i]) + fc[i];
     }
     dst[v] = o;
   }
@@ -716,9 +720,11 @@ int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void*
 int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* dx, void* ws, cudaStream_t st) {
   const int row_vec = (int)((size_t)s.d * s.elt / 16);
   const int slot_blocks = (s.E * s.C + 7) / 8;
-  const int blocks = slot_blocks + (s.residual ? (s.T + 7) / 8 : 0);
+  // (top-2 routing: dx rows are formed by the kernel that sums the two assignments, and `y` is the per-assignment
+  // output buffer already)
+  const int blocks = slot_blocks + ((s.residual && !s.top2) ? (s.T + 7) / 8 : 0);
   // with the skip path inside the layer, y holds x + g . E(x): the gate's gradient needs the copy without x
-  const void* ysrc = s.residual ? ws_ptr<char>(ws, p.layer_y) : y;
+  const void* ysrc = (s.residual && !s.top2) ? ws_ptr<char>(ws, p.layer_y) : y;
   if (s.dtype == SWITCH_MOE_BF16)
     launch_k(gather_dy_kernel<true>, dim3(blocks), dim3(256), 0, st, static_cast<const uint4*>(dy),
              static_cast<const uint4*>(ysrc), ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.token_of_slot),
@@ -738,14 +744,15 @@ int launch_top2_choice(const Shape& s, const Plan& p, void* ws, cudaStream_t st)
   return launch_status();
 }
 
-int launch_top2_sum(const Shape& s, const Plan& p, const void* per_assignment, void* out, void* ws, cudaStream_t st) {
+int launch_top2_sum(const Shape& s, const Plan& p, const void* per_assignment, const void* skip, void* out, void* ws,
+                    cudaStream_t st) {
   const int row_vec = (int)((size_t)s.d * s.elt / 16);
   if (s.dtype == SWITCH_MOE_BF16)
     launch_k(top2_sum_kernel<true>, dim3((s.T + 7) / 8), dim3(256), 0, st, static_cast<const uint4*>(per_assignment),
-             ws_ptr<int>(ws, p.slot), s.T, row_vec, static_cast<uint4*>(out));
+             static_cast<const uint4*>(skip), ws_ptr<int>(ws, p.slot), s.T, row_vec, static_cast<uint4*>(out));
   else
     launch_k(top2_sum_kernel<false>, dim3((s.T + 7) / 8), dim3(256), 0, st, static_cast<const uint4*>(per_assignment),
-             ws_ptr<int>(ws, p.slot), s.T, row_vec, static_cast<uint4*>(out));
+             static_cast<const uint4*>(skip), ws_ptr<int>(ws, p.slot), s.T, row_vec, static_cast<uint4*>(out));
   return launch_status();
 }
 

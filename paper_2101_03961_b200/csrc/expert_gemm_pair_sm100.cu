@@ -698,7 +698,9 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
       q.token_op = 1; q.a_mn_major = 1; q.Mw = s.d; K = s.f;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 64); rc2 = make_token_maps(&bm, h, s.E, s.C, s.f);
       q.out = static_cast<__nv_bfloat16*>(a.y); q.ld_out = s.d;
-      if (s.residual) { q.res = static_cast<const __nv_bfloat16*>(a.x); q.out2 = ws_ptr<__nv_bfloat16>(ws, p.layer_y); }
+      if (s.residual && !s.top2) {   // (top-2 routing adds the skip path where the two assignments' rows are summed)
+        q.res = static_cast<const __nv_bfloat16*>(a.x); q.out2 = ws_ptr<__nv_bfloat16>(ws, p.layer_y);
+      }
       break;
     case kDgrad2Mask:      // A = W_out [E][f (m)][d (k)] K-major; B = dY_d [E][C][d] K-major
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.f; K = s.d;
@@ -708,7 +710,7 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.d; K = fin;
       rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 128); rc2 = make_token_maps(&bm, du, s.E, s.C, fin);
       q.out = static_cast<__nv_bfloat16*>(a.dx); q.ld_out = s.d;
-      if (s.residual) q.res = static_cast<const __nv_bfloat16*>(a.dy);
+      if (s.residual && !s.top2) q.res = static_cast<const __nv_bfloat16*>(a.dy);
       break;
     case kWgrad2:          // dW_out [f][d] = H^T dY_d: A = H [E][C (k)][f (m)] MN-major; B = dY_d [E][C (k)][d (n)]
       q.token_op = 0; q.a_mn_major = 1; q.Mw = s.f; q.Nfix = s.d;

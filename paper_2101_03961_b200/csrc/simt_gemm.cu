@@ -147,8 +147,9 @@ int launch_t(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, void* 
       max_m = s.d; break;
     default: return SWITCH_MOE_INVALID_ARGUMENT;
   }
-  if (s.residual && op == kGemm2Combine) { pr.res = a.x; pr.out2 = ws_ptr<char>(ws, p.layer_y); }
-  if (s.residual && op == kDgrad1Scatter) pr.res = a.dy;
+  // (top-2 routing adds the skip path where the two assignments' rows are summed, not here)
+  if (s.residual && !s.top2 && op == kGemm2Combine) { pr.res = a.x; pr.out2 = ws_ptr<char>(ws, p.layer_y); }
+  if (s.residual && !s.top2 && op == kDgrad1Scatter) pr.res = a.dy;
   dim3 grid((pr.N + kBN - 1) / kBN, (max_m + kBM - 1) / kBM, s.E);
   switch (op) {
     case kGemm1Relu: simt_grouped_gemm_kernel<ET, kGemm1Relu><<<grid, 256, 0, st>>>(pr); break;

@@ -107,7 +107,7 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
     s->keep_scale = 1.f / (1.f - cfg->expert_dropout);
   }
   s->top2 = (cfg->flags & SWITCH_MOE_FLAG_TOP2) ? 1 : 0;
-  if (s->top2 && (s->residual || (cfg->flags & SWITCH_MOE_FLAG_REROUTE) || G > 1 || cfg->T % kPlanBlockTokens != 0))
+  if (s->top2 && ((cfg->flags & SWITCH_MOE_FLAG_REROUTE) || G > 1 || cfg->T % kPlanBlockTokens != 0))
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
   s->Tv = s->top2 ? 2 * cfg->T : cfg->T;
   s->jitter = (cfg->flags & SWITCH_MOE_FLAG_INPUT_JITTER) ? 1 : 0;
@@ -233,7 +233,10 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
 int launch_gather_x(const Shape& s, const Plan& p, const void* x, void* y, void* ws, cudaStream_t st);
 // Top-2 routing: second choices (expert and weight) of every token; sums of the two assignments' rows.
 int launch_top2_choice(const Shape& s, const Plan& p, void* ws, cudaStream_t st);
-int launch_top2_sum(const Shape& s, const Plan& p, const void* per_assignment, void* out, void* ws, cudaStream_t st);
+// `skip` (may be null): rows added to the sum, the layer's input (forward) or dy (backward) when the layer carries its
+// own residual connection.
+int launch_top2_sum(const Shape& s, const Plan& p, const void* per_assignment, const void* skip, void* out, void* ws,
+                    cudaStream_t st);
 int launch_gather_dy(const Shape& s, const Plan& p, const void* dy, const void* y, void* dx, void* ws, cudaStream_t st);
 int launch_router_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, const float* dgate, float d_aux,
                       void* ws, void* dx, bool accumulate_dx, float* dW_r, cudaStream_t st);

@@ -2,7 +2,7 @@
 
 Integer work (expert counts, slots, drop masks, inverse maps) must match bit for bit.  Floating point is held to
 the tolerances in gpu_helpers (router 1e-5; bf16 tensors 2e-2; all-fp32 layer 2e-4), each tensor by its relative
-Frobenius error and element by element, |a - b| <= tol (rms(b) + |b|).
+Frobenius error and element by element, |a - b| <= 2 tol (rms_i(b) + |b|) with the local rms of gpu_helpers.
 Argmax flips are counted and allowed only inside a top-2 probability gap of 1e-4; the oracle then follows the
 device's expert choice, because a single flip moves every later slot of two experts.  The sign decision of the
 ReLU derivative is treated the same way (gpu_helpers.follow_relu_flips).
@@ -567,10 +567,10 @@ def test_extreme_shapes_match_oracle(cfg):
 
 
 # ---------------------------------------------------------------------------------------------- top-2 routing
-def _check_top2(cfg, gemm_path, tol, seed=0, d_aux=0.7):
+def _check_top2(cfg, gemm_path, tol, seed=0, d_aux=0.7, residual=False):
     from tests.gpu_helpers import check_second_choice
     data = si.gen_layer(cfg, seed=seed)
-    g = GpuLayer(cfg, data, gemm_path=gemm_path, top2=True)
+    g = GpuLayer(cfg, data, gemm_path=gemm_path, top2=True, residual=residual)
     g.fwd()
     T, E, C = cfg.T, cfg.E, g.C
     gpu_e = g.expert_index()
@@ -581,7 +581,8 @@ def _check_top2(cfg, gemm_path, tol, seed=0, d_aux=0.7):
     check_flips(first, probe)
     second = check_second_choice(second, probe["p"], first, np.ones(T, dtype=bool))
     fwd = so.top2_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
-                          router_bias=data.get("router_bias"), first_index=first, second_index=second)
+                          router_bias=data.get("router_bias"), first_index=first, second_index=second,
+                          residual=residual)
     assert C == fwd["C"]
     keep = fwd["keep"]
     assert keep[T:].any() and (~keep).any()                   # second choices do get slots, and some assignments overflow
@@ -607,13 +608,20 @@ def _check_top2(cfg, gemm_path, tol, seed=0, d_aux=0.7):
     y = to_np(g.y)
     assert np.isfinite(y).all()
     both_dropped = ~keep[:T] & ~keep[T:]
-    assert np.all(y[both_dropped] == 0.0)
-    errs["y"] = rel_err(y, fwd["y"])
+    if residual:                                               # such a token leaves the layer unchanged, bit for bit
+        np.testing.assert_array_equal(y[both_dropped], to_np(g.x)[both_dropped])
+        assert skip_path_ok(y, fwd["y"], fwd["layer_y"], tol, cfg.dtype)
+    else:
+        assert np.all(y[both_dropped] == 0.0)
+        errs["y"] = rel_err(y, fwd["y"])
     g.bwd(d_aux=d_aux)
     bwd = so.top2_backward(fwd, data["x"], data["W_r"], data["W_in"], data["W_out"], data["dy"], d_aux=d_aux)
     kept_v = np.flatnonzero(keep)
     errs["dgate"] = rel_err(to_np(g.view(sm.WS_DGATE))[kept_v], bwd["dgate"][kept_v])
-    errs["dx"] = rel_err(to_np(g.dx), bwd["dx"])
+    if residual:
+        assert skip_path_ok(to_np(g.dx), bwd["dx"], bwd["dx"] - np.asarray(data["dy"], dtype=np.float64), tol, cfg.dtype)
+    else:
+        errs["dx"] = rel_err(to_np(g.dx), bwd["dx"])
     errs["dW_r"] = rel_err(to_np(g.dW_r), bwd["dW_r"])
     errs["dW_in"] = rel_err(to_np(g.dW_in), _stack(bwd["dW_in"]))
     errs["dW_out"] = rel_err(to_np(g.dW_out), _stack(bwd["dW_out"]))
@@ -636,7 +644,7 @@ def test_top2_routing_matches_oracle(cfg, path, tol):
 
 
 def test_top2_is_refused_with_the_options_it_does_not_combine_with():
-    for kw in (dict(residual=True), dict(reroute=True), dict(groups=2), dict(T=2000)):
+    for kw in (dict(reroute=True), dict(groups=2), dict(T=2000)):
         base = dict(T=2048, d_model=128, d_ff=256, E=8, capacity_factor=1.5, top2=True)
         base.update(kw)
         with pytest.raises(sm.SwitchMoeError):
