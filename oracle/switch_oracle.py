@@ -132,18 +132,38 @@ def second_choice(p, e):
     return np.argmax(q, axis=1).astype(np.int64)
 
 
+def next_choice(p, prev):
+    """The expert that follows prev[t] in token t's ranking of the experts: by probability, highest first, equal
+    probabilities by index, lowest first.  From the argmax this is the second choice, from there the third, and so
+    on; -1 once prev[t] was the last expert of the ranking (or is itself -1)."""
+    p = np.asarray(p, dtype=F64)
+    prev = np.asarray(prev, dtype=np.int64)
+    T, E = p.shape
+    out = np.full(T, -1, dtype=np.int64)
+    for t in range(T):
+        if prev[t] < 0:
+            continue
+        ranking = sorted(range(E), key=lambda i: (-p[t, i], i))
+        place = ranking.index(int(prev[t]))
+        if place + 1 < E:
+            out[t] = ranking[place + 1]
+    return out
+
+
 def reroute_overflow(plan, e, alt, E: int, C: int):
-    """Stage 2 of No-Token-Left-Behind routing (Appendix B, its figure): every token that overflowed its first
-    expert is offered, in token order, to its second-choice expert `alt[t]` and takes that expert's next free slot
-    if it still has one; tokens kept in stage 1 keep their slots.  Returns the updated plan plus "e_proc", the
-    expert that processes each token (its first choice unless it was rerouted)."""
+    """One more stage of No-Token-Left-Behind routing (Appendix B, its figure): every token that has no slot yet is
+    offered, in token order, to its next-choice expert `alt[t]` and takes that expert's next free slot if it still
+    has one; tokens placed in an earlier stage keep their slots.  Applied to the plan of stage 1 with the second
+    choices this is the figure's stage 2; applied again with the third choices it is the iteration the figure's
+    caption mentions.  An `alt[t]` of -1 (no expert left to try) leaves the token where it is.  Returns the updated
+    plan plus "e_proc", the expert that processes each token (its first choice unless it was rerouted)."""
     e = np.asarray(e, dtype=np.int64)
     alt = np.asarray(alt, dtype=np.int64)
     keep, pos, kept = plan["keep"].copy(), plan["pos"].copy(), plan["kept"].copy()
-    e_proc = e.copy()
+    e_proc = np.array(plan.get("e_proc", e), dtype=np.int64, copy=True)
     for t in np.flatnonzero(~plan["keep"]):
         i = alt[t]
-        if kept[i] < C:
+        if i >= 0 and kept[i] < C:
             pos[t] = kept[i]
             kept[i] += 1
             keep[t] = True
@@ -153,14 +173,14 @@ def reroute_overflow(plan, e, alt, E: int, C: int):
     token_of_slot[slot[keep]] = np.flatnonzero(keep)
     out = dict(plan)
     out.update({"pos": pos, "keep": keep, "slot": slot, "token_of_slot": token_of_slot, "kept": kept,
-                "e_proc": e_proc, "rerouted": keep & ~plan["keep"]})
+                "e_proc": e_proc, "rerouted": plan.get("rerouted", False) | (keep & ~plan["keep"])})
     return out
 
 
 def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, router_bias=None,
                    capacity: int | None = None, expert_index=None, experts=None, residual: bool = False,
                    reroute: bool = False, alt_index=None, router_noise=None, router_jitter=None, storage_round=None,
-                   geglu: bool = False, expert_keep=None, expert_dropout: float = 0.0):
+                   geglu: bool = False, expert_keep=None, expert_dropout: float = 0.0, reroute_stages: int = 1):
     """Forward of the Switch FFN layer for one routing group.
 
     x [T, d]; W_r [d, E]; W_in [E, d, f]; W_out [E, f, d].  `capacity` overrides Eq. 3 when given.
@@ -173,8 +193,10 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     layer unchanged (Section 2.2).  "layer_y" always holds the output without it.
     `reroute` adds stage 2 of No-Token-Left-Behind routing (Appendix B): overflowed tokens go to their second-choice
     expert where it has room, and their gate is that expert's probability (Eq. 2 with the expert that processes the
-    token); f in the auxiliary loss still counts the argmax (Eq. 5).  `alt_index`, when given, replaces the second
-    choice (to follow a legitimate near-tie flip of the device).
+    token); f in the auxiliary loss still counts the argmax (Eq. 5).  `reroute_stages` > 1 iterates (the figure's
+    caption: the process can be repeated until virtually no token is dropped): stage 3 offers the tokens that are
+    still without a slot to their third choice, and so on.  `alt_index`, when given, replaces the choices (to follow
+    a legitimate near-tie flip of the device): [T] for one stage, [stages, T] otherwise.
     `router_jitter` [T, d], when given, multiplies the router's input element by element (input jitter as the text
     describes it, Appendix C): the router sees x . u, the experts see x.  It is an
     input (the caller draws it).  `storage_round`, when given, is applied to x . u: the router's input is a tensor
@@ -208,11 +230,16 @@ def switch_forward(x, W_r, W_in, W_out, capacity_factor: float, alpha: float, ro
     plan = dispatch_plan(e, E, C)
     e_proc = e
     if reroute:
-        alt = second_choice(p, e) if alt_index is None else np.asarray(alt_index, dtype=np.int64)
-        plan = reroute_overflow(plan, e, alt, E, C)
+        given = None if alt_index is None else np.asarray(alt_index, dtype=np.int64).reshape(reroute_stages, T)
+        alts, prev = [], e
+        for s in range(reroute_stages):
+            alt = next_choice(p, prev) if given is None else given[s]
+            plan = reroute_overflow(plan, e, alt, E, C)
+            alts.append(alt)
+            prev = alt
         e_proc = plan["e_proc"]
         g = p[np.arange(T), e_proc]
-        plan["alt"] = alt
+        plan["alt"] = alts[0] if reroute_stages == 1 else np.stack(alts)
     keep = plan["keep"]
 
     y = np.zeros((T, d), dtype=F64)

@@ -591,6 +591,117 @@ def test_reroute_layer_gate_and_gradient():
         assert np.linalg.norm(num - grad) / np.linalg.norm(grad) < 1e-7, name
 
 
+# ------------------------------------------------------------------ No-Token-Left-Behind, iterated (Appendix B, figure caption)
+def test_next_choice_walks_every_expert_once_in_order_of_probability():
+    rng = np.random.default_rng(61)
+    p = so.router_probs(rng.standard_normal((40, 7)) * 2.0)
+    p[3, 2] = p[3, 5]                                                    # an exact tie: the lower index comes first
+    p[9] = 1.0 / 7                                                       # all equal: the ranking is 0, 1, .., 6
+    e, _ = so.top1(p)
+    np.testing.assert_array_equal(so.next_choice(p, e), so.second_choice(p, e))
+    seen, prev = [e], e
+    for _ in range(6):
+        prev = so.next_choice(p, prev)
+        seen.append(prev)
+    seen = np.stack(seen, axis=1)                                        # [T, E]: the whole ranking
+    assert np.array_equal(np.sort(seen, axis=1), np.tile(np.arange(7), (40, 1)))
+    ranked = np.take_along_axis(p, seen, axis=1)
+    assert (np.diff(ranked, axis=1) <= 0).all()
+    assert seen[9].tolist() == list(range(7))
+    i2, i5 = seen[3].tolist().index(2), seen[3].tolist().index(5)
+    assert i5 == i2 + 1
+    assert (so.next_choice(p, prev) == -1).all()                         # nothing after the last
+    assert (so.next_choice(p, np.full(40, -1)) == -1).all()
+    hand = np.array([[.1, .4, .2, .3]])
+    assert [int(so.next_choice(hand, np.array([k]))[0]) for k in (1, 3, 2, 0)] == [3, 2, 0, -1]
+
+
+def _iterated_reroute_brute_force(p, E, C, stages):
+    """Stage 1 for everybody; then, stage after stage, the tokens still without a slot try the next expert of their
+    own ranking, in token order (written with preference lists and plain Python lists)."""
+    T = p.shape[0]
+    prefs = [sorted(range(E), key=lambda i: (-p[t, i], i)) for t in range(T)]
+    load = [[] for _ in range(E)]
+    waiting = list(range(T))
+    for s in range(stages + 1):
+        still = []
+        for t in waiting:
+            i = prefs[t][s] if s < E else None
+            if i is not None and len(load[i]) < C:
+                load[i].append(t)
+            else:
+                still.append(t)
+        waiting = still
+    return load, waiting
+
+
+@pytest.mark.parametrize("T,E,cf,stages,seed", [(60, 4, 0.75, 2, 0), (80, 8, 1.0, 3, 1), (33, 3, 0.5, 2, 2),
+                                                (90, 6, 1.0, 5, 3), (50, 5, 0.6, 4, 4), (40, 4, 1.0, 6, 5)])
+def test_iterated_reroute_matches_brute_force(T, E, cf, stages, seed):
+    rng = np.random.default_rng(seed)
+    p = so.router_probs(rng.standard_normal((T, E)) * 2.0 + np.linspace(2.5, 0.0, E))
+    e, _ = so.top1(p)
+    C = so.expert_capacity(T, E, cf)
+    plan, prev, kept_before = so.dispatch_plan(e, E, C), e, None
+    first = plan
+    for s in range(stages):
+        prev = so.next_choice(p, prev)
+        before = plan
+        plan = so.reroute_overflow(plan, e, prev, E, C)
+        assert np.array_equal(plan["slot"][before["keep"]], before["slot"][before["keep"]])   # earlier stages untouched
+        load, waiting = _iterated_reroute_brute_force(p, E, C, s + 1)
+        for i in range(E):
+            assert plan["token_of_slot"][i * C:i * C + len(load[i])].tolist() == load[i]
+            assert plan["kept"][i] == len(load[i]) <= C
+        assert np.flatnonzero(~plan["keep"]).tolist() == waiting
+    assert np.array_equal(plan["rerouted"], plan["keep"] & ~first["keep"])
+    assert np.array_equal(plan["e_proc"][first["keep"]], e[first["keep"]])
+    moved = plan["rerouted"]
+    assert np.array_equal(plan["slot"][moved] // C, plan["e_proc"][moved])
+    if stages >= E - 1:                                                  # every token has tried every expert:
+        assert plan["keep"].sum() == min(T, E * C)                       # a token is dropped only if all slots are taken
+
+
+def test_iterated_reroute_in_the_layer_gate_and_gradient():
+    T, d, f, E, cf, alpha, d_aux, stages = 20, 5, 8, 4, 0.8, 0.03, 1.1, 3
+    rng = np.random.default_rng(43)
+    x, W_r, W_in, W_out = _rand_layer(T, d, f, E, seed=43, scale=2.0)
+    b = np.array([1.5, 0.8, 0.0, -0.5])                                  # experts 0 and 1 overflow
+    R = rng.standard_normal((T, d))
+    one = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_bias=b, reroute=True)
+    fwd = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_bias=b, reroute=True, reroute_stages=stages)
+    assert fwd["keep"].sum() == min(T, E * fwd["C"]) > one["keep"].sum()          # E - 1 extra stages fill every slot
+    assert fwd["aux"] == one["aux"]
+    np.testing.assert_array_equal(fwd["y"][one["keep"]], one["y"][one["keep"]])   # stage 2's tokens stay where they were
+    later = fwd["keep"] & ~one["keep"]
+    assert later.sum() >= 1
+    for t in np.flatnonzero(later):
+        i = fwd["e_proc"][t]
+        want = fwd["p"][t, i] * (np.maximum(x[t] @ W_in[i], 0.0) @ W_out[i])
+        np.testing.assert_allclose(fwd["y"][t], want, rtol=1e-12, atol=1e-14)
+        assert fwd["p"][t, i] <= np.sort(fwd["p"][t])[-3]                          # third choice or later
+    assert fwd["alt"].shape == (stages, T)
+    bwd = so.switch_backward(fwd, x, W_r, W_in, W_out, R, d_aux=d_aux)
+    e_frozen, alt_frozen, eps = fwd["e"], fwd["alt"], 1e-6       # the routing is frozen: the loss is smooth in x, W_r
+
+    def loss():
+        out = so.switch_forward(x, W_r, W_in, W_out, cf, alpha, router_bias=b, expert_index=e_frozen, reroute=True,
+                                reroute_stages=stages, alt_index=alt_frozen)
+        return float(np.sum(out["y"] * R) + d_aux * out["aux"])
+
+    for name, arr, grad in [("dx", x, bwd["dx"]), ("dW_r", W_r, bwd["dW_r"])]:
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            old = arr[idx]
+            arr[idx] = old + eps
+            lp = loss()
+            arr[idx] = old - eps
+            lm = loss()
+            arr[idx] = old
+            num[idx] = (lp - lm) / (2 * eps)
+        assert np.linalg.norm(num - grad) / np.linalg.norm(grad) < 1e-7, name
+
+
 # ------------------------------------------------------------------ exploration noise on the router logits (appendix pseudo-code)
 def test_logit_noise_is_additive_and_its_mean_cancels_in_the_softmax():
     T, d, f, E = 24, 6, 8, 5
