@@ -338,7 +338,7 @@ def run_ours(args, cfg):
 
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, dtype=cfg.dtype,
                           residual=args.residual, groups=args.groups, reroute=args.reroute,
-                          input_jitter=args.input_jitter > 0.0, geglu=cfg.geglu, top2=args.top2,
+                          reroute_stages=args.reroute_stages, input_jitter=args.input_jitter > 0.0, geglu=cfg.geglu, top2=args.top2,
                           expert_dropout=args.expert_dropout if args.expert_dropout > 0.0 else None)
     noise = None
     if args.router_noise > 0.0:                              # exploration noise on the logits: an input of the layer
@@ -635,7 +635,7 @@ def run_ours(args, cfg):
                    "geglu_experts": cfg.geglu,
                    "capacity_factor": cfg.capacity_factor, "alpha": cfg.alpha, "capacity": sm.switch_moe_capacity(mcfg),
                    "kept_tokens": kept, "parallelism": "replicas" if world > 1 else "single",
-                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "top2_routing": bool(args.top2), "expert_dropout": args.expert_dropout, "router_noise_eps": args.router_noise, "input_jitter_eps": args.input_jitter,
+                   "skip_path_inside_layer": bool(args.residual), "routing_groups": args.groups, "reroute_overflow": bool(args.reroute), "reroute_stages": args.reroute_stages if args.reroute else 0, "top2_routing": bool(args.top2), "expert_dropout": args.expert_dropout, "router_noise_eps": args.router_noise, "input_jitter_eps": args.input_jitter,
                    "l2": "inputs larger than L2 (weights 2 x %.0f MB per pass), no flush" %
                          (cfg.E * cfg.d_model * cfg.d_ff * elt / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": sm.switch_moe_launches_per_step(mcfg) * args.steps,
@@ -690,6 +690,8 @@ def main():
     ap.add_argument("--reroute", action="store_true",
                     help="offer tokens that overflow their expert to their second choice (stage 2 of "
                          "No-Token-Left-Behind routing); not the headline configuration")
+    ap.add_argument("--reroute-stages", type=int, default=1,
+                    help="with --reroute: how many stages follow stage 1 (stage k offers the k-th choice)")
     ap.add_argument("--residual", action="store_true",
                     help="time the variant that adds the layer's input to its output inside the combine step "
                          "(y = x + layer(x), dx = dy + ...); not the headline configuration")

@@ -53,7 +53,9 @@ enum switch_moe_gemm_path {
    Section 2.2, every token that overflowed its expert is offered, in token order, to the expert with its
    second-highest probability and takes that expert's next free slot if one is left; its gate is that expert's
    probability.  Tokens kept by the first stage keep their slots, and f in the auxiliary loss still counts the
-   argmax.  One routing group only.
+   argmax.  switch_moe_config.reroute_stages repeats the step with the third, fourth, .. choices (the figure's
+   caption: the process can be iterated); equal probabilities are ranked by index, lowest first.  One routing group
+   only.
    SWITCH_MOE_FLAG_INPUT_JITTER: the router's input is x . u, element by element, with u = router_jitter (input
    jitter as the text describes it, Appendix C); the experts still see x.  The product
    is rounded to the activation dtype (the router's input is a tensor of that type) and kept in the workspace for
@@ -106,7 +108,11 @@ typedef struct switch_moe_config {
                                 expert's rows in the slot buffers are numbered group by group, each group's kept
                                 tokens in token order, G x capacity rows per expert.  G > 1 needs T / G to be a
                                 multiple of 256, T <= 65536 and G <= 64. */
-  int32_t reserved[3];       /* must be 0 */
+  int32_t reroute_stages;    /* SWITCH_MOE_FLAG_REROUTE: how many further stages follow stage 1 (0 or 1: the figure's
+                                stage 2 alone; n: stages 2 .. n + 1, stage k offering the tokens still without a slot
+                                to the expert with their k-th highest probability; at most 16).  Ignored without
+                                the flag.  SWITCH_MOE_WS_SECOND_CHOICE then holds one int32[T] array per stage. */
+  int32_t reserved[2];       /* must be 0 */
   void* const* stage_events; /* HOST array of SWITCH_MOE_STAGE_EVENTS cudaEvent_t handles, or NULL (default).
                                 When set, fwd records event i on the stream before its stage i (0 router, 1 dispatch
                                 plan, 2 gather, 3 GEMM1+ReLU, 4 GEMM2+combine) and event 5 after the last one; bwd

@@ -94,7 +94,7 @@ int switch_moe_workspace_view(const switch_moe_config* cfg, void* workspace, int
       off = p.expert_proc; bytes = T * 4; break;
     case SWITCH_MOE_WS_SECOND_CHOICE:
       if (!s.reroute) return SWITCH_MOE_INVALID_ARGUMENT;
-      off = p.alt; bytes = T * 4; break;
+      off = p.alt; bytes = T * 4 * (size_t)s.reroute_stages; break;
     case SWITCH_MOE_WS_LAYER_Y:
       if (!s.residual) return SWITCH_MOE_INVALID_ARGUMENT;
       off = p.layer_y; bytes = T * s.d * s.elt; break;
@@ -325,7 +325,7 @@ int switch_moe_stage_launches(const switch_moe_config* cfg, int32_t* launches_ou
   n[0] = (s.router_tc ? (s.Epad64 <= 128 ? 2 : 3) : 1) + (s.jitter ? 1 : 0) + (s.top2 ? 1 : 0);
   // plan: one fused kernel when the router left the histograms and there is one routing group; else (histogram,)
   // scan, assign; stage 2 of rerouting adds four
-  n[1] = (s.router_hist ? (s.G == 1 ? 1 : 2) : 3) + (s.reroute ? 4 : 0);
+  n[1] = (s.router_hist ? (s.G == 1 ? 1 : 2) : 3) + 4 * s.reroute_stages;
   n[2] = 1;                                           // gather
   n[3] = 1 + (s.geglu ? 1 : 0) + (s.dropout ? 1 : 0); // GEMM1 (+ GEGLU gating, + expert dropout)
   n[4] = 1 + (s.top2 ? 1 : 0);                        // GEMM2 + combine (+ sum of the two assignments' rows)

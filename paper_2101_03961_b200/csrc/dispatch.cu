@@ -359,27 +359,31 @@ plan_fused_kernel(const int* __restrict__ expert_index, const int* __restrict__ 
   }
 }
 
-// ---- stage 2 of No-Token-Left-Behind routing (Appendix B) ----------------------------------------------------
-// alt[t] = the expert with the second-highest probability of an overflowed token (lowest index on ties), -1 for a
-// token that kept its slot.  One warp per token.
+// ---- further stages of No-Token-Left-Behind routing (Appendix B) ---------------------------------------------
+// alt[t] = the expert that follows prev[t] in the token's ranking of the experts (probability, highest first; equal
+// probabilities by index, lowest first) for a token that has no slot yet; -1 for a token that has one, and when no
+// expert is left.  With prev = the argmax this is the second choice (stage 2), with prev = the previous stage's
+// choices the third, and so on.  One warp per token.
 __global__ void __launch_bounds__(256)
-reroute_choice_kernel(const float* __restrict__ probs, const int* __restrict__ expert_index,
-                      const int* __restrict__ slot, int T, int E, int* __restrict__ alt) {
+reroute_choice_kernel(const float* __restrict__ probs, const int* __restrict__ prev, const int* __restrict__ slot,
+                      int T, int E, int* __restrict__ alt) {
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31;
   const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (t >= T) return;
-  if (slot[t] >= 0) {
+  const int e1 = prev[t];
+  if (slot[t] >= 0 || e1 < 0 || e1 >= E) {
     if (lane == 0) alt[t] = -1;
     return;
   }
-  const int e1 = expert_index[t];
+  const float v1 = probs[(size_t)t * E + e1];
   float best = -1.f;
   int arg = 0x7fffffff;
   for (int e = lane; e < E; e += 32) {
     const float v = probs[(size_t)t * E + e];
-    if (e != e1 && v > best) { best = v; arg = e; }          // ascending e: the first maximum wins
+    const bool later = v < v1 || (v == v1 && e > e1);         // ranked after prev[t]
+    if (later && v > best) { best = v; arg = e; }             // ascending e: the first maximum wins
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
@@ -387,10 +391,10 @@ reroute_choice_kernel(const float* __restrict__ probs, const int* __restrict__ e
     const int oa = __shfl_xor_sync(0xffffffffu, arg, off);
     if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
   }
-  if (lane == 0) alt[t] = arg < E ? arg : -1;                  // E == 1: there is no second choice
+  if (lane == 0) alt[t] = arg < E ? arg : -1;                  // nothing ranked after prev[t]
 }
 
-// Position bases of the second stage: the rerouted tokens of expert e queue up behind its kept[e] first-stage tokens.
+// Position bases of a further stage: the rerouted tokens of expert e queue up behind the kept[e] tokens it has so far.
 // One thread per expert; also rewrites kept[] and the tile lists for the grown experts.
 __global__ void __launch_bounds__(kMaxExperts)
 reroute_scan_kernel(const int* __restrict__ hist, int plan_blocks, int E, int C, int* __restrict__ hist_base,
@@ -425,7 +429,7 @@ __global__ void __launch_bounds__(kPlanBlockTokens)
 reroute_assign_kernel(const int* __restrict__ alt, const int* __restrict__ expert_index,
                       const int* __restrict__ hist_base, const float* __restrict__ probs, int T, int E, int C,
                       int* __restrict__ slot, int* __restrict__ token_of_slot, float* __restrict__ gate,
-                      int* __restrict__ expert_proc) {
+                      int* __restrict__ expert_proc, int first_stage) {
   pdl_launch_dependents();
   pdl_wait();
   __shared__ int warp_cnt[kPlanBlockTokens / 32][kMaxExperts];
@@ -442,7 +446,7 @@ reroute_assign_kernel(const int* __restrict__ alt, const int* __restrict__ exper
   if (a >= 0 && rank == 0) warp_cnt[warp][a] = __popc(same);
   __syncthreads();
   if (t < T) {
-    int proc = expert_index[t];
+    bool moved = false;
     if (a >= 0) {
       int pos = hist_base[(size_t)blockIdx.x * E + a] + rank;
       for (int w = 0; w < warp; ++w) pos += warp_cnt[w][a];
@@ -451,10 +455,12 @@ reroute_assign_kernel(const int* __restrict__ alt, const int* __restrict__ exper
         slot[t] = s;
         token_of_slot[s] = t;
         gate[t] = probs[(size_t)t * E + a];
-        proc = a;
+        moved = true;
       }
     }
-    expert_proc[t] = proc;
+    // the expert that processes the token: its first choice until a stage moves it
+    if (moved) expert_proc[t] = a;
+    else if (first_stage) expert_proc[t] = expert_index[t];
   }
 }
 
@@ -687,12 +693,15 @@ int launch_dispatch_plan(const Shape& s, const Plan& p, const int32_t* expert_in
   return launch_reroute(s, p, ws, st);
 }
 
-// Stage 2 of No-Token-Left-Behind routing, after either form of the first-stage plan.
+// The further stages of No-Token-Left-Behind routing, after either form of the first-stage plan: per stage the next
+// choices of the tokens still without a slot, their block histograms, the position bases behind the rows every
+// expert already holds, and the slots.
 int launch_reroute(const Shape& s, const Plan& p, void* ws, cudaStream_t st) {
   int* ei = ws_ptr<int>(ws, p.expert_index);
-  if (s.reroute) {
-    int* alt = ws_ptr<int>(ws, p.alt);
-    launch_k(reroute_choice_kernel, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs), ei,
+  for (int stage = 0; stage < s.reroute_stages; ++stage) {
+    int* alt = ws_ptr<int>(ws, p.alt) + (size_t)stage * s.T;
+    const int* prev = stage == 0 ? ei : alt - s.T;
+    launch_k(reroute_choice_kernel, dim3((s.T + 7) / 8), dim3(256), 0, st, ws_ptr<float>(ws, p.probs), prev,
              ws_ptr<int>(ws, p.slot), s.T, s.E, alt);
     launch_k(plan_hist_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, alt, s.T, s.E,
              ws_ptr<int>(ws, p.hist));
@@ -701,7 +710,8 @@ int launch_reroute(const Shape& s, const Plan& p, void* ws, cudaStream_t st) {
              ws_ptr<int>(ws, p.tile_row0), ws_ptr<int4>(ws, p.ntile));
     launch_k(reroute_assign_kernel, dim3(s.plan_blocks), dim3(kPlanBlockTokens), 0, st, alt, ei,
              ws_ptr<int>(ws, p.hist_base), ws_ptr<float>(ws, p.probs), s.T, s.E, s.C, ws_ptr<int>(ws, p.slot),
-             ws_ptr<int>(ws, p.token_of_slot), ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.expert_proc));
+             ws_ptr<int>(ws, p.token_of_slot), ws_ptr<float>(ws, p.gate), ws_ptr<int>(ws, p.expert_proc),
+             stage == 0 ? 1 : 0);
   }
   return launch_status();
 }

@@ -36,6 +36,7 @@ struct Shape {
   int router_blocks, plan_blocks, max_mtiles, dwr_chunks;
   int residual;     // 1: y = x + layer(x), dx = dy + d layer / dx (SWITCH_MOE_FLAG_RESIDUAL)
   int reroute;      // 1: overflowed tokens are offered to their second-choice expert (SWITCH_MOE_FLAG_REROUTE)
+  int reroute_stages;   // stages after the first (0 without the flag): stage k + 1 offers the k-th next choice
   int geglu;        // 1: GEGLU experts: W_in is [E, d, 2 f] (SWITCH_MOE_FLAG_GEGLU)
   int fin;          // columns of W_in per expert: f, or 2 f for GEGLU
   int dropout;      // 1: expert dropout on the hidden activations (SWITCH_MOE_FLAG_EXPERT_DROPOUT)
@@ -64,8 +65,9 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (cfg->gemm_path != SWITCH_MOE_GEMM_DEFAULT && cfg->gemm_path != SWITCH_MOE_GEMM_SIMT &&
       cfg->gemm_path != SWITCH_MOE_GEMM_TC_1CTA)
     return SWITCH_MOE_INVALID_ARGUMENT;
-  for (int i = 0; i < 3; ++i)
+  for (int i = 0; i < 2; ++i)
     if (cfg->reserved[i] != 0) return SWITCH_MOE_INVALID_ARGUMENT;
+  if (cfg->reroute_stages < 0 || cfg->reroute_stages > 16) return SWITCH_MOE_INVALID_ARGUMENT;
   if (cfg->groups < 0) return SWITCH_MOE_INVALID_ARGUMENT;
   const int G = cfg->groups > 1 ? cfg->groups : 1;
   if (cfg->T % G != 0) return SWITCH_MOE_INVALID_ARGUMENT;
@@ -113,6 +115,7 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   s->jitter = (cfg->flags & SWITCH_MOE_FLAG_INPUT_JITTER) ? 1 : 0;
   s->jitter_u = s->jitter ? cfg->router_jitter : nullptr;
   s->reroute = (cfg->flags & SWITCH_MOE_FLAG_REROUTE) ? 1 : 0;
+  s->reroute_stages = s->reroute ? (cfg->reroute_stages > 1 ? cfg->reroute_stages : 1) : 0;
   if (s->reroute && G > 1) return SWITCH_MOE_UNSUPPORTED_SHAPE;
   int ne = (cfg->E + 31) / 32;
   int ne_pow2 = 1;
@@ -172,7 +175,7 @@ inline void make_plan(const Shape& s, Plan* p) {
   p->dhsplit = take(3 * T * (size_t)s.Epad64 * 2);
   p->hmask = take(E * C * ((f + 31) / 32) * 4);            // one bit per element of H: [H > 0]
   p->layer_y = s.residual ? take(T * d * s.elt) : 0;       // g . E(x) without the skip path (for the gate's gradient)
-  p->alt = s.reroute ? take(T * 4) : 0;                     // second choice of overflowed tokens, -1 for the others
+  p->alt = s.reroute ? take(T * 4 * (size_t)s.reroute_stages) : 0;   // per stage: next choice of the tokens without a slot, -1 for the others
   p->expert_proc = s.reroute ? take(T * 4) : p->expert_index;   // the expert that processes each token
   p->xr = s.jitter ? take(T * d * s.elt) : 0;               // the router's input x . u, rounded to the activation dtype
   p->ab = s.geglu ? take(E * C * 2 * f * s.elt) : 0;        // GEGLU: [a | b] = X_d [W_0 | W_1] per slot

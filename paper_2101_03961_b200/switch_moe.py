@@ -42,7 +42,8 @@ class SwitchMoeConfig(ctypes.Structure):
         ("T", ctypes.c_int32), ("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("E", ctypes.c_int32),
         ("capacity_factor", ctypes.c_float), ("alpha", ctypes.c_float),
         ("capacity_override", ctypes.c_int32), ("dtype", ctypes.c_int32), ("gemm_path", ctypes.c_int32),
-        ("flags", ctypes.c_int32), ("groups", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
+        ("flags", ctypes.c_int32), ("groups", ctypes.c_int32), ("reroute_stages", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 2),
         ("stage_events", ctypes.POINTER(ctypes.c_void_p)),
         ("router_noise", ctypes.c_void_p),
         ("router_jitter", ctypes.c_void_p),
@@ -96,7 +97,7 @@ def load_library() -> ctypes.CDLL:
 
 
 def make_config(T, d_model, d_ff, E, capacity_factor, alpha=0.01, dtype=BF16, capacity_override=0,
-                gemm_path=GEMM_DEFAULT, residual=False, groups=1, reroute=False, input_jitter=False, geglu=False, top2=False, expert_dropout=None) -> SwitchMoeConfig:
+                gemm_path=GEMM_DEFAULT, residual=False, groups=1, reroute=False, input_jitter=False, geglu=False, top2=False, expert_dropout=None, reroute_stages=1) -> SwitchMoeConfig:
     cfg = SwitchMoeConfig()
     cfg.T, cfg.d_model, cfg.d_ff, cfg.E = int(T), int(d_model), int(d_ff), int(E)
     cfg.capacity_factor, cfg.alpha = float(capacity_factor), float(alpha)
@@ -106,6 +107,7 @@ def make_config(T, d_model, d_ff, E, capacity_factor, alpha=0.01, dtype=BF16, ca
                  | (FLAG_TOP2 if top2 else 0) | (FLAG_EXPERT_DROPOUT if expert_dropout is not None else 0))
     cfg.expert_dropout = float(expert_dropout or 0.0)              # set cfg.expert_keep to the device pointer of the mask     # set cfg.router_jitter to the device pointer of u
     cfg.groups = int(groups)
+    cfg.reroute_stages = int(reroute_stages) if reroute else 0
     return cfg
 
 

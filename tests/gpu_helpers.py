@@ -96,7 +96,7 @@ class GpuLayer:
     """Device buffers of one layer call plus the library calls on them."""
 
     def __init__(self, cfg: si.SwitchConfig, data: dict, gemm_path=sm.GEMM_DEFAULT, capacity_override=0,
-                 residual=False, groups=1, reroute=False, geglu=False, top2=False):
+                 residual=False, groups=1, reroute=False, geglu=False, top2=False, reroute_stages=1):
         sbuild.build()
         keep = data.get("expert_keep")
         geglu = geglu or cfg.geglu
@@ -105,7 +105,7 @@ class GpuLayer:
         self.cfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha,
                                   dtype=cfg.dtype, capacity_override=capacity_override, gemm_path=gemm_path,
                                   residual=residual, groups=groups, reroute=reroute, input_jitter=jit is not None,
-                                  geglu=geglu, top2=top2,
+                                  geglu=geglu, top2=top2, reroute_stages=reroute_stages,
                                   expert_dropout=data.get("expert_dropout") if keep is not None else None)
         dt = cfg.dtype
         self.x = to_dev(data["x"], dt)
@@ -219,6 +219,39 @@ def check_second_choice(gpu_alt: np.ndarray, p: np.ndarray, e: np.ndarray, overf
     return np.where(overflowed, gpu_alt, want)
 
 
+def check_next_choices(gpu_alt: np.ndarray, p: np.ndarray, e: np.ndarray, plan: dict, E: int, C: int) -> np.ndarray:
+    """The further stages of No-Token-Left-Behind routing, stage by stage.  gpu_alt [stages, T]: the device's next
+    choice of every token that had no slot when the stage began must be the expert with the highest probability
+    among those the token has not tried yet (lowest index on ties) -- the oracle's next_choice, as long as no
+    near-tie has flipped -- except where the two probabilities are closer than FLIP_GAP; tokens that have a slot
+    carry -1.  The oracle's plan then follows the device's choices.  Returns the choices to follow, [stages, T]."""
+    T = e.shape[0]
+    gpu_alt = gpu_alt.reshape(-1, T)
+    tried = np.zeros(p.shape, dtype=bool)
+    tried[np.arange(T), e] = True
+    prev, flipped, follow = e, False, []
+    for got in gpu_alt:
+        waiting = ~plan["keep"]
+        left = np.where(tried, -np.inf, p)
+        want = np.where(np.isfinite(left.max(axis=1)), np.argmax(left, axis=1), -1)
+        if not flipped:
+            np.testing.assert_array_equal(want, so.next_choice(p, prev))
+        assert np.all(got[~waiting] == -1)
+        diff = np.flatnonzero(waiting & (got != want))
+        if diff.size:
+            flipped = True
+            assert np.all(got[diff] >= 0) and not tried[diff, got[diff]].any()
+            gap = p[diff, want[diff]] - p[diff, got[diff]]
+            assert np.all(np.abs(gap) < FLIP_GAP), f"{diff.size} next-choice flips, largest gap {np.abs(gap).max():.3e}"
+        nxt = np.where(waiting, got, want)
+        ok = nxt >= 0
+        tried[np.flatnonzero(ok), nxt[ok]] = True
+        plan = so.reroute_overflow(plan, e, nxt, E, C)
+        follow.append(nxt)
+        prev = nxt
+    return np.stack(follow)
+
+
 def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capacity=None, experts=None,
                      residual=False, groups=1, gpu_alt=None, geglu=False):
     """Oracle forward with the device's expert choice (identical unless a near-tie flipped), after checking flips."""
@@ -244,15 +277,17 @@ def oracle_following(cfg: si.SwitchConfig, data: dict, gpu_e: np.ndarray, capaci
                               router_noise=data.get("router_noise"), **jit_kw)
     flips = check_flips(gpu_e, first)
     alt = None
-    if gpu_alt is not None:                                   # stage 2 of No-Token-Left-Behind routing
+    stages = 1
+    if gpu_alt is not None:                                   # the further stages of No-Token-Left-Behind routing
         stage1 = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor,
                                    cfg.alpha, router_bias=data.get("router_bias"), capacity=capacity,
                                    expert_index=gpu_e, experts=[], router_noise=data.get("router_noise"), **jit_kw)
-        alt = check_second_choice(gpu_alt, stage1["p"], gpu_e, ~stage1["keep"])
+        alt = check_next_choices(gpu_alt, stage1["p"], gpu_e, stage1, cfg.E, stage1["C"])
+        stages = alt.shape[0]
     fwd = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
                             router_bias=data.get("router_bias"), capacity=capacity, expert_index=gpu_e,
                             experts=experts, residual=residual, reroute=gpu_alt is not None, alt_index=alt,
-                            router_noise=data.get("router_noise"), **jit_kw)
+                            reroute_stages=stages, router_noise=data.get("router_noise"), **jit_kw)
     fwd["flips"] = flips
     return fwd
 

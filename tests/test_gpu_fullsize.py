@@ -14,7 +14,7 @@ from oracle import switch_oracle as so
 from paper_2101_03961_b200 import build as sbuild
 from paper_2101_03961_b200 import inputs as si
 from paper_2101_03961_b200 import switch_moe as sm
-from tests.gpu_helpers import (TOL_BF16, TOL_ROUTER, check_flips, check_second_choice, expert_hidden,
+from tests.gpu_helpers import (TOL_BF16, TOL_ROUTER, check_flips, check_next_choices, check_second_choice, expert_hidden,
                                follow_relu_flips, rel_err, skip_path_ok, to_np)
 
 pytestmark = pytest.mark.gpu
@@ -35,7 +35,7 @@ class _ExpertWeights:
         return si.from_bf16_bits(self.bits[i])
 
 
-def _run_fullsize(name, seed=0, n_extra=None, residual=False, groups=1, reroute=False):
+def _run_fullsize(name, seed=0, n_extra=None, residual=False, groups=1, reroute=False, reroute_stages=1):
     sbuild.build()
     cfg = si.CONFIGS[name]
     assert cfg.dtype == si.DTYPE_BF16
@@ -48,7 +48,7 @@ def _run_fullsize(name, seed=0, n_extra=None, residual=False, groups=1, reroute=
     W_r = torch.from_numpy(W_r_np).cuda()
     bias = None if b_np is None else torch.from_numpy(b_np).cuda()
     mcfg = sm.make_config(cfg.T, cfg.d_model, cfg.d_ff, cfg.E, cfg.capacity_factor, cfg.alpha, residual=residual,
-                          groups=groups, reroute=reroute, geglu=cfg.geglu)
+                          groups=groups, reroute=reroute, geglu=cfg.geglu, reroute_stages=reroute_stages)
     ws = sm.allocate_workspace(mcfg)
     ws.fill_(0xFF)
     y, dx = torch.full_like(x, float("nan")), torch.full_like(x, float("nan"))
@@ -73,12 +73,14 @@ def _run_fullsize(name, seed=0, n_extra=None, residual=False, groups=1, reroute=
     if groups == 1:
         plan = so.dispatch_plan(gpu_e, E, so.expert_capacity(T, E, cfg.capacity_factor))
         aux_ref, _, _ = so.load_balance_loss(p, gpu_e, cfg.alpha)
-        if reroute:                                          # stage 2: second choices, then the grown plan
+        if reroute:                                          # further stages: next choices, then the grown plan
             gpu_alt = view(sm.WS_SECOND_CHOICE).cpu().numpy().astype(np.int64)
-            alt = check_second_choice(gpu_alt, p, gpu_e, ~plan["keep"])
-            first_kept = int(plan["keep"].sum())
-            plan = so.reroute_overflow(plan, gpu_e, alt, E, so.expert_capacity(T, E, cfg.capacity_factor))
-            assert int(plan["keep"].sum()) > first_kept
+            cap = so.expert_capacity(T, E, cfg.capacity_factor)
+            alt = check_next_choices(gpu_alt, p, gpu_e, plan, E, cap)
+            for stage_alt in alt:
+                before = int(plan["keep"].sum())
+                plan = so.reroute_overflow(plan, gpu_e, stage_alt, E, cap)
+                assert int(plan["keep"].sum()) > before
             np.testing.assert_array_equal(view(sm.WS_EXPERT_PROC).cpu().numpy(), plan["e_proc"])
     else:                                                    # every group on its own; no expert FFN work here
         plan = so.switch_forward_groups(x_np, W_r_np, {}, {}, cfg.capacity_factor, cfg.alpha, groups,
@@ -107,7 +109,7 @@ def _run_fullsize(name, seed=0, n_extra=None, residual=False, groups=1, reroute=
     if groups == 1:
         fwd = so.switch_forward(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, router_bias=b_np,
                                 expert_index=gpu_e, experts=sample, residual=residual, reroute=reroute, alt_index=alt,
-                                geglu=cfg.geglu)
+                                reroute_stages=reroute_stages, geglu=cfg.geglu)
     else:
         fwd = so.switch_forward_groups(x_np, W_r_np, W_in_s, W_out_s, cfg.capacity_factor, cfg.alpha, groups,
                                        router_bias=b_np, expert_index=gpu_e, experts=sample, residual=residual)
@@ -204,6 +206,12 @@ def test_overflow_stress_with_rerouting_full_size():
     out = _run_fullsize("stress_calibrated", reroute=True)
     # capacity factor 1: the experts' slots add up to exactly T, so only part of the 31% overflow finds a second home
     assert out["dropped"] < 0.25 * 32768
+
+
+def test_overflow_stress_with_three_rerouting_stages_full_size():
+    out = _run_fullsize("stress_calibrated", reroute=True, reroute_stages=3)
+    # the second, third and fourth choices together leave fewer tokens without a slot than the second alone
+    assert out["dropped"] < 0.15 * 32768
 
 
 def test_geglu_experts_at_the_papers_switch_base_shape_full_size():

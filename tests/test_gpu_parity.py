@@ -124,7 +124,7 @@ def test_dispatch_plan_is_deterministic():
 
 # ---------------------------------------------------------------------------------------------- whole layer
 def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, residual=False, groups=1,
-                 reroute=False, noise_eps=0.0, jitter_eps=0.0, geglu=False, dropout=0.0):
+                 reroute=False, noise_eps=0.0, jitter_eps=0.0, geglu=False, dropout=0.0, reroute_stages=1):
     if geglu:                                                  # W_in = [W_0 | W_1]: twice the columns
         cfg = cfg.with_(geglu=True)
     data = si.gen_layer(cfg, seed=seed)
@@ -136,7 +136,7 @@ def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, re
     if noise_eps:
         data["router_noise"] = si.gen_router_noise(cfg, noise_eps, seed)
     g = GpuLayer(cfg, data, gemm_path=gemm_path, capacity_override=capacity_override, residual=residual,
-                 groups=groups, reroute=reroute, geglu=geglu)
+                 groups=groups, reroute=reroute, geglu=geglu, reroute_stages=reroute_stages)
     g.fwd()
     gpu_e = g.expert_index()
     cap = capacity_override if capacity_override else None
@@ -203,7 +203,11 @@ def _check_layer(cfg, gemm_path, tol, seed=0, d_aux=1.0, capacity_override=0, re
             assert np.all(dW_in[i] == 0) and np.all(dW_out[i] == 0)
     bad = {k: v for k, v in errs.items() if not v <= tol}
     assert not bad, (bad, errs)
+    LAST_ORACLE["fwd"] = fwd                                   # for tests that assert more about the routing
     return errs
+
+
+LAST_ORACLE = {}
 
 
 def test_tiny_fp32_layer_matches_oracle():
@@ -273,6 +277,31 @@ def test_rerouting_of_overflowed_tokens_matches_oracle(cfg, path, tol, residual)
                               router_bias=data.get("router_bias"), experts=[])
     assert (~plain["keep"]).sum() > 0.03 * cfg.T               # the case does overflow
     _check_layer(cfg, path, tol, reroute=True, residual=residual, d_aux=0.7)
+
+
+@pytest.mark.parametrize("cfg,path,tol,stages", [
+    (OVERFLOW_F32, sm.GEMM_DEFAULT, TOL_F32, 2), (OVERFLOW, sm.GEMM_SIMT, TOL_BF16, 3),
+    (OVERFLOW, sm.GEMM_DEFAULT, TOL_BF16, 3), (MANY, sm.GEMM_DEFAULT, TOL_BF16, 4),
+    (RAGGED, sm.GEMM_DEFAULT, TOL_BF16, 16)],
+    ids=["f32_2", "fma_3", "tc_3", "many_tc_4", "ragged_tc_16"])
+def test_iterated_rerouting_matches_oracle(cfg, path, tol, stages):
+    """No-Token-Left-Behind routing repeated (Appendix B, the figure's caption): stage k offers the tokens still
+    without a slot to the expert with their k-th highest probability.  Each stage must keep more tokens than the
+    one before while any are waiting and slots are free; the whole layer is compared as everywhere else."""
+    _check_layer(cfg, path, tol, reroute=True, reroute_stages=stages, d_aux=0.7)
+    fwd = LAST_ORACLE["fwd"]
+    data = si.gen_layer(cfg, seed=0)
+    one = so.switch_forward(data["x"], data["W_r"], data["W_in"], data["W_out"], cfg.capacity_factor, cfg.alpha,
+                            router_bias=data.get("router_bias"), experts=[], reroute=True)
+    assert fwd["keep"].sum() > one["keep"].sum()               # the later stages placed tokens stage 2 could not
+    if stages >= cfg.E - 1:                                    # every token has tried every expert
+        assert fwd["keep"].sum() == min(cfg.T, cfg.E * fwd["C"])
+
+
+def test_more_rerouting_stages_than_the_config_allows_are_refused():
+    with pytest.raises(sm.SwitchMoeError):
+        sm.switch_moe_workspace_bytes(sm.make_config(2048, 128, 256, 8, 1.0, reroute=True, reroute_stages=17))
+    assert sm.switch_moe_workspace_bytes(sm.make_config(2048, 128, 256, 8, 1.0, reroute_stages=17)) > 0   # ignored without the flag
 
 
 @pytest.mark.parametrize("cfg,path,tol", [(TINY, sm.GEMM_DEFAULT, TOL_F32), (MID, sm.GEMM_SIMT, TOL_BF16),
