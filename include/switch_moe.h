@@ -62,8 +62,11 @@ enum switch_moe_gemm_path {
    the backward pass, where dW_r uses it and the router's part of dx is multiplied by u.
    SWITCH_MOE_FLAG_GEGLU: the experts are GEGLU FFNs (Table 9: two expansion matrices whose outputs are combined
    non-linearly): W_in is [E, d_model, 2 d_ff] = [W_0 | W_1] per expert (and dW_in likewise), hidden = GELU(x W_0) . (x W_1) with the exact GELU z Phi(z), y = hidden W_out.  The two products are
-   one grouped GEMM with 2 d_ff output columns; the gating and its derivative are element-wise kernels over the
-   kept rows.  Not available on SWITCH_MOE_GEMM_TC_1CTA.
+   one grouped GEMM with 2 d_ff output columns.  On the default path its epilogue also gates (a CTA multiplies 64
+   columns of W_0 and the same 64 columns of W_1, the two epilogue warps that hold a and b of a hidden unit exchange
+   them through shared memory) and writes the hidden activations beside [a | b]; the derivative of the gating, and
+   the gating itself on the other paths, are element-wise kernels over the kept rows.  Not available on
+   SWITCH_MOE_GEMM_TC_1CTA.
    SWITCH_MOE_FLAG_TOP2: top-2 routing, the Mixture-of-Experts layer the paper compares with (Eq. 1-2 with the two
    highest-probability experts): y_t = p_a E_a(x_t) + p_b E_b(x_t) with the softmax probabilities of Eq. 1 as they
    are.  Every token's first choice is placed before any second choice (token order within each round), all against

@@ -145,7 +145,8 @@ int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r
   a.W_in = W_in; a.W_out = W_out; a.y = y_rows; a.x = x;
   SWMOE_TRY(mark(cfg, 3, st));
   SWMOE_TRY(run_gemm(kGemm1Relu, c, a, workspace, st));
-  if (c.s.geglu) SWMOE_TRY(launch_geglu_fwd(c.s, c.p, workspace, st));     // hidden = GELU(a) . b
+  // hidden = GELU(a) . b: inside GEMM1's epilogue on the CTA-pair path, an element-wise kernel otherwise
+  if (c.s.geglu && c.s.gemm_path != 0) SWMOE_TRY(launch_geglu_fwd(c.s, c.p, workspace, st));
   if (c.s.dropout) SWMOE_TRY(launch_expert_dropout(c.s, c.p, false, workspace, st));
   SWMOE_TRY(mark(cfg, 4, st));
   SWMOE_TRY(run_gemm(kGemm2Combine, c, a, workspace, st));
@@ -327,7 +328,7 @@ int switch_moe_stage_launches(const switch_moe_config* cfg, int32_t* launches_ou
   // scan, assign; stage 2 of rerouting adds four
   n[1] = (s.router_hist ? (s.G == 1 ? 1 : 2) : 3) + 4 * s.reroute_stages;
   n[2] = 1;                                           // gather
-  n[3] = 1 + (s.geglu ? 1 : 0) + (s.dropout ? 1 : 0); // GEMM1 (+ GEGLU gating, + expert dropout)
+  n[3] = 1 + (s.geglu && s.gemm_path != 0 ? 1 : 0) + (s.dropout ? 1 : 0);   // GEMM1 (+ GEGLU gating kernel, + expert dropout)
   n[4] = 1 + (s.top2 ? 1 : 0);                        // GEMM2 + combine (+ sum of the two assignments' rows)
   // backward.  With the paired-CTA path the two products of dH are one launch (stage 9).
   n[6] = 1;

@@ -48,6 +48,10 @@ constexpr int kPCacheBytes = kPKeptCache * 4 + kPTileCache * 16;
 constexpr int kPSmemBytes = 1024 + kPRingBytes + kPTransBytes + kPAuxBytes + 256 + kPCacheBytes;
 constexpr int kPThreads = 320;
 constexpr uint32_t kPeerMask = 0xFEFFFFFFu;            // clears the CTA-rank bit of a shared::cluster address
+// GEMM1 of GEGLU experts with the gating in its epilogue (a seventh instantiation beside the six GemmOp products):
+// a CTA's 128 weight rows are 64 columns of W_0 and the same 64 columns of W_1, so a_j and b_j of one hidden unit sit
+// in TMEM lanes j and 64 + j of one CTA, i.e. with epilogue warps two lane groups apart.
+constexpr int kGemm1Gated = 6;
 
 struct PairParams {
   int op;                  // GemmOp
@@ -71,6 +75,7 @@ struct PairParams {
   const __nv_bfloat16* res;   // combine / scatter with the skip path inside the layer: rows added to the output (x or dy)
   __nv_bfloat16* out2;        // combine with the skip path: second copy of the output without it
   int plain;                  // GEMM1 / dgrad2 without ReLU and without the ReLU mask (GEGLU experts gate elsewhere)
+  int gate_f;                 // gated GEMM1: d_ff (W_in has 2 d_ff columns [W_0 | W_1]); out = [a | b], out2 = hidden
   int stages, stage_bytes;    // operand ring: token products size a stage for the widest tile the capacity allows
   // ceil(2^32 / divisor) for the three divisions of the tile decode (n_mpairs; n_mpairs * n_ntiles_fixed;
   // n_ntiles_fixed): id / d = umulhi(id, magic) as long as id * d < 2^32
@@ -169,8 +174,9 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
 template <int OP>
 __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet& bm, const PairParams& p,
                                           const int pair, const int n_pairs) {
-  constexpr bool kTok = OP <= kDgrad1Scatter;                 // tokens on N, transposed epilogue
-  constexpr bool kAMn = (OP == kGemm1Relu || OP == kGemm2Combine || OP == kWgrad2 || OP == kWgrad1);
+  constexpr bool kGated = OP == kGemm1Gated;
+  constexpr bool kTok = OP <= kDgrad1Scatter || kGated;       // tokens on N, transposed epilogue
+  constexpr bool kAMn = (OP == kGemm1Relu || kGated || OP == kGemm2Combine || OP == kWgrad2 || OP == kWgrad1);
   constexpr bool kBMn = !kTok;
   pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
@@ -180,9 +186,12 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
   uint8_t* aux_gen = trans_gen + kPTransBytes;
   uint8_t* bar_gen = aux_gen + kPAuxBytes;
   const uint32_t bar_base = smem_base + kPRingBytes + kPTransBytes + kPAuxBytes;
-  // barrier block: full[S] | empty[S] | tmem_full[2] | tmem_empty[2] | tmem_mid[2] | tmem_ptr | abort   (S = kPMaxStages)
+  // barrier block: full[S] | empty[S] | tmem_full[2] | tmem_empty[2] | tmem_mid[2] | tmem_ptr | abort | gate[4]
+  // (S = kPMaxStages; gate[i] at byte 192 + 8 i: the handshake of the two epilogue warps that hold a and b of the
+  // same hidden units, gated GEMM1 only)
   const uint32_t full0 = bar_base, empty0 = bar_base + 8u * kPMaxStages;
   const uint32_t tfull0 = bar_base + 16u * kPMaxStages, tempty0 = tfull0 + 16u, tmid0 = tfull0 + 32u;
+  const uint32_t gate0 = bar_base + 192u;
   volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kPMaxStages + 6));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kPMaxStages + 6) + 4);
   int* kept_s = reinterpret_cast<int*>(bar_gen + 256);
@@ -198,6 +207,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 16); mbar_init(tmid0 + 8u * a, 16);
     }
+    if (kGated)
+      for (int a = 0; a < 4; ++a) mbar_init(gate0 + 8u * a, 2);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -227,7 +238,9 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
       for (int id = pair; id < n_tiles && ok; id += n_pairs) {
         const PTile t = p_decode(p, id, kept_s, tile_s);
         // coordinates of this CTA's boxes; only the contraction coordinate moves inside the tile
-        const int a_m = t.m0 + 128 * (int)rank;
+        // gated GEMM1: 64 columns of W_0 and the same 64 columns of W_1 (a pair covers 128 hidden units)
+        const int a_m = kGated ? (t.m0 >> 1) + 64 * (int)rank : t.m0 + 128 * (int)rank;
+        const int a_m2 = kGated ? p.gate_f + a_m : a_m + 64;
         const int e = t.e, kbs = t.k_blocks;
         // token products: this CTA's half of each column segment's token rows, in boxes of exactly that height;
         // weight gradients: this CTA's 128 of the 256 output columns
@@ -250,7 +263,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
           if (rank == 0) mbar_arrive_expect_tx(fb, tx_bytes);
           if (kAMn) {
             tma_load_3d_pair(a_dst, &tmA, lead_full, a_m, k0, e);
-            tma_load_3d_pair(a_dst + kAtomBytes, &tmA, lead_full, a_m + 64, k0, e);
+            tma_load_3d_pair(a_dst + kAtomBytes, &tmA, lead_full, a_m2, k0, e);
           } else {
             tma_load_3d_pair(a_dst, &tmA, lead_full, k0, a_m, e);
           }
@@ -340,10 +353,17 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
     float* gate_s = reinterpret_cast<float*>(aux_gen + (warp - 2) * 128);
     uint32_t it = 0;
     bool ok = true;
+    // gated GEMM1: lane groups 0, 1 hold a = x W_0, lane groups 2, 3 hold b = x W_1 of the same 32 hidden units
+    const int role = lg >> 1;
+    const uint8_t* tr_other = trans_gen + (half * 4 + lg) * kPTransWarp;   // the transpose tile of the warp two lane groups away
+    const uint32_t gate_bar = gate0 + 8u * (uint32_t)(half * 2 + (lg & 1));
+    uint32_t gate_phase = 0;
     for (int id = pair; id < n_tiles && ok; id += n_pairs, ++it) {
       const PTile t = p_decode(p, id, kept_s, tile_s);
       const uint32_t side = it & 1u, use = it >> 1;
-      const int m_warp = t.m0 + 128 * (int)rank + 32 * lg;    // first M row (weight row) this warp holds
+      const int unit0 = (t.m0 >> 1) + 64 * (int)rank + 32 * (lg & 1);        // gated GEMM1: first hidden unit of this warp
+      // first M row (weight row = output column) this warp holds
+      const int m_warp = kGated ? role * p.gate_f + unit0 : t.m0 + 128 * (int)rank + 32 * lg;
       const int n_chunks = kTok ? (t.n + 31) >> 5 : 8;
       const bool have_acc = t.k_blocks > 0;
       const int c0 = side ? kTmemCols - t.n : 0;              // first accumulator column of the tile
@@ -353,13 +373,14 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
       // ones the next tile may also use.  Lane i describes token column (chunk's first token) + i: the element offset
       // of its output row (or -1) and its gate.  This warp's chunks are j = n_chunks - 1 - half, then every second
       // one down to 0; their descriptions (and ReLU masks) are fetched before the accumulator is awaited.
-      constexpr bool kSlotRows = (OP == kGemm1Relu || OP == kDgrad2Mask);
+      constexpr bool kSlotRows = (OP == kGemm1Relu || kGated || OP == kDgrad2Mask);
       constexpr int kQueue = 5;                                // (320 / 32) chunks over two warps
       int row_limit = 0;
       long long q_off[kQueue] = {-1, -1, -1, -1, -1};           // head = next chunk to process
       float q_gate[kQueue] = {1.f, 1.f, 1.f, 1.f, 1.f};
       uint32_t q_mw[kQueue] = {0u, 0u, 0u, 0u, 0u};             // dgrad2: ReLU mask bits of weight rows m_warp..+31 per token
       const int mcol = m_warp + (lane & 3) * 8;               // store `it` writes weight rows mcol .. mcol + 7
+      const bool col_ok = kGated ? unit0 + (lane & 3) * 8 < p.gate_f : mcol < p.Mw;
       auto chunk_tok0 = [&](int j) { return side ? t.n - 32 * (j + 1) : 32 * j; };
       auto describe = [&](int j, long long* off, float* g) {
         const int col = chunk_tok0(j) + lane, slot_row = t.row0 + col;
@@ -538,7 +559,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
                   word |= __shfl_xor_sync(0xffffffffu, word, 2);
                   mword[st] = word;                             // the word of token tcol(st), in all four lanes of its group
                 }
-                if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[st] >= 0 && mcol < p.Mw) {
+                if ((OP == kGemm2Combine || OP == kDgrad1Scatter) && p.res != nullptr && offs[st] >= 0 && col_ok) {
                   // skip path inside the layer: y = x + g E(x), dx = dy + dH W_in^T (the expert term is already bf16)
                   if (OP == kGemm2Combine) *reinterpret_cast<uint4*>(p.out2 + offs[st] + mcol) = val;
                   const uint4 r = *reinterpret_cast<const uint4*>(p.res + offs[st] + mcol);
@@ -550,7 +571,51 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
                     vv[q] = __floats2bfloat162_rn(a2.x + b2.x, a2.y + b2.y);
                   }
                 }
-                if (offs[st] >= 0 && mcol < p.Mw) *reinterpret_cast<uint4*>(p.out + offs[st] + mcol) = val;
+                if (offs[st] >= 0 && col_ok) *reinterpret_cast<uint4*>(p.out + offs[st] + mcol) = val;
+              }
+            }
+            if constexpr (kGated) {
+              // hidden = GELU(a) . b from the rounded values just stored (what the backward pass reads back).  The a
+              // warp gates the chunk's token pairs 0-7, the b warp pairs 8-15: each reads the other's transpose tile
+              // between two handshakes, then transposes its 16 tokens x 32 hidden units through its own tile.
+              __syncwarp();
+              if (lane == 0) mbar_arrive(gate_bar);
+              ok = mbar_wait(gate_bar, gate_phase, abort_flag, p.status, 26);     // both tiles are written
+              gate_phase ^= 1u;
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              uint32_t hw[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const int tp = 8 * role + k;
+                const uint32_t mine = *reinterpret_cast<const uint32_t*>(tr + tp * 144 + lane * 4);
+                const uint32_t other = *reinterpret_cast<const uint32_t*>(tr_other + tp * 144 + lane * 4);
+                const uint32_t aw = role ? other : mine, bw = role ? mine : other;
+                const float2 af = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw));
+                const float2 bf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw));
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(gelu_exact(af.x) * bf.x, gelu_exact(af.y) * bf.y);
+                hw[k] = *reinterpret_cast<const uint32_t*>(&h2);
+              }
+              __syncwarp();
+              if (lane == 0) mbar_arrive(gate_bar);
+              ok = mbar_wait(gate_bar, gate_phase, abort_flag, p.status, 27);     // both tiles have been read
+              gate_phase ^= 1u;
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+#pragma unroll
+              for (int k = 0; k < 8; ++k) *reinterpret_cast<uint32_t*>(tr + k * 144 + lane * 4) = hw[k];
+              __syncwarp();
+              const uint8_t* src = tr + (lane >> 2) * 144 + (lane & 3) * 32;
+              const uint4 lo = *reinterpret_cast<const uint4*>(src);
+              const uint4 hi = *reinterpret_cast<const uint4*>(src + 16);
+#pragma unroll
+              for (int tb = 0; tb < 2; ++tb) {
+                const uint32_t sel = tb ? 0x7632u : 0x5410u;
+                const uint4 val = make_uint4(__byte_perm(lo.x, lo.y, sel), __byte_perm(lo.z, lo.w, sel),
+                                             __byte_perm(hi.x, hi.y, sel), __byte_perm(hi.z, hi.w, sel));
+                const long long off = __shfl_sync(0xffffffffu, q_off[0], 16 * role + 2 * (lane >> 2) + tb);
+                // a row of [a | b] has 2 d_ff columns, the hidden row d_ff: half the element offset
+                if (off >= 0 && col_ok) *reinterpret_cast<uint4*>(p.out2 + (off >> 1) + unit0 + (lane & 3) * 8) = val;
               }
             }
             if (OP == kGemm1Relu && !p.plain) {                 // lane i stores the mask word of token row i: one 128-byte line
@@ -693,7 +758,9 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
       q.token_op = 1; q.a_mn_major = 1; q.Mw = fin; K = s.d;   // GEGLU: [a | b], 2 f output columns, no ReLU
       rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 64); rc2 = make_token_maps(&bm, xd, s.E, s.C, s.d);
       q.out = s.geglu ? ws_ptr<__nv_bfloat16>(ws, p.ab) : ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = fin;
-      q.plain = s.geglu; break;
+      q.plain = s.geglu;
+      if (s.geglu) { q.gate_f = s.f; q.out2 = ws_ptr<__nv_bfloat16>(ws, p.h); }   // gating in the epilogue
+      break;
     case kGemm2Combine:    // A = W_out [E][f (k)][d (m)] MN-major; B = H [E][C][f] K-major
       q.token_op = 1; q.a_mn_major = 1; q.Mw = s.d; K = s.f;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 64); rc2 = make_token_maps(&bm, h, s.E, s.C, s.f);
@@ -764,7 +831,9 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   const int rc = pair_problem(op, s, p, a, ws, &q, &tmA, &tmB);
   if (rc != SWITCH_MOE_OK) return rc;
   switch (op) {
-    case kGemm1Relu: return launch_pair_op<kGemm1Relu>(tmA, tmB, q, dev, sm_count, st);
+    case kGemm1Relu:
+      if (s.geglu) return launch_pair_op<kGemm1Gated>(tmA, tmB, q, dev, sm_count, st);
+      return launch_pair_op<kGemm1Relu>(tmA, tmB, q, dev, sm_count, st);
     case kGemm2Combine: return launch_pair_op<kGemm2Combine>(tmA, tmB, q, dev, sm_count, st);
     case kDgrad2Mask: return launch_pair_op<kDgrad2Mask>(tmA, tmB, q, dev, sm_count, st);
     case kDgrad1Scatter: return launch_pair_op<kDgrad1Scatter>(tmA, tmB, q, dev, sm_count, st);

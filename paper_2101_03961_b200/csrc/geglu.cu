@@ -8,7 +8,7 @@
 namespace swmoe {
 namespace {
 
-__device__ __forceinline__ float gelu_f(float z) { return 0.5f * z * (1.f + erff(z * 0.70710678118654752f)); }
+__device__ __forceinline__ float gelu_f(float z) { return gelu_exact(z); }
 __device__ __forceinline__ float gelu_prime_f(float z) {
   return 0.5f * (1.f + erff(z * 0.70710678118654752f)) + z * 0.3989422804014327f * __expf(-0.5f * z * z);
 }

@@ -250,6 +250,10 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
 int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, void* ws, void* dx,
                          bool accumulate_dx, cudaStream_t st);
 
+// GELU(z) = z Phi(z), the exact form (GEGLU experts).  One definition for the element-wise kernels and the GEMM
+// epilogue that gates: both must round identically, the backward pass recomputes what the forward pass used.
+__device__ __forceinline__ float gelu_exact(float z) { return 0.5f * z * (1.f + erff(z * 0.70710678118654752f)); }
+
 // The six expert GEMMs (Section 5: h = x W_in, y = ReLU(h) W_out, and their derivatives).
 enum GemmOp {
   kGemm1Relu = 0,     // H = ReLU(X_d W_in)

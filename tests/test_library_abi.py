@@ -90,6 +90,10 @@ def test_launch_count_is_reported(lib):
     # bf16 default path: the router's epilogue leaves the probabilities' column sums and the plan's histograms, and the
     # two products of dH share one launch
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 14
-    # options add launches: four plan kernels for rerouting, one product kernel for input jitter, two GEGLU gating kernels
+    # options add launches: four plan kernels per rerouting stage, one product kernel for input jitter, one GEGLU gating
+    # kernel (the backward one: the forward gating is in GEMM1's epilogue on this path), two expert-dropout kernels
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, reroute=True, input_jitter=True,
-                                                          geglu=True, expert_dropout=0.4)) == 14 + 4 + 1 + 2 + 2
+                                                          geglu=True, expert_dropout=0.4)) == 14 + 4 + 1 + 1 + 2
+    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, reroute=True, reroute_stages=3)) == 14 + 12
+    # the fp32 path gates in element-wise kernels both ways
+    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, dtype=sm.F32, geglu=True)) == 16 + 2
