@@ -61,7 +61,7 @@ enum switch_moe_gemm_path {
    is rounded to the activation dtype (the router's input is a tensor of that type) and kept in the workspace for
    the backward pass, where dW_r uses it and the router's part of dx is multiplied by u.
    SWITCH_MOE_FLAG_GEGLU: the experts are GEGLU FFNs (Table 9: two expansion matrices whose outputs are combined
-   non-linearly): W_in is [E, d_model, 2 d_ff] = [W_0 | W_1] per expert (and dW_in likewise), hidden = GELU(x W_0) . (x W_1) with the exact GELU z Phi(z), y = hidden W_out.  The two products are
+   non-linearly): W_in is [E, d_model, 2 d_ff] = [W_0 | W_1] per expert (and dW_in likewise), hidden = GELU(x W_0) . (x W_1) with the exact form GELU(z) = z Phi(z) (not the tanh fit; Phi is evaluated to about 3e-7 absolute), y = hidden W_out.  The two products are
    one grouped GEMM with 2 d_ff output columns.  On the default path its epilogue also gates (a CTA multiplies 64
    columns of W_0 and the same 64 columns of W_1, the two epilogue warps that hold a and b of a hidden unit exchange
    them through shared memory) and writes the hidden activations beside [a | b]; the derivative of the gating, and

@@ -9,9 +9,6 @@ namespace swmoe {
 namespace {
 
 __device__ __forceinline__ float gelu_f(float z) { return gelu_exact(z); }
-__device__ __forceinline__ float gelu_prime_f(float z) {
-  return 0.5f * (1.f + erff(z * 0.70710678118654752f)) + z * 0.3989422804014327f * __expf(-0.5f * z * z);
-}
 
 template <typename ET> struct Pack;
 template <> struct Pack<__nv_bfloat16> {
@@ -74,7 +71,13 @@ geglu_kernel(const uint4* __restrict__ ab, const int* __restrict__ kept, int E, 
       float g[N], o2[N];
       Pack<ET>::load(hrow[v], g);
 #pragma unroll
-      for (int i = 0; i < N; ++i) { o[i] = g[i] * b[i] * gelu_prime_f(a[i]); o2[i] = g[i] * gelu_f(a[i]); }
+      for (int i = 0; i < N; ++i) {
+        // one evaluation of Phi and phi serves GELU(a) = a Phi(a) and GELU'(a) = Phi(a) + a phi(a)
+        float cdf, pdf;
+        gelu_cdf_pdf(a[i], &cdf, &pdf);
+        o[i] = g[i] * b[i] * fmaf(a[i], pdf, cdf);
+        o2[i] = g[i] * (a[i] * cdf);
+      }
       uint4* drow = dab + (size_t)s * 2 * f_vec;
       drow[v] = Pack<ET>::store(o);
       drow[f_vec + v] = Pack<ET>::store(o2);

@@ -511,6 +511,7 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const uint32_t tfull0 = bar_base + 16u * kStages, tempty0 = tfull0 + 16u;
   volatile uint32_t* tmem_ptr_s = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * kStages + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kStages + 4) + 4);
+  volatile int* fail_s = reinterpret_cast<volatile int*>(bar_gen + 8 * (2 * kStages + 4) + 8);   // an epilogue warp gave up
   int* hist_s = reinterpret_cast<int*>(bar_gen + 1024);        // kMaxExperts counters
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -518,6 +519,7 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 8); }
     *abort_flag = 0;
+    *fail_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -611,12 +613,15 @@ router_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int et = threadIdx.x - 64;                          // 0..255 over the epilogue warps
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
-    for (int id = blockIdx.x; id < n_tiles && ok; id += gridDim.x) {
+    for (int id = blockIdx.x; id < n_tiles; id += gridDim.x) {
       const int tok0 = id * 2 * kTileM + ti * kTileM + lg * 32;
       const int tok = tok0 + lane;                            // the token whose logits this lane holds
       ok = mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag, p.status, 34);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
+      // the eight warps meet at barriers below: all of them leave together if the bounded wait of any gave up
+      if (!ok && lane == 0) *fail_s = 1;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (*fail_s != 0) break;
       tc_fence_after();
       const uint32_t t_addr = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * (uint32_t)kBN + (uint32_t)ti * 128u;
       float h[NCH * 32];

@@ -250,9 +250,31 @@ int launch_router_tc_fwd(const Shape& s, const Plan& p, const void* x, const flo
 int launch_router_tc_bwd(const Shape& s, const Plan& p, const void* x, const float* W_r, void* ws, void* dx,
                          bool accumulate_dx, cudaStream_t st);
 
-// GELU(z) = z Phi(z), the exact form (GEGLU experts).  One definition for the element-wise kernels and the GEMM
-// epilogue that gates: both must round identically, the backward pass recomputes what the forward pass used.
-__device__ __forceinline__ float gelu_exact(float z) { return 0.5f * z * (1.f + erff(z * 0.70710678118654752f)); }
+// GELU(z) = z Phi(z), the exact form (GEGLU experts), and what its derivative needs.  Phi(z) = (1 + erf(z / sqrt 2)) / 2
+// with the rational approximation 7.1.26 of Abramowitz and Stegun for erf (absolute error below 1.5e-7, i.e. the
+// resolution of a float32 near 1): erf(x) = 1 - (a1 t + .. + a5 t^5) exp(-x^2), t = 1 / (1 + p x), x >= 0.  Its
+// exponential exp(-z^2 / 2) is the one the density phi(z) needs, so one exp2 and one reciprocal serve the value
+// and the derivative; the library erff costs about three times the instructions, and the gating is bound by the
+// number of instructions it issues.  One definition for the element-wise kernels and the GEMM epilogue that gates:
+// both must round identically.
+__device__ __forceinline__ void gelu_cdf_pdf(float z, float* cdf, float* pdf) {
+  const float az = fabsf(z);
+  const float e = __expf(-0.5f * z * z);
+  float t;                                                    // the hardware's approximate reciprocal (1 ulp)
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f * 0.70710678118654752f, az, 1.f)));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float tail = 0.5f * poly * t * e;                     // Phi(-|z|)
+  *cdf = z >= 0.f ? 1.f - tail : tail;
+  *pdf = 0.3989422804014327f * e;
+}
+__device__ __forceinline__ float gelu_exact(float z) {
+  float cdf, pdf;
+  gelu_cdf_pdf(z, &cdf, &pdf);
+  return z * cdf;
+}
 
 // The six expert GEMMs (Section 5: h = x W_in, y = ReLU(h) W_out, and their derivatives).
 enum GemmOp {
