@@ -66,6 +66,9 @@ CONFIGS = {
     "switch_base_quarter": SwitchConfig("switch_base_quarter", 8192, 768, 3072, 32, 1.25),
     # the paper's own Switch-Base layer shape with GEGLU experts (its hyper-parameter table: d_model 768, d_ff 2048)
     "geglu_base": SwitchConfig("geglu_base", 32768, 768, 2048, 128, 1.25, geglu=True),
+    # the same table's Switch-Large (d_model 1024, d_ff 2816) and Switch-XXL (d_model 4096, d_ff 10240, 64 experts)
+    "geglu_large": SwitchConfig("geglu_large", 32768, 1024, 2816, 128, 1.25, geglu=True),
+    "geglu_xxl": SwitchConfig("geglu_xxl", 16384, 4096, 10240, 64, 1.25, geglu=True),
     # many tokens, narrow layer: exercises the token-count limits of the router's partial sums and of the plan's scan
     "long_batch": SwitchConfig("long_batch", 131072, 256, 512, 128, 1.25),
 }

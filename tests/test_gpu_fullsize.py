@@ -218,6 +218,14 @@ def test_geglu_experts_at_the_papers_switch_base_shape_full_size():
     _run_fullsize("geglu_base")
 
 
+def test_geglu_experts_at_the_papers_switch_large_shape_full_size():
+    _run_fullsize("geglu_large")                              # d_ff 2816 = 11 weight-row tiles of 256: an odd count
+
+
+def test_geglu_experts_at_the_papers_switch_xxl_shape_full_size():
+    _run_fullsize("geglu_xxl", n_extra=1)                     # sampled experts: the oracle pass would take minutes
+
+
 def test_batch_of_131072_tokens_full_size():
     out = _run_fullsize("long_batch")
     assert out["dropped"] < 0.05 * 131072
