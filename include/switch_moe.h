@@ -64,9 +64,11 @@ enum switch_moe_gemm_path {
    non-linearly): W_in is [E, d_model, 2 d_ff] = [W_0 | W_1] per expert (and dW_in likewise), hidden = GELU(x W_0) . (x W_1) with the exact form GELU(z) = z Phi(z) (not the tanh fit; Phi is evaluated to about 3e-7 absolute), y = hidden W_out.  The two products are
    one grouped GEMM with 2 d_ff output columns.  On the default path its epilogue also gates (a CTA multiplies 64
    columns of W_0 and the same 64 columns of W_1, the two epilogue warps that hold a and b of a hidden unit exchange
-   them through shared memory) and writes the hidden activations beside [a | b]; the derivative of the gating, and
-   the gating itself on the other paths, are element-wise kernels over the kept rows.  Not available on
-   SWITCH_MOE_GEMM_TC_1CTA.
+   them through shared memory): it writes the hidden activations and, for the backward pass, the two factors
+   GELU(a) and b GELU'(a) of every hidden unit (rounded to the activation dtype) instead of a and b; dgrad2's
+   epilogue multiplies dH by them and writes d[a | b] directly.  With expert dropout, and on the other paths, the
+   derivative of the gating (and on the other paths the gating itself) is an element-wise kernel over the kept
+   rows.  Not available on SWITCH_MOE_GEMM_TC_1CTA.
    SWITCH_MOE_FLAG_TOP2: top-2 routing, the Mixture-of-Experts layer the paper compares with (Eq. 1-2 with the two
    highest-probability experts): y_t = p_a E_a(x_t) + p_b E_b(x_t) with the softmax probabilities of Eq. 1 as they
    are.  Every token's first choice is placed before any second choice (token order within each round), all against

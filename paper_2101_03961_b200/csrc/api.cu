@@ -177,7 +177,9 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
   SWMOE_TRY(mark(cfg, 7, st));
   SWMOE_TRY(run_gemm(kDgrad2Mask, c, a, workspace, st));
   if (c.s.dropout) SWMOE_TRY(launch_expert_dropout(c.s, c.p, true, workspace, st));   // same factors on the way back
-  if (c.s.geglu) SWMOE_TRY(launch_geglu_bwd(c.s, c.p, workspace, st));     // d[a | b] from dH
+  // d[a | b] from dH: inside dgrad2's epilogue on the CTA-pair path (unless expert dropout has to touch dH first),
+  // an element-wise kernel otherwise
+  if (c.s.geglu && (c.s.gemm_path != 0 || c.s.dropout)) SWMOE_TRY(launch_geglu_bwd(c.s, c.p, workspace, st));
   SWMOE_TRY(mark(cfg, 8, st));
   SWMOE_TRY(run_gemm(kWgrad2, c, a, workspace, st));
   SWMOE_TRY(mark(cfg, 9, st));
@@ -332,7 +334,7 @@ int switch_moe_stage_launches(const switch_moe_config* cfg, int32_t* launches_ou
   n[4] = 1 + (s.top2 ? 1 : 0);                        // GEMM2 + combine (+ sum of the two assignments' rows)
   // backward.  With the paired-CTA path the two products of dH are one launch (stage 9).
   n[6] = 1;
-  n[7] = 1 + (s.dropout ? 1 : 0) + (s.geglu ? 1 : 0);
+  n[7] = 1 + (s.dropout ? 1 : 0) + (s.geglu && (s.gemm_path != 0 || s.dropout) ? 1 : 0);
   n[8] = 1;
   n[9] = 1;
   n[10] = (s.gemm_path == 0 ? 0 : 1) + (s.top2 ? 1 : 0);

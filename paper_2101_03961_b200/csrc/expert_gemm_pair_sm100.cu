@@ -52,6 +52,9 @@ constexpr uint32_t kPeerMask = 0xFEFFFFFFu;            // clears the CTA-rank bi
 // a CTA's 128 weight rows are 64 columns of W_0 and the same 64 columns of W_1, so a_j and b_j of one hidden unit sit
 // in TMEM lanes j and 64 + j of one CTA, i.e. with epilogue warps two lane groups apart.
 constexpr int kGemm1Gated = 6;
+// dgrad2 of GEGLU experts with the derivative of the gating in its epilogue: d a = dH . (b GELU'(a)), d b = dH . GELU(a),
+// the two factors read back from what the gated GEMM1 saved.
+constexpr int kDgrad2Gated = 7;
 
 struct PairParams {
   int op;                  // GemmOp
@@ -75,7 +78,10 @@ struct PairParams {
   const __nv_bfloat16* res;   // combine / scatter with the skip path inside the layer: rows added to the output (x or dy)
   __nv_bfloat16* out2;        // combine with the skip path: second copy of the output without it
   int plain;                  // GEMM1 / dgrad2 without ReLU and without the ReLU mask (GEGLU experts gate elsewhere)
-  int gate_f;                 // gated GEMM1: d_ff (W_in has 2 d_ff columns [W_0 | W_1]); out = [a | b], out2 = hidden
+  int gate_f;                 // gated products: d_ff.  Gated GEMM1: W_in has 2 d_ff columns [W_0 | W_1]; out = the saved
+                              // factors, one 32-bit word {GELU(a), b GELU'(a)} per hidden unit and slot row; out2 = hidden.
+                              // Gated dgrad2: out = d[a | b] (2 d_ff columns), gate_in = those words.
+  const uint32_t* gate_in;
   int stages, stage_bytes;    // operand ring: token products size a stage for the widest tile the capacity allows
   // ceil(2^32 / divisor) for the three divisions of the tile decode (n_mpairs; n_mpairs * n_ntiles_fixed;
   // n_ntiles_fixed): id / d = umulhi(id, magic) as long as id * d < 2^32
@@ -174,8 +180,8 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
 template <int OP>
 __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet& bm, const PairParams& p,
                                           const int pair, const int n_pairs) {
-  constexpr bool kGated = OP == kGemm1Gated;
-  constexpr bool kTok = OP <= kDgrad1Scatter || kGated;       // tokens on N, transposed epilogue
+  constexpr bool kGated = OP == kGemm1Gated, kDGated = OP == kDgrad2Gated;
+  constexpr bool kTok = OP <= kDgrad1Scatter || kGated || kDGated;   // tokens on N, transposed epilogue
   constexpr bool kAMn = (OP == kGemm1Relu || kGated || OP == kGemm2Combine || OP == kWgrad2 || OP == kWgrad1);
   constexpr bool kBMn = !kTok;
   pdl_launch_dependents();
@@ -373,7 +379,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
       // ones the next tile may also use.  Lane i describes token column (chunk's first token) + i: the element offset
       // of its output row (or -1) and its gate.  This warp's chunks are j = n_chunks - 1 - half, then every second
       // one down to 0; their descriptions (and ReLU masks) are fetched before the accumulator is awaited.
-      constexpr bool kSlotRows = (OP == kGemm1Relu || kGated || OP == kDgrad2Mask);
+      constexpr bool kSlotRows = (OP == kGemm1Relu || kGated || OP == kDgrad2Mask || kDGated);
       constexpr int kQueue = 5;                                // (320 / 32) chunks over two warps
       int row_limit = 0;
       long long q_off[kQueue] = {-1, -1, -1, -1, -1};           // head = next chunk to process
@@ -414,6 +420,23 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
                                 chunk_tok0(n_chunks - 1 - half - 2 * k) + lane];
         }
       }
+      // gated dgrad2: the saved factors of this lane's hidden unit for the 32 tokens of a chunk, one word per token
+      // ({GELU(a), b GELU'(a)} as two bfloat16), fetched one chunk ahead; 0 for columns that hold no token
+      uint32_t gg[kDGated ? 32 : 1];
+      auto fetch_factors = [&](int j, uint32_t* dst) {
+        if constexpr (kDGated) {
+          const int tok_first = chunk_tok0(j);
+          const bool unit_ok = m_warp < p.Mw;
+          const uint32_t* src = p.gate_in + ((long long)t.e * p.C + t.row0 + tok_first) * p.gate_f + m_warp + lane;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int col = tok_first + i;
+            const bool valid = unit_ok && j >= 0 && col >= 0 && col < t.n && t.row0 + col < row_limit;
+            dst[i] = valid ? src[(long long)i * p.gate_f] : 0u;
+          }
+        }
+      };
+      fetch_factors(n_chunks - 1 - half, gg);
       ok = mbar_wait(tfull0 + 8u * side, use & 1u, abort_flag, p.status, 24);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -499,15 +522,100 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
             if (lane == 0) mbar_arrive_remote(tempty0 + 8u * side, 0);
             released = true;
           }
+          uint32_t gn[kDGated ? 32 : 1];                        // gated dgrad2: the next chunk's factors, in flight meanwhile
+          fetch_factors(j - 2, gn);
           {
             // Store `st` of this lane writes weight rows mcol .. mcol + 7 of token column tcol(st) of the chunk:
             // eight lanes' token pairs x four row groups per instruction.
             auto tcol = [&](int st) { return 16 * (st >> 1) + 2 * (lane >> 2) + (st & 1); };
+            uint32_t mword[4] = {0u, 0u, 0u, 0u};
+            if constexpr (kGated) {
+              // GEGLU gating.  Both warps of a pair round their values (a or b of 32 hidden units x 32 tokens) into
+              // their transpose tiles; between two handshakes the a warp takes b of the chunk's tokens 0-15 from the
+              // other tile and the b warp a of tokens 16-31.  Each then has a and b of one hidden unit per lane for 16
+              // tokens and forms GELU(a), b GELU'(a) (saved for the backward pass as one word per unit and row) and the
+              // hidden activation GELU(a) b, and transposes both through its own tile.
+              uint32_t pk[16];
+#pragma unroll
+              for (int k = 0; k < 16; ++k) {
+                const __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1]));
+                pk[k] = *reinterpret_cast<const uint32_t*>(&t2);
+                *reinterpret_cast<uint32_t*>(tr + k * 144 + lane * 4) = pk[k];
+              }
+              __syncwarp();
+              if (lane == 0) mbar_arrive(gate_bar);
+              ok = mbar_wait(gate_bar, gate_phase, abort_flag, p.status, 26);     // both tiles are written
+              gate_phase ^= 1u;
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              uint32_t other[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k)
+                other[k] = *reinterpret_cast<const uint32_t*>(tr_other + (8 * role + k) * 144 + lane * 4);
+              __syncwarp();
+              if (lane == 0) mbar_arrive(gate_bar);
+              ok = mbar_wait(gate_bar, gate_phase, abort_flag, p.status, 27);     // both tiles have been read
+              gate_phase ^= 1u;
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              uint32_t hw[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {                     // this warp's token pair k: tokens 16 role + 2 k, + 1
+                const uint32_t mine = role ? pk[8 + k] : pk[k];
+                const uint32_t aw = role ? other[k] : mine, bw = role ? mine : other[k];
+                const float2 af = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw));
+                const float2 bf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw));
+                float cdf0, pdf0, cdf1, pdf1;
+                gelu_cdf_pdf(af.x, &cdf0, &pdf0);
+                gelu_cdf_pdf(af.y, &cdf1, &pdf1);
+                const float ga0 = af.x * cdf0, ga1 = af.y * cdf1;
+                const __nv_bfloat162 s0 = __floats2bfloat162_rn(ga0, bf.x * fmaf(af.x, pdf0, cdf0));
+                const __nv_bfloat162 s1 = __floats2bfloat162_rn(ga1, bf.y * fmaf(af.y, pdf1, cdf1));
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(ga0 * bf.x, ga1 * bf.y);
+                hw[k] = *reinterpret_cast<const uint32_t*>(&h2);
+                // saved factors: tile row = token of this warp (0..15), one word per lane
+                *reinterpret_cast<uint32_t*>(tr + (2 * k) * 144 + lane * 4) = *reinterpret_cast<const uint32_t*>(&s0);
+                *reinterpret_cast<uint32_t*>(tr + (2 * k + 1) * 144 + lane * 4) = *reinterpret_cast<const uint32_t*>(&s1);
+              }
+              __syncwarp();
+              const bool warp_ok = unit0 < p.gate_f;
+#pragma unroll
+              for (int pass = 0; pass < 4; ++pass) {            // a store writes 4 tokens x 32 hidden units x 4 bytes
+                const int trow = 4 * pass + (lane >> 3);
+                const uint4 val = *reinterpret_cast<const uint4*>(tr + trow * 144 + (lane & 7) * 16);
+                const long long off = __shfl_sync(0xffffffffu, q_off[0], 16 * role + trow);
+                // the saved row has one word (two bfloat16) per hidden unit: d_ff words = the 2 d_ff elements of q_off's row
+                if (off >= 0 && warp_ok)
+                  *reinterpret_cast<uint4*>(p.out + off + 2 * (unit0 + (lane & 7) * 4)) = val;
+              }
+              __syncwarp();
+#pragma unroll
+              for (int k = 0; k < 8; ++k) *reinterpret_cast<uint32_t*>(tr + k * 144 + lane * 4) = hw[k];
+              __syncwarp();
+              const uint8_t* src = tr + (lane >> 2) * 144 + (lane & 3) * 32;
+              const uint4 lo = *reinterpret_cast<const uint4*>(src);
+              const uint4 hi = *reinterpret_cast<const uint4*>(src + 16);
+#pragma unroll
+              for (int tb = 0; tb < 2; ++tb) {
+                const uint32_t sel = tb ? 0x7632u : 0x5410u;
+                const uint4 val = make_uint4(__byte_perm(lo.x, lo.y, sel), __byte_perm(lo.z, lo.w, sel),
+                                             __byte_perm(hi.x, hi.y, sel), __byte_perm(hi.z, hi.w, sel));
+                const long long off = __shfl_sync(0xffffffffu, q_off[0], 16 * role + 2 * (lane >> 2) + tb);
+                // the saved row has 2 d_ff elements, the hidden row d_ff: half the element offset
+                if (off >= 0 && col_ok) *reinterpret_cast<uint4*>(p.out2 + (off >> 1) + unit0 + (lane & 3) * 8) = val;
+              }
+            } else {
             long long offs[4];
 #pragma unroll
             for (int st = 0; st < 4; ++st) offs[st] = __shfl_sync(0xffffffffu, q_off[0], tcol(st));
             if (OP == kGemm2Combine) gate_s[lane] = q_gate[0];
             __syncwarp();
+            // gated dgrad2 writes two sets of columns from one accumulator: d a = dH . (b GELU'(a)) at column j, then
+            // d b = dH . GELU(a) at column d_ff + j
+#pragma unroll
+            for (int rnd = 0; rnd < (kDGated ? 2 : 1); ++rnd) {
+            if (rnd > 0) __syncwarp();                          // the tile's readers of the first set are done
+            const int mcol_r = mcol + rnd * p.gate_f;
             // transpose: this lane holds weight row m_warp + lane for 32 tokens.  Two tokens are packed into one
             // 32-bit word, tr[token pair][lane]: half the shared-memory stores of a 16-bit layout, each a full
             // 128-byte wavefront; a reader takes the words of eight rows (32 bytes) and separates the two tokens.
@@ -524,12 +632,13 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
                 a[u] = __uint_as_float(v[i4 + u]);
                 if (OP == kGemm2Combine) a[u] *= g[u];
                 if (OP == kGemm1Relu && !p.plain) a[u] = fmaxf(a[u], 0.f);
+                if (kDGated)                                    // high half: b GELU'(a); low half: GELU(a)
+                  a[u] *= __uint_as_float(rnd == 0 ? (gg[kDGated ? i4 + u : 0] & 0xFFFF0000u) : (gg[kDGated ? i4 + u : 0] << 16));
               }
               *reinterpret_cast<__nv_bfloat162*>(tr + (i4 >> 1) * 144 + lane * 4) = __floats2bfloat162_rn(a[0], a[1]);
               *reinterpret_cast<__nv_bfloat162*>(tr + ((i4 >> 1) + 1) * 144 + lane * 4) = __floats2bfloat162_rn(a[2], a[3]);
             }
             __syncwarp();
-            uint32_t mword[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
             for (int pass = 0; pass < 2; ++pass) {
               const uint8_t* src = tr + (8 * pass + (lane >> 2)) * 144 + (lane & 3) * 32;
@@ -571,52 +680,14 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
                     vv[q] = __floats2bfloat162_rn(a2.x + b2.x, a2.y + b2.y);
                   }
                 }
-                if (offs[st] >= 0 && col_ok) *reinterpret_cast<uint4*>(p.out + offs[st] + mcol) = val;
+                if (offs[st] >= 0 && col_ok) *reinterpret_cast<uint4*>(p.out + offs[st] + mcol_r) = val;
               }
             }
-            if constexpr (kGated) {
-              // hidden = GELU(a) . b from the rounded values just stored (what the backward pass reads back).  The a
-              // warp gates the chunk's token pairs 0-7, the b warp pairs 8-15: each reads the other's transpose tile
-              // between two handshakes, then transposes its 16 tokens x 32 hidden units through its own tile.
-              __syncwarp();
-              if (lane == 0) mbar_arrive(gate_bar);
-              ok = mbar_wait(gate_bar, gate_phase, abort_flag, p.status, 26);     // both tiles are written
-              gate_phase ^= 1u;
-              ok = __all_sync(0xffffffffu, ok);
-              if (!ok) break;
-              uint32_t hw[8];
+            }
+            }
+            if constexpr (kDGated) {
 #pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const int tp = 8 * role + k;
-                const uint32_t mine = *reinterpret_cast<const uint32_t*>(tr + tp * 144 + lane * 4);
-                const uint32_t other = *reinterpret_cast<const uint32_t*>(tr_other + tp * 144 + lane * 4);
-                const uint32_t aw = role ? other : mine, bw = role ? mine : other;
-                const float2 af = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw));
-                const float2 bf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw));
-                const __nv_bfloat162 h2 = __floats2bfloat162_rn(gelu_exact(af.x) * bf.x, gelu_exact(af.y) * bf.y);
-                hw[k] = *reinterpret_cast<const uint32_t*>(&h2);
-              }
-              __syncwarp();
-              if (lane == 0) mbar_arrive(gate_bar);
-              ok = mbar_wait(gate_bar, gate_phase, abort_flag, p.status, 27);     // both tiles have been read
-              gate_phase ^= 1u;
-              ok = __all_sync(0xffffffffu, ok);
-              if (!ok) break;
-#pragma unroll
-              for (int k = 0; k < 8; ++k) *reinterpret_cast<uint32_t*>(tr + k * 144 + lane * 4) = hw[k];
-              __syncwarp();
-              const uint8_t* src = tr + (lane >> 2) * 144 + (lane & 3) * 32;
-              const uint4 lo = *reinterpret_cast<const uint4*>(src);
-              const uint4 hi = *reinterpret_cast<const uint4*>(src + 16);
-#pragma unroll
-              for (int tb = 0; tb < 2; ++tb) {
-                const uint32_t sel = tb ? 0x7632u : 0x5410u;
-                const uint4 val = make_uint4(__byte_perm(lo.x, lo.y, sel), __byte_perm(lo.z, lo.w, sel),
-                                             __byte_perm(hi.x, hi.y, sel), __byte_perm(hi.z, hi.w, sel));
-                const long long off = __shfl_sync(0xffffffffu, q_off[0], 16 * role + 2 * (lane >> 2) + tb);
-                // a row of [a | b] has 2 d_ff columns, the hidden row d_ff: half the element offset
-                if (off >= 0 && col_ok) *reinterpret_cast<uint4*>(p.out2 + (off >> 1) + unit0 + (lane & 3) * 8) = val;
-              }
+              for (int i = 0; i < 32; ++i) gg[i] = gn[i];
             }
             if (OP == kGemm1Relu && !p.plain) {                 // lane i stores the mask word of token row i: one 128-byte line
               // token `lane` was handled as st = 2 (lane / 16) + (lane & 1) by the four lanes 4 ((lane / 2) & 7) ..
@@ -772,7 +843,12 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
     case kDgrad2Mask:      // A = W_out [E][f (m)][d (k)] K-major; B = dY_d [E][C][d] K-major
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.f; K = s.d;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 128); rc2 = make_token_maps(&bm, dyd, s.E, s.C, s.d);
-      q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.ld_out = s.f; q.plain = s.geglu; break;
+      q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.ld_out = s.f; q.plain = s.geglu;
+      if (s.geglu && !s.dropout) {   // the derivative of the gating in the epilogue: d[a | b] is written, dH never is
+        q.out = ws_ptr<__nv_bfloat16>(ws, p.dab); q.ld_out = fin; q.gate_f = s.f;
+        q.gate_in = ws_ptr<uint32_t>(ws, p.ab);
+      }
+      break;
     case kDgrad1Scatter:   // A = W_in [E][d (m)][f (k)] K-major; B = dH [E][C][f] K-major  (GEGLU: d[a | b], K = 2 f)
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.d; K = fin;
       rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 128); rc2 = make_token_maps(&bm, du, s.E, s.C, fin);
@@ -835,7 +911,9 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
       if (s.geglu) return launch_pair_op<kGemm1Gated>(tmA, tmB, q, dev, sm_count, st);
       return launch_pair_op<kGemm1Relu>(tmA, tmB, q, dev, sm_count, st);
     case kGemm2Combine: return launch_pair_op<kGemm2Combine>(tmA, tmB, q, dev, sm_count, st);
-    case kDgrad2Mask: return launch_pair_op<kDgrad2Mask>(tmA, tmB, q, dev, sm_count, st);
+    case kDgrad2Mask:
+      if (s.geglu && !s.dropout) return launch_pair_op<kDgrad2Gated>(tmA, tmB, q, dev, sm_count, st);
+      return launch_pair_op<kDgrad2Mask>(tmA, tmB, q, dev, sm_count, st);
     case kDgrad1Scatter: return launch_pair_op<kDgrad1Scatter>(tmA, tmB, q, dev, sm_count, st);
     case kWgrad2: return launch_pair_op<kWgrad2>(tmA, tmB, q, dev, sm_count, st);
     default: return launch_pair_op<kWgrad1>(tmA, tmB, q, dev, sm_count, st);

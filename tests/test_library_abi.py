@@ -91,9 +91,12 @@ def test_launch_count_is_reported(lib):
     # two products of dH share one launch
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 14
     # options add launches: four plan kernels per rerouting stage, one product kernel for input jitter, one GEGLU gating
-    # kernel (the backward one: the forward gating is in GEMM1's epilogue on this path), two expert-dropout kernels
+    # kernel (the backward one, because expert dropout has to touch dH first; the forward gating is in GEMM1's epilogue
+    # on this path), two expert-dropout kernels
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, reroute=True, input_jitter=True,
                                                           geglu=True, expert_dropout=0.4)) == 14 + 4 + 1 + 1 + 2
+    # GEGLU experts alone: both gatings are in the epilogues
+    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, geglu=True)) == 14
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, reroute=True, reroute_stages=3)) == 14 + 12
     # the fp32 path gates in element-wise kernels both ways
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, dtype=sm.F32, geglu=True)) == 16 + 2
