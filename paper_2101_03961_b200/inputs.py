@@ -67,6 +67,7 @@ CONFIGS = {
     # the paper's own Switch-Base layer shape with GEGLU experts (its hyper-parameter table: d_model 768, d_ff 2048)
     "geglu_base": SwitchConfig("geglu_base", 32768, 768, 2048, 128, 1.25, geglu=True),
     # the same table's Switch-Large (d_model 1024, d_ff 2816) and Switch-XXL (d_model 4096, d_ff 10240, 64 experts)
+    "geglu_base_quarter": SwitchConfig("geglu_base_quarter", 8192, 768, 2048, 32, 1.25, geglu=True),   # for profiler captures
     "geglu_large": SwitchConfig("geglu_large", 32768, 1024, 2816, 128, 1.25, geglu=True),
     "geglu_xxl": SwitchConfig("geglu_xxl", 16384, 4096, 10240, 64, 1.25, geglu=True),
     # many tokens, narrow layer: exercises the token-count limits of the router's partial sums and of the plan's scan
