@@ -75,12 +75,12 @@ enum switch_moe_gemm_path {
    the capacity of Eq. 3; f in the auxiliary loss counts the first choice.  The library numbers the 2T assignments
    v = t (first choice of token t) and v = T + t (second choice): the workspace regions EXPERT_INDEX, GATE, SLOT and
    DGATE then have 2T entries and TOKEN_OF_SLOT holds v.  Needs T to be a multiple of 256; not together with
-   REROUTE or several routing groups.  With RESIDUAL the input row is added where the two assignments' rows are
+   REROUTE, several routing groups, GEGLU experts, expert dropout, input jitter or logit noise (UNSUPPORTED_SHAPE).  With RESIDUAL the input row is added where the two assignments' rows are
    summed (one rounding of the three-term sum), and dy likewise on the way back.
    SWITCH_MOE_FLAG_EXPERT_DROPOUT: expert dropout (the fine-tuning regularisation of Section 2.4: a larger dropout
    rate on the hidden activations inside every expert): the experts' hidden activations are
    multiplied by keep / (1 - expert_dropout), and so is their gradient on the way back.  The keep mask is an input
-   (expert_keep), one bit per hidden unit of every slot row; the caller draws it. */
+   (expert_keep), one bit per hidden unit of every slot row; the caller draws it.  One routing group only. */
 enum switch_moe_flags {
   SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2, SWITCH_MOE_FLAG_INPUT_JITTER = 4, SWITCH_MOE_FLAG_GEGLU = 8,
   SWITCH_MOE_FLAG_TOP2 = 16, SWITCH_MOE_FLAG_EXPERT_DROPOUT = 32

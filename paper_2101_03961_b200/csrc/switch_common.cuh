@@ -106,10 +106,14 @@ inline int resolve_shape(const switch_moe_config* cfg, Shape* s) {
   if (s->dropout) {
     if (!(cfg->expert_dropout >= 0.f) || !(cfg->expert_dropout < 1.f)) return SWITCH_MOE_INVALID_ARGUMENT;
     if (cfg->d_ff % 32 != 0) return SWITCH_MOE_UNSUPPORTED_SHAPE;
+    if (G > 1) return SWITCH_MOE_UNSUPPORTED_SHAPE;          // built and checked for one routing group
     s->keep_scale = 1.f / (1.f - cfg->expert_dropout);
   }
   s->top2 = (cfg->flags & SWITCH_MOE_FLAG_TOP2) ? 1 : 0;
-  if (s->top2 && ((cfg->flags & SWITCH_MOE_FLAG_REROUTE) || G > 1 || cfg->T % kPlanBlockTokens != 0))
+  // top-2 routing is built and checked for the plain ReLU layer (with or without the skip path) only
+  if (s->top2 && ((cfg->flags & (SWITCH_MOE_FLAG_REROUTE | SWITCH_MOE_FLAG_GEGLU | SWITCH_MOE_FLAG_EXPERT_DROPOUT |
+                                 SWITCH_MOE_FLAG_INPUT_JITTER)) ||
+                  cfg->router_noise != nullptr || G > 1 || cfg->T % kPlanBlockTokens != 0))
     return SWITCH_MOE_UNSUPPORTED_SHAPE;
   s->Tv = s->top2 ? 2 * cfg->T : cfg->T;
   s->jitter = (cfg->flags & SWITCH_MOE_FLAG_INPUT_JITTER) ? 1 : 0;

@@ -254,7 +254,8 @@ def test_several_routing_groups_in_one_call_match_oracle(cfg, path, tol, groups,
 
 
 def test_group_count_limits_are_enforced():
-    for kw in (dict(T=2048, groups=3), dict(T=2048 + 256, groups=2), dict(T=1000, groups=2)):
+    for kw in (dict(T=2048, groups=3), dict(T=2048 + 256, groups=2), dict(T=1000, groups=2),
+               dict(groups=2, expert_dropout=0.2)):          # expert dropout: one routing group only
         base = dict(T=2048, d_model=128, d_ff=256, E=8, capacity_factor=1.0)
         base.update(kw)
         with pytest.raises(sm.SwitchMoeError):
@@ -673,7 +674,8 @@ def test_top2_routing_matches_oracle(cfg, path, tol):
 
 
 def test_top2_is_refused_with_the_options_it_does_not_combine_with():
-    for kw in (dict(reroute=True), dict(groups=2), dict(T=2000)):
+    for kw in (dict(reroute=True), dict(groups=2), dict(T=2000), dict(geglu=True), dict(expert_dropout=0.2),
+               dict(input_jitter=True)):
         base = dict(T=2048, d_model=128, d_ff=256, E=8, capacity_factor=1.5, top2=True)
         base.update(kw)
         with pytest.raises(sm.SwitchMoeError):
@@ -706,7 +708,8 @@ def test_results_are_bitwise_reproducible(kw):
 
 
 def test_options_combine():
-    """Rerouting + the skip path + GEGLU experts + logit noise + input jitter in one call; several groups + GEGLU."""
+    """Rerouting + the skip path + GEGLU experts + logit noise + input jitter in one call; several groups + GEGLU;
+    several groups + the skip path + input jitter."""
     cfg = si.SwitchConfig("combo", 2048, 128, 256, 8, 1.0, bias_std=0.5)
     _check_layer(cfg, sm.GEMM_DEFAULT, TOL_BF16, reroute=True, residual=True, geglu=True, noise_eps=0.3, jitter_eps=0.2,
                  d_aux=0.4)
@@ -714,6 +717,8 @@ def test_options_combine():
                  d_aux=0.4)
     _check_layer(si.SwitchConfig("combo_groups", 2048, 128, 256, 8, 1.0, bias_std=0.3), sm.GEMM_DEFAULT, TOL_BF16,
                  groups=4, geglu=True, noise_eps=0.3, d_aux=0.4)
+    _check_layer(si.SwitchConfig("combo_groups", 2048, 128, 256, 8, 1.0, bias_std=0.3), sm.GEMM_DEFAULT, TOL_BF16,
+                 groups=2, residual=True, jitter_eps=0.2, d_aux=0.4)
 
 
 def test_top2_with_a_single_expert_has_no_second_choice():
@@ -734,8 +739,9 @@ def test_top2_with_a_single_expert_has_no_second_choice():
 
 @pytest.mark.parametrize("cfg,path,tol,kw", [
     (TINY, sm.GEMM_DEFAULT, TOL_F32, {}), (MID, sm.GEMM_SIMT, TOL_BF16, {}), (MID, sm.GEMM_DEFAULT, TOL_BF16, {}),
-    (RAGGED, sm.GEMM_DEFAULT, TOL_BF16, dict(reroute=True)), (MANY, sm.GEMM_DEFAULT, TOL_BF16, dict(geglu=True, residual=True))],
-    ids=["tiny_f32", "mid_fma", "mid_tc", "ragged_tc_reroute", "many_tc_geglu_skip"])
+    (RAGGED, sm.GEMM_DEFAULT, TOL_BF16, dict(reroute=True)), (MANY, sm.GEMM_DEFAULT, TOL_BF16, dict(geglu=True, residual=True)),
+    (MID, sm.GEMM_SIMT, TOL_BF16, dict(geglu=True)), (MID, sm.GEMM_DEFAULT, TOL_BF16, dict(geglu=True, reroute=True, reroute_stages=2))],
+    ids=["tiny_f32", "mid_fma", "mid_tc", "ragged_tc_reroute", "many_tc_geglu_skip", "mid_fma_geglu", "mid_tc_geglu_reroute2"])
 def test_expert_dropout_matches_oracle(cfg, path, tol, kw):
     """Hidden activations and their gradient are multiplied by keep / (1 - rate); the mask is a seeded input."""
     _check_layer(cfg, path, tol, dropout=0.4, d_aux=0.7, **kw)
