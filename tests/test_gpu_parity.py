@@ -344,7 +344,9 @@ def test_jitter_flag_without_the_factors_is_refused():
     (RAGGED, sm.GEMM_DEFAULT, TOL_BF16, False), (MANY, sm.GEMM_DEFAULT, TOL_BF16, True)],
     ids=["tiny_f32", "mid_fma", "mid_tc", "ragged_tc", "many_tc_skip"])
 def test_geglu_experts_match_oracle(cfg, path, tol, residual):
-    """hidden = GELU(x W_0) . (x W_1) (Table 9): one grouped GEMM with 2 d_ff columns, gating and its derivative after."""
+    """hidden = GELU(x W_0) . (x W_1) (Table 9): one grouped GEMM with 2 d_ff columns; the gating and its derivative
+    sit in the GEMM epilogues on the CTA-pair path and in element-wise kernels on the others.  The ragged case has
+    d_ff = 320: the last CTA pair of the gated GEMM1 holds hidden units beyond d_ff, which must not be stored."""
     _check_layer(cfg, path, tol, geglu=True, residual=residual, d_aux=0.7)
 
 
