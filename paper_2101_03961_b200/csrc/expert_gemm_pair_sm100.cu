@@ -1,7 +1,8 @@
 // Grouped expert GEMMs on pairs of SMs (tcgen05 cta_group::2, M = 256), bfloat16 in, float32 accumulate, bfloat16
 // out: the expert FFN h = x W_in, y = ReLU(h) W_out (Section 5, FFN review) and its derivatives, with the layer's
 // element-wise steps fused into the epilogues (ReLU, the gate of Eq. 2 with the scatter back to token order, the
-// ReLU mask of the backward pass).
+// ReLU mask of the backward pass; for GEGLU experts the gating GELU(a) . b in GEMM1's epilogue and its derivative in
+// dgrad2's, two more instantiations of the same kernel).
 //
 // Orientation.  An expert has about 256 tokens but thousands of weight rows, so the weight matrix sits on the MMA's
 // M side (256 rows per CTA pair, 128 per CTA) and the expert's tokens on the N side, whose granularity is 16:
@@ -77,7 +78,7 @@ struct PairParams {
   int* status;
   const __nv_bfloat16* res;   // combine / scatter with the skip path inside the layer: rows added to the output (x or dy)
   __nv_bfloat16* out2;        // combine with the skip path: second copy of the output without it
-  int plain;                  // GEMM1 / dgrad2 without ReLU and without the ReLU mask (GEGLU experts gate elsewhere)
+  int plain;                  // GEMM1 / dgrad2 without ReLU and without the ReLU mask (GEGLU experts)
   int gate_f;                 // gated products: d_ff.  Gated GEMM1: W_in has 2 d_ff columns [W_0 | W_1]; out = the saved
                               // factors, one 32-bit word {GELU(a), b GELU'(a)} per hidden unit and slot row; out2 = hidden.
                               // Gated dgrad2: out = d[a | b] (2 d_ff columns), gate_in = those words.
@@ -826,7 +827,7 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
   int K = 0;
   switch (op) {
     case kGemm1Relu:       // A = W_in [E][d (k)][f (m)]: m contiguous -> MN-major; B = X_d [E][C][d] K-major
-      q.token_op = 1; q.a_mn_major = 1; q.Mw = fin; K = s.d;   // GEGLU: [a | b], 2 f output columns, no ReLU
+      q.token_op = 1; q.a_mn_major = 1; q.Mw = fin; K = s.d;   // GEGLU: 2 f weight columns [W_0 | W_1], no ReLU
       rc = make_map(&tmA, a.W_in, s.E, s.d, fin, 64); rc2 = make_token_maps(&bm, xd, s.E, s.C, s.d);
       q.out = s.geglu ? ws_ptr<__nv_bfloat16>(ws, p.ab) : ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = fin;
       q.plain = s.geglu;
