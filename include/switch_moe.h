@@ -66,9 +66,8 @@ enum switch_moe_gemm_path {
    columns of W_0 and the same 64 columns of W_1, the two epilogue warps that hold a and b of a hidden unit exchange
    them through shared memory): it writes the hidden activations and, for the backward pass, the two factors
    GELU(a) and b GELU'(a) of every hidden unit (rounded to the activation dtype) instead of a and b; dgrad2's
-   epilogue multiplies dH by them and writes d[a | b] directly.  With expert dropout, and on the other paths, the
-   derivative of the gating (and on the other paths the gating itself) is an element-wise kernel over the kept
-   rows.  Not available on SWITCH_MOE_GEMM_TC_1CTA.
+   epilogue multiplies dH by them and writes d[a | b] directly.  On the other paths the gating and its derivative
+   are element-wise kernels over the kept rows.  Not available on SWITCH_MOE_GEMM_TC_1CTA.
    SWITCH_MOE_FLAG_TOP2: top-2 routing, the Mixture-of-Experts layer the paper compares with (Eq. 1-2 with the two
    highest-probability experts): y_t = p_a E_a(x_t) + p_b E_b(x_t) with the softmax probabilities of Eq. 1 as they
    are.  Every token's first choice is placed before any second choice (token order within each round), all against
@@ -80,7 +79,10 @@ enum switch_moe_gemm_path {
    SWITCH_MOE_FLAG_EXPERT_DROPOUT: expert dropout (the fine-tuning regularisation of Section 2.4: a larger dropout
    rate on the hidden activations inside every expert): the experts' hidden activations are
    multiplied by keep / (1 - expert_dropout), and so is their gradient on the way back.  The keep mask is an input
-   (expert_keep), one bit per hidden unit of every slot row; the caller draws it.  One routing group only. */
+   (expert_keep), one bit per hidden unit of every slot row; the caller draws it.  On the default path both happen in
+   GEMM epilogues (GEMM1 applies the factor before it rounds; the ReLU mask bits it saves then say "kept and
+   positive", so dgrad2 only multiplies by 1 / (1 - rate); with GEGLU experts the factors saved for the backward pass
+   carry it), on the other paths in element-wise kernels.  One routing group only. */
 enum switch_moe_flags {
   SWITCH_MOE_FLAG_RESIDUAL = 1, SWITCH_MOE_FLAG_REROUTE = 2, SWITCH_MOE_FLAG_INPUT_JITTER = 4, SWITCH_MOE_FLAG_GEGLU = 8,
   SWITCH_MOE_FLAG_TOP2 = 16, SWITCH_MOE_FLAG_EXPERT_DROPOUT = 32

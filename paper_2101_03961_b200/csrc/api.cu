@@ -147,7 +147,8 @@ int switch_moe_fwd(const switch_moe_config* cfg, const void* x, const float* W_r
   SWMOE_TRY(run_gemm(kGemm1Relu, c, a, workspace, st));
   // hidden = GELU(a) . b: inside GEMM1's epilogue on the CTA-pair path, an element-wise kernel otherwise
   if (c.s.geglu && c.s.gemm_path != 0) SWMOE_TRY(launch_geglu_fwd(c.s, c.p, workspace, st));
-  if (c.s.dropout) SWMOE_TRY(launch_expert_dropout(c.s, c.p, false, workspace, st));
+  // expert dropout: in GEMM1's epilogue on the CTA-pair path, an element-wise kernel otherwise
+  if (c.s.dropout && c.s.gemm_path != 0) SWMOE_TRY(launch_expert_dropout(c.s, c.p, false, workspace, st));
   SWMOE_TRY(mark(cfg, 4, st));
   SWMOE_TRY(run_gemm(kGemm2Combine, c, a, workspace, st));
   if (c.s.top2)                                                                   // Eq. 2: sum over the two experts
@@ -176,10 +177,10 @@ int switch_moe_bwd(const switch_moe_config* cfg, const void* dy, float d_aux, co
   SWMOE_TRY(launch_gather_dy(c.s, c.p, dy, c.s.top2 ? ws_ptr<void>(workspace, c.p.yv) : y, dx, workspace, st));
   SWMOE_TRY(mark(cfg, 7, st));
   SWMOE_TRY(run_gemm(kDgrad2Mask, c, a, workspace, st));
-  if (c.s.dropout) SWMOE_TRY(launch_expert_dropout(c.s, c.p, true, workspace, st));   // same factors on the way back
-  // d[a | b] from dH: inside dgrad2's epilogue on the CTA-pair path (unless expert dropout has to touch dH first),
-  // an element-wise kernel otherwise
-  if (c.s.geglu && (c.s.gemm_path != 0 || c.s.dropout)) SWMOE_TRY(launch_geglu_bwd(c.s, c.p, workspace, st));
+  // the dropout factors on the way back and d[a | b] from dH: inside dgrad2's epilogue on the CTA-pair path,
+  // element-wise kernels otherwise
+  if (c.s.dropout && c.s.gemm_path != 0) SWMOE_TRY(launch_expert_dropout(c.s, c.p, true, workspace, st));
+  if (c.s.geglu && c.s.gemm_path != 0) SWMOE_TRY(launch_geglu_bwd(c.s, c.p, workspace, st));
   SWMOE_TRY(mark(cfg, 8, st));
   SWMOE_TRY(run_gemm(kWgrad2, c, a, workspace, st));
   SWMOE_TRY(mark(cfg, 9, st));
@@ -330,11 +331,12 @@ int switch_moe_stage_launches(const switch_moe_config* cfg, int32_t* launches_ou
   // scan, assign; stage 2 of rerouting adds four
   n[1] = (s.router_hist ? (s.G == 1 ? 1 : 2) : 3) + 4 * s.reroute_stages;
   n[2] = 1;                                           // gather
-  n[3] = 1 + (s.geglu && s.gemm_path != 0 ? 1 : 0) + (s.dropout ? 1 : 0);   // GEMM1 (+ GEGLU gating kernel, + expert dropout)
+  const int slow = s.gemm_path != 0 ? 1 : 0;   // gating and dropout are element-wise kernels off the CTA-pair path
+  n[3] = 1 + (s.geglu ? slow : 0) + (s.dropout ? slow : 0);   // GEMM1 (+ GEGLU gating kernel, + expert dropout kernel)
   n[4] = 1 + (s.top2 ? 1 : 0);                        // GEMM2 + combine (+ sum of the two assignments' rows)
   // backward.  With the paired-CTA path the two products of dH are one launch (stage 9).
   n[6] = 1;
-  n[7] = 1 + (s.dropout ? 1 : 0) + (s.geglu && (s.gemm_path != 0 || s.dropout) ? 1 : 0);
+  n[7] = 1 + (s.dropout ? slow : 0) + (s.geglu ? slow : 0);
   n[8] = 1;
   n[9] = 1;
   n[10] = (s.gemm_path == 0 ? 0 : 1) + (s.top2 ? 1 : 0);

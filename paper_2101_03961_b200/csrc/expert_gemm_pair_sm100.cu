@@ -83,6 +83,12 @@ struct PairParams {
                               // factors, one 32-bit word {GELU(a), b GELU'(a)} per hidden unit and slot row; out2 = hidden.
                               // Gated dgrad2: out = d[a | b] (2 d_ff columns), gate_in = those words.
   const uint32_t* gate_in;
+  // expert dropout (Section 2.4) in the epilogues: GEMM1 multiplies the hidden activations by keep / (1 - rate) before
+  // it rounds them and takes the mask bits (the gated GEMM1: the hidden activations and both saved factors); dgrad2
+  // multiplies by 1 / (1 - rate), its mask bits already say "kept and positive".
+  const uint32_t* keep_bits;  // [E * C][d_ff / 32]: bit i of word [row][w] = keep hidden unit 32 w + i; or null
+  int keep_words;             // d_ff / 32
+  float keep_scale;           // 1 / (1 - rate); 1 without dropout
   int stages, stage_bytes;    // operand ring: token products size a stage for the widest tile the capacity allows
   // ceil(2^32 / divisor) for the three divisions of the tile decode (n_mpairs; n_mpairs * n_ntiles_fixed;
   // n_ntiles_fixed): id / d = umulhi(id, magic) as long as id * d < 2^32
@@ -178,7 +184,7 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
 //
 // `pair` of `n_pairs` is this CTA pair's place among the pairs that work on this product: the whole grid for a
 // launch of one product, a share of it when two products run side by side in one launch (below).
-template <int OP>
+template <int OP, bool DROP = false>                          // DROP: expert dropout in this product's epilogue
 __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet& bm, const PairParams& p,
                                           const int pair, const int n_pairs) {
   constexpr bool kGated = OP == kGemm1Gated, kDGated = OP == kDgrad2Gated;
@@ -413,6 +419,14 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
         // everything the epilogue needs from global memory is requested here, before the accumulator is awaited
 #pragma unroll
         for (int k = 0; k < kQueue; ++k) describe(n_chunks - 1 - half - 2 * k, &q_off[k], &q_gate[k]);
+        if (DROP && (OP == kGemm1Relu || kGated) && (kGated ? unit0 < p.gate_f : m_warp < p.Mw)) {
+          const int unit_word = (kGated ? unit0 : m_warp) >> 5;   // this warp's 32 hidden units are one word per row
+#pragma unroll
+          for (int k = 0; k < kQueue; ++k)
+            if (q_off[k] >= 0)
+              q_mw[k] = p.keep_bits[((long long)t.e * p.C + t.row0 + chunk_tok0(n_chunks - 1 - half - 2 * k) + lane) *
+                                        p.keep_words + unit_word];
+        }
         if (OP == kDgrad2Mask && !p.plain && m_warp < p.Mw) {
 #pragma unroll
           for (int k = 0; k < kQueue; ++k)
@@ -569,9 +583,16 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
                 float cdf0, pdf0, cdf1, pdf1;
                 gelu_cdf_pdf(af.x, &cdf0, &pdf0);
                 gelu_cdf_pdf(af.y, &cdf1, &pdf1);
-                const float ga0 = af.x * cdf0, ga1 = af.y * cdf1;
-                const __nv_bfloat162 s0 = __floats2bfloat162_rn(ga0, bf.x * fmaf(af.x, pdf0, cdf0));
-                const __nv_bfloat162 s1 = __floats2bfloat162_rn(ga1, bf.y * fmaf(af.y, pdf1, cdf1));
+                float ga0 = af.x * cdf0, ga1 = af.y * cdf1;
+                float gp0 = bf.x * fmaf(af.x, pdf0, cdf0), gp1 = bf.y * fmaf(af.y, pdf1, cdf1);
+                if (DROP) {                                     // expert dropout: the hidden unit's factor on all three
+                  const uint32_t kw0 = __shfl_sync(0xffffffffu, q_mw[0], 16 * role + 2 * k);
+                  const uint32_t kw1 = __shfl_sync(0xffffffffu, q_mw[0], 16 * role + 2 * k + 1);
+                  const float f0 = (kw0 >> lane) & 1u ? p.keep_scale : 0.f, f1 = (kw1 >> lane) & 1u ? p.keep_scale : 0.f;
+                  ga0 *= f0; gp0 *= f0; ga1 *= f1; gp1 *= f1;
+                }
+                const __nv_bfloat162 s0 = __floats2bfloat162_rn(ga0, gp0);
+                const __nv_bfloat162 s1 = __floats2bfloat162_rn(ga1, gp1);
                 const __nv_bfloat162 h2 = __floats2bfloat162_rn(ga0 * bf.x, ga1 * bf.y);
                 hw[k] = *reinterpret_cast<const uint32_t*>(&h2);
                 // saved factors: tile row = token of this warp (0..15), one word per lane
@@ -633,6 +654,11 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
                 a[u] = __uint_as_float(v[i4 + u]);
                 if (OP == kGemm2Combine) a[u] *= g[u];
                 if (OP == kGemm1Relu && !p.plain) a[u] = fmaxf(a[u], 0.f);
+                if (DROP && OP == kGemm1Relu) {                 // expert dropout before the rounding and the mask bits
+                  const uint32_t kw = __shfl_sync(0xffffffffu, q_mw[0], i4 + u);
+                  a[u] = (kw >> lane) & 1u ? a[u] * p.keep_scale : 0.f;
+                }
+                if (DROP && OP == kDgrad2Mask) a[u] *= p.keep_scale;
                 if (kDGated)                                    // high half: b GELU'(a); low half: GELU(a)
                   a[u] *= __uint_as_float(rnd == 0 ? (gg[kDGated ? i4 + u : 0] & 0xFFFF0000u) : (gg[kDGated ? i4 + u : 0] << 16));
               }
@@ -734,11 +760,11 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmA, const BMapSet&
   }
 }
 
-template <int OP>
+template <int OP, bool DROP = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
 expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ BMapSet bm,
                         const PairParams p) {
-  pair_body<OP>(tmA, bm, p, (int)(blockIdx.x >> 1), (int)(gridDim.x >> 1));
+  pair_body<OP, DROP>(tmA, bm, p, (int)(blockIdx.x >> 1), (int)(gridDim.x >> 1));
 }
 
 // Two products that read the same activations, side by side in one launch: the first `split` CTA pairs work on
@@ -782,14 +808,14 @@ int pair_grid(Kernel kernel, int* cached_grid, int dev, int sm_count, cudaStream
   return SWITCH_MOE_OK;
 }
 
-template <int OP>
+template <int OP, bool DROP = false>
 int launch_pair_op(const CUtensorMap& tmA, const BMapSet& tmB, const PairParams& q, int dev, int sm_count,
                    cudaStream_t st) {
   static int cached_grid[64] = {0};
   int grid = 0;
-  const int rc = pair_grid(expert_gemm_pair_kernel<OP>, cached_grid, dev, sm_count, st, &grid);
+  const int rc = pair_grid(expert_gemm_pair_kernel<OP, DROP>, cached_grid, dev, sm_count, st, &grid);
   if (rc != SWITCH_MOE_OK) return rc;
-  launch_k(expert_gemm_pair_kernel<OP>, dim3(grid), dim3(kPThreads), kPSmemBytes, st, tmA, tmB, q);
+  launch_k(expert_gemm_pair_kernel<OP, DROP>, dim3(grid), dim3(kPThreads), kPSmemBytes, st, tmA, tmB, q);
   return launch_status();
 }
 
@@ -820,6 +846,7 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
   q.status = ws_ptr<int>(ws, p.status);
   q.hmask = ws_ptr<uint32_t>(ws, p.hmask);
   q.hmask_rows = (long long)s.E * s.C;
+  q.keep_scale = 1.f;
   CUtensorMap& tmA = *tmA_out;
   BMapSet& bm = *tmB_out;
   CUtensorMap& tmB = bm.m[0];
@@ -832,6 +859,10 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
       q.out = s.geglu ? ws_ptr<__nv_bfloat16>(ws, p.ab) : ws_ptr<__nv_bfloat16>(ws, p.h); q.ld_out = fin;
       q.plain = s.geglu;
       if (s.geglu) { q.gate_f = s.f; q.out2 = ws_ptr<__nv_bfloat16>(ws, p.h); }   // gating in the epilogue
+      if (s.dropout) {
+        if (s.keep_bits == nullptr || (reinterpret_cast<uintptr_t>(s.keep_bits) & 3u) != 0) return SWITCH_MOE_INVALID_ARGUMENT;
+        q.keep_bits = s.keep_bits; q.keep_words = s.f / 32; q.keep_scale = s.keep_scale;
+      }
       break;
     case kGemm2Combine:    // A = W_out [E][f (k)][d (m)] MN-major; B = H [E][C][f] K-major
       q.token_op = 1; q.a_mn_major = 1; q.Mw = s.d; K = s.f;
@@ -845,7 +876,8 @@ int pair_problem(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a, vo
       q.token_op = 1; q.a_mn_major = 0; q.Mw = s.f; K = s.d;
       rc = make_map(&tmA, a.W_out, s.E, s.f, s.d, 128); rc2 = make_token_maps(&bm, dyd, s.E, s.C, s.d);
       q.out = ws_ptr<__nv_bfloat16>(ws, p.dh); q.ld_out = s.f; q.plain = s.geglu;
-      if (s.geglu && !s.dropout) {   // the derivative of the gating in the epilogue: d[a | b] is written, dH never is
+      if (s.dropout && !s.geglu) q.keep_scale = s.keep_scale;   // (GEGLU: the saved factors carry the dropout factor)
+      if (s.geglu) {   // the derivative of the gating in the epilogue: d[a | b] is written, dH never is
         q.out = ws_ptr<__nv_bfloat16>(ws, p.dab); q.ld_out = fin; q.gate_f = s.f;
         q.gate_in = ws_ptr<uint32_t>(ws, p.ab);
       }
@@ -909,12 +941,15 @@ int launch_pair_gemm(GemmOp op, const Shape& s, const Plan& p, const GemmArgs& a
   if (rc != SWITCH_MOE_OK) return rc;
   switch (op) {
     case kGemm1Relu:
-      if (s.geglu) return launch_pair_op<kGemm1Gated>(tmA, tmB, q, dev, sm_count, st);
-      return launch_pair_op<kGemm1Relu>(tmA, tmB, q, dev, sm_count, st);
+      if (s.geglu) return s.dropout ? launch_pair_op<kGemm1Gated, true>(tmA, tmB, q, dev, sm_count, st)
+                                    : launch_pair_op<kGemm1Gated>(tmA, tmB, q, dev, sm_count, st);
+      return s.dropout ? launch_pair_op<kGemm1Relu, true>(tmA, tmB, q, dev, sm_count, st)
+                       : launch_pair_op<kGemm1Relu>(tmA, tmB, q, dev, sm_count, st);
     case kGemm2Combine: return launch_pair_op<kGemm2Combine>(tmA, tmB, q, dev, sm_count, st);
     case kDgrad2Mask:
-      if (s.geglu && !s.dropout) return launch_pair_op<kDgrad2Gated>(tmA, tmB, q, dev, sm_count, st);
-      return launch_pair_op<kDgrad2Mask>(tmA, tmB, q, dev, sm_count, st);
+      if (s.geglu) return launch_pair_op<kDgrad2Gated>(tmA, tmB, q, dev, sm_count, st);
+      return s.dropout ? launch_pair_op<kDgrad2Mask, true>(tmA, tmB, q, dev, sm_count, st)
+                       : launch_pair_op<kDgrad2Mask>(tmA, tmB, q, dev, sm_count, st);
     case kDgrad1Scatter: return launch_pair_op<kDgrad1Scatter>(tmA, tmB, q, dev, sm_count, st);
     case kWgrad2: return launch_pair_op<kWgrad2>(tmA, tmB, q, dev, sm_count, st);
     default: return launch_pair_op<kWgrad1>(tmA, tmB, q, dev, sm_count, st);

@@ -112,38 +112,6 @@ expert_dropout_kernel(const uint32_t* __restrict__ keep_bits, const int* __restr
   }
 }
 
-// Backward gating from the factors the gated GEMM1 saved (CTA-pair path): word [row][j] = {GELU(a), b GELU'(a)} as two
-// bfloat16; dab[row][j] = dh . (b GELU'(a)), dab[row][f + j] = dh . GELU(a).  One warp per slot row; a lane takes eight
-// hidden units at a time (16 bytes of dh, 32 bytes of factors).
-__global__ void __launch_bounds__(256)
-geglu_bwd_saved_kernel(const uint4* __restrict__ saved, const int* __restrict__ kept, int E, int C, int f_vec,
-                       const uint4* __restrict__ dh, uint4* __restrict__ dab) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const int lane = threadIdx.x & 31;
-  const int s = blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (s >= E * C) return;
-  const int ex = s / C, pos = s - ex * C;
-  if (pos >= min(C, (kept[ex] + 15) / 16 * 16)) return;
-  const uint4* srow = saved + (size_t)s * 2 * f_vec;
-  const uint4* grow = dh + (size_t)s * f_vec;
-  uint4* drow = dab + (size_t)s * 2 * f_vec;
-  for (int v = lane; v < f_vec; v += 32) {
-    float g[8];
-    Pack<__nv_bfloat16>::load(grow[v], g);
-    const uint4 w0 = srow[2 * v], w1 = srow[2 * v + 1];
-    const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-    float o[8], o2[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      o[i] = g[i] * __uint_as_float(w[i] & 0xFFFF0000u);       // high half: b GELU'(a)
-      o2[i] = g[i] * __uint_as_float(w[i] << 16);              // low half: GELU(a)
-    }
-    drow[v] = Pack<__nv_bfloat16>::store(o);
-    drow[f_vec + v] = Pack<__nv_bfloat16>::store(o2);
-  }
-}
-
 template <bool kBackward>
 int launch(const Shape& s, const Plan& p, void* ws, cudaStream_t st) {
   const int f_vec = (int)((size_t)s.f * s.elt / 16);
@@ -151,11 +119,6 @@ int launch(const Shape& s, const Plan& p, void* ws, cudaStream_t st) {
   const uint4* ab = ws_ptr<uint4>(ws, p.ab);
   uint4* hh = ws_ptr<uint4>(ws, kBackward ? p.dh : p.h);
   uint4* dab = ws_ptr<uint4>(ws, p.dab);
-  if (kBackward && s.gemm_path == 0) {                       // the pair path's GEMM1 saved the factors, not [a | b]
-    launch_k(geglu_bwd_saved_kernel, dim3(blocks), dim3(256), 0, st, ab, ws_ptr<int>(ws, p.kept), s.E, s.C, f_vec,
-             static_cast<const uint4*>(hh), dab);
-    return launch_status();
-  }
   if (s.dtype == SWITCH_MOE_BF16)
     launch_k(geglu_kernel<__nv_bfloat16, kBackward>, dim3(blocks), dim3(256), 0, st, ab, ws_ptr<int>(ws, p.kept), s.E, s.C,
              f_vec, hh, dab);

@@ -90,13 +90,13 @@ def test_launch_count_is_reported(lib):
     # bf16 default path: the router's epilogue leaves the probabilities' column sums and the plan's histograms, and the
     # two products of dH share one launch
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0)) == 14
-    # options add launches: four plan kernels per rerouting stage, one product kernel for input jitter, one GEGLU gating
-    # kernel (the backward one, because expert dropout has to touch dH first; the forward gating is in GEMM1's epilogue
-    # on this path), two expert-dropout kernels
+    # options add launches: four plan kernels per rerouting stage, one product kernel for input jitter; GEGLU gating and
+    # expert dropout live in the GEMM epilogues on this path and add none
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, reroute=True, input_jitter=True,
-                                                          geglu=True, expert_dropout=0.4)) == 14 + 4 + 1 + 1 + 2
-    # GEGLU experts alone: both gatings are in the epilogues
+                                                          geglu=True, expert_dropout=0.4)) == 14 + 4 + 1
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, geglu=True)) == 14
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, reroute=True, reroute_stages=3)) == 14 + 12
-    # the fp32 path gates in element-wise kernels both ways
+    # the fp32 path gates, and drops hidden units, in element-wise kernels both ways
     assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, dtype=sm.F32, geglu=True)) == 16 + 2
+    assert sm.switch_moe_launches_per_step(sm.make_config(512, 64, 256, 8, 1.0, dtype=sm.F32, geglu=True,
+                                                          expert_dropout=0.4)) == 16 + 2 + 2
