@@ -234,8 +234,9 @@ def check_next_choices(gpu_alt: np.ndarray, p: np.ndarray, e: np.ndarray, plan: 
         waiting = ~plan["keep"]
         left = np.where(tried, -np.inf, p)
         want = np.where(np.isfinite(left.max(axis=1)), np.argmax(left, axis=1), -1)
-        if not flipped:
-            np.testing.assert_array_equal(want, so.next_choice(p, prev))
+        if not flipped:                                       # (a token whose first choice flipped inside the gap has
+            same = e == np.argmax(p, axis=1)                  # the oracle's own argmax still untried: its ranking walk
+            np.testing.assert_array_equal(want[same], so.next_choice(p, prev)[same])   # starts one place later)
         assert np.all(got[~waiting] == -1)
         diff = np.flatnonzero(waiting & (got != want))
         if diff.size:

@@ -599,7 +599,7 @@ def test_extreme_shapes_match_oracle(cfg):
 
 
 # ---------------------------------------------------------------------------------------------- top-2 routing
-def _check_top2(cfg, gemm_path, tol, seed=0, d_aux=0.7, residual=False):
+def _check_top2(cfg, gemm_path, tol, seed=0, d_aux=0.7, residual=False, expect_mix=True):
     from tests.gpu_helpers import check_second_choice
     data = si.gen_layer(cfg, seed=seed)
     g = GpuLayer(cfg, data, gemm_path=gemm_path, top2=True, residual=residual)
@@ -617,7 +617,8 @@ def _check_top2(cfg, gemm_path, tol, seed=0, d_aux=0.7, residual=False):
                           residual=residual)
     assert C == fwd["C"]
     keep = fwd["keep"]
-    assert keep[T:].any() and (~keep).any()                   # second choices do get slots, and some assignments overflow
+    if expect_mix:                                             # the case is meant to exercise both:
+        assert keep[T:].any() and (~keep).any()               # second choices do get slots, and some assignments overflow
     np.testing.assert_array_equal(g.view(sm.WS_SLOT).cpu().numpy(), fwd["slot"])
     np.testing.assert_array_equal(g.view(sm.WS_TOKEN_OF_SLOT).cpu().numpy(), fwd["token_of_slot"])
     np.testing.assert_array_equal(g.view(sm.WS_COUNT).cpu().numpy(), fwd["count_first"])   # f counts first choices
